@@ -1,0 +1,124 @@
+"""ctypes front end of the C oracle (test infrastructure; the product never imports this).
+
+Arrays are numpy: fp16 data travels as uint16 bit patterns so nothing is converted on the
+way in, results come back as float64.
+"""
+from __future__ import annotations
+
+import ctypes
+from typing import Optional
+
+import numpy as np
+
+from . import build as _build
+
+_lib = None
+
+
+def _load() -> ctypes.CDLL:
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(str(_build.build()))
+        i32, i64, ptr = ctypes.c_int32, ctypes.c_int64, ctypes.c_void_p
+        lib.oracle_num_threads.restype = ctypes.c_int
+        lib.oracle_num_threads.argtypes = []
+        lib.oracle_kv_append.restype = ctypes.c_int
+        lib.oracle_kv_append.argtypes = [ptr, ptr, ptr, ptr, ptr, ptr, i32, i32, i64,
+                                         i32, i32, i32, i32]
+        lib.oracle_decode_attention.restype = ctypes.c_int
+        lib.oracle_decode_attention.argtypes = [ptr, ptr, ptr, i64, ptr, ptr, ptr, ptr, ptr,
+                                                i32, i32, i64, i32, i32, i32, i32,
+                                                ctypes.c_float]
+        _lib = lib
+    return _lib
+
+
+def num_threads() -> int:
+    """Threads the oracle's (sequence, head) loop runs on."""
+    return int(_load().oracle_num_threads())
+
+
+def _bits(a: np.ndarray, writable: bool = False) -> np.ndarray:
+    """View an fp16 / uint16 array as contiguous uint16 bit patterns (no copy if possible)."""
+    if a.dtype == np.float16:
+        a = a.view(np.uint16)
+    if a.dtype != np.uint16:
+        raise TypeError(f"expected float16 or uint16 bits, got {a.dtype}")
+    if not a.flags.c_contiguous or (writable and not a.flags.writeable):
+        raise ValueError("oracle arrays must be C-contiguous (and writable where mutated)")
+    return a
+
+
+def _p(a: Optional[np.ndarray]):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+class OracleError(RuntimeError):
+    """Raised with the C oracle's negative return code."""
+
+    def __init__(self, code: int):
+        super().__init__({-1: "bad argument", -2: "seq_len out of range",
+                          -3: "block id out of range"}.get(code, f"code {code}"))
+        self.code = code
+
+
+def _table(block_table, batch):
+    if block_table is None:
+        return None, 0
+    t = np.ascontiguousarray(block_table, dtype=np.int32)
+    if t.ndim != 2 or t.shape[0] != batch:
+        raise ValueError("block_table must be [batch, max_blocks_per_seq]")
+    return t, t.shape[1]
+
+
+def kv_append(k_cache: np.ndarray, v_cache: np.ndarray, k_new: np.ndarray, v_new: np.ndarray,
+              seq_lens: np.ndarray, block_table: Optional[np.ndarray] = None) -> None:
+    """In-place append of the new token's k,v at logical position seq_lens[b]-1.
+
+    contiguous: caches are [B,H,s_max,D]; paged: pools are [P,H,T,D] and block_table [B,M].
+    """
+    kb, vb = _bits(k_cache, True), _bits(v_cache, True)
+    kn, vn = _bits(np.ascontiguousarray(k_new)), _bits(np.ascontiguousarray(v_new))
+    batch, heads, head_dim = kn.shape
+    lens = np.ascontiguousarray(seq_lens, dtype=np.int32)
+    table, max_blocks = _table(block_table, batch)
+    if table is None:
+        s_max, block_tokens, phys = kb.shape[2], 0, 0
+    else:
+        s_max, block_tokens, phys = 0, kb.shape[2], kb.shape[0]
+    rc = _load().oracle_kv_append(_p(kb), _p(vb), _p(kn), _p(vn), _p(lens), _p(table),
+                                  max_blocks, block_tokens, phys, batch, heads, head_dim, s_max)
+    if rc:
+        raise OracleError(rc)
+
+
+def decode_attention(q: np.ndarray, k_cache: np.ndarray, v_cache: np.ndarray,
+                     seq_lens: np.ndarray, scale: float,
+                     block_table: Optional[np.ndarray] = None, want_weights: bool = False):
+    """softmax(scale * q K^T) V per (sequence, head) in fp64.
+
+    Returns (out [B,H,D] float64, lse [B,H] float64, weights [B,H,max(seq_lens)] or None).
+    """
+    qb = _bits(np.ascontiguousarray(q))
+    kb, vb = _bits(k_cache), _bits(v_cache)
+    batch, heads, head_dim = qb.shape
+    lens = np.ascontiguousarray(seq_lens, dtype=np.int32)
+    table, max_blocks = _table(block_table, batch)
+    if table is None:
+        s_max, block_tokens, phys = kb.shape[2], 0, 0
+    else:
+        s_max, block_tokens, phys = 0, kb.shape[2], kb.shape[0]
+    out = np.zeros((batch, heads, head_dim), dtype=np.float64)
+    lse = np.zeros((batch, heads), dtype=np.float64)
+    weights, stride = None, 0
+    if want_weights:
+        stride = int(lens.max()) if batch else 0
+        weights = np.zeros((batch, heads, max(stride, 1)), dtype=np.float64)
+        stride = max(stride, 1)
+    rc = _load().oracle_decode_attention(_p(out), _p(lse), _p(weights), stride, _p(qb), _p(kb),
+                                         _p(vb), _p(lens), _p(table), max_blocks, block_tokens,
+                                         phys, batch, heads, head_dim, s_max,
+                                         ctypes.c_float(scale))
+    if rc:
+        raise OracleError(rc)
+    return out, lse, weights
