@@ -1,0 +1,145 @@
+/*
+ * instinfer.h -- C ABI of the decode-attention library (sm_100a).
+ *
+ * One decode step of one transformer layer, per (sequence, head): the newest token's k,v
+ * are appended to that sequence's fp16 KV cache, then its single query row computes
+ * q.K^T over every cached key, a softmax scaled by `scale`, and the weighted sum of V.
+ * This is the work the paper moves into the storage drive together with the KV cache:
+ * the decode-phase "Logit" and "Attend" operators (Sec. III-B) of
+ * Attention(Q,K,V) = softmax(Q K^T / sqrt(d_k)) V (Sec. II-A) with a KV cache (Sec. II-B).
+ *
+ * Conventions common to every entry point
+ * ---------------------------------------
+ * - Every pointer is a DEVICE pointer unless a comment says "host".  Data pointers must be
+ *   16-byte aligned.  The library allocates nothing, never synchronises, and only enqueues
+ *   work on `cuda_stream` (a cudaStream_t passed as void*; NULL = the default stream).  The
+ *   caller owns every buffer, the workspace included, and must keep it alive until the
+ *   enqueued work has run.
+ * - fp16 = IEEE binary16.  heads = number of attention heads (query heads == KV heads,
+ *   multi-head attention, Sec. II-A).  head_dim must be 128 (the paper's head size,
+ *   Sec. IV-C).
+ * - seq_lens[b] (int32, device, [batch]) is the length of sequence b AFTER this step's
+ *   append: the append writes logical position seq_lens[b]-1, attention covers positions
+ *   [0, seq_lens[b]) -- the new token attends to itself (Sec. II-B).  seq_lens[b] == 0
+ *   marks an inactive slot: nothing is appended, its output rows are 0 and its lse -inf.
+ * - Contiguous layout: K and V caches are [batch, heads, s_max, head_dim], row-major.
+ * - Paged layout (the counterpart of the paper's token-indexed page groups, Sec. IV-C):
+ *   K pool and V pool are each [num_phys_blocks, heads, block_tokens, head_dim]; logical
+ *   token i of sequence b lives in physical block block_table[b][i / block_tokens] at slot
+ *   i % block_tokens; block_table is int32 [batch, max_blocks_per_seq], shared by K and V.
+ *   Entries past a sequence's last block are never read.  block_tokens must be a positive
+ *   multiple of 8.
+ * - Cache slots outside [0, seq_lens[b]) are never read and never influence a result.
+ * - Return value: an instinfer_status.  Everything the host can check (null or misaligned
+ *   pointers, non-positive sizes, unsupported head_dim or block_tokens, a workspace that is
+ *   too small) fails before anything is enqueued.  A failed launch gives INSTINFER_ERR_CUDA.
+ * - Data-dependent violations are found on the device and never fault it: a bit is OR-ed
+ *   into *status_flags (int32, device, nullable; the caller zeroes it and reads it back
+ *   when it wants to know).  A sequence whose length is out of range is treated as
+ *   inactive (nothing appended, zero output).  A block-table entry outside
+ *   [0, num_phys_blocks) is not dereferenced: the append skips that sequence, attention
+ *   reads that block's rows as zeros (the sequence's output is then meaningless but finite).
+ *   No kernel traps, asserts or waits on another kernel.
+ * - batch == 0 is a valid empty call: INSTINFER_OK, nothing enqueued.
+ */
+#ifndef INSTINFER_H_
+#define INSTINFER_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    INSTINFER_OK = 0,
+    INSTINFER_ERR_INVALID_ARG = 1,   /* null / misaligned pointer, non-positive size, bad bound */
+    INSTINFER_ERR_UNSUPPORTED = 2,   /* head_dim != 128, block_tokens not a multiple of 8       */
+    INSTINFER_ERR_WORKSPACE = 3,     /* workspace null or smaller than instinfer_workspace_bytes */
+    INSTINFER_ERR_CUDA = 4           /* the CUDA runtime refused a launch                        */
+} instinfer_status;
+
+/* Bits OR-ed into *status_flags by the kernels. */
+#define INSTINFER_FLAG_SEQ_LEN_RANGE 1  /* seq_lens[b] < 0, beyond the cache capacity, or beyond max_seq_len */
+#define INSTINFER_FLAG_BLOCK_RANGE   2  /* a block_table entry that had to be read lies outside [0, num_phys_blocks) */
+
+/*
+ * Append (Sec. II-B: the new token's k,v join the cache; Sec. IV-C, batch writing of the
+ * decode phase's new vectors).  Copies the bit patterns of k_new[b][h][:] and v_new[b][h][:]
+ * (fp16 [batch, heads, head_dim]) into logical position seq_lens[b]-1 of the caches.
+ *   block_table == NULL : contiguous caches [batch, heads, s_max, head_dim];
+ *                         max_blocks_per_seq, block_tokens, num_phys_blocks are ignored.
+ *   block_table != NULL : paged pools; s_max is ignored.
+ * k_cache / v_cache are the only buffers this call mutates, and only those rows.
+ */
+int instinfer_kv_append(void *k_cache, void *v_cache,
+                        const void *k_new, const void *v_new,
+                        const int32_t *seq_lens,
+                        const int32_t *block_table, int32_t max_blocks_per_seq,
+                        int32_t block_tokens, int64_t num_phys_blocks,
+                        int32_t batch, int32_t heads, int32_t head_dim, int32_t s_max,
+                        int32_t *status_flags, void *cuda_stream);
+
+/*
+ * Decode attention over a contiguous cache (Sec. II-A definition, Sec. II-B/III-B decode
+ * form): out[b][h][:] = softmax_i(scale * q[b][h].K[b][h][i]) . V[b][h][i], i < seq_lens[b].
+ *   out          fp16 [batch, heads, head_dim]; fp32 accumulation, rounded once (nearest even)
+ *   lse          fp32 [batch, heads], nullable: max_i s_i + ln sum_i exp(s_i - max), s = scale*q.k
+ *   q            fp16 [batch, heads, head_dim]
+ *   max_seq_len  host upper bound on every seq_lens[b], 1 <= max_seq_len <= s_max; a longer
+ *                sequence is treated as inactive and flagged
+ *   workspace    at least instinfer_workspace_bytes(batch, heads, head_dim, max_seq_len) bytes;
+ *                holds the per-split partial outputs between the two kernels; contents are
+ *                scratch before and after the call
+ */
+int instinfer_decode_attention(void *out, float *lse, const void *q,
+                               const void *k_cache, const void *v_cache,
+                               const int32_t *seq_lens,
+                               int32_t batch, int32_t heads, int32_t head_dim,
+                               int32_t s_max, int32_t max_seq_len, float scale,
+                               void *workspace, size_t workspace_bytes,
+                               int32_t *status_flags, void *cuda_stream);
+
+/*
+ * The same over block-paged pools with a block table (Sec. IV-C token-indexed groups).
+ * max_seq_len <= max_blocks_per_seq * block_tokens.  The split of a sequence into partial
+ * results follows logical token positions only, so the result does not depend on which
+ * physical blocks hold the tokens.
+ */
+int instinfer_decode_attention_paged(void *out, float *lse, const void *q,
+                                     const void *k_pool, const void *v_pool,
+                                     const int32_t *block_table, const int32_t *seq_lens,
+                                     int32_t batch, int32_t heads, int32_t head_dim,
+                                     int32_t block_tokens, int32_t max_blocks_per_seq,
+                                     int64_t num_phys_blocks, int32_t max_seq_len, float scale,
+                                     void *workspace, size_t workspace_bytes,
+                                     int32_t *status_flags, void *cuda_stream);
+
+/*
+ * Workspace size (bytes, host computation only) for a call with these sizes under the
+ * current split plan; 0 if an argument is invalid.
+ */
+size_t instinfer_workspace_bytes(int32_t batch, int32_t heads, int32_t head_dim,
+                                 int32_t max_seq_len);
+
+/*
+ * Split plan.  A sequence is cut at multiples of `chunk_tokens` logical positions; each
+ * chunk of each (sequence, head) is reduced by one thread block and the partial results are
+ * merged by log-sum-exp (no counterpart in the paper, whose engine streams token groups
+ * through parallel GeMV units, Sec. IV-B).  instinfer_plan_chunk_tokens returns the chunk
+ * the library would use for these sizes (0 if an argument is invalid).
+ * instinfer_set_chunk_tokens(n) forces chunk_tokens = n for later calls of this process
+ * (n > 0, a multiple of 64), n == 0 restores the automatic choice; it returns
+ * INSTINFER_OK or INSTINFER_ERR_INVALID_ARG.  Not thread-safe against concurrent calls.
+ */
+int32_t instinfer_plan_chunk_tokens(int32_t batch, int32_t heads, int32_t max_seq_len);
+int instinfer_set_chunk_tokens(int32_t chunk_tokens);
+
+/* Static, human-readable text for a status value (host pointer, never NULL). */
+const char *instinfer_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* INSTINFER_H_ */
