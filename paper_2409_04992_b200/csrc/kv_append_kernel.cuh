@@ -1,0 +1,64 @@
+// KV append for sm_100a: the new token's k,v rows join the cache (Sec. II-B; the decode
+// phase's incremental writes of Sec. IV-C).  A pure bit copy: one thread moves one 16-byte
+// segment of K and one of V, 16 threads cover a (sequence, head) row pair.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace instinfer {
+
+struct AppendParams {
+    uint4 *k_cache;
+    uint4 *v_cache;
+    const uint4 *k_new;           // [batch, heads, 128] fp16 = 16 uint4 per row
+    const uint4 *v_new;
+    const int32_t *seq_lens;
+    const int32_t *block_table;   // nullptr: contiguous
+    int32_t *status;              // nullable
+    int64_t num_phys_blocks;
+    int32_t batch;
+    int32_t heads;
+    int32_t s_max;
+    int32_t block_tokens;
+    int32_t max_blocks_per_seq;
+};
+
+constexpr int kAppendThreads = 128;
+constexpr int kSegsPerRow = 16;   // 256 B / 16 B
+
+__global__ void __launch_bounds__(kAppendThreads)
+kv_append_kernel(const AppendParams p)
+{
+    const int64_t idx = (int64_t)blockIdx.x * kAppendThreads + threadIdx.x;
+    const int64_t pair = idx / kSegsPerRow;
+    if (pair >= (int64_t)p.batch * p.heads) return;
+    const int seg = (int)(idx % kSegsPerRow);
+    const int b = (int)(pair / p.heads), h = (int)(pair % p.heads);
+    const bool reporter = seg == 0 && h == 0 && p.status != nullptr;
+
+    const int len = p.seq_lens[b];
+    if (len == 0) return;                                   // inactive slot
+    const int64_t capacity = p.block_table ? (int64_t)p.max_blocks_per_seq * p.block_tokens
+                                           : (int64_t)p.s_max;
+    if (len < 0 || len > capacity) {
+        if (reporter) atomicOr(p.status, 1);                // seq_len out of range
+        return;
+    }
+    const int pos = len - 1;
+    int64_t row;
+    if (p.block_table) {
+        const int phys = p.block_table[(int64_t)b * p.max_blocks_per_seq + pos / p.block_tokens];
+        if (phys < 0 || (int64_t)phys >= p.num_phys_blocks) {
+            if (reporter) atomicOr(p.status, 2);            // block id out of range
+            return;
+        }
+        row = ((int64_t)phys * p.heads + h) * p.block_tokens + pos % p.block_tokens;
+    } else {
+        row = pair * p.s_max + pos;
+    }
+    p.k_cache[row * kSegsPerRow + seg] = p.k_new[idx];
+    p.v_cache[row * kSegsPerRow + seg] = p.v_new[idx];
+}
+
+}  // namespace instinfer
