@@ -1,0 +1,144 @@
+"""Thin ctypes layer over libinstinfer.so: argument marshalling only.
+
+Function names mirror the C ABI (see include/instinfer.h for what each argument means).
+Tensors are torch CUDA tensors used as device memory; every step of the path runs in the
+library's kernels.  There is no fallback: if the library has not been built, loading fails.
+"""
+from __future__ import annotations
+
+import ctypes
+from pathlib import Path
+from typing import Optional
+
+import torch
+
+LIBRARY = Path(__file__).resolve().parent / "libinstinfer.so"
+
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA = range(5)
+FLAG_SEQ_LEN_RANGE, FLAG_BLOCK_RANGE = 1, 2
+
+_lib: Optional[ctypes.CDLL] = None
+
+
+class InstInferError(RuntimeError):
+    def __init__(self, status: int):
+        super().__init__(f"instinfer status {status}: {status_string(status)}")
+        self.status = status
+
+
+def load() -> ctypes.CDLL:
+    """dlopen the CUDA library; raises if it is missing (build it with paper_2409_04992_b200.build)."""
+    global _lib
+    if _lib is None:
+        if not LIBRARY.exists():
+            raise RuntimeError(f"{LIBRARY} is missing: run `python -m paper_2409_04992_b200.build` "
+                               "(there is no CPU or PyTorch fallback)")
+        lib = ctypes.CDLL(str(LIBRARY))
+        i32, i64, ptr, f32, sz = (ctypes.c_int32, ctypes.c_int64, ctypes.c_void_p,
+                                  ctypes.c_float, ctypes.c_size_t)
+        lib.instinfer_kv_append.restype = ctypes.c_int
+        lib.instinfer_kv_append.argtypes = [ptr, ptr, ptr, ptr, ptr, ptr, i32, i32, i64,
+                                            i32, i32, i32, i32, ptr, ptr]
+        lib.instinfer_decode_attention.restype = ctypes.c_int
+        lib.instinfer_decode_attention.argtypes = [ptr, ptr, ptr, ptr, ptr, ptr, i32, i32, i32,
+                                                   i32, i32, f32, ptr, sz, ptr, ptr]
+        lib.instinfer_decode_attention_paged.restype = ctypes.c_int
+        lib.instinfer_decode_attention_paged.argtypes = [ptr, ptr, ptr, ptr, ptr, ptr, ptr,
+                                                         i32, i32, i32, i32, i32, i64, i32, f32,
+                                                         ptr, sz, ptr, ptr]
+        lib.instinfer_workspace_bytes.restype = sz
+        lib.instinfer_workspace_bytes.argtypes = [i32, i32, i32, i32]
+        lib.instinfer_plan_chunk_tokens.restype = i32
+        lib.instinfer_plan_chunk_tokens.argtypes = [i32, i32, i32]
+        lib.instinfer_set_chunk_tokens.restype = ctypes.c_int
+        lib.instinfer_set_chunk_tokens.argtypes = [i32]
+        lib.instinfer_status_string.restype = ctypes.c_char_p
+        lib.instinfer_status_string.argtypes = [ctypes.c_int]
+        _lib = lib
+    return _lib
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    return None if t is None else t.data_ptr()
+
+
+def _stream(stream: Optional[torch.cuda.Stream]) -> Optional[int]:
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return s.cuda_stream or None
+
+
+def _check(status: int) -> None:
+    if status != OK:
+        raise InstInferError(status)
+
+
+def status_string(status: int) -> str:
+    return load().instinfer_status_string(int(status)).decode()
+
+
+def workspace_bytes(batch: int, heads: int, head_dim: int, max_seq_len: int) -> int:
+    return int(load().instinfer_workspace_bytes(batch, heads, head_dim, max_seq_len))
+
+
+def plan_chunk_tokens(batch: int, heads: int, max_seq_len: int) -> int:
+    return int(load().instinfer_plan_chunk_tokens(batch, heads, max_seq_len))
+
+
+def set_chunk_tokens(chunk_tokens: int) -> None:
+    _check(load().instinfer_set_chunk_tokens(int(chunk_tokens)))
+
+
+def kv_append(k_cache: torch.Tensor, v_cache: torch.Tensor, k_new: torch.Tensor,
+              v_new: torch.Tensor, seq_lens: torch.Tensor,
+              block_table: Optional[torch.Tensor] = None,
+              status_flags: Optional[torch.Tensor] = None,
+              stream: Optional[torch.cuda.Stream] = None) -> None:
+    """instinfer_kv_append.  Caches: [B,H,s_max,D] (block_table None) or pools [P,H,T,D]."""
+    batch, heads, head_dim = k_new.shape
+    if block_table is None:
+        max_blocks, block_tokens, phys, s_max = 0, 0, 0, k_cache.shape[2]
+    else:
+        max_blocks, block_tokens, phys, s_max = (block_table.shape[1], k_cache.shape[2],
+                                                 k_cache.shape[0], 0)
+    _check(load().instinfer_kv_append(
+        _ptr(k_cache), _ptr(v_cache), _ptr(k_new), _ptr(v_new), _ptr(seq_lens),
+        _ptr(block_table), max_blocks, block_tokens, phys, batch, heads, head_dim, s_max,
+        _ptr(status_flags), _stream(stream)))
+
+
+def decode_attention(out: torch.Tensor, lse: Optional[torch.Tensor], q: torch.Tensor,
+                     k_cache: torch.Tensor, v_cache: torch.Tensor, seq_lens: torch.Tensor,
+                     max_seq_len: int, scale: float, workspace: torch.Tensor,
+                     status_flags: Optional[torch.Tensor] = None,
+                     stream: Optional[torch.cuda.Stream] = None) -> None:
+    """instinfer_decode_attention over contiguous caches [B,H,s_max,D]."""
+    batch, heads, head_dim = q.shape
+    _check(load().instinfer_decode_attention(
+        _ptr(out), _ptr(lse), _ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(seq_lens),
+        batch, heads, head_dim, k_cache.shape[2], int(max_seq_len), float(scale),
+        _ptr(workspace), workspace.numel() * workspace.element_size(),
+        _ptr(status_flags), _stream(stream)))
+
+
+def decode_attention_paged(out: torch.Tensor, lse: Optional[torch.Tensor], q: torch.Tensor,
+                           k_pool: torch.Tensor, v_pool: torch.Tensor,
+                           block_table: torch.Tensor, seq_lens: torch.Tensor,
+                           max_seq_len: int, scale: float, workspace: torch.Tensor,
+                           status_flags: Optional[torch.Tensor] = None,
+                           stream: Optional[torch.cuda.Stream] = None) -> None:
+    """instinfer_decode_attention_paged over pools [P,H,T,D] with block_table [B,M]."""
+    batch, heads, head_dim = q.shape
+    _check(load().instinfer_decode_attention_paged(
+        _ptr(out), _ptr(lse), _ptr(q), _ptr(k_pool), _ptr(v_pool), _ptr(block_table),
+        _ptr(seq_lens), batch, heads, head_dim, k_pool.shape[2], block_table.shape[1],
+        k_pool.shape[0], int(max_seq_len), float(scale), _ptr(workspace),
+        workspace.numel() * workspace.element_size(), _ptr(status_flags), _stream(stream)))
+
+
+def alloc_workspace(batch: int, heads: int, head_dim: int, max_seq_len: int,
+                    device: torch.device | str = "cuda") -> torch.Tensor:
+    """A byte tensor of the size the library asks for under the current split plan."""
+    need = workspace_bytes(batch, heads, head_dim, max_seq_len)
+    if need == 0:
+        raise InstInferError(ERR_INVALID_ARG)
+    return torch.empty(need, dtype=torch.uint8, device=device)

@@ -1,0 +1,281 @@
+// C ABI of the decode-attention library: argument checks, the split plan, the workspace
+// layout and the launches.  Nothing here allocates or synchronises; all work is enqueued on
+// the caller's stream.
+#include "../../include/instinfer.h"
+
+#include <cmath>
+
+#include "decode_attention_kernels.cuh"
+#include "kv_append_kernel.cuh"
+
+namespace {
+
+using namespace instinfer;
+
+constexpr int kMaxDevices = 64;
+constexpr int kChunkGranule = 64;        // chunk_tokens is a multiple of this
+constexpr int kChunkCeiling = 2048;      // automatic plan: chunk never longer than this ...
+constexpr int kChunkFloor = 256;         // ... nor shorter than this, sequence permitting
+constexpr int kTargetWaves = 8;          // automatic plan: aim for this many waves of blocks
+
+int g_forced_chunk = 0;
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+bool usable(const void *p) { return p != nullptr && aligned16(p); }
+
+int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
+
+// SM count of the current device; 148 (B200) when no device can be asked.
+int sm_count()
+{
+    static int cached[kMaxDevices] = {0};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+        (void)cudaGetLastError();
+        return 148;
+    }
+    if (cached[dev] == 0) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) {
+            (void)cudaGetLastError();
+            n = 148;
+        }
+        cached[dev] = n;
+    }
+    return cached[dev];
+}
+
+struct SplitPlan {
+    int32_t chunk_tokens;
+    int32_t n_splits;
+};
+
+// Cuts are at multiples of chunk_tokens in logical token positions, the same for every
+// sequence, so a result never depends on the physical placement of blocks.
+SplitPlan make_plan(int64_t pairs, int32_t max_seq_len)
+{
+    int64_t chunk;
+    if (g_forced_chunk > 0) {
+        chunk = g_forced_chunk;
+    } else {
+        const int64_t slots = (int64_t)sm_count() * kCtasPerSm;
+        const int64_t fewest = ceil_div(max_seq_len, kChunkCeiling);
+        const int64_t most = ceil_div(max_seq_len, kChunkFloor);
+        int64_t n = ceil_div(slots * kTargetWaves, pairs);
+        if (n > most) n = most;
+        if (n < fewest) n = fewest;
+        chunk = ceil_div(ceil_div(max_seq_len, n), kChunkGranule) * kChunkGranule;
+    }
+    SplitPlan plan;
+    plan.chunk_tokens = (int32_t)chunk;
+    plan.n_splits = (int32_t)ceil_div(max_seq_len, chunk);
+    return plan;
+}
+
+size_t workspace_for(int64_t pairs, const SplitPlan &plan)
+{
+    const size_t floats = (size_t)pairs * (size_t)plan.n_splits * (kHeadDim + 1);
+    return (floats * sizeof(float) + 255) / 256 * 256 + 256;
+}
+
+bool sizes_ok(int32_t batch, int32_t heads, int32_t max_seq_len)
+{
+    if (batch < 0 || heads <= 0 || max_seq_len <= 0) return false;
+    return (int64_t)batch * heads <= (int64_t)1 << 24;     // keeps every grid below 2^31 blocks
+}
+
+int ensure_split_smem(bool paged)
+{
+    static bool done[kMaxDevices][2] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return INSTINFER_ERR_CUDA;
+    if (!done[dev][paged]) {
+        const cudaError_t err = paged
+            ? cudaFuncSetAttribute(decode_attn_split_kernel<true>,
+                                   cudaFuncAttributeMaxDynamicSharedMemorySize, kSplitSmemBytes)
+            : cudaFuncSetAttribute(decode_attn_split_kernel<false>,
+                                   cudaFuncAttributeMaxDynamicSharedMemorySize, kSplitSmemBytes);
+        if (err != cudaSuccess) {
+            (void)cudaGetLastError();
+            return INSTINFER_ERR_CUDA;
+        }
+        done[dev][paged] = true;
+    }
+    return INSTINFER_OK;
+}
+
+int launch_attention(AttnParams p, bool paged, int32_t batch, void *workspace,
+                     size_t workspace_bytes, cudaStream_t stream)
+{
+    const int64_t pairs = (int64_t)batch * p.heads;
+    const SplitPlan plan = make_plan(pairs, p.max_seq_len);
+    if (workspace == nullptr || !aligned16(workspace) || workspace_bytes < workspace_for(pairs, plan))
+        return INSTINFER_ERR_WORKSPACE;
+    if (pairs * plan.n_splits >= (int64_t)1 << 31) return INSTINFER_ERR_INVALID_ARG;
+    p.chunk_tokens = plan.chunk_tokens;
+    p.n_splits = plan.n_splits;
+    p.part_o = static_cast<float *>(workspace);
+    p.part_lse = p.part_o + (size_t)pairs * plan.n_splits * kHeadDim;
+
+    const int rc = ensure_split_smem(paged);
+    if (rc != INSTINFER_OK) return rc;
+    const unsigned grid = (unsigned)(pairs * plan.n_splits);
+    if (paged)
+        decode_attn_split_kernel<true><<<grid, kThreads, kSplitSmemBytes, stream>>>(p);
+    else
+        decode_attn_split_kernel<false><<<grid, kThreads, kSplitSmemBytes, stream>>>(p);
+    if (cudaGetLastError() != cudaSuccess) return INSTINFER_ERR_CUDA;
+    if (plan.n_splits > 1) {
+        lse_merge_kernel<<<(unsigned)pairs, kHeadDim, 0, stream>>>(p);
+        if (cudaGetLastError() != cudaSuccess) return INSTINFER_ERR_CUDA;
+    }
+    return INSTINFER_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int instinfer_kv_append(void *k_cache, void *v_cache, const void *k_new, const void *v_new,
+                        const int32_t *seq_lens, const int32_t *block_table,
+                        int32_t max_blocks_per_seq, int32_t block_tokens, int64_t num_phys_blocks,
+                        int32_t batch, int32_t heads, int32_t head_dim, int32_t s_max,
+                        int32_t *status_flags, void *cuda_stream)
+{
+    if (batch < 0 || heads <= 0 || head_dim <= 0) return INSTINFER_ERR_INVALID_ARG;
+    if (head_dim != kHeadDim) return INSTINFER_ERR_UNSUPPORTED;
+    if ((int64_t)batch * heads > (int64_t)1 << 24) return INSTINFER_ERR_INVALID_ARG;
+    if (block_table != nullptr) {
+        if (max_blocks_per_seq <= 0 || block_tokens <= 0 || num_phys_blocks <= 0)
+            return INSTINFER_ERR_INVALID_ARG;
+        if (block_tokens % 8 != 0) return INSTINFER_ERR_UNSUPPORTED;
+    } else if (s_max <= 0) {
+        return INSTINFER_ERR_INVALID_ARG;
+    }
+    if (batch == 0) return INSTINFER_OK;
+    if (!usable(k_cache) || !usable(v_cache) || !usable(k_new) || !usable(v_new) || seq_lens == nullptr)
+        return INSTINFER_ERR_INVALID_ARG;
+
+    AppendParams p;
+    p.k_cache = static_cast<uint4 *>(k_cache);
+    p.v_cache = static_cast<uint4 *>(v_cache);
+    p.k_new = static_cast<const uint4 *>(k_new);
+    p.v_new = static_cast<const uint4 *>(v_new);
+    p.seq_lens = seq_lens;
+    p.block_table = block_table;
+    p.status = status_flags;
+    p.num_phys_blocks = num_phys_blocks;
+    p.batch = batch;
+    p.heads = heads;
+    p.s_max = s_max;
+    p.block_tokens = block_tokens;
+    p.max_blocks_per_seq = max_blocks_per_seq;
+    const int64_t threads = (int64_t)batch * heads * kSegsPerRow;
+    const unsigned grid = (unsigned)ceil_div(threads, kAppendThreads);
+    kv_append_kernel<<<grid, kAppendThreads, 0, static_cast<cudaStream_t>(cuda_stream)>>>(p);
+    return cudaGetLastError() == cudaSuccess ? INSTINFER_OK : INSTINFER_ERR_CUDA;
+}
+
+int instinfer_decode_attention(void *out, float *lse, const void *q, const void *k_cache,
+                               const void *v_cache, const int32_t *seq_lens, int32_t batch,
+                               int32_t heads, int32_t head_dim, int32_t s_max,
+                               int32_t max_seq_len, float scale, void *workspace,
+                               size_t workspace_bytes, int32_t *status_flags, void *cuda_stream)
+{
+    if (head_dim <= 0 || !sizes_ok(batch, heads, max_seq_len) || s_max <= 0 || max_seq_len > s_max)
+        return INSTINFER_ERR_INVALID_ARG;
+    if (head_dim != kHeadDim) return INSTINFER_ERR_UNSUPPORTED;
+    if (!std::isfinite(scale)) return INSTINFER_ERR_INVALID_ARG;
+    if (batch == 0) return INSTINFER_OK;
+    if (!usable(out) || !usable(q) || !usable(k_cache) || !usable(v_cache) || seq_lens == nullptr)
+        return INSTINFER_ERR_INVALID_ARG;
+
+    AttnParams p = {};
+    p.q = static_cast<const __half *>(q);
+    p.k = static_cast<const __half *>(k_cache);
+    p.v = static_cast<const __half *>(v_cache);
+    p.seq_lens = seq_lens;
+    p.out = static_cast<__half *>(out);
+    p.lse = lse;
+    p.status = status_flags;
+    p.heads = heads;
+    p.s_max = s_max;
+    p.max_seq_len = max_seq_len;
+    p.scale_log2e = scale * 1.44269504088896340736f;
+    return launch_attention(p, false, batch, workspace, workspace_bytes,
+                            static_cast<cudaStream_t>(cuda_stream));
+}
+
+int instinfer_decode_attention_paged(void *out, float *lse, const void *q, const void *k_pool,
+                                     const void *v_pool, const int32_t *block_table,
+                                     const int32_t *seq_lens, int32_t batch, int32_t heads,
+                                     int32_t head_dim, int32_t block_tokens,
+                                     int32_t max_blocks_per_seq, int64_t num_phys_blocks,
+                                     int32_t max_seq_len, float scale, void *workspace,
+                                     size_t workspace_bytes, int32_t *status_flags,
+                                     void *cuda_stream)
+{
+    if (head_dim <= 0 || !sizes_ok(batch, heads, max_seq_len) || block_tokens <= 0 ||
+        max_blocks_per_seq <= 0 || num_phys_blocks <= 0)
+        return INSTINFER_ERR_INVALID_ARG;
+    if (head_dim != kHeadDim || block_tokens % 8 != 0) return INSTINFER_ERR_UNSUPPORTED;
+    if ((int64_t)max_seq_len > (int64_t)max_blocks_per_seq * block_tokens || !std::isfinite(scale))
+        return INSTINFER_ERR_INVALID_ARG;
+    if (batch == 0) return INSTINFER_OK;
+    if (!usable(out) || !usable(q) || !usable(k_pool) || !usable(v_pool) || seq_lens == nullptr ||
+        block_table == nullptr)
+        return INSTINFER_ERR_INVALID_ARG;
+
+    AttnParams p = {};
+    p.q = static_cast<const __half *>(q);
+    p.k = static_cast<const __half *>(k_pool);
+    p.v = static_cast<const __half *>(v_pool);
+    p.seq_lens = seq_lens;
+    p.block_table = block_table;
+    p.out = static_cast<__half *>(out);
+    p.lse = lse;
+    p.status = status_flags;
+    p.num_phys_blocks = num_phys_blocks;
+    p.heads = heads;
+    p.block_tokens = block_tokens;
+    p.max_blocks_per_seq = max_blocks_per_seq;
+    p.max_seq_len = max_seq_len;
+    p.scale_log2e = scale * 1.44269504088896340736f;
+    return launch_attention(p, true, batch, workspace, workspace_bytes,
+                            static_cast<cudaStream_t>(cuda_stream));
+}
+
+size_t instinfer_workspace_bytes(int32_t batch, int32_t heads, int32_t head_dim, int32_t max_seq_len)
+{
+    if (head_dim != kHeadDim || !sizes_ok(batch, heads, max_seq_len)) return 0;
+    const int64_t pairs = (int64_t)batch * heads;
+    if (pairs == 0) return 256;
+    return workspace_for(pairs, make_plan(pairs, max_seq_len));
+}
+
+int32_t instinfer_plan_chunk_tokens(int32_t batch, int32_t heads, int32_t max_seq_len)
+{
+    if (!sizes_ok(batch, heads, max_seq_len) || batch == 0) return 0;
+    return make_plan((int64_t)batch * heads, max_seq_len).chunk_tokens;
+}
+
+int instinfer_set_chunk_tokens(int32_t chunk_tokens)
+{
+    if (chunk_tokens < 0 || chunk_tokens % kChunkGranule != 0) return INSTINFER_ERR_INVALID_ARG;
+    g_forced_chunk = chunk_tokens;
+    return INSTINFER_OK;
+}
+
+const char *instinfer_status_string(int status)
+{
+    switch (status) {
+    case INSTINFER_OK: return "ok";
+    case INSTINFER_ERR_INVALID_ARG: return "invalid argument";
+    case INSTINFER_ERR_UNSUPPORTED: return "unsupported head_dim or block_tokens";
+    case INSTINFER_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case INSTINFER_ERR_CUDA: return "CUDA launch failed";
+    default: return "unknown status";
+    }
+}
+
+}  // extern "C"
