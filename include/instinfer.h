@@ -136,6 +136,15 @@ size_t instinfer_workspace_bytes(int32_t batch, int32_t heads, int32_t head_dim,
 int32_t instinfer_plan_chunk_tokens(int32_t batch, int32_t heads, int32_t max_seq_len);
 int instinfer_set_chunk_tokens(int32_t chunk_tokens);
 
+/*
+ * Measurement aid (no counterpart in the paper).  Given two cudaEvent_t (as void*, owned by
+ * the caller), later attention calls of this process record `before_split` on the stream
+ * just before the split-KV kernel and `after_split` just after it, so that the caller can
+ * time that one kernel where it runs; (NULL, NULL) switches this off, one NULL is invalid.
+ * Each call overwrites the previous recording of the same events.  Not thread-safe.
+ */
+int instinfer_set_timing_events(void *before_split, void *after_split);
+
 /* Static, human-readable text for a status value (host pointer, never NULL). */
 const char *instinfer_status_string(int status);
 

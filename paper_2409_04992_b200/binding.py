@@ -52,6 +52,8 @@ def load() -> ctypes.CDLL:
         lib.instinfer_plan_chunk_tokens.argtypes = [i32, i32, i32]
         lib.instinfer_set_chunk_tokens.restype = ctypes.c_int
         lib.instinfer_set_chunk_tokens.argtypes = [i32]
+        lib.instinfer_set_timing_events.restype = ctypes.c_int
+        lib.instinfer_set_timing_events.argtypes = [ptr, ptr]
         lib.instinfer_status_string.restype = ctypes.c_char_p
         lib.instinfer_status_string.argtypes = [ctypes.c_int]
         _lib = lib
@@ -86,6 +88,14 @@ def plan_chunk_tokens(batch: int, heads: int, max_seq_len: int) -> int:
 
 def set_chunk_tokens(chunk_tokens: int) -> None:
     _check(load().instinfer_set_chunk_tokens(int(chunk_tokens)))
+
+
+def set_timing_events(before_split: Optional[torch.cuda.Event],
+                      after_split: Optional[torch.cuda.Event]) -> None:
+    """instinfer_set_timing_events with torch events (already created, i.e. recorded once)."""
+    _check(load().instinfer_set_timing_events(
+        None if before_split is None else before_split.cuda_event,
+        None if after_split is None else after_split.cuda_event))
 
 
 def kv_append(k_cache: torch.Tensor, v_cache: torch.Tensor, k_new: torch.Tensor,

@@ -19,6 +19,8 @@ constexpr int kChunkFloor = 256;         // ... nor shorter than this, sequence 
 constexpr int kTargetWaves = 8;          // automatic plan: aim for this many waves of blocks
 
 int g_forced_chunk = 0;
+cudaEvent_t g_before_split = nullptr;    // measurement aid, see instinfer_set_timing_events
+cudaEvent_t g_after_split = nullptr;
 
 bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 bool usable(const void *p) { return p != nullptr && aligned16(p); }
@@ -120,10 +122,12 @@ int launch_attention(AttnParams p, bool paged, int32_t batch, void *workspace,
     const int rc = ensure_split_smem(paged);
     if (rc != INSTINFER_OK) return rc;
     const unsigned grid = (unsigned)(pairs * plan.n_splits);
+    if (g_before_split) cudaEventRecord(g_before_split, stream);
     if (paged)
         decode_attn_split_kernel<true><<<grid, kThreads, kSplitSmemBytes, stream>>>(p);
     else
         decode_attn_split_kernel<false><<<grid, kThreads, kSplitSmemBytes, stream>>>(p);
+    if (g_after_split) cudaEventRecord(g_after_split, stream);
     if (cudaGetLastError() != cudaSuccess) return INSTINFER_ERR_CUDA;
     if (plan.n_splits > 1) {
         lse_merge_kernel<<<(unsigned)pairs, kHeadDim, 0, stream>>>(p);
@@ -263,6 +267,14 @@ int instinfer_set_chunk_tokens(int32_t chunk_tokens)
 {
     if (chunk_tokens < 0 || chunk_tokens % kChunkGranule != 0) return INSTINFER_ERR_INVALID_ARG;
     g_forced_chunk = chunk_tokens;
+    return INSTINFER_OK;
+}
+
+int instinfer_set_timing_events(void *before_split, void *after_split)
+{
+    if ((before_split == nullptr) != (after_split == nullptr)) return INSTINFER_ERR_INVALID_ARG;
+    g_before_split = static_cast<cudaEvent_t>(before_split);
+    g_after_split = static_cast<cudaEvent_t>(after_split);
     return INSTINFER_OK;
 }
 
