@@ -117,6 +117,41 @@ int instinfer_decode_attention_paged(void *out, float *lse, const void *q,
                                      int32_t *status_flags, void *cuda_stream);
 
 /*
+ * Decode attention without a caller-supplied workspace (the paper has no counterpart: its
+ * engine has no split partials to park).  For callers that have no device memory of their
+ * own to hand over and may not ask the driver for any: a serving engine that gave its whole
+ * memory budget to the KV pool at start-up, a plug-in that runs under someone else's
+ * allocator, a latency-critical loop in which an allocation's implicit device
+ * synchronisation is not acceptable.  The partial results live in a 16 MiB array that is
+ * part of the library image, so every GPU context that loads the library carries those
+ * 16 MiB until it exits.
+ *   block_table == NULL : contiguous caches, arguments as instinfer_decode_attention
+ *                         (block_tokens, max_blocks_per_seq, num_phys_blocks ignored);
+ *   block_table != NULL : paged pools, arguments as instinfer_decode_attention_paged
+ *                         (s_max ignored).
+ * Results are those of the two entry points above, bit for bit.
+ * Limits and rules:
+ * - instinfer_workspace_bytes(batch, heads, head_dim, max_seq_len) must not exceed
+ *   INSTINFER_STATIC_WORKSPACE_BYTES; otherwise INSTINFER_ERR_WORKSPACE, nothing enqueued.
+ * - The first call on each device looks up the array's device address (the device must be
+ *   current); make that first call outside any stream capture.  No call allocates or frees.
+ * - All calls on a device share the one array, which keeps whatever the last call left in
+ *   it.  Nothing in it needs to start at zero: a call only reads back the slots it has
+ *   itself just written.  Two calls that can run at the same time on the GPU (different
+ *   streams, no dependency between them) race on it and corrupt each other's results:
+ *   order them on one stream or with events.
+ */
+#define INSTINFER_STATIC_WORKSPACE_BYTES ((size_t)16 << 20)
+int instinfer_decode_attention_static(void *out, float *lse, const void *q,
+                                      const void *k_cache, const void *v_cache,
+                                      const int32_t *block_table, const int32_t *seq_lens,
+                                      int32_t batch, int32_t heads, int32_t head_dim,
+                                      int32_t s_max, int32_t block_tokens,
+                                      int32_t max_blocks_per_seq, int64_t num_phys_blocks,
+                                      int32_t max_seq_len, float scale,
+                                      int32_t *status_flags, void *cuda_stream);
+
+/*
  * Workspace size (bytes, host computation only) for a call with these sizes under the
  * current split plan; 0 if an argument is invalid.
  */

@@ -16,6 +16,7 @@ LIBRARY = Path(__file__).resolve().parent / "libinstinfer.so"
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA = range(5)
 FLAG_SEQ_LEN_RANGE, FLAG_BLOCK_RANGE = 1, 2
+STATIC_WORKSPACE_BYTES = 16 << 20
 
 _lib: Optional[ctypes.CDLL] = None
 
@@ -46,6 +47,10 @@ def load() -> ctypes.CDLL:
         lib.instinfer_decode_attention_paged.argtypes = [ptr, ptr, ptr, ptr, ptr, ptr, ptr,
                                                          i32, i32, i32, i32, i32, i64, i32, f32,
                                                          ptr, sz, ptr, ptr]
+        lib.instinfer_decode_attention_static.restype = ctypes.c_int
+        lib.instinfer_decode_attention_static.argtypes = [ptr, ptr, ptr, ptr, ptr, ptr, ptr,
+                                                          i32, i32, i32, i32, i32, i32, i64, i32,
+                                                          f32, ptr, ptr]
         lib.instinfer_workspace_bytes.restype = sz
         lib.instinfer_workspace_bytes.argtypes = [i32, i32, i32, i32]
         lib.instinfer_plan_chunk_tokens.restype = i32
@@ -143,6 +148,26 @@ def decode_attention_paged(out: torch.Tensor, lse: Optional[torch.Tensor], q: to
         _ptr(seq_lens), batch, heads, head_dim, k_pool.shape[2], block_table.shape[1],
         k_pool.shape[0], int(max_seq_len), float(scale), _ptr(workspace),
         workspace.numel() * workspace.element_size(), _ptr(status_flags), _stream(stream)))
+
+
+def decode_attention_static(out: torch.Tensor, lse: Optional[torch.Tensor], q: torch.Tensor,
+                            k_cache: torch.Tensor, v_cache: torch.Tensor,
+                            block_table: Optional[torch.Tensor], seq_lens: torch.Tensor,
+                            max_seq_len: int, scale: float,
+                            status_flags: Optional[torch.Tensor] = None,
+                            stream: Optional[torch.cuda.Stream] = None) -> None:
+    """instinfer_decode_attention_static: attention in the library's built-in scratch array,
+    for callers that cannot provide a workspace (block_table None = contiguous caches)."""
+    batch, heads, head_dim = q.shape
+    if block_table is None:
+        s_max, block_tokens, max_blocks, phys = k_cache.shape[2], 0, 0, 0
+    else:
+        s_max, block_tokens, max_blocks, phys = (0, k_cache.shape[2], block_table.shape[1],
+                                                 k_cache.shape[0])
+    _check(load().instinfer_decode_attention_static(
+        _ptr(out), _ptr(lse), _ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(block_table),
+        _ptr(seq_lens), batch, heads, head_dim, s_max, block_tokens, max_blocks, phys,
+        int(max_seq_len), float(scale), _ptr(status_flags), _stream(stream)))
 
 
 def alloc_workspace(batch: int, heads: int, head_dim: int, max_seq_len: int,

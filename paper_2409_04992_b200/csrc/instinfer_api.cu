@@ -136,6 +136,33 @@ int launch_attention(AttnParams p, bool paged, int32_t batch, void *workspace,
     return INSTINFER_OK;
 }
 
+// Built-in scratch for instinfer_decode_attention_static: lives in every GPU context that
+// loads the library, from load until exit.  In host code this name is only a handle for
+// cudaGetSymbolAddress, never a device address.
+constexpr size_t kStaticWorkspaceBytes = INSTINFER_STATIC_WORKSPACE_BYTES;
+static __device__ __align__(256) unsigned char g_static_workspace[kStaticWorkspaceBytes];
+
+// Device address of the built-in scratch on the current device, looked up once per device.
+int static_workspace(void **address)
+{
+    static void *cached[kMaxDevices] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+        (void)cudaGetLastError();
+        return INSTINFER_ERR_CUDA;
+    }
+    if (cached[dev] == nullptr) {
+        void *ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_static_workspace) != cudaSuccess || ptr == nullptr) {
+            (void)cudaGetLastError();
+            return INSTINFER_ERR_CUDA;
+        }
+        cached[dev] = ptr;
+    }
+    *address = cached[dev];
+    return INSTINFER_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -247,6 +274,35 @@ int instinfer_decode_attention_paged(void *out, float *lse, const void *q, const
     p.scale_log2e = scale * 1.44269504088896340736f;
     return launch_attention(p, true, batch, workspace, workspace_bytes,
                             static_cast<cudaStream_t>(cuda_stream));
+}
+
+int instinfer_decode_attention_static(void *out, float *lse, const void *q, const void *k_cache,
+                                      const void *v_cache, const int32_t *block_table,
+                                      const int32_t *seq_lens, int32_t batch, int32_t heads,
+                                      int32_t head_dim, int32_t s_max, int32_t block_tokens,
+                                      int32_t max_blocks_per_seq, int64_t num_phys_blocks,
+                                      int32_t max_seq_len, float scale, int32_t *status_flags,
+                                      void *cuda_stream)
+{
+    // Size check first: it needs no device and must not depend on the set-up below.
+    if (head_dim == kHeadDim && sizes_ok(batch, heads, max_seq_len) && batch > 0 &&
+        workspace_for((int64_t)batch * heads, make_plan((int64_t)batch * heads, max_seq_len)) >
+            kStaticWorkspaceBytes)
+        return INSTINFER_ERR_WORKSPACE;
+    void *scratch = nullptr;
+    if (batch > 0) {
+        const int rc = static_workspace(&scratch);
+        if (rc != INSTINFER_OK) return rc;
+    }
+    if (block_table == nullptr)
+        return instinfer_decode_attention(out, lse, q, k_cache, v_cache, seq_lens, batch, heads,
+                                          head_dim, s_max, max_seq_len, scale, scratch,
+                                          kStaticWorkspaceBytes, status_flags, cuda_stream);
+    return instinfer_decode_attention_paged(out, lse, q, k_cache, v_cache, block_table, seq_lens,
+                                            batch, heads, head_dim, block_tokens,
+                                            max_blocks_per_seq, num_phys_blocks, max_seq_len,
+                                            scale, scratch, kStaticWorkspaceBytes, status_flags,
+                                            cuda_stream);
 }
 
 size_t instinfer_workspace_bytes(int32_t batch, int32_t heads, int32_t head_dim, int32_t max_seq_len)
