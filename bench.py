@@ -404,10 +404,8 @@ def cpu_baseline(w: wl.Workload, seconds: float) -> dict:
             "kv_tokens_per_s": case.kv_tokens * case.workload.heads / wl.HEADS_13B / elapsed}
 
 
-def reference_arm(args, ranks: Ranks) -> None:
+def reference_arm(args, world: int) -> None:
     """--impl reference: the CPU oracle, as it stands, timed on host cores (rank 0 only)."""
-    if ranks.rank != 0:
-        return
     w = wl.by_name(args.workload)
     per_step = min(3.0, 120.0 / max(args.steps + args.warmup, 1))
     case, threads = oracle_sample(w, per_step)
@@ -417,7 +415,7 @@ def reference_arm(args, ranks: Ranks) -> None:
     used = min(threads, case.workload.batch * case.workload.heads)
     value = case.kv_bytes_read * args.steps / seconds / 1e9
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT,
-            "n_gpus": ranks.world, "steps": args.steps, "warmup": args.warmup,
+            "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": seconds / args.steps * 1e3, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
             "config": {"workload": w.name, "sample": sample_text(case)},
@@ -468,11 +466,12 @@ def measure_workload(w: wl.Workload, ranks: Ranks, device, steps: int, warmup: i
 
 def main(argv=None) -> int:
     args = parse_args(argv)
+    if args.impl == "reference":          # CPU only: no process group; ranks other than 0 do nothing
+        if int(os.environ.get("RANK", "0")) == 0:
+            reference_arm(args, int(os.environ.get("WORLD_SIZE", "1")))
+        return 0
     ranks = Ranks(args.gpus)
     try:
-        if args.impl == "reference":
-            reference_arm(args, ranks)
-            return 0
         from paper_2409_04992_b200 import binding, build
         if not build.is_current() and ranks.local_rank == 0:
             build.build()
