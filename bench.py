@@ -47,7 +47,10 @@ def parse_args(argv=None):
     ap.add_argument("--no-others", action="store_true",
                     help="skip the short extra measurements of the other long-context workloads")
     ap.add_argument("--no-graph", action="store_true", help="do not replay the step from a CUDA graph")
-    ap.add_argument("--cpu-seconds", type=float, default=15.0, help="CPU budget of the oracle baseline")
+    ap.add_argument("--cpu-seconds", type=float, default=15.0,
+                    help="CPU budget of the oracle baseline (0 skips it)")
+    ap.add_argument("--layers", type=int, default=0,
+                    help="override the workload's layer count (profiling a small case)")
     return ap.parse_args(argv)
 
 
@@ -482,6 +485,8 @@ def main(argv=None) -> int:
         device = torch.device("cuda", ranks.local_rank)
         torch.cuda.set_device(device)
         w = wl.by_name(args.workload)
+        if args.layers > 0:
+            w = w.replace(layers=args.layers)
         graph = not args.no_graph
         main_res = measure_workload(w, ranks, device, args.steps, args.warmup, graph, True)
 
@@ -513,7 +518,7 @@ def main(argv=None) -> int:
                          "algorithmic_bytes_per_launch": main_res["split_bytes"],
                          "avg_launch_ms": main_res["split_seconds"] * 1e3},
         }
-        if ranks.rank == 0 and ranks.world == 1:
+        if ranks.rank == 0 and ranks.world == 1 and args.cpu_seconds > 0:
             line["cpu_baseline"] = cpu_baseline(w, args.cpu_seconds)
         if not args.no_others and ranks.world == 1:
             others = {}
