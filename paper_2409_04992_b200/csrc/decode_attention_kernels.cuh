@@ -51,6 +51,7 @@ struct AttnParams {
     int32_t *status;      // nullable
     int64_t num_phys_blocks;
     int32_t heads;
+    int32_t pairs;        // batch * heads
     int32_t s_max;
     int32_t block_tokens;
     int32_t max_blocks_per_seq;
@@ -106,8 +107,11 @@ decode_attn_split_kernel(const AttnParams p)
     extern __shared__ __align__(128) unsigned char smem[];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int col = lane & 15, half_warp = lane >> 4;
-    const int split = blockIdx.x % p.n_splits;
-    const int pair = blockIdx.x / p.n_splits;
+    // Grid order: split slowest, then sequence, head fastest.  Blocks that run together then
+    // cover all heads of a few sequences (one paged block's heads are adjacent in memory),
+    // and the short last chunks of ragged sequences are scheduled last.
+    const int split = blockIdx.x / p.pairs;
+    const int pair = blockIdx.x - split * p.pairs;
     const int b = pair / p.heads, h = pair - b * p.heads;
     const bool final_writer = p.n_splits == 1;
 

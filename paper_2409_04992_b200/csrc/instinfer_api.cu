@@ -116,6 +116,7 @@ int launch_attention(AttnParams p, bool paged, int32_t batch, void *workspace,
     if (pairs * plan.n_splits >= (int64_t)1 << 31) return INSTINFER_ERR_INVALID_ARG;
     p.chunk_tokens = plan.chunk_tokens;
     p.n_splits = plan.n_splits;
+    p.pairs = (int32_t)pairs;
     p.part_o = static_cast<float *>(workspace);
     p.part_lse = p.part_o + (size_t)pairs * plan.n_splits * kHeadDim;
 
