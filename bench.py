@@ -195,9 +195,8 @@ class Layer:
         self.workspace = binding.alloc_workspace(B, H, D, self.max_len, dev)
         self.host_in = [t.cpu().pin_memory() for t in (case.q, case.k_new, case.v_new)]
         self.host_out = torch.empty((B, H, D), dtype=torch.float16).pin_memory()
-        chunk = binding.plan_chunk_tokens(B, H, self.max_len)
-        self.n_splits = -(-self.max_len // chunk)
-        self.chunk_tokens = chunk
+        self.chunk_tokens = binding.plan_chunk_tokens(B, H, self.max_len)
+        self.n_splits = binding.plan_num_splits(B, H, self.max_len)
 
     @property
     def launches(self) -> int:

@@ -159,16 +159,20 @@ size_t instinfer_workspace_bytes(int32_t batch, int32_t heads, int32_t head_dim,
                                  int32_t max_seq_len);
 
 /*
- * Split plan.  A sequence is cut at multiples of `chunk_tokens` logical positions; each
- * chunk of each (sequence, head) is reduced by one thread block and the partial results are
- * merged by log-sum-exp (no counterpart in the paper, whose engine streams token groups
- * through parallel GeMV units, Sec. IV-B).  instinfer_plan_chunk_tokens returns the chunk
- * the library would use for these sizes (0 if an argument is invalid).
- * instinfer_set_chunk_tokens(n) forces chunk_tokens = n for later calls of this process
- * (n > 0, a multiple of 64), n == 0 restores the automatic choice; it returns
+ * Split plan.  A sequence is cut at fixed logical token positions, the same for every
+ * sequence: first chunks of `chunk_tokens`, then, near the end of the longest admissible
+ * sequence, shorter chunks (they are scheduled last and keep the tail of the launch short).
+ * Each chunk of each (sequence, head) is reduced by one thread block and the partial results
+ * are merged by log-sum-exp (no counterpart in the paper, whose engine streams token groups
+ * through parallel GeMV units, Sec. IV-B).  instinfer_plan_chunk_tokens returns the first
+ * chunk size the library would use for these sizes and instinfer_plan_num_splits the number
+ * of chunks per sequence (0 if an argument is invalid).
+ * instinfer_set_chunk_tokens(n) forces uniform chunks of n tokens for later calls of this
+ * process (n > 0, a multiple of 64), n == 0 restores the automatic choice; it returns
  * INSTINFER_OK or INSTINFER_ERR_INVALID_ARG.  Not thread-safe against concurrent calls.
  */
 int32_t instinfer_plan_chunk_tokens(int32_t batch, int32_t heads, int32_t max_seq_len);
+int32_t instinfer_plan_num_splits(int32_t batch, int32_t heads, int32_t max_seq_len);
 int instinfer_set_chunk_tokens(int32_t chunk_tokens);
 
 /*

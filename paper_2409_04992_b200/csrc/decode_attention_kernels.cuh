@@ -55,8 +55,10 @@ struct AttnParams {
     int32_t s_max;
     int32_t block_tokens;
     int32_t max_blocks_per_seq;
-    int32_t chunk_tokens;
-    int32_t n_splits;
+    int32_t chunk_tokens; // tokens per chunk for the first n_big chunks of a sequence ...
+    int32_t n_big;
+    int32_t tail_chunk;   // ... and per chunk after that (scheduled last: short tail of the launch)
+    int32_t n_splits;     // n_big + number of tail chunks
     int32_t max_seq_len;
     float scale_log2e;    // scale * log2(e): logits are kept in the base-2 domain
 };
@@ -89,6 +91,26 @@ __device__ __forceinline__ int checked_seq_len(const AttnParams &p, int b, bool 
     return len;
 }
 
+// Logical token range [begin, begin + size) of chunk `split`.
+__device__ __forceinline__ void chunk_range(const AttnParams &p, int split, int &begin, int &size)
+{
+    if (split < p.n_big) {
+        begin = split * p.chunk_tokens;
+        size = p.chunk_tokens;
+    } else {
+        begin = p.n_big * p.chunk_tokens + (split - p.n_big) * p.tail_chunk;
+        size = p.tail_chunk;
+    }
+}
+
+// Number of chunks of a sequence of `len` tokens that hold at least one token.
+__device__ __forceinline__ int live_chunks(const AttnParams &p, int len)
+{
+    const int big_span = p.n_big * p.chunk_tokens;
+    if (len <= big_span) return (len + p.chunk_tokens - 1) / p.chunk_tokens;
+    return p.n_big + (len - big_span + p.tail_chunk - 1) / p.tail_chunk;
+}
+
 __device__ __forceinline__ void unpack8(const uint4 &raw, float (&f)[8])
 {
     const __half2 *h = reinterpret_cast<const __half2 *>(&raw);
@@ -117,7 +139,8 @@ decode_attn_split_kernel(const AttnParams p)
 
     // With several splits the merge kernel reports a bad length; here only the lone writer does.
     const int len = checked_seq_len(p, b, threadIdx.x == 0 && h == 0 && final_writer);
-    const int begin = split * p.chunk_tokens;
+    int begin, chunk_size;
+    chunk_range(p, split, begin, chunk_size);
     if (begin >= len) {
         if (final_writer) {            // inactive slot: zero output, lse = -inf
             p.out[(int64_t)pair * kHeadDim + threadIdx.x] = __float2half_rn(0.f);
@@ -125,7 +148,7 @@ decode_attn_split_kernel(const AttnParams p)
         }
         return;
     }
-    const int end = min(begin + p.chunk_tokens, len);
+    const int end = min(begin + chunk_size, len);
     const int n_tiles = (end - begin + kTileRows - 1) / kTileRows;
     const int my_tiles = warp < n_tiles ? (n_tiles - warp + kWarps - 1) / kWarps : 0;
 
@@ -287,7 +310,7 @@ lse_merge_kernel(const AttnParams p)
     const int pair = blockIdx.x;
     const int b = pair / p.heads;
     const int len = checked_seq_len(p, b, threadIdx.x == 0 && pair == b * p.heads);
-    const int live = (len + p.chunk_tokens - 1) / p.chunk_tokens;
+    const int live = live_chunks(p, len);
     if (live == 0) {
         p.out[(int64_t)pair * kHeadDim + threadIdx.x] = __float2half_rn(0.f);
         if (p.lse && threadIdx.x == 0) p.lse[pair] = -INFINITY;

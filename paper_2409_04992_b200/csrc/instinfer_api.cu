@@ -17,6 +17,8 @@ constexpr int kChunkGranule = 64;        // chunk_tokens is a multiple of this
 constexpr int kChunkCeiling = 2048;      // automatic plan: chunk never longer than this ...
 constexpr int kChunkFloor = 256;         // ... nor shorter than this, sequence permitting
 constexpr int kTargetWaves = 8;          // automatic plan: aim for this many waves of blocks
+constexpr int kTailChunk = 256;          // automatic plan: chunk size at the end of long sequences
+constexpr int kTailWaves = 2;            // ... covering about this many waves of blocks
 
 int g_forced_chunk = 0;
 cudaEvent_t g_before_split = nullptr;    // measurement aid, see instinfer_set_timing_events
@@ -48,29 +50,47 @@ int sm_count()
 }
 
 struct SplitPlan {
-    int32_t chunk_tokens;
+    int32_t chunk_tokens;   // size of the first n_big chunks
+    int32_t n_big;
+    int32_t tail_chunk;     // size of the chunks after them
     int32_t n_splits;
 };
 
-// Cuts are at multiples of chunk_tokens in logical token positions, the same for every
-// sequence, so a result never depends on the physical placement of blocks.
+// Cuts are at fixed logical token positions, the same for every sequence, so a result never
+// depends on the physical placement of blocks.  Blocks are scheduled chunk-major, so the
+// chunks at the end of the longest sequences run last: making those short keeps the tail of
+// a launch (SMs idling while the last blocks finish) short without paying the per-block
+// overhead of small chunks everywhere.
 SplitPlan make_plan(int64_t pairs, int32_t max_seq_len)
 {
-    int64_t chunk;
-    if (g_forced_chunk > 0) {
-        chunk = g_forced_chunk;
-    } else {
-        const int64_t slots = (int64_t)sm_count() * kCtasPerSm;
-        const int64_t fewest = ceil_div(max_seq_len, kChunkCeiling);
-        const int64_t most = ceil_div(max_seq_len, kChunkFloor);
-        int64_t n = ceil_div(slots * kTargetWaves, pairs);
-        if (n > most) n = most;
-        if (n < fewest) n = fewest;
-        chunk = ceil_div(ceil_div(max_seq_len, n), kChunkGranule) * kChunkGranule;
-    }
     SplitPlan plan;
+    if (g_forced_chunk > 0) {
+        plan.chunk_tokens = plan.tail_chunk = g_forced_chunk;
+        plan.n_big = (int32_t)ceil_div(max_seq_len, g_forced_chunk);
+        plan.n_splits = plan.n_big;
+        return plan;
+    }
+    const int64_t slots = (int64_t)sm_count() * kCtasPerSm;
+    const int64_t fewest = ceil_div(max_seq_len, kChunkCeiling);
+    const int64_t most = ceil_div(max_seq_len, kChunkFloor);
+    int64_t n = ceil_div(slots * kTargetWaves, pairs);
+    if (n > most) n = most;
+    if (n < fewest) n = fewest;
+    int64_t chunk = ceil_div(ceil_div(max_seq_len, n), kChunkGranule) * kChunkGranule;
+    // Tail region: about kTailWaves waves of kTailChunk-token blocks at the end of the longest
+    // sequences, at most a quarter of the sequence; none when the chunks are that short anyway.
+    int64_t tail_tokens = ceil_div(slots * kTailWaves, pairs) * kTailChunk;
+    if (tail_tokens > max_seq_len / 4) tail_tokens = max_seq_len / 4 / kTailChunk * kTailChunk;
+    if (chunk <= 2 * kTailChunk || tail_tokens < kTailChunk) tail_tokens = 0;
+    if (tail_tokens > 0)      // rounded down, so that at least tail_tokens are left for the tail
+        chunk = (max_seq_len - tail_tokens) / n / kChunkGranule * kChunkGranule;
+    int64_t big_span = n * chunk;
+    while (big_span - chunk >= max_seq_len) big_span -= chunk;
     plan.chunk_tokens = (int32_t)chunk;
-    plan.n_splits = (int32_t)ceil_div(max_seq_len, chunk);
+    plan.n_big = (int32_t)(big_span / chunk);
+    plan.tail_chunk = tail_tokens > 0 ? kTailChunk : (int32_t)chunk;
+    plan.n_splits = plan.n_big + (big_span < max_seq_len
+                                      ? (int32_t)ceil_div(max_seq_len - big_span, plan.tail_chunk) : 0);
     return plan;
 }
 
@@ -115,6 +135,8 @@ int launch_attention(AttnParams p, bool paged, int32_t batch, void *workspace,
         return INSTINFER_ERR_WORKSPACE;
     if (pairs * plan.n_splits >= (int64_t)1 << 31) return INSTINFER_ERR_INVALID_ARG;
     p.chunk_tokens = plan.chunk_tokens;
+    p.n_big = plan.n_big;
+    p.tail_chunk = plan.tail_chunk;
     p.n_splits = plan.n_splits;
     p.pairs = (int32_t)pairs;
     p.part_o = static_cast<float *>(workspace);
@@ -318,6 +340,12 @@ int32_t instinfer_plan_chunk_tokens(int32_t batch, int32_t heads, int32_t max_se
 {
     if (!sizes_ok(batch, heads, max_seq_len) || batch == 0) return 0;
     return make_plan((int64_t)batch * heads, max_seq_len).chunk_tokens;
+}
+
+int32_t instinfer_plan_num_splits(int32_t batch, int32_t heads, int32_t max_seq_len)
+{
+    if (!sizes_ok(batch, heads, max_seq_len) || batch == 0) return 0;
+    return make_plan((int64_t)batch * heads, max_seq_len).n_splits;
 }
 
 int instinfer_set_chunk_tokens(int32_t chunk_tokens)

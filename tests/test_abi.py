@@ -45,7 +45,8 @@ def test_plan_and_workspace_are_consistent(lib):
     for batch, heads, L in [(1, 40, 1024), (16, 40, 4096), (64, 40, 16384), (8, 40, 131072), (3, 5, 1)]:
         chunk = binding.plan_chunk_tokens(batch, heads, L)
         assert chunk > 0 and chunk % 64 == 0
-        splits = -(-L // chunk)
+        splits = binding.plan_num_splits(batch, heads, L)
+        assert splits >= -(-L // chunk)
         need = binding.workspace_bytes(batch, heads, 128, L)
         assert need >= batch * heads * splits * 129 * 4
         assert need % 256 == 0
