@@ -10,10 +10,13 @@
 //   * each warp streams its own 8-token tiles of K and V through a private ring of shared
 //     memory stages filled by 16-byte cp.async copies (coalesced 512 B per warp instruction),
 //     with no block-wide barrier and no spin-wait anywhere in the main loop;
-//   * a half-warp (16 lanes x 8 dims) owns one row at a time: dot product in fp32, a 4-step
-//     shuffle reduction, then an fp32 online softmax (base-2 exponent) and the p.V update;
-//   * the 8 half-warp states of a block are merged once at the end of the chunk; chunk
-//     partials go to the workspace and a small second kernel merges them.
+//   * logits: 4 lanes share a key row (32 dims each, fp32 FMA, 2 xor-shuffles), so a warp
+//     scores the 8 rows of a tile at once; the running maximum is uniform over the warp and
+//     each row's exponential (base 2, fp32) is computed once;
+//   * weighted sum: 16 lanes share a value row (8 dims each), the half-warps take alternate
+//     rows and fetch the row's weight with one shuffle;
+//   * the 4 warp states of a block are merged once at the end of the chunk; chunk partials
+//     go to the workspace and a small second kernel merges them.
 #pragma once
 
 #include <cuda_fp16.h>
@@ -28,9 +31,12 @@ constexpr int kWarps = 4;
 constexpr int kThreads = kWarps * 32;
 constexpr int kTileRows = 8;                       // tokens per warp tile
 constexpr int kStages = 4;                         // ring depth per warp
-constexpr int kTileBytes = kTileRows * kRowBytes;  // 2 KiB of K, same of V
-constexpr int kStageBytes = 2 * kTileBytes;
-constexpr int kSplitSmemBytes = kWarps * kStages * kStageBytes;   // 64 KiB
+constexpr int kKRowStride = kRowBytes + 16;        // K rows padded in shared memory: 4 lanes per
+                                                   // row read 8 rows at once without bank conflicts
+constexpr int kKTileBytes = kTileRows * kKRowStride;
+constexpr int kVTileBytes = kTileRows * kRowBytes;
+constexpr int kStageBytes = kKTileBytes + kVTileBytes;
+constexpr int kSplitSmemBytes = kWarps * kStages * kStageBytes;   // 66 KiB
 constexpr int kCtasPerSm = 3;
 constexpr float kMinusHuge = -1.0e30f;             // finite stand-in for "no row seen yet"
 constexpr float kLn2 = 0.69314718055994530942f;
@@ -70,9 +76,8 @@ __device__ __forceinline__ float fast_exp2(float x)
     return y;
 }
 
-__device__ __forceinline__ void cp_async_16(void *smem_dst, const void *gmem_src, int src_bytes)
+__device__ __forceinline__ void cp_async_16(unsigned dst, const void *gmem_src, int src_bytes)
 {
-    const unsigned dst = static_cast<unsigned>(__cvta_generic_to_shared(smem_dst));
     asm volatile("cp.async.cg.shared.global.L2::128B [%0], [%1], 16, %2;\n"
                  :: "r"(dst), "l"(gmem_src), "r"(src_bytes) : "memory");
 }
@@ -111,6 +116,32 @@ __device__ __forceinline__ int live_chunks(const AttnParams &p, int len)
     return p.n_big + (len - big_span + p.tail_chunk - 1) / p.tail_chunk;
 }
 
+// d = a * b + c with fp16 a, b and fp32 c, d: the product of two fp16 values is exact in
+// fp32, so this is one rounding, and one full-rate instruction with no conversion.
+__device__ __forceinline__ float fma_h(unsigned short a, unsigned short b, float c)
+{
+    float d;
+    asm("fma.rn.f32.f16 %0, %1, %2, %3;" : "=f"(d) : "h"(a), "h"(b), "f"(c));
+    return d;
+}
+
+__device__ __forceinline__ void halves(unsigned packed, unsigned short &lo, unsigned short &hi)
+{
+    asm("mov.b32 {%0, %1}, %2;" : "=h"(lo), "=h"(hi) : "r"(packed));
+}
+
+// A softmax weight w in [0, 1] as two fp16 numbers hi + lo ~ w * 2^14 (packed lo | hi << 16).
+// The scaling keeps weights down to 2^-38 of the maximum representable; hi + lo carries
+// about 22 significant bits, the precision of the exponential itself.
+constexpr float kWeightScale = 16384.f;
+__device__ __forceinline__ unsigned split_weight(float w)
+{
+    const float scaled = w * kWeightScale;
+    const __half hi = __float2half_rn(scaled);
+    const __half lo = __float2half_rn(scaled - __half2float(hi));
+    return (unsigned)__half_as_ushort(hi) << 16 | (unsigned)__half_as_ushort(lo);
+}
+
 __device__ __forceinline__ void unpack8(const uint4 &raw, float (&f)[8])
 {
     const __half2 *h = reinterpret_cast<const __half2 *>(&raw);
@@ -122,12 +153,26 @@ __device__ __forceinline__ void unpack8(const uint4 &raw, float (&f)[8])
     }
 }
 
+__device__ __forceinline__ uint4 lds128(unsigned shared_addr)
+{
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(shared_addr));
+    return v;
+}
+
 template <bool kPaged>
 __global__ void __launch_bounds__(kThreads, kCtasPerSm)
 decode_attn_split_kernel(const AttnParams p)
 {
     extern __shared__ __align__(128) unsigned char smem[];
+    static_assert((kStages & (kStages - 1)) == 0, "ring depth must be a power of two");
+    constexpr int kStepTokens = kWarps * kTileRows;      // a warp's next tile is this far ahead
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // Logit phase: 4 lanes per key row, lane (row = lane & 7, quarter = lane >> 3) owns 32 dims.
+    // Attend phase: 16 lanes per value row, lane (col = lane & 15) owns 8 dims, half-warps
+    // take alternate rows.
+    const int row = lane & 7, quarter = lane >> 3;
     const int col = lane & 15, half_warp = lane >> 4;
     // Grid order: split slowest, then sequence, head fastest.  Blocks that run together then
     // cover all heads of a few sequences (one paged block's heads are adjacent in memory),
@@ -151,146 +196,222 @@ decode_attn_split_kernel(const AttnParams p)
     const int end = min(begin + chunk_size, len);
     const int n_tiles = (end - begin + kTileRows - 1) / kTileRows;
     const int my_tiles = warp < n_tiles ? (n_tiles - warp + kWarps - 1) / kWarps : 0;
+    // Only the chunk's very last tile can be ragged; it belongs to exactly one warp.
+    const int last_rows = warp == (n_tiles - 1) % kWarps ? (end - begin) - (n_tiles - 1) * kTileRows
+                                                         : kTileRows;
 
-    // This lane's 8 query dims, pre-multiplied by scale*log2(e).
-    float qf[8];
+    // This lane's 32 query dims, kept in fp16 (16 registers): products with fp16 keys are
+    // exact in fp32 and the scale is applied to the finished dot product.
+    uint4 qh[4];
     {
-        const uint4 raw = *reinterpret_cast<const uint4 *>(p.q + (int64_t)pair * kHeadDim + col * 8);
-        unpack8(raw, qf);
+        const uint4 *src = reinterpret_cast<const uint4 *>(p.q + (int64_t)pair * kHeadDim + quarter * 32);
 #pragma unroll
-        for (int i = 0; i < 8; ++i) qf[i] *= p.scale_log2e;
+        for (int i = 0; i < 4; ++i) qh[i] = src[i];
     }
 
-    unsigned char *ring = smem + warp * (kStages * kStageBytes);
-    const int64_t contiguous_base = (int64_t)pair * p.s_max;          // rows
-    const int32_t *table_row = kPaged ? p.block_table + (int64_t)b * p.max_blocks_per_seq : nullptr;
+    // Shared-memory addresses (shared window, 32 bit).  K rows are padded to kKRowStride.
+    const unsigned ring = static_cast<unsigned>(__cvta_generic_to_shared(smem)) +
+                          warp * (kStages * kStageBytes);
+    // copies: 16-byte segment lane + 32 i, i < 4, lies in row 2 i + half_warp at column segment col
+    const unsigned k_dst = half_warp * kKRowStride + col * 16;
+    const unsigned v_dst = kKTileBytes + lane * 16;
+    const unsigned k_rd = row * kKRowStride + quarter * 64;
+    const unsigned v_rd = kKTileBytes + lane * 16;
 
-    // Block-table entries for this warp's next 32 tiles live one per lane (paged only).
-    auto table_entry = [&](int j) -> int {
-        if (j >= my_tiles) return 0;
-        const int token0 = begin + (warp + j * kWarps) * kTileRows;
-        return __ldg(table_row + token0 / p.block_tokens);
-    };
-    int table_now = 0, table_next = 0;
+    // ---- copy-issue side: walks this warp's tiles incrementally (no division per tile) ----
+    const unsigned char *k_lane = reinterpret_cast<const unsigned char *>(p.k) + lane * 16;
+    const unsigned char *v_lane = reinterpret_cast<const unsigned char *>(p.v) + lane * 16;
+    const int first_token = begin + warp * kTileRows;
+    int64_t src_off = 0;                       // contiguous: byte offset of the next tile
+    int blk = 0, rem = 0, win_base = 0;        // paged: block index, row inside it, window start
+    int window_now = 0, window_next = 0;       // block-table entries win_base + lane (+ 32)
+    int64_t block_stride = 0, head_off = 0;
+    int step_blk = 0, step_rem = 0, blocks_needed = 0;
+    const int32_t *table_row = nullptr;
     if (kPaged) {
-        table_now = table_entry(lane);
-        table_next = table_entry(32 + lane);
+        const int tokens = p.block_tokens;
+        table_row = p.block_table + (int64_t)b * p.max_blocks_per_seq;
+        blocks_needed = (end + tokens - 1) / tokens;
+        blk = first_token / tokens;
+        rem = first_token - blk * tokens;
+        step_blk = kStepTokens / tokens;
+        step_rem = kStepTokens - step_blk * tokens;
+        block_stride = (int64_t)p.heads * tokens * kRowBytes;
+        head_off = (int64_t)h * tokens * kRowBytes;
+        win_base = blk;
+    } else {
+        src_off = ((int64_t)pair * p.s_max + first_token) * kRowBytes;
+    }
+    auto load_window = [&](int base) -> int {
+        const int idx = base + lane;
+        return idx < blocks_needed ? __ldg(table_row + idx) : 0;
+    };
+    if (kPaged && my_tiles > 0) {
+        window_now = load_window(win_base);
+        window_next = load_window(win_base + 32);
     }
 
-    auto issue = [&](int j) {
-        if (j < my_tiles) {
-            const int token0 = begin + (warp + j * kWarps) * kTileRows;
-            int64_t row0;
+    int issue_j = 0;
+    unsigned issue_stage = 0;
+    auto issue = [&]() {
+        if (issue_j < my_tiles) {
+            const int rows = issue_j == my_tiles - 1 ? last_rows : kTileRows;
             bool usable = true;
+            int64_t off;
             if (kPaged) {
-                if ((j & 31) == 0 && j > 0) {
-                    table_now = table_next;
-                    table_next = table_entry(j + 32 + lane);
+                int idx = blk - win_base;
+                if (idx >= 32) {               // uniform: slide the window of table entries
+                    idx -= 32;
+                    win_base += 32;
+                    window_now = window_next;
+                    window_next = load_window(win_base + 32);
                 }
-                const int phys = __shfl_sync(0xffffffffu, table_now, j & 31);
+                const int phys = __shfl_sync(0xffffffffu, window_now, idx);
                 usable = phys >= 0 && (int64_t)phys < p.num_phys_blocks;
                 if (!usable && lane == 0 && p.status) atomicOr(p.status, kFlagBlockRange);
-                row0 = usable ? ((int64_t)phys * p.heads + h) * p.block_tokens + token0 % p.block_tokens : 0;
+                off = usable ? (int64_t)phys * block_stride + head_off + rem * kRowBytes : 0;
+                blk += step_blk;
+                rem += step_rem;
+                if (rem >= p.block_tokens) {
+                    rem -= p.block_tokens;
+                    ++blk;
+                }
             } else {
-                row0 = contiguous_base + token0;
+                off = src_off;
+                src_off += kStepTokens * kRowBytes;
             }
-            const unsigned char *k_src = reinterpret_cast<const unsigned char *>(p.k) + row0 * kRowBytes;
-            const unsigned char *v_src = reinterpret_cast<const unsigned char *>(p.v) + row0 * kRowBytes;
-            unsigned char *dst = ring + (j % kStages) * kStageBytes;
+            const unsigned char *ks = k_lane + off, *vs = v_lane + off;
+            const unsigned dst = ring + issue_stage * kStageBytes;
+            if (usable && rows == kTileRows) {                 // full tile: no predicates
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const int seg = lane + 32 * i;                 // 16-byte segment of the tile
-                const bool valid = usable && (token0 + (seg >> 4) < end);
-                const int off = valid ? seg * 16 : 0;          // masked rows are zero-filled
-                cp_async_16(dst + seg * 16, k_src + off, valid ? 16 : 0);
-                cp_async_16(dst + kTileBytes + seg * 16, v_src + off, valid ? 16 : 0);
+                for (int i = 0; i < 4; ++i) {
+                    cp_async_16(dst + k_dst + i * 2 * kKRowStride, ks + i * 512, 16);
+                    cp_async_16(dst + v_dst + i * 512, vs + i * 512, 16);
+                }
+            } else {                                           // ragged tail: masked rows are zero-filled
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const bool valid = usable && (2 * i + half_warp < rows);
+                    const int src = valid ? i * 512 : 0;
+                    cp_async_16(dst + k_dst + i * 2 * kKRowStride, ks + src, valid ? 16 : 0);
+                    cp_async_16(dst + v_dst + i * 512, vs + src, valid ? 16 : 0);
+                }
             }
         }
         cp_async_commit();                                     // empty groups keep the count uniform
+        ++issue_j;
+        issue_stage = (issue_stage + 1) & (kStages - 1);
     };
 
+    // Running softmax state.  m is uniform over the warp; l is a per-lane partial sum (lanes
+    // of one row hold equal values); acc covers this half-warp's rows and carries kWeightScale.
     float m = kMinusHuge, l = 0.f, acc[8];
 #pragma unroll
     for (int i = 0; i < 8; ++i) acc[i] = 0.f;
 
 #pragma unroll
-    for (int j = 0; j < kStages - 1; ++j) issue(j);
+    for (int j = 0; j < kStages - 1; ++j) issue();
 
+    unsigned stage = 0;
     for (int j = 0; j < my_tiles; ++j) {
         cp_async_wait<kStages - 2>();
         __syncwarp();                    // tile j visible to the warp; everyone is done with tile j-1
-        issue(j + kStages - 1);          // refills the slot tile j-1 used
+        issue();                         // refills the slot tile j-1 used
+        const unsigned base = ring + stage * kStageBytes;
+        stage = (stage + 1) & (kStages - 1);
 
-        const unsigned char *stage = ring + (j % kStages) * kStageBytes;
-        const int token0 = begin + (warp + j * kWarps) * kTileRows;
-        float s[4];
+        // Logit: this lane's quarter of row `row`, four independent fp32 chains.
+        float part[4];
 #pragma unroll
-        for (int r = 0; r < 4; ++r) {
-            float kf[8];
-            unpack8(*reinterpret_cast<const uint4 *>(stage + r * 512 + lane * 16), kf);
+        for (int i = 0; i < 4; ++i) {
+            const uint4 kr = lds128(base + k_rd + i * 16);
+            const unsigned kw[4] = {kr.x, kr.y, kr.z, kr.w};
+            const unsigned qw[4] = {qh[i].x, qh[i].y, qh[i].z, qh[i].w};
             float dot = 0.f;
 #pragma unroll
-            for (int i = 0; i < 8; ++i) dot = fmaf(kf[i], qf[i], dot);
-            s[r] = dot;
+            for (int e = 0; e < 4; ++e) {
+                unsigned short k0, k1, q0, q1;
+                halves(kw[e], k0, k1);
+                halves(qw[e], q0, q1);
+                dot = fma_h(k0, q0, dot);
+                dot = fma_h(k1, q1, dot);
+            }
+            part[i] = dot;
         }
+        float s = ((part[0] + part[1]) + (part[2] + part[3])) * p.scale_log2e;
+        s += __shfl_xor_sync(0xffffffffu, s, 8);
+        s += __shfl_xor_sync(0xffffffffu, s, 16);
+        const int rows = j == my_tiles - 1 ? last_rows : kTileRows;
+        if (row >= rows) s = -INFINITY;
+
+        // Online softmax with a warp-uniform running max.
+        float tile_max = s;
+        tile_max = fmaxf(tile_max, __shfl_xor_sync(0xffffffffu, tile_max, 1));
+        tile_max = fmaxf(tile_max, __shfl_xor_sync(0xffffffffu, tile_max, 2));
+        tile_max = fmaxf(tile_max, __shfl_xor_sync(0xffffffffu, tile_max, 4));
+        if (__any_sync(0xffffffffu, tile_max > m)) {     // rare once the maximum has settled
+            const float alpha = fast_exp2(m - tile_max);
+            l *= alpha;
 #pragma unroll
-        for (int off = 8; off >= 1; off >>= 1) {
-#pragma unroll
-            for (int r = 0; r < 4; ++r) s[r] += __shfl_xor_sync(0xffffffffu, s[r], off);
+            for (int i = 0; i < 8; ++i) acc[i] *= alpha;
+            m = tile_max;
         }
-        float m_new = m;
+        const float pw = fast_exp2(s - m);
+        l += pw;
+
+        // Attend: rows 2 r + half_warp, r < 4.
+        const unsigned packed = split_weight(pw);
 #pragma unroll
         for (int r = 0; r < 4; ++r) {
-            if (token0 + 2 * r + half_warp >= end) s[r] = -INFINITY;
-            m_new = fmaxf(m_new, s[r]);
-        }
-        const float alpha = fast_exp2(m - m_new);
-        float pw[4], psum = 0.f;
+            unsigned short w_lo, w_hi;
+            halves(__shfl_sync(0xffffffffu, packed, 2 * r + half_warp), w_lo, w_hi);
+            const uint4 vr = lds128(base + v_rd + r * 512);
+            const unsigned vw[4] = {vr.x, vr.y, vr.z, vr.w};
 #pragma unroll
-        for (int r = 0; r < 4; ++r) {
-            pw[r] = fast_exp2(s[r] - m_new);
-            psum += pw[r];
-        }
-        l = fmaf(l, alpha, psum);
-        m = m_new;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) acc[i] *= alpha;
-#pragma unroll
-        for (int r = 0; r < 4; ++r) {
-            float vf[8];
-            unpack8(*reinterpret_cast<const uint4 *>(stage + kTileBytes + r * 512 + lane * 16), vf);
-#pragma unroll
-            for (int i = 0; i < 8; ++i) acc[i] = fmaf(pw[r], vf[i], acc[i]);
+            for (int e = 0; e < 4; ++e) {
+                unsigned short v0, v1;
+                halves(vw[e], v0, v1);
+                acc[2 * e] = fma_h(v0, w_hi, acc[2 * e]);
+                acc[2 * e + 1] = fma_h(v1, w_hi, acc[2 * e + 1]);
+                acc[2 * e] = fma_h(v0, w_lo, acc[2 * e]);
+                acc[2 * e + 1] = fma_h(v1, w_lo, acc[2 * e + 1]);
+            }
         }
     }
     cp_async_wait<0>();
+
+    // One state per warp: sum l over the 8 rows, fold the two half-warps' accumulators.
+    l += __shfl_xor_sync(0xffffffffu, l, 1);
+    l += __shfl_xor_sync(0xffffffffu, l, 2);
+    l += __shfl_xor_sync(0xffffffffu, l, 4);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) acc[i] += __shfl_xor_sync(0xffffffffu, acc[i], 16);
     __syncthreads();                     // every ring is idle: reuse shared memory for the merge
 
-    // Merge the 8 half-warp states of this block.
-    constexpr int kStates = 2 * kWarps;
     float *sm_m = reinterpret_cast<float *>(smem);
-    float *sm_l = sm_m + kStates;
-    float *sm_acc = sm_l + kStates;                      // [kStates][kHeadDim]
-    const int state = warp * 2 + half_warp;
-    if (col == 0) {
-        sm_m[state] = m;
-        sm_l[state] = l;
+    float *sm_l = sm_m + kWarps;
+    float *sm_acc = sm_l + kWarps;                       // [kWarps][kHeadDim]
+    if (lane == 0) {
+        sm_m[warp] = m;
+        sm_l[warp] = l;
     }
+    if (half_warp == 0) {
 #pragma unroll
-    for (int i = 0; i < 8; ++i) sm_acc[state * kHeadDim + col * 8 + i] = acc[i];
+        for (int i = 0; i < 8; ++i) sm_acc[warp * kHeadDim + col * 8 + i] = acc[i];
+    }
     __syncthreads();
 
     float top = kMinusHuge;
 #pragma unroll
-    for (int i = 0; i < kStates; ++i) top = fmaxf(top, sm_m[i]);
+    for (int i = 0; i < kWarps; ++i) top = fmaxf(top, sm_m[i]);
     float total = 0.f, o = 0.f;
 #pragma unroll
-    for (int i = 0; i < kStates; ++i) {
+    for (int i = 0; i < kWarps; ++i) {
         const float w = fast_exp2(sm_m[i] - top);
         total = fmaf(w, sm_l[i], total);
         o = fmaf(w, sm_acc[i * kHeadDim + threadIdx.x], o);
     }
-    o /= total;
+    o /= total * kWeightScale;
     const float lse2 = top + log2f(total);
     if (final_writer) {
         p.out[(int64_t)pair * kHeadDim + threadIdx.x] = __float2half_rn(o);
