@@ -54,6 +54,28 @@ def parse_args(argv=None):
     return ap.parse_args(argv)
 
 
+def kernel_source_hash() -> str:
+    """sha256 of the file that holds the split kernel (identifies the profiled revision)."""
+    import hashlib
+    path = os.path.join(ROOT, "paper_2409_04992_b200", "csrc", "decode_attention_kernels.cuh")
+    with open(path, "rb") as fh:
+        return hashlib.sha256(fh.read()).hexdigest()
+
+
+def profiled_traffic(workload_name: str, algorithmic_bytes: float):
+    """DRAM bytes per launch of the split kernel from the committed ncu summary, scaled by
+    the algorithmic bytes of this launch; None if the kernel source changed since."""
+    try:
+        with open(os.path.join(ROOT, "profiles", "split_kernel_traffic.json")) as fh:
+            rec = json.load(fh)
+        if rec["kernel_source_sha256"] != kernel_source_hash():
+            return None
+        scale = algorithmic_bytes / rec["algorithmic_bytes_per_launch"]
+        return (rec["dram_bytes_read"] + rec["dram_bytes_write"]) * scale
+    except Exception:
+        return None
+
+
 def measured_peak_gbs():
     """HBM copy bandwidth measured on this machine, else the documented fallback."""
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
@@ -193,7 +215,10 @@ class Layer:
         self.out = torch.empty((B, H, D), dtype=torch.float16, device=dev)
         self.lse = torch.empty((B, H), dtype=torch.float32, device=dev)
         self.workspace = binding.alloc_workspace(B, H, D, self.max_len, dev)
-        self.host_in = [t.cpu().pin_memory() for t in (case.q, case.k_new, case.v_new)]
+        # q, k_new, v_new live in one device buffer so that a host caller uploads them in one copy
+        self.qkv = torch.stack([case.q, case.k_new, case.v_new]).contiguous()
+        case.q, case.k_new, case.v_new = self.qkv[0], self.qkv[1], self.qkv[2]
+        self.host_qkv = self.qkv.cpu().pin_memory()
         self.host_out = torch.empty((B, H, D), dtype=torch.float16).pin_memory()
         self.chunk_tokens = binding.plan_chunk_tokens(B, H, self.max_len)
         self.n_splits = binding.plan_num_splits(B, H, self.max_len)
@@ -218,15 +243,13 @@ class Layer:
         """The same step as a caller with host-resident q,k,v sees it: the three new vectors
         go up from pinned memory, the attention output comes back (the KV cache stays on the
         device, which is the point of the method: Sec. IV-D)."""
-        c = self.case
-        for dst, src in zip((c.q, c.k_new, c.v_new), self.host_in):
-            dst.copy_(src, non_blocking=True)
+        self.qkv.copy_(self.host_qkv, non_blocking=True)
         self.run(flags)
         self.host_out.copy_(self.out, non_blocking=True)
 
     @property
     def h2d_bytes(self) -> int:
-        return sum(t.numel() * t.element_size() for t in self.host_in)
+        return self.host_qkv.numel() * self.host_qkv.element_size()
 
     @property
     def d2h_bytes(self) -> int:
@@ -399,11 +422,14 @@ def sample_text(case: wl.Case) -> str:
 
 def cpu_baseline(w: wl.Workload, seconds: float) -> dict:
     case, threads = oracle_sample(w, seconds)
-    elapsed = oracle_pass(case)
+    first = oracle_pass(case)
+    passes = 1 + max(0, min(30, int(seconds / max(first, 1e-3)) - 1))   # fill the budget, bounded
+    elapsed = first + sum(oracle_pass(case) for _ in range(passes - 1))
     used = min(threads, case.workload.batch * case.workload.heads)
-    return {"value": case.kv_bytes_read / elapsed / 1e9, "unit": UNIT, "cores": used,
-            "kind": "oracle", "sample": sample_text(case), "seconds": round(elapsed, 2),
-            "kv_tokens_per_s": case.kv_tokens * case.workload.heads / wl.HEADS_13B / elapsed}
+    return {"value": case.kv_bytes_read * passes / elapsed / 1e9, "unit": UNIT, "cores": used,
+            "kind": "oracle", "sample": f"{passes} passes over " + sample_text(case),
+            "seconds": round(elapsed, 2),
+            "kv_tokens_per_s": case.kv_tokens * passes * case.workload.heads / wl.HEADS_13B / elapsed}
 
 
 def reference_arm(args, world: int) -> None:
@@ -513,7 +539,8 @@ def main(argv=None) -> int:
             "status_flags": main_res["flags"],
             "roofline": {"kernel": "decode_attn_split_kernel", "bound": "hbm",
                          "achieved": achieved, "peak": peak, "peak_kind": peak_kind,
-                         "unit": UNIT, "frac": achieved / peak, "traffic": None,
+                         "unit": UNIT, "frac": achieved / peak,
+                         "traffic": profiled_traffic(w.name, main_res["split_bytes"]),
                          "algorithmic_bytes_per_launch": main_res["split_bytes"],
                          "avg_launch_ms": main_res["split_seconds"] * 1e3},
         }

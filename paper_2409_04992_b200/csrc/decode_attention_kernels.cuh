@@ -166,7 +166,6 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm)
 decode_attn_split_kernel(const AttnParams p)
 {
     extern __shared__ __align__(128) unsigned char smem[];
-    static_assert((kStages & (kStages - 1)) == 0, "ring depth must be a power of two");
     constexpr int kStepTokens = kWarps * kTileRows;      // a warp's next tile is this far ahead
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     // Logit phase: 4 lanes per key row, lane (row = lane & 7, quarter = lane >> 3) owns 32 dims.
@@ -300,7 +299,7 @@ decode_attn_split_kernel(const AttnParams p)
         }
         cp_async_commit();                                     // empty groups keep the count uniform
         ++issue_j;
-        issue_stage = (issue_stage + 1) & (kStages - 1);
+        issue_stage = issue_stage + 1 == kStages ? 0 : issue_stage + 1;
     };
 
     // Running softmax state.  m is uniform over the warp; l is a per-lane partial sum (lanes
@@ -318,7 +317,7 @@ decode_attn_split_kernel(const AttnParams p)
         __syncwarp();                    // tile j visible to the warp; everyone is done with tile j-1
         issue();                         // refills the slot tile j-1 used
         const unsigned base = ring + stage * kStageBytes;
-        stage = (stage + 1) & (kStages - 1);
+        stage = stage + 1 == kStages ? 0 : stage + 1;
 
         // Logit: this lane's quarter of row `row`, four independent fp32 chains.
         float part[4];
