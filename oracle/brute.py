@@ -72,3 +72,42 @@ def kv_append(k_cache, v_cache, k_new, v_new, seq_lens: Sequence[int],
         for h in range(len(k_new[b])):
             _row(k_cache, b, h, length - 1, block_table, block_tokens)[:] = list(k_new[b][h])
             _row(v_cache, b, h, length - 1, block_table, block_tokens)[:] = list(v_new[b][h])
+
+
+def sparf_attention(q, k_rows, v_rows, r: int, k: int, l: int, scale: float):
+    """Algorithm 1 (SparF / SparQ arithmetic) for ONE head in pure Python.
+
+    q: [D] fp16 bit patterns; k_rows, v_rows: [S][D] bit patterns (already gathered in token
+    order).  vbar is the plain mean of the V rows.  Returns (out [D], alpha, J ascending).
+    Ties in both top-k selections go to the lower index.
+    """
+    scale = struct.unpack("<f", struct.pack("<f", scale))[0]
+    qv = [half_value(x) for x in q]
+    K = [[half_value(x) for x in row] for row in k_rows]
+    V = [[half_value(x) for x in row] for row in v_rows]
+    S, D = len(K), len(qv)
+    if S == 0:
+        return [0.0] * D, 0.0, []
+    k = min(k, S)
+    l = min(l, k)
+    dims = sorted(range(D), key=lambda d: (-abs(qv[d]), d))[:r]
+    q_l1 = math.fsum(abs(x) for x in qv)
+    ratio = math.fsum(abs(qv[d]) for d in dims) / q_l1 if q_l1 > 0 else 1.0
+    approx = [scale / math.sqrt(ratio) * math.fsum(qv[d] * K[i][d] for d in dims) for i in range(S)]
+    top = max(approx)
+    e = [math.exp(x - top) for x in approx]
+    z = math.fsum(e)
+    s_hat = [x / z for x in e]
+    keyed = [s_hat[i] + (1.0 if i >= S - l else 0.0) for i in range(S)]
+    J = sorted(sorted(range(S), key=lambda i: (-keyed[i], i))[:k])
+    alpha = math.fsum(s_hat[j] for j in J)
+    vbar = [math.fsum(V[i][d] for i in range(S)) / S for d in range(D)]
+    if not J:
+        return vbar, 0.0, []
+    logits = [scale * math.fsum(qv[d] * K[j][d] for d in range(D)) for j in J]
+    top = max(logits)
+    w = [math.exp(x - top) for x in logits]
+    zw = math.fsum(w)
+    out = [alpha * math.fsum(w[t] / zw * V[j][d] for t, j in enumerate(J)) + (1.0 - alpha) * vbar[d]
+           for d in range(D)]
+    return out, alpha, J

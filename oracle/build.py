@@ -11,16 +11,18 @@ from pathlib import Path
 
 _HERE = Path(__file__).resolve().parent
 SOURCE = _HERE / "decode_attention_oracle.c"
+SOURCES = [SOURCE, _HERE / "sparf_oracle.c"]
 LIBRARY = _HERE / "liboracle.so"
 
 
 def build(force: bool = False) -> Path:
     """gcc -O2 -fopenmp; rebuilt when the source is newer than the library."""
-    if not force and LIBRARY.exists() and LIBRARY.stat().st_mtime >= SOURCE.stat().st_mtime:
+    if not force and LIBRARY.exists() and all(LIBRARY.stat().st_mtime >= f.stat().st_mtime
+                                               for f in SOURCES):
         return LIBRARY
     tmp = LIBRARY.with_suffix(f".{os.getpid()}.tmp.so")
     cmd = ["gcc", "-O2", "-std=c11", "-fopenmp", "-fPIC", "-shared", "-Wall", "-Wextra",
-           "-fno-fast-math", "-ffp-contract=off", str(SOURCE), "-o", str(tmp), "-lm"]
+           "-fno-fast-math", "-ffp-contract=off", *map(str, SOURCES), "-o", str(tmp), "-lm"]
     subprocess.run(cmd, check=True)
     os.replace(tmp, LIBRARY)
     return LIBRARY

@@ -29,6 +29,13 @@ def _load() -> ctypes.CDLL:
         lib.oracle_decode_attention.argtypes = [ptr, ptr, ptr, i64, ptr, ptr, ptr, ptr, ptr,
                                                 i32, i32, i64, i32, i32, i32, i32,
                                                 ctypes.c_float]
+        lib.oracle_sparf_append.restype = ctypes.c_int
+        lib.oracle_sparf_append.argtypes = [ptr, ptr, ptr, ptr, ptr, ptr, ptr, ptr, i32, i32, i64,
+                                            i32, i32, i32]
+        lib.oracle_sparf_attention.restype = ctypes.c_int
+        lib.oracle_sparf_attention.argtypes = [ptr, ptr, ptr, i64, ptr, ptr, i64, ptr, ptr, ptr, ptr,
+                                               ptr, ptr, ptr, ptr, i32, i32, i64, i32, i32, i32,
+                                               i32, i32, ctypes.c_float]
         _lib = lib
     return _lib
 
@@ -122,3 +129,54 @@ def decode_attention(q: np.ndarray, k_cache: np.ndarray, v_cache: np.ndarray,
     if rc:
         raise OracleError(rc)
     return out, lse, weights
+
+
+def sparf_append(k_pool: np.ndarray, v_pool: np.ndarray, kt_pool: np.ndarray, v_sum: np.ndarray,
+                 k_new: np.ndarray, v_new: np.ndarray, seq_lens: np.ndarray,
+                 block_table: np.ndarray) -> None:
+    """In-place append for the SparF state: pools [P,H,T,D], K^T pool [P,H,D,T], v_sum f32 [B,H,D]."""
+    kb, vb, ktb = _bits(k_pool, True), _bits(v_pool, True), _bits(kt_pool, True)
+    kn, vn = _bits(np.ascontiguousarray(k_new)), _bits(np.ascontiguousarray(v_new))
+    if v_sum.dtype != np.float32 or not v_sum.flags.c_contiguous:
+        raise TypeError("v_sum must be contiguous float32")
+    batch, heads, head_dim = kn.shape
+    lens = np.ascontiguousarray(seq_lens, dtype=np.int32)
+    table, max_blocks = _table(block_table, batch)
+    rc = _load().oracle_sparf_append(_p(kb), _p(vb), _p(ktb), _p(v_sum), _p(kn), _p(vn), _p(lens),
+                                     _p(table), max_blocks, kb.shape[2], kb.shape[0], batch, heads,
+                                     head_dim)
+    if rc:
+        raise OracleError(rc)
+
+
+def sparf_attention(q: np.ndarray, k_pool: np.ndarray, v_pool: np.ndarray, kt_pool: np.ndarray,
+                    v_sum: np.ndarray, seq_lens: np.ndarray, k_tokens: np.ndarray,
+                    block_table: np.ndarray, r: int, l: int, scale: float,
+                    given: Optional[np.ndarray] = None, want_weights: bool = False):
+    """Algorithm 1 per (sequence, head).  Returns (out f64 [B,H,D], alpha f64 [B,H],
+    selected int32 [B,H,max k] ascending / -1 padded, approximate weights or None)."""
+    qb = _bits(np.ascontiguousarray(q))
+    kb, vb, ktb = _bits(k_pool), _bits(v_pool), _bits(kt_pool)
+    batch, heads, head_dim = qb.shape
+    lens = np.ascontiguousarray(seq_lens, dtype=np.int32)
+    ks = np.ascontiguousarray(k_tokens, dtype=np.int32)
+    table, max_blocks = _table(block_table, batch)
+    vs = np.ascontiguousarray(v_sum, dtype=np.float32)
+    stride_k = max(int(np.minimum(ks, lens).max()) if batch else 0, 1)
+    stride_s = max(int(lens.max()) if batch else 0, 1)
+    out = np.zeros((batch, heads, head_dim), dtype=np.float64)
+    alpha = np.zeros((batch, heads), dtype=np.float64)
+    selected = np.full((batch, heads, stride_k), -1, dtype=np.int32)
+    weights = np.zeros((batch, heads, stride_s), dtype=np.float64) if want_weights else None
+    giv = None
+    if given is not None:
+        giv = np.full((batch, heads, stride_k), -1, dtype=np.int32)
+        giv[:, :, :min(stride_k, given.shape[2])] = given[:, :, :stride_k]
+    rc = _load().oracle_sparf_attention(_p(out), _p(alpha), _p(weights), stride_s, _p(selected),
+                                        _p(giv), stride_k, _p(qb), _p(kb), _p(vb), _p(ktb), _p(vs),
+                                        _p(lens), _p(ks), _p(table), max_blocks, kb.shape[2],
+                                        kb.shape[0], batch, heads, head_dim, int(r), int(l),
+                                        ctypes.c_float(scale))
+    if rc:
+        raise OracleError(rc)
+    return out, alpha, selected, weights

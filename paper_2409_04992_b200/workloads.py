@@ -235,3 +235,34 @@ def gather_rows(case: Case, b: int, h: int):
     k = case.k_cache[blocks, h].reshape(-1, case.workload.head_dim)[:n].contiguous()
     v = case.v_cache[blocks, h].reshape(-1, case.workload.head_dim)[:n].contiguous()
     return k, v
+
+
+@dataclasses.dataclass
+class SparfState:
+    """Extra per-layer state of the sparse (SparF) path for a paged case."""
+
+    kt_pool: torch.Tensor           # fp16 [P,H,D,T]: the embedding-major copy of the K pool
+    v_sum: torch.Tensor             # fp32 [B,H,D]: running sum of each sequence's V rows
+    k_tokens: torch.Tensor          # int32 [B]: tokens to keep per sequence
+    k_tokens_host: List[int]
+
+
+def make_sparf_state(case: Case, keep_fraction: float = 0.125) -> SparfState:
+    """The embedding-major K copy is a pure re-layout of the K pool (poison included).  v_sum
+    is an input of the algorithm (it enters as the mean value vector): it is drawn as
+    N(0, L) per element, the distribution of a sum of L unit normals, not computed from V."""
+    if case.block_table is None:
+        raise ValueError("the sparse path is defined on the paged layout")
+    w = case.workload
+    dev = case.q.device
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(BASE_SEED + 5000 + w.index + 1000 * case.layer)
+    kt_pool = case.k_cache.transpose(2, 3).contiguous()
+    lens = torch.tensor(case.seq_lens_host, dtype=torch.float32, device=dev)
+    v_sum = torch.randn((w.batch, w.heads, w.head_dim), dtype=torch.float32, device=dev,
+                        generator=gen) * lens.clamp(min=1).sqrt()[:, None, None]
+    keep = [0 if n == 0 else max(1, -(-n * int(round(keep_fraction * 1024)) // 1024))
+            for n in case.seq_lens_host]
+    return SparfState(kt_pool=kt_pool, v_sum=v_sum.contiguous(),
+                      k_tokens=torch.tensor(keep, dtype=torch.int32, device=dev),
+                      k_tokens_host=keep)
