@@ -152,6 +152,61 @@ int instinfer_decode_attention_static(void *out, float *lse, const void *q,
                                       int32_t *status_flags, void *cuda_stream);
 
 /*
+ * ---- Sparse decode attention (the paper's Algorithm 1, SparF; SparQ's arithmetic) ----
+ * Paged layout only.  Besides the K and V pools the cache keeps
+ *   kt_pool  fp16 [num_phys_blocks, heads, head_dim, block_tokens]: K a second time,
+ *            embedding-major inside each block (Sec. IV-C, hidden-embedding-indexed copy);
+ *   v_sum    fp32 [batch, heads, head_dim]: the sum of all cached V rows of each sequence;
+ *            Algorithm 1's mean value vector is v_sum / seq_lens[b].
+ *
+ * instinfer_sparf_append does what instinfer_kv_append does on the paged pools and also
+ * writes k_new into kt_pool and adds v_new to v_sum (one fp32 rounding per element).
+ */
+int instinfer_sparf_append(void *k_pool, void *v_pool, void *kt_pool, float *v_sum,
+                           const void *k_new, const void *v_new, const int32_t *seq_lens,
+                           const int32_t *block_table, int32_t max_blocks_per_seq,
+                           int32_t block_tokens, int64_t num_phys_blocks,
+                           int32_t batch, int32_t heads, int32_t head_dim,
+                           int32_t *status_flags, void *cuda_stream);
+
+/*
+ * Algorithm 1 per (sequence, head), S = seq_lens[b]:
+ *   1     I = the r dims of largest |q_d| (ties: lower d)
+ *   2-4   approximate weights s^ = softmax_i(q_I . K^T[I, i] * scale / sqrt(|q_I|_1 / |q|_1)),
+ *         read from kt_pool (scale = 1/sqrt(head_dim) gives the printed temperature)
+ *   5-6   J = the k positions of largest s^, the last `local_window` positions always kept
+ *         (ties: lower position); k = k_tokens[b] clipped to S, local_window clipped to k
+ *   7     alpha = sum of s^ over J
+ *   8-10  exact softmax over J of scale * q . K[j]
+ *   11    out = alpha * (weights . V[J]) + (1 - alpha) * v_sum / S
+ * The page-then-filter loading of steps 2-3 and 8-9 is a property of flash pages; here rows
+ * are gathered directly, which gives the same values.
+ *   out       fp16 [batch, heads, head_dim]
+ *   alpha     fp32 [batch, heads], nullable
+ *   selected  int32 [batch, heads, max_k], nullable: J in ascending order, -1 padded
+ *   k_tokens  int32 [batch], device; max_k is a host upper bound (1 <= max_k <= max_seq_len);
+ *             a larger k_tokens[b] is clipped to max_k
+ *   r         1 <= r <= head_dim
+ *   workspace at least instinfer_sparf_workspace_bytes(batch, heads, head_dim, max_seq_len, max_k)
+ * Scores and the selection are computed in fp32; two scores closer than fp32 rounding may be
+ * ordered differently than in exact arithmetic.  num_phys_blocks * heads * block_tokens must
+ * be below 2^31.  S == 0 gives a zero row.
+ */
+int instinfer_sparf_decode_attention(void *out, float *alpha, int32_t *selected, const void *q,
+                                     const void *k_pool, const void *v_pool, const void *kt_pool,
+                                     const float *v_sum, const int32_t *block_table,
+                                     const int32_t *seq_lens, const int32_t *k_tokens,
+                                     int32_t batch, int32_t heads, int32_t head_dim,
+                                     int32_t block_tokens, int32_t max_blocks_per_seq,
+                                     int64_t num_phys_blocks, int32_t max_seq_len, int32_t max_k,
+                                     int32_t r, int32_t local_window, float scale,
+                                     void *workspace, size_t workspace_bytes,
+                                     int32_t *status_flags, void *cuda_stream);
+
+size_t instinfer_sparf_workspace_bytes(int32_t batch, int32_t heads, int32_t head_dim,
+                                       int32_t max_seq_len, int32_t max_k);
+
+/*
  * Workspace size (bytes, host computation only) for a call with these sizes under the
  * current split plan; 0 if an argument is invalid.
  */

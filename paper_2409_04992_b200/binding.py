@@ -51,6 +51,15 @@ def load() -> ctypes.CDLL:
         lib.instinfer_decode_attention_static.argtypes = [ptr, ptr, ptr, ptr, ptr, ptr, ptr,
                                                           i32, i32, i32, i32, i32, i32, i64, i32,
                                                           f32, ptr, ptr]
+        lib.instinfer_sparf_append.restype = ctypes.c_int
+        lib.instinfer_sparf_append.argtypes = [ptr, ptr, ptr, ptr, ptr, ptr, ptr, ptr, i32, i32, i64,
+                                               i32, i32, i32, ptr, ptr]
+        lib.instinfer_sparf_decode_attention.restype = ctypes.c_int
+        lib.instinfer_sparf_decode_attention.argtypes = [ptr, ptr, ptr, ptr, ptr, ptr, ptr, ptr, ptr,
+                                                         ptr, ptr, i32, i32, i32, i32, i32, i64,
+                                                         i32, i32, i32, i32, f32, ptr, sz, ptr, ptr]
+        lib.instinfer_sparf_workspace_bytes.restype = sz
+        lib.instinfer_sparf_workspace_bytes.argtypes = [i32, i32, i32, i32, i32]
         lib.instinfer_workspace_bytes.restype = sz
         lib.instinfer_workspace_bytes.argtypes = [i32, i32, i32, i32]
         lib.instinfer_plan_chunk_tokens.restype = i32
@@ -174,6 +183,41 @@ def decode_attention_static(out: torch.Tensor, lse: Optional[torch.Tensor], q: t
         _ptr(out), _ptr(lse), _ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(block_table),
         _ptr(seq_lens), batch, heads, head_dim, s_max, block_tokens, max_blocks, phys,
         int(max_seq_len), float(scale), _ptr(status_flags), _stream(stream)))
+
+
+def sparf_append(k_pool: torch.Tensor, v_pool: torch.Tensor, kt_pool: torch.Tensor,
+                 v_sum: torch.Tensor, k_new: torch.Tensor, v_new: torch.Tensor,
+                 seq_lens: torch.Tensor, block_table: torch.Tensor,
+                 status_flags: Optional[torch.Tensor] = None,
+                 stream: Optional[torch.cuda.Stream] = None) -> None:
+    """instinfer_sparf_append: pools [P,H,T,D], kt_pool [P,H,D,T], v_sum fp32 [B,H,D]."""
+    batch, heads, head_dim = k_new.shape
+    _check(load().instinfer_sparf_append(
+        _ptr(k_pool), _ptr(v_pool), _ptr(kt_pool), _ptr(v_sum), _ptr(k_new), _ptr(v_new),
+        _ptr(seq_lens), _ptr(block_table), block_table.shape[1], k_pool.shape[2], k_pool.shape[0],
+        batch, heads, head_dim, _ptr(status_flags), _stream(stream)))
+
+
+def sparf_workspace_bytes(batch: int, heads: int, head_dim: int, max_seq_len: int, max_k: int) -> int:
+    return int(load().instinfer_sparf_workspace_bytes(batch, heads, head_dim, max_seq_len, max_k))
+
+
+def sparf_decode_attention(out: torch.Tensor, alpha: Optional[torch.Tensor],
+                           selected: Optional[torch.Tensor], q: torch.Tensor,
+                           k_pool: torch.Tensor, v_pool: torch.Tensor, kt_pool: torch.Tensor,
+                           v_sum: torch.Tensor, block_table: torch.Tensor, seq_lens: torch.Tensor,
+                           k_tokens: torch.Tensor, max_seq_len: int, max_k: int, r: int,
+                           local_window: int, scale: float, workspace: torch.Tensor,
+                           status_flags: Optional[torch.Tensor] = None,
+                           stream: Optional[torch.cuda.Stream] = None) -> None:
+    """instinfer_sparf_decode_attention (Algorithm 1) over paged pools."""
+    batch, heads, head_dim = q.shape
+    _check(load().instinfer_sparf_decode_attention(
+        _ptr(out), _ptr(alpha), _ptr(selected), _ptr(q), _ptr(k_pool), _ptr(v_pool), _ptr(kt_pool),
+        _ptr(v_sum), _ptr(block_table), _ptr(seq_lens), _ptr(k_tokens), batch, heads, head_dim,
+        k_pool.shape[2], block_table.shape[1], k_pool.shape[0], int(max_seq_len), int(max_k),
+        int(r), int(local_window), float(scale), _ptr(workspace),
+        workspace.numel() * workspace.element_size(), _ptr(status_flags), _stream(stream)))
 
 
 def alloc_workspace(batch: int, heads: int, head_dim: int, max_seq_len: int,

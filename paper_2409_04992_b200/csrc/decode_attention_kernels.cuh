@@ -67,7 +67,14 @@ struct AttnParams {
     int32_t n_splits;     // n_big + number of tail chunks
     int32_t max_seq_len;
     float scale_log2e;    // scale * log2(e): logits are kept in the base-2 domain
+    // gathered mode only (sparse attention over a list of selected rows):
+    const int32_t *row_ids;    // [pairs, row_stride] physical row index (phys * H + h) * T + slot
+    const int32_t *k_tokens;   // [batch] rows to attend per sequence (clipped to its length)
+    int32_t row_stride;
 };
+
+// Where a (sequence, head)'s rows come from.
+enum class Rows { kContiguous, kPaged, kGathered };
 
 __device__ __forceinline__ float fast_exp2(float x)
 {
@@ -94,6 +101,12 @@ __device__ __forceinline__ int checked_seq_len(const AttnParams &p, int b, bool 
         len = 0;
     }
     return len;
+}
+
+// Gathered mode: number of listed rows of sequence b (its k, clipped to its length and to the list).
+__device__ __forceinline__ int gathered_count(const AttnParams &p, int b, int len)
+{
+    return min(len, min(max(p.k_tokens[b], 0), p.row_stride));
 }
 
 // Logical token range [begin, begin + size) of chunk `split`.
@@ -161,10 +174,12 @@ __device__ __forceinline__ uint4 lds128(unsigned shared_addr)
     return v;
 }
 
-template <bool kPaged>
+template <Rows kRows>
 __global__ void __launch_bounds__(kThreads, kCtasPerSm)
 decode_attn_split_kernel(const AttnParams p)
 {
+    constexpr bool kPaged = kRows == Rows::kPaged;
+    constexpr bool kGathered = kRows == Rows::kGathered;
     extern __shared__ __align__(128) unsigned char smem[];
     constexpr int kStepTokens = kWarps * kTileRows;      // a warp's next tile is this far ahead
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -179,10 +194,11 @@ decode_attn_split_kernel(const AttnParams p)
     const int split = blockIdx.x / p.pairs;
     const int pair = blockIdx.x - split * p.pairs;
     const int b = pair / p.heads, h = pair - b * p.heads;
-    const bool final_writer = p.n_splits == 1;
+    const bool final_writer = !kGathered && p.n_splits == 1;
 
     // With several splits the merge kernel reports a bad length; here only the lone writer does.
-    const int len = checked_seq_len(p, b, threadIdx.x == 0 && h == 0 && final_writer);
+    int len = checked_seq_len(p, b, threadIdx.x == 0 && h == 0 && final_writer);
+    if (kGathered) len = gathered_count(p, b, len);           // rows in this pair's list
     int begin, chunk_size;
     chunk_range(p, split, begin, chunk_size);
     if (begin >= len) {
@@ -227,7 +243,19 @@ decode_attn_split_kernel(const AttnParams p)
     int64_t block_stride = 0, head_off = 0;
     int step_blk = 0, step_rem = 0, blocks_needed = 0;
     const int32_t *table_row = nullptr;
-    if (kPaged) {
+    // gathered: row ids of this warp's next 4 tiles, one per lane (tile = lane >> 3, row = lane & 7)
+    const int32_t *row_list = kGathered ? p.row_ids + (int64_t)pair * p.row_stride : nullptr;
+    int rows_now = 0, rows_next = 0;
+    auto load_rows = [&](int tile_base) -> int {
+        const int idx = begin + (warp + (tile_base + (lane >> 3)) * kWarps) * kTileRows + (lane & 7);
+        return idx < end ? __ldg(row_list + idx) : 0;
+    };
+    if (kGathered) {
+        if (my_tiles > 0) {
+            rows_now = load_rows(0);
+            rows_next = load_rows(4);
+        }
+    } else if (kPaged) {
         const int tokens = p.block_tokens;
         table_row = p.block_table + (int64_t)b * p.max_blocks_per_seq;
         blocks_needed = (end + tokens - 1) / tokens;
@@ -256,8 +284,24 @@ decode_attn_split_kernel(const AttnParams p)
         if (issue_j < my_tiles) {
             const int rows = issue_j == my_tiles - 1 ? last_rows : kTileRows;
             bool usable = true;
-            int64_t off;
-            if (kPaged) {
+            int64_t off = 0;
+            if (kGathered) {
+                if ((issue_j & 3) == 0 && issue_j > 0) {       // uniform: next window of 4 tiles
+                    rows_now = rows_next;
+                    rows_next = load_rows(issue_j + 4);
+                }
+                const unsigned dst = ring + issue_stage * kStageBytes;
+                const unsigned char *k_col = reinterpret_cast<const unsigned char *>(p.k) + col * 16;
+                const unsigned char *v_col = reinterpret_cast<const unsigned char *>(p.v) + col * 16;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int rid = __shfl_sync(0xffffffffu, rows_now, (issue_j & 3) * 8 + 2 * i + half_warp);
+                    const bool valid = 2 * i + half_warp < rows;
+                    const int64_t src = valid ? (int64_t)rid * kRowBytes : 0;
+                    cp_async_16(dst + k_dst + i * 2 * kKRowStride, k_col + src, valid ? 16 : 0);
+                    cp_async_16(dst + v_dst + i * 512, v_col + src, valid ? 16 : 0);
+                }
+            } else if (kPaged) {
                 int idx = blk - win_base;
                 if (idx >= 32) {               // uniform: slide the window of table entries
                     idx -= 32;
@@ -281,7 +325,9 @@ decode_attn_split_kernel(const AttnParams p)
             }
             const unsigned char *ks = k_lane + off, *vs = v_lane + off;
             const unsigned dst = ring + issue_stage * kStageBytes;
-            if (usable && rows == kTileRows) {                 // full tile: no predicates
+            if (kGathered) {
+                // copies already issued above
+            } else if (usable && rows == kTileRows) {          // full tile: no predicates
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
                     cp_async_16(dst + k_dst + i * 2 * kKRowStride, ks + i * 512, 16);

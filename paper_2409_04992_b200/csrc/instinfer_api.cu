@@ -7,6 +7,7 @@
 
 #include "decode_attention_kernels.cuh"
 #include "kv_append_kernel.cuh"
+#include "sparf_kernels.cuh"
 
 namespace {
 
@@ -113,9 +114,9 @@ int ensure_split_smem(bool paged)
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return INSTINFER_ERR_CUDA;
     if (!done[dev][paged]) {
         const cudaError_t err = paged
-            ? cudaFuncSetAttribute(decode_attn_split_kernel<true>,
+            ? cudaFuncSetAttribute(decode_attn_split_kernel<Rows::kPaged>,
                                    cudaFuncAttributeMaxDynamicSharedMemorySize, kSplitSmemBytes)
-            : cudaFuncSetAttribute(decode_attn_split_kernel<false>,
+            : cudaFuncSetAttribute(decode_attn_split_kernel<Rows::kContiguous>,
                                    cudaFuncAttributeMaxDynamicSharedMemorySize, kSplitSmemBytes);
         if (err != cudaSuccess) {
             (void)cudaGetLastError();
@@ -147,9 +148,9 @@ int launch_attention(AttnParams p, bool paged, int32_t batch, void *workspace,
     const unsigned grid = (unsigned)(pairs * plan.n_splits);
     if (g_before_split) cudaEventRecord(g_before_split, stream);
     if (paged)
-        decode_attn_split_kernel<true><<<grid, kThreads, kSplitSmemBytes, stream>>>(p);
+        decode_attn_split_kernel<Rows::kPaged><<<grid, kThreads, kSplitSmemBytes, stream>>>(p);
     else
-        decode_attn_split_kernel<false><<<grid, kThreads, kSplitSmemBytes, stream>>>(p);
+        decode_attn_split_kernel<Rows::kContiguous><<<grid, kThreads, kSplitSmemBytes, stream>>>(p);
     if (g_after_split) cudaEventRecord(g_after_split, stream);
     if (cudaGetLastError() != cudaSuccess) return INSTINFER_ERR_CUDA;
     if (plan.n_splits > 1) {
@@ -326,6 +327,191 @@ int instinfer_decode_attention_static(void *out, float *lse, const void *q, cons
                                             max_blocks_per_seq, num_phys_blocks, max_seq_len,
                                             scale, scratch, kStaticWorkspaceBytes, status_flags,
                                             cuda_stream);
+}
+
+namespace {
+
+struct SparfLayout {
+    size_t scores, row_ids, stats, partials, total;
+    int32_t score_stride;
+    SplitPlan plan;
+};
+
+size_t round256(size_t n) { return (n + 255) / 256 * 256; }
+
+SparfLayout sparf_layout(int64_t pairs, int32_t max_seq_len, int32_t max_k)
+{
+    SparfLayout w;
+    w.score_stride = (max_seq_len + 3) / 4 * 4;
+    w.plan = make_plan(pairs, max_k);
+    w.scores = 0;
+    w.row_ids = w.scores + round256((size_t)pairs * w.score_stride * sizeof(float));
+    w.stats = w.row_ids + round256((size_t)pairs * max_k * sizeof(int32_t));
+    w.partials = w.stats + round256((size_t)pairs * sizeof(float2));
+    w.total = w.partials + workspace_for(pairs, w.plan);
+    return w;
+}
+
+bool sparf_sizes_ok(int32_t batch, int32_t heads, int32_t head_dim, int32_t block_tokens,
+                    int32_t max_blocks_per_seq, int64_t num_phys_blocks)
+{
+    if (batch < 0 || heads <= 0 || head_dim <= 0 || block_tokens <= 0 || max_blocks_per_seq <= 0 ||
+        num_phys_blocks <= 0 || (int64_t)batch * heads > (int64_t)1 << 24)
+        return false;
+    return true;
+}
+
+}  // namespace
+
+int instinfer_sparf_append(void *k_pool, void *v_pool, void *kt_pool, float *v_sum,
+                           const void *k_new, const void *v_new, const int32_t *seq_lens,
+                           const int32_t *block_table, int32_t max_blocks_per_seq,
+                           int32_t block_tokens, int64_t num_phys_blocks, int32_t batch,
+                           int32_t heads, int32_t head_dim, int32_t *status_flags,
+                           void *cuda_stream)
+{
+    if (!sparf_sizes_ok(batch, heads, head_dim, block_tokens, max_blocks_per_seq, num_phys_blocks))
+        return INSTINFER_ERR_INVALID_ARG;
+    if (head_dim != kHeadDim || block_tokens % 8 != 0) return INSTINFER_ERR_UNSUPPORTED;
+    if (batch == 0) return INSTINFER_OK;
+    if (!usable(k_pool) || !usable(v_pool) || !usable(kt_pool) || !usable(v_sum) || !usable(k_new) ||
+        !usable(v_new) || seq_lens == nullptr || block_table == nullptr)
+        return INSTINFER_ERR_INVALID_ARG;
+    SparfParams p = {};
+    p.k_pool = static_cast<__half *>(k_pool);
+    p.v_pool = static_cast<__half *>(v_pool);
+    p.kt_pool = static_cast<__half *>(kt_pool);
+    p.v_sum = v_sum;
+    p.k_new = static_cast<const __half *>(k_new);
+    p.v_new = static_cast<const __half *>(v_new);
+    p.seq_lens = seq_lens;
+    p.block_table = block_table;
+    p.status = status_flags;
+    p.num_phys_blocks = num_phys_blocks;
+    p.batch = batch;
+    p.heads = heads;
+    p.block_tokens = block_tokens;
+    p.max_blocks_per_seq = max_blocks_per_seq;
+    sparf_append_kernel<<<(unsigned)((int64_t)batch * heads), kSparfThreads, 0,
+                          static_cast<cudaStream_t>(cuda_stream)>>>(p);
+    return cudaGetLastError() == cudaSuccess ? INSTINFER_OK : INSTINFER_ERR_CUDA;
+}
+
+size_t instinfer_sparf_workspace_bytes(int32_t batch, int32_t heads, int32_t head_dim,
+                                       int32_t max_seq_len, int32_t max_k)
+{
+    if (head_dim != kHeadDim || !sizes_ok(batch, heads, max_seq_len) || max_k <= 0 ||
+        max_k > max_seq_len)
+        return 0;
+    if (batch == 0) return 256;
+    return sparf_layout((int64_t)batch * heads, max_seq_len, max_k).total;
+}
+
+int instinfer_sparf_decode_attention(void *out, float *alpha, int32_t *selected, const void *q,
+                                     const void *k_pool, const void *v_pool, const void *kt_pool,
+                                     const float *v_sum, const int32_t *block_table,
+                                     const int32_t *seq_lens, const int32_t *k_tokens,
+                                     int32_t batch, int32_t heads, int32_t head_dim,
+                                     int32_t block_tokens, int32_t max_blocks_per_seq,
+                                     int64_t num_phys_blocks, int32_t max_seq_len, int32_t max_k,
+                                     int32_t r, int32_t local_window, float scale,
+                                     void *workspace, size_t workspace_bytes,
+                                     int32_t *status_flags, void *cuda_stream)
+{
+    if (!sparf_sizes_ok(batch, heads, head_dim, block_tokens, max_blocks_per_seq, num_phys_blocks) ||
+        max_seq_len <= 0 || (int64_t)max_seq_len > (int64_t)max_blocks_per_seq * block_tokens ||
+        max_k <= 0 || max_k > max_seq_len || local_window < 0 || !std::isfinite(scale))
+        return INSTINFER_ERR_INVALID_ARG;
+    if (head_dim != kHeadDim || block_tokens % 8 != 0) return INSTINFER_ERR_UNSUPPORTED;
+    if (r <= 0 || r > head_dim) return INSTINFER_ERR_INVALID_ARG;
+    if (num_phys_blocks * heads * block_tokens >= (int64_t)1 << 31) return INSTINFER_ERR_UNSUPPORTED;
+    if (batch == 0) return INSTINFER_OK;
+    if (!usable(out) || !usable(q) || !usable(k_pool) || !usable(v_pool) || !usable(kt_pool) ||
+        !usable(v_sum) || block_table == nullptr || seq_lens == nullptr || k_tokens == nullptr)
+        return INSTINFER_ERR_INVALID_ARG;
+    const int64_t pairs = (int64_t)batch * heads;
+    const SparfLayout w = sparf_layout(pairs, max_seq_len, max_k);
+    if (workspace == nullptr || !aligned16(workspace) || workspace_bytes < w.total)
+        return INSTINFER_ERR_WORKSPACE;
+    const int64_t score_chunks = ceil_div(max_seq_len, kScoreChunk);
+    if (pairs * score_chunks >= (int64_t)1 << 31 || pairs * w.plan.n_splits >= (int64_t)1 << 31)
+        return INSTINFER_ERR_INVALID_ARG;
+    unsigned char *ws = static_cast<unsigned char *>(workspace);
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+
+    SparfParams sp = {};
+    sp.k_pool = const_cast<__half *>(static_cast<const __half *>(k_pool));
+    sp.v_pool = const_cast<__half *>(static_cast<const __half *>(v_pool));
+    sp.kt_pool = const_cast<__half *>(static_cast<const __half *>(kt_pool));
+    sp.v_sum = const_cast<float *>(v_sum);
+    sp.q = static_cast<const __half *>(q);
+    sp.seq_lens = seq_lens;
+    sp.k_tokens = k_tokens;
+    sp.block_table = block_table;
+    sp.status = status_flags;
+    sp.scores = reinterpret_cast<float *>(ws + w.scores);
+    sp.row_ids = reinterpret_cast<int32_t *>(ws + w.row_ids);
+    sp.stats = reinterpret_cast<float2 *>(ws + w.stats);
+    sp.alpha_out = alpha;
+    sp.selected = selected;
+    sp.num_phys_blocks = num_phys_blocks;
+    sp.batch = batch;
+    sp.heads = heads;
+    sp.block_tokens = block_tokens;
+    sp.max_blocks_per_seq = max_blocks_per_seq;
+    sp.max_seq_len = max_seq_len;
+    sp.max_k = max_k;
+    sp.score_stride = w.score_stride;
+    sp.score_chunks = (int32_t)score_chunks;
+    sp.r = r;
+    sp.window = local_window;
+    sp.scale_log2e = scale * 1.44269504088896340736f;
+
+    sparf_scores_kernel<<<(unsigned)(pairs * score_chunks), kSparfThreads, 0, stream>>>(sp);
+    if (cudaGetLastError() != cudaSuccess) return INSTINFER_ERR_CUDA;
+    sparf_select_kernel<<<(unsigned)pairs, kSelectThreads, 0, stream>>>(sp);
+    if (cudaGetLastError() != cudaSuccess) return INSTINFER_ERR_CUDA;
+
+    SparfMergeParams mp = {};
+    AttnParams &ap = mp.attn;
+    ap.q = sp.q;
+    ap.k = sp.k_pool;
+    ap.v = sp.v_pool;
+    ap.seq_lens = seq_lens;
+    ap.out = static_cast<__half *>(out);
+    ap.status = nullptr;                 // the select kernel has already reported
+    ap.heads = heads;
+    ap.pairs = (int32_t)pairs;
+    ap.max_seq_len = max_seq_len;
+    ap.scale_log2e = sp.scale_log2e;
+    ap.chunk_tokens = w.plan.chunk_tokens;
+    ap.n_big = w.plan.n_big;
+    ap.tail_chunk = w.plan.tail_chunk;
+    ap.n_splits = w.plan.n_splits;
+    ap.part_o = reinterpret_cast<float *>(ws + w.partials);
+    ap.part_lse = ap.part_o + (size_t)pairs * w.plan.n_splits * kHeadDim;
+    ap.row_ids = sp.row_ids;
+    ap.k_tokens = k_tokens;
+    ap.row_stride = max_k;
+    mp.stats = sp.stats;
+    mp.v_sum = v_sum;
+
+    static bool smem_set[kMaxDevices] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return INSTINFER_ERR_CUDA;
+    if (!smem_set[dev]) {
+        if (cudaFuncSetAttribute(decode_attn_split_kernel<Rows::kGathered>,
+                                 cudaFuncAttributeMaxDynamicSharedMemorySize, kSplitSmemBytes) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return INSTINFER_ERR_CUDA;
+        }
+        smem_set[dev] = true;
+    }
+    decode_attn_split_kernel<Rows::kGathered>
+        <<<(unsigned)(pairs * w.plan.n_splits), kThreads, kSplitSmemBytes, stream>>>(ap);
+    if (cudaGetLastError() != cudaSuccess) return INSTINFER_ERR_CUDA;
+    sparf_merge_kernel<<<(unsigned)pairs, kHeadDim, 0, stream>>>(mp);
+    return cudaGetLastError() == cudaSuccess ? INSTINFER_OK : INSTINFER_ERR_CUDA;
 }
 
 size_t instinfer_workspace_bytes(int32_t batch, int32_t heads, int32_t head_dim, int32_t max_seq_len)

@@ -1,0 +1,346 @@
+// Sparse decode attention after the paper's Algorithm 1 (SparF: SparQ's arithmetic with
+// page-granular loading), on the block-paged cache, for sm_100a.
+//
+//   sparf_append_kernel   the new token's k,v go to the token-major pools, k also to the
+//                         embedding-major K copy (Sec. IV-C: K is stored twice), and v is
+//                         added to the running V sum that gives the mean value vector.
+//   sparf_scores_kernel   step 1 (the r largest |q_d|) and steps 2-4 without the softmax
+//                         normalisation: approximate logits from the embedding-major copy.
+//   sparf_select_kernel   softmax statistics of the approximate logits, steps 5-7: the k
+//                         largest scores with the last l tokens forced in (radix select on
+//                         order-preserving keys, ties to the lower index), alpha, and the
+//                         ascending list of selected rows as physical row ids.
+//   (steps 8-10 run in decode_attn_split_kernel<Rows::kGathered>)
+//   sparf_merge_kernel    log-sum-exp merge of the chunk partials and step 11:
+//                         out = alpha * attended + (1 - alpha) * v_sum / S.
+#pragma once
+
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "decode_attention_kernels.cuh"
+
+namespace instinfer {
+
+struct SparfParams {
+    // cache
+    __half *k_pool;
+    __half *v_pool;
+    __half *kt_pool;           // [P, H, D, T]
+    float *v_sum;              // [B, H, D]
+    const __half *q;
+    const __half *k_new;
+    const __half *v_new;
+    const int32_t *seq_lens;
+    const int32_t *k_tokens;
+    const int32_t *block_table;
+    int32_t *status;
+    // scratch
+    float *scores;             // [pairs, score_stride] approximate logits, base-2 domain
+    int32_t *row_ids;          // [pairs, max_k]
+    float2 *stats;             // [pairs] (alpha, number of selected rows)
+    // outputs
+    float *alpha_out;          // nullable [pairs]
+    int32_t *selected;         // nullable [pairs, max_k] logical token index, ascending, -1 padded
+    int64_t num_phys_blocks;
+    int32_t batch, heads, block_tokens, max_blocks_per_seq;
+    int32_t max_seq_len, max_k, score_stride, score_chunks, r, window;
+    float scale_log2e;
+};
+
+constexpr int kSparfThreads = 128;       // append and scores: one thread per head dim
+constexpr int kScoreChunk = 2048;        // tokens per scores block
+constexpr int kSelectThreads = 1024;
+
+__device__ __forceinline__ int sparf_seq_len(const SparfParams &p, int b, bool report)
+{
+    int len = p.seq_lens[b];
+    if (len < 0 || len > p.max_seq_len) {
+        if (report && p.status) atomicOr(p.status, kFlagSeqLenRange);
+        len = 0;
+    }
+    return len;
+}
+
+__global__ void __launch_bounds__(kSparfThreads)
+sparf_append_kernel(const SparfParams p)
+{
+    const int pair = blockIdx.x, d = threadIdx.x;
+    const int b = pair / p.heads, h = pair - b * p.heads;
+    const int len = p.seq_lens[b];
+    if (len == 0) return;
+    if (len < 0 || (int64_t)len > (int64_t)p.max_blocks_per_seq * p.block_tokens) {
+        if (d == 0 && h == 0 && p.status) atomicOr(p.status, kFlagSeqLenRange);
+        return;
+    }
+    const int pos = len - 1, T = p.block_tokens;
+    const int phys = p.block_table[(int64_t)b * p.max_blocks_per_seq + pos / T];
+    if (phys < 0 || (int64_t)phys >= p.num_phys_blocks) {
+        if (d == 0 && h == 0 && p.status) atomicOr(p.status, kFlagBlockRange);
+        return;
+    }
+    const int slot = pos % T;
+    const int64_t base = ((int64_t)phys * p.heads + h) * T * kHeadDim;      // elements
+    const __half k = p.k_new[(int64_t)pair * kHeadDim + d];
+    const __half v = p.v_new[(int64_t)pair * kHeadDim + d];
+    p.k_pool[base + (int64_t)slot * kHeadDim + d] = k;
+    p.v_pool[base + (int64_t)slot * kHeadDim + d] = v;
+    p.kt_pool[base + (int64_t)d * T + slot] = k;
+    p.v_sum[(int64_t)pair * kHeadDim + d] += __half2float(v);
+}
+
+// grid pairs * score_chunks: approximate logits of the tokens of one chunk of one (sequence, head).
+__global__ void __launch_bounds__(kSparfThreads)
+sparf_scores_kernel(const SparfParams p)
+{
+    __shared__ float sm_abs[kHeadDim];
+    __shared__ float sm_q[kHeadDim];        // q of the selected dims, in rank order
+    __shared__ int sm_dim[kHeadDim];
+    __shared__ float sm_red[2][kSparfThreads / 32];
+    const int pair = blockIdx.x / p.score_chunks, d = threadIdx.x;
+    const int b = pair / p.heads, h = pair - b * p.heads;
+    const int len = sparf_seq_len(p, b, false);
+    const int begin = (blockIdx.x - pair * p.score_chunks) * kScoreChunk;
+    if (begin >= len) return;
+    const int end = min(begin + kScoreChunk, len);
+
+    // Step 1: rank of |q_d| (exact comparisons of fp16 magnitudes, ties to the lower index).
+    const float qd = __half2float(p.q[(int64_t)pair * kHeadDim + d]);
+    sm_abs[d] = fabsf(qd);
+    __syncthreads();
+    int rank = 0;
+    for (int e = 0; e < kHeadDim; ++e) {
+        const float other = sm_abs[e];
+        rank += (other > sm_abs[d]) || (other == sm_abs[d] && e < d);
+    }
+    const bool kept = rank < p.r;
+    if (kept) {
+        sm_dim[rank] = d;
+        sm_q[rank] = qd;
+    }
+    // |q|_1 and |q_I|_1
+    float all = sm_abs[d], sel = kept ? sm_abs[d] : 0.f;
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) {
+        all += __shfl_xor_sync(0xffffffffu, all, off);
+        sel += __shfl_xor_sync(0xffffffffu, sel, off);
+    }
+    if ((d & 31) == 0) {
+        sm_red[0][d >> 5] = all;
+        sm_red[1][d >> 5] = sel;
+    }
+    __syncthreads();
+    all = sm_red[0][0] + sm_red[0][1] + sm_red[0][2] + sm_red[0][3];
+    sel = sm_red[1][0] + sm_red[1][1] + sm_red[1][2] + sm_red[1][3];
+    const float ratio = all > 0.f ? sel / all : 1.f;
+    const float approx_scale = p.scale_log2e * rsqrtf(ratio);
+
+    // Steps 2-4: one thread per token; the selected dims' rows of the K^T block are T apart.
+    const int T = p.block_tokens;
+    const int32_t *table_row = p.block_table + (int64_t)b * p.max_blocks_per_seq;
+    float *dst = p.scores + (int64_t)pair * p.score_stride;
+    for (int i = begin + d; i < end; i += kSparfThreads) {
+        const int blk = i / T, slot = i - blk * T;
+        const int phys = table_row[blk];
+        float dot = 0.f;
+        if (phys >= 0 && (int64_t)phys < p.num_phys_blocks) {
+            const __half *kt = p.kt_pool + ((int64_t)phys * p.heads + h) * T * kHeadDim + slot;
+            for (int t = 0; t < p.r; ++t)
+                dot = fmaf(sm_q[t], __half2float(kt[(int64_t)sm_dim[t] * T]), dot);
+        } else if (p.status) {
+            atomicOr(p.status, kFlagBlockRange);
+        }
+        dst[i] = dot * approx_scale;
+    }
+}
+
+// Order-preserving map float -> uint32 (larger float, larger key).
+__device__ __forceinline__ unsigned ordered_key(float x)
+{
+    const unsigned u = __float_as_uint(x);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+template <typename T>
+__device__ __forceinline__ T block_sum(T v, T *scratch)      // scratch: 32 entries
+{
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0) scratch[threadIdx.x >> 5] = v;
+    __syncthreads();
+    T total = 0;
+    for (int w = 0; w < (int)(blockDim.x >> 5); ++w) total += scratch[w];
+    return total;
+}
+
+// One block per (sequence, head).
+__global__ void __launch_bounds__(kSelectThreads)
+sparf_select_kernel(const SparfParams p)
+{
+    __shared__ unsigned hist[256];
+    __shared__ float red_f[32];
+    __shared__ int warp_gt[32], warp_eq[32];
+    __shared__ unsigned sm_prefix;
+    __shared__ int sm_remaining;
+    const int pair = blockIdx.x, tid = threadIdx.x;
+    const int b = pair / p.heads, h = pair - b * p.heads;
+    const int S = sparf_seq_len(p, b, tid == 0 && h == 0);
+    const int k = min(S, min(max(p.k_tokens[b], 0), p.max_k));
+    const int window = min(p.window, k);
+    int32_t *rows = p.row_ids + (int64_t)pair * p.max_k;
+    int32_t *sel = p.selected ? p.selected + (int64_t)pair * p.max_k : nullptr;
+    if (sel) for (int t = k + tid; t < p.max_k; t += kSelectThreads) sel[t] = -1;
+    if (k == 0) {
+        if (tid == 0) {
+            p.stats[pair] = make_float2(0.f, 0.f);
+            if (p.alpha_out) p.alpha_out[pair] = 0.f;
+        }
+        return;
+    }
+    const float *a = p.scores + (int64_t)pair * p.score_stride;
+
+    // softmax statistics of the approximate logits (base-2 domain)
+    float top = kMinusHuge;
+    for (int i = tid; i < S; i += kSelectThreads) top = fmaxf(top, a[i]);
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) top = fmaxf(top, __shfl_xor_sync(0xffffffffu, top, off));
+    if ((tid & 31) == 0) red_f[tid >> 5] = top;
+    __syncthreads();
+    top = red_f[0];
+    for (int w = 1; w < kSelectThreads / 32; ++w) top = fmaxf(top, red_f[w]);
+    float z = 0.f;
+    for (int i = tid; i < S; i += kSelectThreads) z += fast_exp2(a[i] - top);
+    z = block_sum(z, red_f);
+
+    // Step 5: the last `window` positions get the largest key (s^ + 1 beats every s^).
+    auto key_of = [&](int i) -> unsigned { return i >= S - window ? 0xffffffffu : ordered_key(a[i]); };
+
+    // Step 6: radix select of the k-th largest key, 8 bits per pass from the top.
+    if (tid == 0) {
+        sm_prefix = 0u;
+        sm_remaining = k;
+    }
+    for (int pass = 0; pass < 4; ++pass) {
+        const int shift = 24 - 8 * pass;
+        const unsigned mask = pass == 0 ? 0u : 0xffffffffu << (shift + 8);
+        if (tid < 256) hist[tid] = 0u;
+        __syncthreads();
+        const unsigned prefix = sm_prefix;
+        for (int i = tid; i < S; i += kSelectThreads) {
+            const unsigned key = key_of(i);
+            if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
+        }
+        __syncthreads();
+        if (tid == 0) {
+            int remaining = sm_remaining, bucket = 255;
+            for (; bucket > 0; --bucket) {
+                const int c = (int)hist[bucket];
+                if (c >= remaining) break;
+                remaining -= c;
+            }
+            sm_prefix = prefix | ((unsigned)bucket << shift);
+            sm_remaining = remaining;
+        }
+        __syncthreads();
+    }
+    const unsigned tau = sm_prefix;          // key of the k-th largest
+    const int take_equal = sm_remaining;     // how many keys equal to tau belong to the top k
+
+    // Ordered compaction: position = #greater before + min(#equal before, take_equal).
+    const int T = p.block_tokens;
+    const int32_t *table_row = p.block_table + (int64_t)b * p.max_blocks_per_seq;
+    int base_gt = 0, base_eq = 0;
+    float mass = 0.f;
+    const int lane = tid & 31, warp = tid >> 5;
+    for (int start = 0; start < S; start += kSelectThreads) {
+        const int i = start + tid;
+        unsigned key = 0u;
+        bool gt = false, eq = false;
+        if (i < S) {
+            key = key_of(i);
+            gt = key > tau;
+            eq = key == tau;
+        }
+        const unsigned bal_gt = __ballot_sync(0xffffffffu, gt), bal_eq = __ballot_sync(0xffffffffu, eq);
+        if (lane == 0) {
+            warp_gt[warp] = __popc(bal_gt);
+            warp_eq[warp] = __popc(bal_eq);
+        }
+        __syncthreads();
+        int gt_before = base_gt, eq_before = base_eq, gt_tile = 0, eq_tile = 0;
+        for (int w = 0; w < kSelectThreads / 32; ++w) {
+            if (w < warp) {
+                gt_before += warp_gt[w];
+                eq_before += warp_eq[w];
+            }
+            gt_tile += warp_gt[w];
+            eq_tile += warp_eq[w];
+        }
+        const unsigned below = (1u << lane) - 1u;
+        gt_before += __popc(bal_gt & below);
+        eq_before += __popc(bal_eq & below);
+        if (gt || (eq && eq_before < take_equal)) {
+            const int pos = gt_before + min(eq_before, take_equal);
+            const int blk = i / T, slot = i - blk * T;
+            const int phys = table_row[blk];
+            const bool ok = phys >= 0 && (int64_t)phys < p.num_phys_blocks;
+            if (!ok && p.status) atomicOr(p.status, kFlagBlockRange);
+            rows[pos] = ok ? (phys * p.heads + h) * T + slot : 0;
+            if (sel) sel[pos] = i;
+            mass += fast_exp2(a[i] - top);
+        }
+        base_gt += gt_tile;
+        base_eq += eq_tile;
+        __syncthreads();
+    }
+    mass = block_sum(mass, red_f);
+    if (tid == 0) {
+        const float alpha = mass / z;
+        p.stats[pair] = make_float2(alpha, (float)k);
+        if (p.alpha_out) p.alpha_out[pair] = alpha;
+    }
+}
+
+// Merge of the gathered-attention partials and step 11.
+struct SparfMergeParams {
+    AttnParams attn;
+    const float2 *stats;
+    const float *v_sum;
+};
+
+__global__ void __launch_bounds__(kHeadDim)
+sparf_merge_kernel(const SparfMergeParams m)
+{
+    const AttnParams &p = m.attn;
+    const int pair = blockIdx.x;
+    const int b = pair / p.heads;
+    const int S = checked_seq_len(p, b, false);
+    __half *out = p.out + (int64_t)pair * kHeadDim + threadIdx.x;
+    if (S == 0) {
+        *out = __float2half_rn(0.f);
+        return;
+    }
+    const float alpha = m.stats[pair].x;
+    const int count = gathered_count(p, b, S);
+    const float vbar = m.v_sum[(int64_t)pair * kHeadDim + threadIdx.x] / (float)S;
+    const int live = live_chunks(p, count);
+    float attended = 0.f;
+    if (live > 0) {
+        const float *lse2 = p.part_lse + (int64_t)pair * p.n_splits;
+        const float *po = p.part_o + (int64_t)pair * p.n_splits * kHeadDim + threadIdx.x;
+        float top = kMinusHuge;
+        for (int s = 0; s < live; ++s) top = fmaxf(top, lse2[s]);
+        float total = 0.f, o = 0.f;
+        for (int s = 0; s < live; ++s) {
+            const float w = fast_exp2(lse2[s] - top);
+            total += w;
+            o = fmaf(w, po[(int64_t)s * kHeadDim], o);
+        }
+        attended = o / total;
+    }
+    *out = __float2half_rn(alpha * attended + (1.f - alpha) * vbar);
+}
+
+}  // namespace instinfer
