@@ -156,6 +156,8 @@ int instinfer_decode_attention_static(void *out, float *lse, const void *q,
  * Paged layout only.  Besides the K and V pools the cache keeps
  *   kt_pool  fp16 [num_phys_blocks, heads, head_dim, block_tokens]: K a second time,
  *            embedding-major inside each block (Sec. IV-C, hidden-embedding-indexed copy);
+ *            slots past a sequence's end inside its last block may be read (in groups of 8
+ *            tokens) but never influence a result;
  *   v_sum    fp32 [batch, heads, head_dim]: the sum of all cached V rows of each sequence;
  *            Algorithm 1's mean value vector is v_sum / seq_lens[b].
  *

@@ -342,7 +342,7 @@ size_t round256(size_t n) { return (n + 255) / 256 * 256; }
 SparfLayout sparf_layout(int64_t pairs, int32_t max_seq_len, int32_t max_k)
 {
     SparfLayout w;
-    w.score_stride = (max_seq_len + 3) / 4 * 4;
+    w.score_stride = (max_seq_len + 7) / 8 * 8;      // whole 8-token groups, 32-byte aligned rows
     w.plan = make_plan(pairs, max_k);
     w.scores = 0;
     w.row_ids = w.scores + round256((size_t)pairs * w.score_stride * sizeof(float));

@@ -136,22 +136,44 @@ sparf_scores_kernel(const SparfParams p)
     const float ratio = all > 0.f ? sel / all : 1.f;
     const float approx_scale = p.scale_log2e * rsqrtf(ratio);
 
-    // Steps 2-4: one thread per token; the selected dims' rows of the K^T block are T apart.
+    // Steps 2-4: one thread per group of 8 consecutive tokens (one 16-byte load per selected
+    // dim; block_tokens is a multiple of 8, so a group never straddles a block).  The loads
+    // of 8 dims are issued together to keep enough bytes in flight.
     const int T = p.block_tokens;
     const int32_t *table_row = p.block_table + (int64_t)b * p.max_blocks_per_seq;
     float *dst = p.scores + (int64_t)pair * p.score_stride;
-    for (int i = begin + d; i < end; i += kSparfThreads) {
+    for (int i = begin + d * 8; i < end; i += kSparfThreads * 8) {
         const int blk = i / T, slot = i - blk * T;
         const int phys = table_row[blk];
-        float dot = 0.f;
+        float dot[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) dot[e] = 0.f;
         if (phys >= 0 && (int64_t)phys < p.num_phys_blocks) {
             const __half *kt = p.kt_pool + ((int64_t)phys * p.heads + h) * T * kHeadDim + slot;
-            for (int t = 0; t < p.r; ++t)
-                dot = fmaf(sm_q[t], __half2float(kt[(int64_t)sm_dim[t] * T]), dot);
+            for (int t0 = 0; t0 < p.r; t0 += 8) {
+                uint4 raw[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    const int t = min(t0 + u, p.r - 1);            // clamped: extra loads repeat the last dim
+                    raw[u] = __ldg(reinterpret_cast<const uint4 *>(kt + (int64_t)sm_dim[t] * T));
+                }
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    const float qv = t0 + u < p.r ? sm_q[t0 + u] : 0.f;
+                    float kf[8];
+                    unpack8(raw[u], kf);
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) dot[e] = fmaf(qv, kf[e], dot[e]);
+                }
+            }
         } else if (p.status) {
             atomicOr(p.status, kFlagBlockRange);
         }
-        dst[i] = dot * approx_scale;
+        // score_stride is a multiple of 8 and rows start 32-byte aligned; entries past `end`
+        // inside the last group are scratch nobody reads.
+        float4 *out4 = reinterpret_cast<float4 *>(dst + i);
+        out4[0] = make_float4(dot[0] * approx_scale, dot[1] * approx_scale, dot[2] * approx_scale, dot[3] * approx_scale);
+        out4[1] = make_float4(dot[4] * approx_scale, dot[5] * approx_scale, dot[6] * approx_scale, dot[7] * approx_scale);
     }
 }
 
