@@ -7,8 +7,9 @@
 //   sparf_scores_kernel   step 1 (the r largest |q_d|) and steps 2-4 without the softmax
 //                         normalisation: approximate logits from the embedding-major copy.
 //   sparf_select_kernel   softmax statistics of the approximate logits, steps 5-7: the k
-//                         largest scores with the last l tokens forced in (radix select on
-//                         order-preserving keys, ties to the lower index), alpha, and the
+//                         largest scores with the last l tokens forced in (a monotone
+//                         linear histogram finds the threshold bin, its members are
+//                         resolved exactly; ties to the lower index), alpha, and the
 //                         ascending list of selected rows as physical row ids.
 //   (steps 8-10 run in decode_attn_split_kernel<Rows::kGathered>)
 //   sparf_merge_kernel    log-sum-exp merge of the chunk partials and step 11:
@@ -197,16 +198,95 @@ __device__ __forceinline__ T block_sum(T v, T *scratch)      // scratch: 32 entr
     return total;
 }
 
+constexpr int kLinearBins = 2048;        // select: linear bins between the smallest and largest logit
+constexpr int kCandidates = 8192;        // select: keys of the threshold bin resolved in shared memory
+
+struct SelectShared {
+    unsigned hist[kLinearBins + 1];      // bin kLinearBins: the forced local window
+    unsigned cand[kCandidates];
+    float red_f[32];
+    unsigned red_u[2][32];
+    int scan_gt[32], scan_eq[32];
+    unsigned tau;
+    int take_equal, bin, above, n_cand;
+};
+
+// Exact k-th largest among the keys key_at(i) of the members i < n (member(i) true), 8 bits
+// per pass from the top.  Bytes on which all members agree are skipped without counting, so
+// a set of (nearly) equal keys costs nothing.  Returns through sh.tau / sh.take_equal the
+// threshold key and how many keys equal to it are among the `need` largest.
+template <typename Member, typename KeyAt>
+__device__ __forceinline__ void exact_threshold(SelectShared &sh, int n, int need, Member member, KeyAt key_at)
+{
+    const int tid = threadIdx.x;
+    unsigned any = 0u, all = 0xffffffffu;
+    for (int i = tid; i < n; i += kSelectThreads) {
+        if (member(i)) {
+            const unsigned key = key_at(i);
+            any |= key;
+            all &= key;
+        }
+    }
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) {
+        any |= __shfl_xor_sync(0xffffffffu, any, off);
+        all &= __shfl_xor_sync(0xffffffffu, all, off);
+    }
+    __syncthreads();
+    if ((tid & 31) == 0) {
+        sh.red_u[0][tid >> 5] = any;
+        sh.red_u[1][tid >> 5] = all;
+    }
+    __syncthreads();
+    any = 0u;
+    all = 0xffffffffu;
+    for (int w = 0; w < kSelectThreads / 32; ++w) {
+        any |= sh.red_u[0][w];
+        all &= sh.red_u[1][w];
+    }
+    const unsigned differ = any ^ all;           // bits on which members disagree
+    unsigned prefix = 0u;
+    int remaining = need;
+    for (int pass = 0; pass < 4; ++pass) {
+        const int shift = 24 - 8 * pass;
+        const unsigned done_mask = pass == 0 ? 0u : 0xffffffffu << (shift + 8);
+        if (((differ >> shift) & 255u) == 0u) {  // every member has the same byte here
+            prefix |= all & (255u << shift);
+            continue;
+        }
+        __syncthreads();
+        if (tid < 256) sh.hist[tid] = 0u;
+        __syncthreads();
+        for (int i = tid; i < n; i += kSelectThreads) {
+            if (member(i)) {
+                const unsigned key = key_at(i);
+                if ((key & done_mask) == prefix) atomicAdd(&sh.hist[(key >> shift) & 255u], 1u);
+            }
+        }
+        __syncthreads();
+        int bucket = 255;
+        for (; bucket > 0; --bucket) {           // every thread walks the same 256 counters
+            const int c = (int)sh.hist[bucket];
+            if (c >= remaining) break;
+            remaining -= c;
+        }
+        prefix |= (unsigned)bucket << shift;
+    }
+    __syncthreads();
+    if (tid == 0) {
+        sh.tau = prefix;
+        sh.take_equal = remaining;
+    }
+    __syncthreads();
+}
+
 // One block per (sequence, head).
 __global__ void __launch_bounds__(kSelectThreads)
 sparf_select_kernel(const SparfParams p)
 {
-    __shared__ unsigned hist[256];
-    __shared__ float red_f[32];
-    __shared__ int warp_gt[32], warp_eq[32];
-    __shared__ unsigned sm_prefix;
-    __shared__ int sm_remaining;
+    __shared__ SelectShared sh;
     const int pair = blockIdx.x, tid = threadIdx.x;
+    const int lane = tid & 31, warp = tid >> 5;
     const int b = pair / p.heads, h = pair - b * p.heads;
     const int S = sparf_seq_len(p, b, tid == 0 && h == 0);
     const int k = min(S, min(max(p.k_tokens[b], 0), p.max_k));
@@ -223,86 +303,135 @@ sparf_select_kernel(const SparfParams p)
     }
     const float *a = p.scores + (int64_t)pair * p.score_stride;
 
-    // softmax statistics of the approximate logits (base-2 domain)
-    float top = kMinusHuge;
-    for (int i = tid; i < S; i += kSelectThreads) top = fmaxf(top, a[i]);
+    // Pass 1: largest and smallest approximate logit (base-2 domain).
+    float top = kMinusHuge, low = -kMinusHuge;
+    for (int i = tid; i < S; i += kSelectThreads) {
+        const float x = a[i];
+        top = fmaxf(top, x);
+        low = fminf(low, x);
+    }
 #pragma unroll
-    for (int off = 16; off >= 1; off >>= 1) top = fmaxf(top, __shfl_xor_sync(0xffffffffu, top, off));
-    if ((tid & 31) == 0) red_f[tid >> 5] = top;
+    for (int off = 16; off >= 1; off >>= 1) {
+        top = fmaxf(top, __shfl_xor_sync(0xffffffffu, top, off));
+        low = fminf(low, __shfl_xor_sync(0xffffffffu, low, off));
+    }
+    if (lane == 0) {
+        sh.red_f[warp] = top;
+        sh.red_u[0][warp] = __float_as_uint(low);
+    }
+    for (int t = tid; t <= kLinearBins; t += kSelectThreads) sh.hist[t] = 0u;
     __syncthreads();
-    top = red_f[0];
-    for (int w = 1; w < kSelectThreads / 32; ++w) top = fmaxf(top, red_f[w]);
+    for (int w = 0; w < kSelectThreads / 32; ++w) {
+        top = fmaxf(top, sh.red_f[w]);
+        low = fminf(low, __uint_as_float(sh.red_u[0][w]));
+    }
+
+    // Step 5: the last `window` positions rank above everything (s^ + 1 beats every s^).
+    // Linear bins are monotone in the logit: a higher bin holds strictly larger logits.
+    const float bin_scale = top > low ? (float)(kLinearBins - 1) / (top - low) : 0.f;
+    auto bin_of = [&](int i, float x) -> int {
+        return i >= S - window ? kLinearBins : min(kLinearBins - 1, (int)((x - low) * bin_scale));
+    };
+    auto key_of = [&](int i, float x) -> unsigned { return i >= S - window ? 0xffffffffu : ordered_key(x); };
+
+    // Pass 2: histogram over the linear bins, and the softmax denominator.
     float z = 0.f;
-    for (int i = tid; i < S; i += kSelectThreads) z += fast_exp2(a[i] - top);
-    z = block_sum(z, red_f);
-
-    // Step 5: the last `window` positions get the largest key (s^ + 1 beats every s^).
-    auto key_of = [&](int i) -> unsigned { return i >= S - window ? 0xffffffffu : ordered_key(a[i]); };
-
-    // Step 6: radix select of the k-th largest key, 8 bits per pass from the top.
-    if (tid == 0) {
-        sm_prefix = 0u;
-        sm_remaining = k;
+    for (int i = tid; i < S; i += kSelectThreads) {
+        const float x = a[i];
+        z += fast_exp2(x - top);
+        atomicAdd(&sh.hist[bin_of(i, x)], 1u);
     }
-    for (int pass = 0; pass < 4; ++pass) {
-        const int shift = 24 - 8 * pass;
-        const unsigned mask = pass == 0 ? 0u : 0xffffffffu << (shift + 8);
-        if (tid < 256) hist[tid] = 0u;
-        __syncthreads();
-        const unsigned prefix = sm_prefix;
-        for (int i = tid; i < S; i += kSelectThreads) {
-            const unsigned key = key_of(i);
-            if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
+    z = block_sum(z, sh.red_f);                  // its barriers also publish the histogram
+
+    // The bin that holds the k-th largest: warp 0, lane L owns bins [64 L, 64 L + 64).
+    if (warp == 0) {
+        int mine = 0;
+        for (int j = 0; j < 64; ++j) mine += (int)sh.hist[64 * lane + ((j + lane) & 63)];
+        int above = (int)sh.hist[kLinearBins];   // members of higher bins
+        for (int src = 31; src >= 0; --src) {
+            const int seg = __shfl_sync(0xffffffffu, mine, src);
+            if (src > lane) above += seg;
         }
-        __syncthreads();
-        if (tid == 0) {
-            int remaining = sm_remaining, bucket = 255;
-            for (; bucket > 0; --bucket) {
-                const int c = (int)hist[bucket];
-                if (c >= remaining) break;
-                remaining -= c;
+        if ((int)sh.hist[kLinearBins] >= k) {
+            if (lane == 0) {
+                sh.bin = kLinearBins;
+                sh.above = 0;
             }
-            sm_prefix = prefix | ((unsigned)bucket << shift);
-            sm_remaining = remaining;
+        } else if (above < k && k <= above + mine) {
+            int bin = 64 * lane + 63;
+            for (; bin > 64 * lane; --bin) {
+                const int c = (int)sh.hist[bin];
+                if (above + c >= k) break;
+                above += c;
+            }
+            sh.bin = bin;
+            sh.above = above;
+        }
+        if (lane == 0) sh.n_cand = 0;
+    }
+    __syncthreads();
+    const int bin = sh.bin, above = sh.above;
+    const int in_bin = (int)sh.hist[bin];
+    __syncthreads();                             // the histogram is reused below
+
+    // Step 6: the exact threshold inside that bin.
+    if (bin == kLinearBins) {                    // the window alone fills k
+        if (tid == 0) {
+            sh.tau = 0xffffffffu;
+            sh.take_equal = k;
         }
         __syncthreads();
+    } else if (in_bin <= kCandidates) {
+        for (int i = tid; i < S; i += kSelectThreads) {
+            const float x = a[i];
+            if (bin_of(i, x) == bin) sh.cand[atomicAdd(&sh.n_cand, 1)] = ordered_key(x);
+        }
+        __syncthreads();
+        exact_threshold(sh, in_bin, k - above, [](int) { return true; },
+                        [&](int i) { return sh.cand[i]; });
+    } else {                                     // very many near-equal logits: work from global memory
+        exact_threshold(sh, S, k - above, [&](int i) { return bin_of(i, a[i]) == bin; },
+                        [&](int i) { return ordered_key(a[i]); });
     }
-    const unsigned tau = sm_prefix;          // key of the k-th largest
-    const int take_equal = sm_remaining;     // how many keys equal to tau belong to the top k
+    const unsigned tau = sh.tau;                 // key of the k-th largest
+    const int take_equal = sh.take_equal;        // how many keys equal to tau belong to the top k
 
     // Ordered compaction: position = #greater before + min(#equal before, take_equal).
     const int T = p.block_tokens;
     const int32_t *table_row = p.block_table + (int64_t)b * p.max_blocks_per_seq;
     int base_gt = 0, base_eq = 0;
     float mass = 0.f;
-    const int lane = tid & 31, warp = tid >> 5;
     for (int start = 0; start < S; start += kSelectThreads) {
         const int i = start + tid;
-        unsigned key = 0u;
         bool gt = false, eq = false;
+        float x = 0.f;
         if (i < S) {
-            key = key_of(i);
+            x = a[i];
+            const unsigned key = key_of(i, x);
             gt = key > tau;
             eq = key == tau;
         }
         const unsigned bal_gt = __ballot_sync(0xffffffffu, gt), bal_eq = __ballot_sync(0xffffffffu, eq);
         if (lane == 0) {
-            warp_gt[warp] = __popc(bal_gt);
-            warp_eq[warp] = __popc(bal_eq);
+            sh.scan_gt[warp] = __popc(bal_gt);
+            sh.scan_eq[warp] = __popc(bal_eq);
         }
         __syncthreads();
-        int gt_before = base_gt, eq_before = base_eq, gt_tile = 0, eq_tile = 0;
-        for (int w = 0; w < kSelectThreads / 32; ++w) {
-            if (w < warp) {
-                gt_before += warp_gt[w];
-                eq_before += warp_eq[w];
+        // every warp scans the 32 per-warp counts with shuffles
+        const int cg = sh.scan_gt[lane], ce = sh.scan_eq[lane];
+        int ig = cg, ie = ce;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const int ug = __shfl_up_sync(0xffffffffu, ig, off), ue = __shfl_up_sync(0xffffffffu, ie, off);
+            if (lane >= off) {
+                ig += ug;
+                ie += ue;
             }
-            gt_tile += warp_gt[w];
-            eq_tile += warp_eq[w];
         }
-        const unsigned below = (1u << lane) - 1u;
-        gt_before += __popc(bal_gt & below);
-        eq_before += __popc(bal_eq & below);
+        const int gt_tile = __shfl_sync(0xffffffffu, ig, 31), eq_tile = __shfl_sync(0xffffffffu, ie, 31);
+        const int below = (1u << lane) - 1u;
+        const int gt_before = base_gt + __shfl_sync(0xffffffffu, ig - cg, warp) + __popc(bal_gt & below);
+        const int eq_before = base_eq + __shfl_sync(0xffffffffu, ie - ce, warp) + __popc(bal_eq & below);
         if (gt || (eq && eq_before < take_equal)) {
             const int pos = gt_before + min(eq_before, take_equal);
             const int blk = i / T, slot = i - blk * T;
@@ -311,13 +440,13 @@ sparf_select_kernel(const SparfParams p)
             if (!ok && p.status) atomicOr(p.status, kFlagBlockRange);
             rows[pos] = ok ? (phys * p.heads + h) * T + slot : 0;
             if (sel) sel[pos] = i;
-            mass += fast_exp2(a[i] - top);
+            mass += fast_exp2(x - top);
         }
         base_gt += gt_tile;
         base_eq += eq_tile;
         __syncthreads();
     }
-    mass = block_sum(mass, red_f);
+    mass = block_sum(mass, sh.red_f);
     if (tid == 0) {
         const float alpha = mass / z;
         p.stats[pair] = make_float2(alpha, (float)k);
