@@ -492,6 +492,57 @@ def measure_workload(w: wl.Workload, ranks: Ranks, device, steps: int, warmup: i
     return res
 
 
+def measure_sparse(w: wl.Workload, device, steps: int, r: int = 16, keep: float = 0.125,
+                   window: int = 16) -> dict:
+    """One layer of `w` through the sparse (Algorithm 1) entry points next to the dense ones on
+    the same data: append + attention per step, CUDA events, inputs far larger than L2."""
+    from paper_2409_04992_b200 import binding
+    case = wl.generate(w.replace(layers=1), device=str(device), poison=False)
+    state = wl.make_sparf_state(case, keep)
+    B, H, D = case.q.shape
+    max_len, max_k = case.max_seq_len, max(state.k_tokens_host)
+    out = torch.empty((B, H, D), dtype=torch.float16, device=device)
+    lse = torch.empty((B, H), dtype=torch.float32, device=device)
+    flags = torch.zeros(1, dtype=torch.int32, device=device)
+    ws_dense = binding.alloc_workspace(B, H, D, max_len, device)
+    ws_sparse = torch.empty(binding.sparf_workspace_bytes(B, H, D, max_len, max_k), dtype=torch.uint8,
+                            device=device)
+
+    def dense():
+        binding.kv_append(case.k_cache, case.v_cache, case.k_new, case.v_new, case.seq_lens,
+                          case.block_table, flags)
+        binding.decode_attention_paged(out, lse, case.q, case.k_cache, case.v_cache, case.block_table,
+                                       case.seq_lens, max_len, case.scale, ws_dense, flags)
+
+    def sparse():
+        binding.sparf_append(case.k_cache, case.v_cache, state.kt_pool, state.v_sum, case.k_new,
+                             case.v_new, case.seq_lens, case.block_table, flags)
+        binding.sparf_decode_attention(out, None, None, case.q, case.k_cache, case.v_cache,
+                                       state.kt_pool, state.v_sum, case.block_table, case.seq_lens,
+                                       state.k_tokens, max_len, max_k, r, window, case.scale,
+                                       ws_sparse, flags)
+
+    def timed(fn):
+        for _ in range(3):
+            fn()
+        a, z = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        a.record()
+        for _ in range(steps):
+            fn()
+        z.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(z) / 1e3 / steps
+
+    t_dense, t_sparse = timed(dense), timed(sparse)
+    moved = case.kv_tokens * H * r * 2 + sum(state.k_tokens_host) * H * 2 * D * 2
+    return {"r": r, "keep_fraction": keep, "local_window": window, "ms_per_step": t_sparse * 1e3,
+            "dense_ms_per_step": t_dense * 1e3, "speedup_over_dense": t_dense / t_sparse,
+            "kv_tokens_per_s": case.kv_tokens / t_sparse,
+            "algorithmic_bytes": moved, "algorithmic_gbs": moved / t_sparse / 1e9,
+            "status_flags": int(flags.item())}
+
+
 def main(argv=None) -> int:
     args = parse_args(argv)
     if args.impl == "reference":          # CPU only: no process group; ranks other than 0 do nothing
@@ -562,6 +613,8 @@ def main(argv=None) -> int:
                     "chunk_tokens": r["chunk_tokens"], "sm_mhz": r["clocks"]["sm_mhz"],
                     "reasons": r["clocks"]["reasons"]}
             line["other_workloads"] = others
+            line["sparse_attention"] = {wl.STANDARD[i].name: measure_sparse(wl.STANDARD[i], device, 10)
+                                        for i in (2, 3)}
         if ranks.rank == 0:
             print(json.dumps(line), flush=True)
         return 0
