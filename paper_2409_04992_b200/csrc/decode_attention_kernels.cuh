@@ -143,10 +143,11 @@ __device__ __forceinline__ void halves(unsigned packed, unsigned short &lo, unsi
     asm("mov.b32 {%0, %1}, %2;" : "=h"(lo), "=h"(hi) : "r"(packed));
 }
 
-// A softmax weight w in [0, 1] as two fp16 numbers hi + lo ~ w * 2^14 (packed lo | hi << 16).
+// A softmax weight w in [0, 2] as two fp16 numbers hi + lo ~ w * 2^14 (packed lo | hi << 16).
 // The scaling keeps weights down to 2^-38 of the maximum representable; hi + lo carries
 // about 22 significant bits, the precision of the exponential itself.
 constexpr float kWeightScale = 16384.f;
+constexpr float kMaxLag = 1.f;          // weights <= 2, so weight * kWeightScale <= 32768 < 65504
 __device__ __forceinline__ unsigned split_weight(float w)
 {
     const float scaled = w * kWeightScale;
@@ -389,12 +390,16 @@ decode_attn_split_kernel(const AttnParams p)
         const int rows = j == my_tiles - 1 ? last_rows : kTileRows;
         if (row >= rows) s = -INFINITY;
 
-        // Online softmax with a warp-uniform running max.
-        float tile_max = s;
-        tile_max = fmaxf(tile_max, __shfl_xor_sync(0xffffffffu, tile_max, 1));
-        tile_max = fmaxf(tile_max, __shfl_xor_sync(0xffffffffu, tile_max, 2));
-        tile_max = fmaxf(tile_max, __shfl_xor_sync(0xffffffffu, tile_max, 4));
-        if (__any_sync(0xffffffffu, tile_max > m)) {     // rare once the maximum has settled
+        // Online softmax with a warp-uniform reference m that may lag the true maximum by up to
+        // kMaxLag (base-2 units): weights then reach at most 2^kMaxLag, which is harmless in
+        // fp32 and inside the range of the fp16 weight split.  The reference only moves (and
+        // the accumulators are only rescaled) when some logit exceeds it by more than that,
+        // so the common tile pays one vote instead of a shuffle reduction.
+        if (__any_sync(0xffffffffu, s > m + kMaxLag)) {
+            float tile_max = s;
+            tile_max = fmaxf(tile_max, __shfl_xor_sync(0xffffffffu, tile_max, 1));
+            tile_max = fmaxf(tile_max, __shfl_xor_sync(0xffffffffu, tile_max, 2));
+            tile_max = fmaxf(tile_max, __shfl_xor_sync(0xffffffffu, tile_max, 4));
             const float alpha = fast_exp2(m - tile_max);
             l *= alpha;
 #pragma unroll
