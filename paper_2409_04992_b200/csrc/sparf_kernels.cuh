@@ -211,6 +211,55 @@ struct SelectShared {
     int take_equal, bin, above, n_cand;
 };
 
+// Streams a score row as float4 with 4 loads in flight per thread; fn(first_index, values[4]).
+template <typename Fn>
+__device__ __forceinline__ void for_each_quad(const float4 *a4, int quads, Fn fn)
+{
+    for (int g0 = threadIdx.x; g0 < quads; g0 += 4 * kSelectThreads) {
+        float4 v[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int g = g0 + u * kSelectThreads;
+            v[u] = g < quads ? a4[g] : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int g = g0 + u * kSelectThreads;
+            if (g < quads) {
+                const float x[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+                fn(4 * g, x);
+            }
+        }
+    }
+}
+
+// Warp 0 finds, among 256 counters, the bucket (from the top) in which the running count
+// reaches `remaining`; returns it with the count of the buckets above through shared memory.
+__device__ __forceinline__ void locate_bucket(const unsigned *hist, int remaining, int *bucket_out, int *above_out)
+{
+    if (threadIdx.x < 32) {
+        const int lane = threadIdx.x;
+        int mine = 0;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) mine += (int)hist[8 * lane + j];
+        int above = 0;
+        for (int src = 31; src >= 0; --src) {
+            const int seg = __shfl_sync(0xffffffffu, mine, src);
+            if (src > lane) above += seg;
+        }
+        if (above < remaining && remaining <= above + mine) {
+            int bucket = 8 * lane + 7;
+            for (; bucket > 8 * lane; --bucket) {
+                const int c = (int)hist[bucket];
+                if (above + c >= remaining) break;
+                above += c;
+            }
+            *bucket_out = bucket;
+            *above_out = above;
+        }
+    }
+}
+
 // Exact k-th largest among the keys key_at(i) of the members i < n (member(i) true), 8 bits
 // per pass from the top.  Bytes on which all members agree are skipped without counting, so
 // a set of (nearly) equal keys costs nothing.  Returns through sh.tau / sh.take_equal the
@@ -264,13 +313,10 @@ __device__ __forceinline__ void exact_threshold(SelectShared &sh, int n, int nee
             }
         }
         __syncthreads();
-        int bucket = 255;
-        for (; bucket > 0; --bucket) {           // every thread walks the same 256 counters
-            const int c = (int)sh.hist[bucket];
-            if (c >= remaining) break;
-            remaining -= c;
-        }
-        prefix |= (unsigned)bucket << shift;
+        locate_bucket(sh.hist, remaining, &sh.bin, &sh.above);
+        __syncthreads();
+        prefix |= (unsigned)sh.bin << shift;
+        remaining -= sh.above;
     }
     __syncthreads();
     if (tid == 0) {
@@ -303,13 +349,22 @@ sparf_select_kernel(const SparfParams p)
     }
     const float *a = p.scores + (int64_t)pair * p.score_stride;
 
+    // The score row is 32-byte aligned and padded to a multiple of 8 floats (padding is
+    // readable scratch), so every pass streams it as float4 and masks the tail by index.
+    const float4 *a4 = reinterpret_cast<const float4 *>(a);
+    const int quads = (S + 3) / 4;
+
     // Pass 1: largest and smallest approximate logit (base-2 domain).
     float top = kMinusHuge, low = -kMinusHuge;
-    for (int i = tid; i < S; i += kSelectThreads) {
-        const float x = a[i];
-        top = fmaxf(top, x);
-        low = fminf(low, x);
-    }
+    for_each_quad(a4, quads, [&](int i0, const float (&x)[4]) {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            if (i0 + e < S) {
+                top = fmaxf(top, x[e]);
+                low = fminf(low, x[e]);
+            }
+        }
+    });
 #pragma unroll
     for (int off = 16; off >= 1; off >>= 1) {
         top = fmaxf(top, __shfl_xor_sync(0xffffffffu, top, off));
@@ -336,11 +391,15 @@ sparf_select_kernel(const SparfParams p)
 
     // Pass 2: histogram over the linear bins, and the softmax denominator.
     float z = 0.f;
-    for (int i = tid; i < S; i += kSelectThreads) {
-        const float x = a[i];
-        z += fast_exp2(x - top);
-        atomicAdd(&sh.hist[bin_of(i, x)], 1u);
-    }
+    for_each_quad(a4, quads, [&](int i0, const float (&x)[4]) {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            if (i0 + e < S) {
+                z += fast_exp2(x[e] - top);
+                atomicAdd(&sh.hist[bin_of(i0 + e, x[e])], 1u);
+            }
+        }
+    });
     z = block_sum(z, sh.red_f);                  // its barriers also publish the histogram
 
     // The bin that holds the k-th largest: warp 0, lane L owns bins [64 L, 64 L + 64).
@@ -382,13 +441,34 @@ sparf_select_kernel(const SparfParams p)
         }
         __syncthreads();
     } else if (in_bin <= kCandidates) {
-        for (int i = tid; i < S; i += kSelectThreads) {
-            const float x = a[i];
-            if (bin_of(i, x) == bin) sh.cand[atomicAdd(&sh.n_cand, 1)] = ordered_key(x);
-        }
+        for_each_quad(a4, quads, [&](int i0, const float (&x)[4]) {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                if (i0 + e < S && bin_of(i0 + e, x[e]) == bin)
+                    sh.cand[atomicAdd(&sh.n_cand, 1)] = ordered_key(x[e]);
+            }
+        });
         __syncthreads();
-        exact_threshold(sh, in_bin, k - above, [](int) { return true; },
-                        [&](int i) { return sh.cand[i]; });
+        if (in_bin <= kSelectThreads) {          // the usual case: rank every candidate directly
+            const int need = k - above;
+            if (tid < in_bin) {
+                const unsigned mine = sh.cand[tid];
+                int greater = 0, equal = 0;
+                for (int j = 0; j < in_bin; ++j) {
+                    const unsigned other = sh.cand[j];
+                    greater += other > mine;
+                    equal += other == mine;
+                }
+                if (greater < need && need <= greater + equal) {     // all holders of this key agree
+                    sh.tau = mine;
+                    sh.take_equal = need - greater;
+                }
+            }
+            __syncthreads();
+        } else {
+            exact_threshold(sh, in_bin, k - above, [](int) { return true; },
+                            [&](int i) { return sh.cand[i]; });
+        }
     } else {                                     // very many near-equal logits: work from global memory
         exact_threshold(sh, S, k - above, [&](int i) { return bin_of(i, a[i]) == bin; },
                         [&](int i) { return ordered_key(a[i]); });
@@ -401,49 +481,64 @@ sparf_select_kernel(const SparfParams p)
     const int32_t *table_row = p.block_table + (int64_t)b * p.max_blocks_per_seq;
     int base_gt = 0, base_eq = 0;
     float mass = 0.f;
-    for (int start = 0; start < S; start += kSelectThreads) {
-        const int i = start + tid;
-        bool gt = false, eq = false;
-        float x = 0.f;
-        if (i < S) {
-            x = a[i];
-            const unsigned key = key_of(i, x);
-            gt = key > tau;
-            eq = key == tau;
-        }
-        const unsigned bal_gt = __ballot_sync(0xffffffffu, gt), bal_eq = __ballot_sync(0xffffffffu, eq);
-        if (lane == 0) {
-            sh.scan_gt[warp] = __popc(bal_gt);
-            sh.scan_eq[warp] = __popc(bal_eq);
-        }
-        __syncthreads();
-        // every warp scans the 32 per-warp counts with shuffles
-        const int cg = sh.scan_gt[lane], ce = sh.scan_eq[lane];
-        int ig = cg, ie = ce;
+    // Each thread takes 4 consecutive positions; counts travel packed (greater | equal << 16).
+    float4 ahead = tid < quads ? a4[tid] : make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int start = 0; start < quads; start += kSelectThreads) {
+        const int g = start + tid;
+        const float4 v = ahead;
+        if (g + kSelectThreads < quads) ahead = a4[g + kSelectThreads];    // next tile's loads fly over the barriers
+        float x[4] = {0.f, 0.f, 0.f, 0.f};
+        bool gt[4] = {false, false, false, false}, eq[4] = {false, false, false, false};
+        int mine = 0;
+        if (g < quads) {
+            x[0] = v.x; x[1] = v.y; x[2] = v.z; x[3] = v.w;
 #pragma unroll
-        for (int off = 1; off < 32; off <<= 1) {
-            const int ug = __shfl_up_sync(0xffffffffu, ig, off), ue = __shfl_up_sync(0xffffffffu, ie, off);
-            if (lane >= off) {
-                ig += ug;
-                ie += ue;
+            for (int e = 0; e < 4; ++e) {
+                const int i = 4 * g + e;
+                if (i < S) {
+                    const unsigned key = key_of(i, x[e]);
+                    gt[e] = key > tau;
+                    eq[e] = key == tau;
+                    mine += (int)gt[e] + ((int)eq[e] << 16);
+                }
             }
         }
-        const int gt_tile = __shfl_sync(0xffffffffu, ig, 31), eq_tile = __shfl_sync(0xffffffffu, ie, 31);
-        const int below = (1u << lane) - 1u;
-        const int gt_before = base_gt + __shfl_sync(0xffffffffu, ig - cg, warp) + __popc(bal_gt & below);
-        const int eq_before = base_eq + __shfl_sync(0xffffffffu, ie - ce, warp) + __popc(bal_eq & below);
-        if (gt || (eq && eq_before < take_equal)) {
-            const int pos = gt_before + min(eq_before, take_equal);
-            const int blk = i / T, slot = i - blk * T;
-            const int phys = table_row[blk];
-            const bool ok = phys >= 0 && (int64_t)phys < p.num_phys_blocks;
-            if (!ok && p.status) atomicOr(p.status, kFlagBlockRange);
-            rows[pos] = ok ? (phys * p.heads + h) * T + slot : 0;
-            if (sel) sel[pos] = i;
-            mass += fast_exp2(x - top);
+        int incl = mine;                          // inclusive scan over the warp
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const int up = __shfl_up_sync(0xffffffffu, incl, off);
+            if (lane >= off) incl += up;
         }
-        base_gt += gt_tile;
-        base_eq += eq_tile;
+        if (lane == 31) sh.scan_gt[warp] = incl;
+        __syncthreads();
+        const int warp_total = sh.scan_gt[lane];  // every warp scans the 32 warp totals
+        int warp_incl = warp_total;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const int up = __shfl_up_sync(0xffffffffu, warp_incl, off);
+            if (lane >= off) warp_incl += up;
+        }
+        const int tile_total = __shfl_sync(0xffffffffu, warp_incl, 31);
+        const int before = __shfl_sync(0xffffffffu, warp_incl - warp_total, warp) + incl - mine;
+        int gt_before = base_gt + (before & 0xffff), eq_before = base_eq + (before >> 16);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            if (gt[e] || (eq[e] && eq_before < take_equal)) {
+                const int i = 4 * g + e;
+                const int pos = gt_before + min(eq_before, take_equal);
+                const int blk = i / T, slot = i - blk * T;
+                const int phys = table_row[blk];
+                const bool ok = phys >= 0 && (int64_t)phys < p.num_phys_blocks;
+                if (!ok && p.status) atomicOr(p.status, kFlagBlockRange);
+                rows[pos] = ok ? (phys * p.heads + h) * T + slot : 0;
+                if (sel) sel[pos] = i;
+                mass += fast_exp2(x[e] - top);
+            }
+            gt_before += (int)gt[e];
+            eq_before += (int)eq[e];
+        }
+        base_gt += tile_total & 0xffff;
+        base_eq += tile_total >> 16;
         __syncthreads();
     }
     mass = block_sum(mass, sh.red_f);
