@@ -29,6 +29,9 @@ def _load() -> ctypes.CDLL:
         lib.oracle_decode_attention.argtypes = [ptr, ptr, ptr, i64, ptr, ptr, ptr, ptr, ptr,
                                                 i32, i32, i64, i32, i32, i32, i32,
                                                 ctypes.c_float]
+        lib.oracle_kv_append_bulk.restype = ctypes.c_int
+        lib.oracle_kv_append_bulk.argtypes = [ptr, ptr, ptr, ptr, ptr, ptr, ptr, i32, i32, i64,
+                                              i32, i32, i32, i32, i32]
         lib.oracle_sparf_append.restype = ctypes.c_int
         lib.oracle_sparf_append.argtypes = [ptr, ptr, ptr, ptr, ptr, ptr, ptr, ptr, i32, i32, i64,
                                             i32, i32, i32]
@@ -95,6 +98,27 @@ def kv_append(k_cache: np.ndarray, v_cache: np.ndarray, k_new: np.ndarray, v_new
         s_max, block_tokens, phys = 0, kb.shape[2], kb.shape[0]
     rc = _load().oracle_kv_append(_p(kb), _p(vb), _p(kn), _p(vn), _p(lens), _p(table),
                                   max_blocks, block_tokens, phys, batch, heads, head_dim, s_max)
+    if rc:
+        raise OracleError(rc)
+
+
+def kv_append_bulk(k_cache: np.ndarray, v_cache: np.ndarray, k_new: np.ndarray, v_new: np.ndarray,
+                   seq_lens: np.ndarray, new_lens: np.ndarray,
+                   block_table: Optional[np.ndarray] = None) -> None:
+    """In-place append of new_lens[b] tokens per sequence; k_new, v_new are [B,N,H,D]."""
+    kb, vb = _bits(k_cache, True), _bits(v_cache, True)
+    kn, vn = _bits(np.ascontiguousarray(k_new)), _bits(np.ascontiguousarray(v_new))
+    batch, max_new, heads, head_dim = kn.shape
+    lens = np.ascontiguousarray(seq_lens, dtype=np.int32)
+    news = np.ascontiguousarray(new_lens, dtype=np.int32)
+    table, max_blocks = _table(block_table, batch)
+    if table is None:
+        s_max, block_tokens, phys = kb.shape[2], 0, 0
+    else:
+        s_max, block_tokens, phys = 0, kb.shape[2], kb.shape[0]
+    rc = _load().oracle_kv_append_bulk(_p(kb), _p(vb), _p(kn), _p(vn), _p(lens), _p(news), _p(table),
+                                       max_blocks, block_tokens, phys, batch, max_new, heads,
+                                       head_dim, s_max)
     if rc:
         raise OracleError(rc)
 

@@ -139,6 +139,42 @@ int oracle_kv_append(uint16_t *k_cache, uint16_t *v_cache,
 }
 
 /*
+ * Bulk append (Sec. IV-D: in the prefill phase the K,V of all prompt tokens of a layer are
+ * produced at once and handed to the cache layer by layer).  Sequence b receives
+ * new_lens[b] tokens, taken from k_new / v_new [batch][max_new][heads][head_dim] (token-major,
+ * as a projection produces them), at logical positions seq_lens[b]-new_lens[b] ..
+ * seq_lens[b]-1.  Bit copy.
+ */
+int oracle_kv_append_bulk(uint16_t *k_cache, uint16_t *v_cache,
+                          const uint16_t *k_new, const uint16_t *v_new,
+                          const int32_t *seq_lens, const int32_t *new_lens,
+                          const int32_t *block_table, int32_t max_blocks_per_seq,
+                          int32_t block_tokens, int64_t num_phys_blocks,
+                          int32_t batch, int32_t max_new, int32_t heads, int32_t head_dim,
+                          int32_t s_max)
+{
+    const cache_geometry g = {block_table, max_blocks_per_seq, block_tokens,
+                              num_phys_blocks, heads, head_dim, s_max};
+    int rc = check_geometry(&g, batch);
+    if (rc) return rc;
+    if (max_new < 0) return -1;
+    for (int32_t b = 0; b < batch; ++b) {
+        const int32_t L = seq_lens[b], n = new_lens[b];
+        if (L < 0 || (int64_t)L > capacity_tokens(&g) || n < 0 || n > max_new || n > L) return -2;
+        for (int32_t t = 0; t < n; ++t) {
+            for (int32_t h = 0; h < heads; ++h) {
+                const int64_t dst = row_offset(&g, b, h, L - n + t);
+                if (dst < 0) return -3;
+                const int64_t src = ((((int64_t)b * max_new + t) * heads) + h) * head_dim;
+                memcpy(k_cache + dst, k_new + src, sizeof(uint16_t) * (size_t)head_dim);
+                memcpy(v_cache + dst, v_new + src, sizeof(uint16_t) * (size_t)head_dim);
+            }
+        }
+    }
+    return 0;
+}
+
+/*
  * One (sequence, head): the definition of Sec. II-A with a single query row.
  *   s_i = scale * sum_d q[d] K[i][d]          ("Logit", Sec. III-B)
  *   w_i = exp(s_i - max_j s_j) / sum_j exp(s_j - max_j s_j)
