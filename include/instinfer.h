@@ -82,6 +82,23 @@ int instinfer_kv_append(void *k_cache, void *v_cache,
                         int32_t *status_flags, void *cuda_stream);
 
 /*
+ * Bulk append (the prefill phase hands a layer's K,V of all prompt tokens to the cache at
+ * once, Sec. IV-D).  Sequence b receives new_lens[b] tokens (0 <= new_lens[b] <= max_new,
+ * new_lens[b] <= seq_lens[b]) from k_new / v_new, fp16 [batch, max_new, heads, head_dim]
+ * (token-major, as a projection produces them), at logical positions
+ * seq_lens[b]-new_lens[b] .. seq_lens[b]-1; seq_lens are the lengths AFTER the append.
+ * Layout selection and the other arguments as in instinfer_kv_append.  A sequence whose
+ * lengths are out of range is skipped and flagged.
+ */
+int instinfer_kv_append_bulk(void *k_cache, void *v_cache,
+                             const void *k_new, const void *v_new,
+                             const int32_t *seq_lens, const int32_t *new_lens,
+                             const int32_t *block_table, int32_t max_blocks_per_seq,
+                             int32_t block_tokens, int64_t num_phys_blocks,
+                             int32_t batch, int32_t max_new, int32_t heads, int32_t head_dim,
+                             int32_t s_max, int32_t *status_flags, void *cuda_stream);
+
+/*
  * Decode attention over a contiguous cache (Sec. II-A definition, Sec. II-B/III-B decode
  * form): out[b][h][:] = softmax_i(scale * q[b][h].K[b][h][i]) . V[b][h][i], i < seq_lens[b].
  *   out          fp16 [batch, heads, head_dim]; fp32 accumulation, rounded once (nearest even)

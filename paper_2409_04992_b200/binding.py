@@ -40,6 +40,9 @@ def load() -> ctypes.CDLL:
         lib.instinfer_kv_append.restype = ctypes.c_int
         lib.instinfer_kv_append.argtypes = [ptr, ptr, ptr, ptr, ptr, ptr, i32, i32, i64,
                                             i32, i32, i32, i32, ptr, ptr]
+        lib.instinfer_kv_append_bulk.restype = ctypes.c_int
+        lib.instinfer_kv_append_bulk.argtypes = [ptr, ptr, ptr, ptr, ptr, ptr, ptr, i32, i32, i64,
+                                                 i32, i32, i32, i32, i32, ptr, ptr]
         lib.instinfer_decode_attention.restype = ctypes.c_int
         lib.instinfer_decode_attention.argtypes = [ptr, ptr, ptr, ptr, ptr, ptr, i32, i32, i32,
                                                    i32, i32, f32, ptr, sz, ptr, ptr]
@@ -133,6 +136,24 @@ def kv_append(k_cache: torch.Tensor, v_cache: torch.Tensor, k_new: torch.Tensor,
     _check(load().instinfer_kv_append(
         _ptr(k_cache), _ptr(v_cache), _ptr(k_new), _ptr(v_new), _ptr(seq_lens),
         _ptr(block_table), max_blocks, block_tokens, phys, batch, heads, head_dim, s_max,
+        _ptr(status_flags), _stream(stream)))
+
+
+def kv_append_bulk(k_cache: torch.Tensor, v_cache: torch.Tensor, k_new: torch.Tensor,
+                   v_new: torch.Tensor, seq_lens: torch.Tensor, new_lens: torch.Tensor,
+                   block_table: Optional[torch.Tensor] = None,
+                   status_flags: Optional[torch.Tensor] = None,
+                   stream: Optional[torch.cuda.Stream] = None) -> None:
+    """instinfer_kv_append_bulk: k_new, v_new are [B, max_new, H, D] (token-major)."""
+    batch, max_new, heads, head_dim = k_new.shape
+    if block_table is None:
+        max_blocks, block_tokens, phys, s_max = 0, 0, 0, k_cache.shape[2]
+    else:
+        max_blocks, block_tokens, phys, s_max = (block_table.shape[1], k_cache.shape[2],
+                                                 k_cache.shape[0], 0)
+    _check(load().instinfer_kv_append_bulk(
+        _ptr(k_cache), _ptr(v_cache), _ptr(k_new), _ptr(v_new), _ptr(seq_lens), _ptr(new_lens),
+        _ptr(block_table), max_blocks, block_tokens, phys, batch, max_new, heads, head_dim, s_max,
         _ptr(status_flags), _stream(stream)))
 
 

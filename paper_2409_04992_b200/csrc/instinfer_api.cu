@@ -231,6 +231,52 @@ int instinfer_kv_append(void *k_cache, void *v_cache, const void *k_new, const v
     return cudaGetLastError() == cudaSuccess ? INSTINFER_OK : INSTINFER_ERR_CUDA;
 }
 
+int instinfer_kv_append_bulk(void *k_cache, void *v_cache, const void *k_new, const void *v_new,
+                             const int32_t *seq_lens, const int32_t *new_lens,
+                             const int32_t *block_table, int32_t max_blocks_per_seq,
+                             int32_t block_tokens, int64_t num_phys_blocks, int32_t batch,
+                             int32_t max_new, int32_t heads, int32_t head_dim, int32_t s_max,
+                             int32_t *status_flags, void *cuda_stream)
+{
+    if (batch < 0 || heads <= 0 || head_dim <= 0 || max_new < 0) return INSTINFER_ERR_INVALID_ARG;
+    if (head_dim != kHeadDim) return INSTINFER_ERR_UNSUPPORTED;
+    if ((int64_t)batch * heads > (int64_t)1 << 24) return INSTINFER_ERR_INVALID_ARG;
+    if (block_table != nullptr) {
+        if (max_blocks_per_seq <= 0 || block_tokens <= 0 || num_phys_blocks <= 0)
+            return INSTINFER_ERR_INVALID_ARG;
+        if (block_tokens % 8 != 0) return INSTINFER_ERR_UNSUPPORTED;
+    } else if (s_max <= 0) {
+        return INSTINFER_ERR_INVALID_ARG;
+    }
+    if (batch == 0 || max_new == 0) return INSTINFER_OK;
+    if (!usable(k_cache) || !usable(v_cache) || !usable(k_new) || !usable(v_new) ||
+        seq_lens == nullptr || new_lens == nullptr)
+        return INSTINFER_ERR_INVALID_ARG;
+    const int64_t threads = (int64_t)batch * max_new * heads * kSegsPerRow;
+    const int64_t grid = ceil_div(threads, kAppendThreads);
+    if (grid >= (int64_t)1 << 31) return INSTINFER_ERR_INVALID_ARG;
+
+    BulkAppendParams q = {};
+    AppendParams &p = q.base;
+    p.k_cache = static_cast<uint4 *>(k_cache);
+    p.v_cache = static_cast<uint4 *>(v_cache);
+    p.k_new = static_cast<const uint4 *>(k_new);
+    p.v_new = static_cast<const uint4 *>(v_new);
+    p.seq_lens = seq_lens;
+    p.block_table = block_table;
+    p.status = status_flags;
+    p.num_phys_blocks = num_phys_blocks;
+    p.batch = batch;
+    p.heads = heads;
+    p.s_max = s_max;
+    p.block_tokens = block_tokens;
+    p.max_blocks_per_seq = max_blocks_per_seq;
+    q.new_lens = new_lens;
+    q.max_new = max_new;
+    kv_append_bulk_kernel<<<(unsigned)grid, kAppendThreads, 0, static_cast<cudaStream_t>(cuda_stream)>>>(q);
+    return cudaGetLastError() == cudaSuccess ? INSTINFER_OK : INSTINFER_ERR_CUDA;
+}
+
 int instinfer_decode_attention(void *out, float *lse, const void *q, const void *k_cache,
                                const void *v_cache, const int32_t *seq_lens, int32_t batch,
                                int32_t heads, int32_t head_dim, int32_t s_max,

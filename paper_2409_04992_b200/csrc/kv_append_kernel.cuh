@@ -61,4 +61,51 @@ kv_append_kernel(const AppendParams p)
     p.v_cache[row * kSegsPerRow + seg] = p.v_new[idx];
 }
 
+// Bulk append (prefill, Sec. IV-D): new_lens[b] tokens per sequence from token-major
+// k_new / v_new [batch, max_new, heads, 128] into positions seq_lens[b]-new_lens[b] ... of the
+// cache.  One thread per 16-byte segment; reads are fully contiguous, each written row is a
+// contiguous 256 bytes.
+struct BulkAppendParams {
+    AppendParams base;            // k_new / v_new point at [batch, max_new, heads, 128]
+    const int32_t *new_lens;
+    int32_t max_new;
+};
+
+__global__ void __launch_bounds__(kAppendThreads)
+kv_append_bulk_kernel(const BulkAppendParams q)
+{
+    const AppendParams &p = q.base;
+    const int64_t idx = (int64_t)blockIdx.x * kAppendThreads + threadIdx.x;
+    const int64_t row = idx / kSegsPerRow;                    // (b, t, h)
+    if (row >= (int64_t)p.batch * q.max_new * p.heads) return;
+    const int seg = (int)(idx % kSegsPerRow);
+    const int h = (int)(row % p.heads);
+    const int64_t bt = row / p.heads;
+    const int t = (int)(bt % q.max_new), b = (int)(bt / q.max_new);
+    const bool reporter = seg == 0 && h == 0 && t == 0 && p.status != nullptr;
+
+    const int len = p.seq_lens[b], fresh = q.new_lens[b];
+    const int64_t capacity = p.block_table ? (int64_t)p.max_blocks_per_seq * p.block_tokens
+                                           : (int64_t)p.s_max;
+    if (len < 0 || len > capacity || fresh < 0 || fresh > q.max_new || fresh > len) {
+        if (reporter) atomicOr(p.status, 1);                // lengths out of range: sequence skipped
+        return;
+    }
+    if (t >= fresh) return;
+    const int pos = len - fresh + t;
+    int64_t dst;
+    if (p.block_table) {
+        const int phys = p.block_table[(int64_t)b * p.max_blocks_per_seq + pos / p.block_tokens];
+        if (phys < 0 || (int64_t)phys >= p.num_phys_blocks) {
+            if (seg == 0 && h == 0 && p.status) atomicOr(p.status, 2);
+            return;
+        }
+        dst = ((int64_t)phys * p.heads + h) * p.block_tokens + pos % p.block_tokens;
+    } else {
+        dst = ((int64_t)b * p.heads + h) * p.s_max + pos;
+    }
+    p.k_cache[dst * kSegsPerRow + seg] = p.k_new[idx];
+    p.v_cache[dst * kSegsPerRow + seg] = p.v_new[idx];
+}
+
 }  // namespace instinfer
