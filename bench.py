@@ -543,6 +543,38 @@ def measure_sparse(w: wl.Workload, device, steps: int, r: int = 16, keep: float 
             "status_flags": int(flags.item())}
 
 
+def measure_bulk_append(device, steps: int = 10, batch: int = 16, new_tokens: int = 4096) -> dict:
+    """Prefill-style append of `new_tokens` tokens per sequence into a paged cache (T=32):
+    bytes read plus bytes written per second, comparable with a device-to-device copy."""
+    from paper_2409_04992_b200 import binding
+    w = wl.STANDARD[4].replace(batch=batch, len_lo=new_tokens, len_hi=new_tokens, layers=1)
+    case = wl.generate(w, device=str(device), poison=False)
+    gen = torch.Generator(device=device)
+    gen.manual_seed(wl.BASE_SEED + 77)
+    fresh = [torch.randn((batch, new_tokens, w.heads, w.head_dim), dtype=torch.float32, device=device,
+                         generator=gen).to(torch.float16) for _ in range(2)]
+    new_lens = torch.full((batch,), new_tokens, dtype=torch.int32, device=device)
+    flags = torch.zeros(1, dtype=torch.int32, device=device)
+
+    def step():
+        binding.kv_append_bulk(case.k_cache, case.v_cache, fresh[0], fresh[1], case.seq_lens, new_lens,
+                               case.block_table, flags)
+
+    for _ in range(3):
+        step()
+    a, z = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    a.record()
+    for _ in range(steps):
+        step()
+    z.record()
+    torch.cuda.synchronize()
+    seconds = a.elapsed_time(z) / 1e3 / steps
+    moved = 2 * 2 * fresh[0].numel() * 2                      # K and V, read and written, fp16
+    return {"tokens_per_sequence": new_tokens, "batch": batch, "ms_per_step": seconds * 1e3,
+            "read_plus_write_gbs": moved / seconds / 1e9, "status_flags": int(flags.item())}
+
+
 def main(argv=None) -> int:
     args = parse_args(argv)
     if args.impl == "reference":          # CPU only: no process group; ranks other than 0 do nothing
@@ -613,6 +645,7 @@ def main(argv=None) -> int:
                     "chunk_tokens": r["chunk_tokens"], "sm_mhz": r["clocks"]["sm_mhz"],
                     "reasons": r["clocks"]["reasons"]}
             line["other_workloads"] = others
+            line["bulk_append"] = measure_bulk_append(device)
             line["sparse_attention"] = {wl.STANDARD[i].name: measure_sparse(wl.STANDARD[i], device, 10)
                                         for i in (2, 3)}
         if ranks.rank == 0:
