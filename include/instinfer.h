@@ -40,6 +40,10 @@
  *   [0, num_phys_blocks) is not dereferenced: the append skips that sequence, attention
  *   reads that block's rows as zeros (the sequence's output is then meaningless but finite).
  *   No kernel traps, asserts or waits on another kernel.
+ * - Stream order is kept: each kernel sees everything enqueued before it on the stream as
+ *   complete.  Internally the launches use programmatic dependent launch, so a kernel's
+ *   blocks may already be resident while the previous kernel drains; they touch no memory
+ *   before that kernel has completed.
  * - batch == 0 is a valid empty call: INSTINFER_OK, nothing enqueued.
  */
 #ifndef INSTINFER_H_

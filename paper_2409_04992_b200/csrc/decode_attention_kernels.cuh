@@ -76,6 +76,12 @@ struct AttnParams {
 // Where a (sequence, head)'s rows come from.
 enum class Rows { kContiguous, kPaged, kGathered };
 
+// Programmatic dependent launch: a kernel first lets the next kernel in the stream start
+// being scheduled, then waits until the kernels before it have completed and their writes
+// are visible.  Both are no-ops for a launch without the attribute.
+__device__ __forceinline__ void allow_next_kernel() { asm volatile("griddepcontrol.launch_dependents;"); }
+__device__ __forceinline__ void wait_for_previous_kernels() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 __device__ __forceinline__ float fast_exp2(float x)
 {
     float y;
@@ -196,6 +202,8 @@ decode_attn_split_kernel(const AttnParams p)
     const int pair = blockIdx.x - split * p.pairs;
     const int b = pair / p.heads, h = pair - b * p.heads;
     const bool final_writer = !kGathered && p.n_splits == 1;
+    allow_next_kernel();
+    wait_for_previous_kernels();
 
     // With several splits the merge kernel reports a bad length; here only the lone writer does.
     int len = checked_seq_len(p, b, threadIdx.x == 0 && h == 0 && final_writer);
@@ -480,6 +488,8 @@ lse_merge_kernel(const AttnParams p)
 {
     const int pair = blockIdx.x;
     const int b = pair / p.heads;
+    allow_next_kernel();
+    wait_for_previous_kernels();
     const int len = checked_seq_len(p, b, threadIdx.x == 0 && pair == b * p.heads);
     const int live = live_chunks(p, len);
     if (live == 0) {

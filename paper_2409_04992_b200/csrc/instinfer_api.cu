@@ -50,6 +50,32 @@ int sm_count()
     return cached[dev];
 }
 
+// Launch with programmatic stream serialization: the kernel may be scheduled while the
+// previous kernel in the stream drains; it orders itself with griddepcontrol.wait.  Falls
+// back to an ordinary launch if the runtime refuses the attribute.
+template <typename Params>
+cudaError_t launch_overlapped(void (*kernel)(Params), unsigned grid, unsigned block, size_t smem,
+                              cudaStream_t stream, const Params &params)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(block);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t err = cudaLaunchKernelEx(&cfg, kernel, params);
+    if (err != cudaSuccess) {
+        (void)cudaGetLastError();
+        cfg.numAttrs = 0;
+        err = cudaLaunchKernelEx(&cfg, kernel, params);
+    }
+    return err;
+}
+
 struct SplitPlan {
     int32_t chunk_tokens;   // size of the first n_big chunks
     int32_t n_big;
@@ -147,15 +173,17 @@ int launch_attention(AttnParams p, bool paged, int32_t batch, void *workspace,
     if (rc != INSTINFER_OK) return rc;
     const unsigned grid = (unsigned)(pairs * plan.n_splits);
     if (g_before_split) cudaEventRecord(g_before_split, stream);
+    const bool timed = g_before_split != nullptr;          // event records break the overlap anyway
+    cudaError_t err;
     if (paged)
-        decode_attn_split_kernel<Rows::kPaged><<<grid, kThreads, kSplitSmemBytes, stream>>>(p);
+        err = launch_overlapped(decode_attn_split_kernel<Rows::kPaged>, grid, kThreads, kSplitSmemBytes, stream, p);
     else
-        decode_attn_split_kernel<Rows::kContiguous><<<grid, kThreads, kSplitSmemBytes, stream>>>(p);
-    if (g_after_split) cudaEventRecord(g_after_split, stream);
-    if (cudaGetLastError() != cudaSuccess) return INSTINFER_ERR_CUDA;
+        err = launch_overlapped(decode_attn_split_kernel<Rows::kContiguous>, grid, kThreads, kSplitSmemBytes, stream, p);
+    if (timed) cudaEventRecord(g_after_split, stream);
+    if (err != cudaSuccess || cudaGetLastError() != cudaSuccess) return INSTINFER_ERR_CUDA;
     if (plan.n_splits > 1) {
-        lse_merge_kernel<<<(unsigned)pairs, kHeadDim, 0, stream>>>(p);
-        if (cudaGetLastError() != cudaSuccess) return INSTINFER_ERR_CUDA;
+        err = launch_overlapped(lse_merge_kernel, (unsigned)pairs, kHeadDim, 0, stream, p);
+        if (err != cudaSuccess || cudaGetLastError() != cudaSuccess) return INSTINFER_ERR_CUDA;
     }
     return INSTINFER_OK;
 }
@@ -227,8 +255,9 @@ int instinfer_kv_append(void *k_cache, void *v_cache, const void *k_new, const v
     p.max_blocks_per_seq = max_blocks_per_seq;
     const int64_t threads = (int64_t)batch * heads * kSegsPerRow;
     const unsigned grid = (unsigned)ceil_div(threads, kAppendThreads);
-    kv_append_kernel<<<grid, kAppendThreads, 0, static_cast<cudaStream_t>(cuda_stream)>>>(p);
-    return cudaGetLastError() == cudaSuccess ? INSTINFER_OK : INSTINFER_ERR_CUDA;
+    const cudaError_t err = launch_overlapped(kv_append_kernel, grid, kAppendThreads, 0,
+                                              static_cast<cudaStream_t>(cuda_stream), p);
+    return err == cudaSuccess && cudaGetLastError() == cudaSuccess ? INSTINFER_OK : INSTINFER_ERR_CUDA;
 }
 
 int instinfer_kv_append_bulk(void *k_cache, void *v_cache, const void *k_new, const void *v_new,

@@ -36,6 +36,8 @@ kv_append_kernel(const AppendParams p)
     const int seg = (int)(idx % kSegsPerRow);
     const int b = (int)(pair / p.heads), h = (int)(pair % p.heads);
     const bool reporter = seg == 0 && h == 0 && p.status != nullptr;
+    asm volatile("griddepcontrol.launch_dependents;");      // the next kernel may start being scheduled
+    asm volatile("griddepcontrol.wait;" ::: "memory");      // earlier kernels' writes are visible from here
 
     const int len = p.seq_lens[b];
     if (len == 0) return;                                   // inactive slot
