@@ -30,14 +30,14 @@ constexpr int kRowBytes = kHeadDim * 2;            // one token's K (or V) row o
 constexpr int kWarps = 4;
 constexpr int kThreads = kWarps * 32;
 constexpr int kTileRows = 8;                       // tokens per warp tile
-constexpr int kStages = 4;                         // ring depth per warp
+constexpr int kStages = 3;                         // ring depth per warp
 constexpr int kKRowStride = kRowBytes + 16;        // K rows padded in shared memory: 4 lanes per
                                                    // row read 8 rows at once without bank conflicts
 constexpr int kKTileBytes = kTileRows * kKRowStride;
 constexpr int kVTileBytes = kTileRows * kRowBytes;
 constexpr int kStageBytes = kKTileBytes + kVTileBytes;
-constexpr int kSplitSmemBytes = kWarps * kStages * kStageBytes;   // 66 KiB
-constexpr int kCtasPerSm = 3;
+constexpr int kSplitSmemBytes = kWarps * kStages * kStageBytes;   // 49.5 KiB
+constexpr int kCtasPerSm = 4;
 constexpr float kMinusHuge = -1.0e30f;             // finite stand-in for "no row seen yet"
 constexpr float kLn2 = 0.69314718055994530942f;
 
