@@ -407,7 +407,7 @@ int instinfer_decode_attention_static(void *out, float *lse, const void *q, cons
 namespace {
 
 struct SparfLayout {
-    size_t scores, row_ids, stats, chunk_range, partials, total;
+    size_t scores, row_ids, stats, partials, total;
     int32_t score_stride;
     SplitPlan plan;
 };
@@ -422,8 +422,7 @@ SparfLayout sparf_layout(int64_t pairs, int32_t max_seq_len, int32_t max_k)
     w.scores = 0;
     w.row_ids = w.scores + round256((size_t)pairs * w.score_stride * sizeof(float));
     w.stats = w.row_ids + round256((size_t)pairs * max_k * sizeof(int32_t));
-    w.chunk_range = w.stats + round256((size_t)pairs * sizeof(float2));
-    w.partials = w.chunk_range + round256((size_t)pairs * ceil_div(max_seq_len, kScoreChunk) * sizeof(float2));
+    w.partials = w.stats + round256((size_t)pairs * sizeof(float2));
     w.total = w.partials + workspace_for(pairs, w.plan);
     return w;
 }
@@ -528,7 +527,6 @@ int instinfer_sparf_decode_attention(void *out, float *alpha, int32_t *selected,
     sp.scores = reinterpret_cast<float *>(ws + w.scores);
     sp.row_ids = reinterpret_cast<int32_t *>(ws + w.row_ids);
     sp.stats = reinterpret_cast<float2 *>(ws + w.stats);
-    sp.chunk_range = reinterpret_cast<float2 *>(ws + w.chunk_range);
     sp.alpha_out = alpha;
     sp.selected = selected;
     sp.num_phys_blocks = num_phys_blocks;

@@ -41,7 +41,6 @@ struct SparfParams {
     float *scores;             // [pairs, score_stride] approximate logits, base-2 domain
     int32_t *row_ids;          // [pairs, max_k]
     float2 *stats;             // [pairs] (alpha, number of selected rows)
-    float2 *chunk_range;       // [pairs, score_chunks] (min, max) logit of each score chunk
     // outputs
     float *alpha_out;          // nullable [pairs]
     int32_t *selected;         // nullable [pairs, max_k] logical token index, ascending, -1 padded
@@ -144,7 +143,6 @@ sparf_scores_kernel(const SparfParams p)
     const int T = p.block_tokens;
     const int32_t *table_row = p.block_table + (int64_t)b * p.max_blocks_per_seq;
     float *dst = p.scores + (int64_t)pair * p.score_stride;
-    float lowest = -kMinusHuge, highest = kMinusHuge;
     for (int i = begin + d * 8; i < end; i += kSparfThreads * 8) {
         const int blk = i / T, slot = i - blk * T;
         const int phys = table_row[blk];
@@ -174,34 +172,9 @@ sparf_scores_kernel(const SparfParams p)
         }
         // score_stride is a multiple of 8 and rows start 32-byte aligned; entries past `end`
         // inside the last group are scratch nobody reads.
-#pragma unroll
-        for (int e = 0; e < 8; ++e) {
-            dot[e] *= approx_scale;
-            if (i + e < end) {
-                lowest = fminf(lowest, dot[e]);
-                highest = fmaxf(highest, dot[e]);
-            }
-        }
         float4 *out4 = reinterpret_cast<float4 *>(dst + i);
-        out4[0] = make_float4(dot[0], dot[1], dot[2], dot[3]);
-        out4[1] = make_float4(dot[4], dot[5], dot[6], dot[7]);
-    }
-    // (min, max) of this chunk for the select kernel
-#pragma unroll
-    for (int off = 16; off >= 1; off >>= 1) {
-        lowest = fminf(lowest, __shfl_xor_sync(0xffffffffu, lowest, off));
-        highest = fmaxf(highest, __shfl_xor_sync(0xffffffffu, highest, off));
-    }
-    __syncthreads();
-    if ((d & 31) == 0) {
-        sm_red[0][d >> 5] = lowest;
-        sm_red[1][d >> 5] = highest;
-    }
-    __syncthreads();
-    if (d == 0) {
-        p.chunk_range[blockIdx.x] = make_float2(
-            fminf(fminf(sm_red[0][0], sm_red[0][1]), fminf(sm_red[0][2], sm_red[0][3])),
-            fmaxf(fmaxf(sm_red[1][0], sm_red[1][1]), fmaxf(sm_red[1][2], sm_red[1][3])));
+        out4[0] = make_float4(dot[0] * approx_scale, dot[1] * approx_scale, dot[2] * approx_scale, dot[3] * approx_scale);
+        out4[1] = make_float4(dot[4] * approx_scale, dot[5] * approx_scale, dot[6] * approx_scale, dot[7] * approx_scale);
     }
 }
 
@@ -227,8 +200,6 @@ __device__ __forceinline__ T block_sum(T v, T *scratch)      // scratch: 32 entr
 
 constexpr int kLinearBins = 2048;        // select: linear bins between the smallest and largest logit
 constexpr int kCandidates = 8192;        // select: keys of the threshold bin resolved in shared memory
-constexpr int kSampleMinTokens = 32768;  // select: rows at least this long estimate the bin from a sample
-constexpr int kSampleSlackBins = 24;     // select: bins kept on either side of the estimate
 
 struct SelectShared {
     unsigned hist[kLinearBins + 1];      // bin kLinearBins: the forced local window
@@ -383,17 +354,17 @@ sparf_select_kernel(const SparfParams p)
     const float4 *a4 = reinterpret_cast<const float4 *>(a);
     const int quads = (S + 3) / 4;
 
-    // Largest and smallest approximate logit (base-2 domain), from the score kernel's chunks.
+    // Pass 1: largest and smallest approximate logit (base-2 domain).
     float top = kMinusHuge, low = -kMinusHuge;
-    {
-        const float2 *range = p.chunk_range + (int64_t)pair * p.score_chunks;
-        const int chunks = (S + kScoreChunk - 1) / kScoreChunk;
-        for (int c = tid; c < chunks; c += kSelectThreads) {
-            const float2 r = range[c];
-            low = fminf(low, r.x);
-            top = fmaxf(top, r.y);
+    for_each_quad(a4, quads, [&](int i0, const float (&x)[4]) {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            if (i0 + e < S) {
+                top = fmaxf(top, x[e]);
+                low = fminf(low, x[e]);
+            }
         }
-    }
+    });
 #pragma unroll
     for (int off = 16; off >= 1; off >>= 1) {
         top = fmaxf(top, __shfl_xor_sync(0xffffffffu, top, off));
@@ -404,10 +375,6 @@ sparf_select_kernel(const SparfParams p)
         sh.red_u[0][warp] = __float_as_uint(low);
     }
     for (int t = tid; t <= kLinearBins; t += kSelectThreads) sh.hist[t] = 0u;
-    if (tid == 0) {
-        sh.n_cand = 0;
-        sh.bin = 0;
-    }
     __syncthreads();
     for (int w = 0; w < kSelectThreads / 32; ++w) {
         top = fmaxf(top, sh.red_f[w]);
@@ -422,95 +389,8 @@ sparf_select_kernel(const SparfParams p)
     };
     auto key_of = [&](int i, float x) -> unsigned { return i >= S - window ? 0xffffffffu : ordered_key(x); };
 
-    // Step 6, long rows: the threshold bin is first estimated from every 8th quad, then one
-    // full pass counts what lies above a window of bins around the estimate and collects the
-    // keys inside it; the exact threshold is found among those.  If the window missed (or
-    // overflowed), the full histogram below decides, so the result never depends on luck.
-    float z = 0.f;
-    bool solved = false;
-    __syncthreads();
-    if (window >= k) {                           // the local window alone fills k
-        if (tid == 0) {
-            sh.tau = 0xffffffffu;
-            sh.take_equal = k;
-        }
-        for_each_quad(a4, quads, [&](int i0, const float (&x)[4]) {
-#pragma unroll
-            for (int e = 0; e < 4; ++e)
-                if (i0 + e < S) z += fast_exp2(x[e] - top);
-        });
-        z = block_sum(z, sh.red_f);
-        solved = true;
-    } else if (S >= kSampleMinTokens) {
-        int sampled = 0;
-        for (int g = 8 * tid; g < quads; g += 8 * kSelectThreads) {
-            const float4 v = a4[g];
-            const float x[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const int i = 4 * g + e;
-                if (i < S - window) {
-                    atomicAdd(&sh.hist[bin_of(i, x[e])], 1u);
-                    ++sampled;
-                }
-            }
-        }
-        sampled = block_sum(sampled, sh.scan_eq);
-        const int target = max(1, min(sampled, (int)(((int64_t)(k - window) * sampled + (S - window) - 1) / (S - window))));
-        if (warp == 0) {
-            int mine = 0;
-            for (int j = 0; j < 64; ++j) mine += (int)sh.hist[64 * lane + ((j + lane) & 63)];
-            int above = 0;
-            for (int src = 31; src >= 0; --src) {
-                const int seg = __shfl_sync(0xffffffffu, mine, src);
-                if (src > lane) above += seg;
-            }
-            if (above < target && target <= above + mine) {
-                int bin = 64 * lane + 63;
-                for (; bin > 64 * lane; --bin) {
-                    const int c = (int)sh.hist[bin];
-                    if (above + c >= target) break;
-                    above += c;
-                }
-                sh.bin = bin;
-            }
-        }
-        __syncthreads();
-        const int lo_bin = max(0, sh.bin - kSampleSlackBins), hi_bin = min(kLinearBins - 1, sh.bin + kSampleSlackBins);
-        int above = 0;
-        for_each_quad(a4, quads, [&](int i0, const float (&x)[4]) {
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const int i = i0 + e;
-                if (i < S) {
-                    z += fast_exp2(x[e] - top);
-                    const int bin = bin_of(i, x[e]);
-                    if (bin > hi_bin) {
-                        ++above;
-                    } else if (bin >= lo_bin) {
-                        const int at = atomicAdd(&sh.n_cand, 1);
-                        if (at < kCandidates) sh.cand[at] = ordered_key(x[e]);
-                    }
-                }
-            }
-        });
-        z = block_sum(z, sh.red_f);
-        above = block_sum(above, sh.scan_eq);
-        const int n_cand = sh.n_cand, need = k - above;
-        if (n_cand <= kCandidates && need >= 1 && need <= n_cand) {
-            exact_threshold(sh, n_cand, need, [](int) { return true; }, [&](int i) { return sh.cand[i]; });
-            solved = true;
-        } else {                                 // start over with the full histogram
-            z = 0.f;
-            __syncthreads();
-            for (int t = tid; t <= kLinearBins; t += kSelectThreads) sh.hist[t] = 0u;
-            if (tid == 0) sh.n_cand = 0;
-            __syncthreads();
-        }
-    }
-
-    if (!solved) {
     // Pass 2: histogram over the linear bins, and the softmax denominator.
+    float z = 0.f;
     for_each_quad(a4, quads, [&](int i0, const float (&x)[4]) {
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
@@ -531,7 +411,12 @@ sparf_select_kernel(const SparfParams p)
             const int seg = __shfl_sync(0xffffffffu, mine, src);
             if (src > lane) above += seg;
         }
-        if (above < k && k <= above + mine) {
+        if ((int)sh.hist[kLinearBins] >= k) {
+            if (lane == 0) {
+                sh.bin = kLinearBins;
+                sh.above = 0;
+            }
+        } else if (above < k && k <= above + mine) {
             int bin = 64 * lane + 63;
             for (; bin > 64 * lane; --bin) {
                 const int c = (int)sh.hist[bin];
@@ -541,14 +426,21 @@ sparf_select_kernel(const SparfParams p)
             sh.bin = bin;
             sh.above = above;
         }
+        if (lane == 0) sh.n_cand = 0;
     }
     __syncthreads();
     const int bin = sh.bin, above = sh.above;
     const int in_bin = (int)sh.hist[bin];
     __syncthreads();                             // the histogram is reused below
 
-    // The exact threshold inside that bin.
-    if (in_bin <= kCandidates) {
+    // Step 6: the exact threshold inside that bin.
+    if (bin == kLinearBins) {                    // the window alone fills k
+        if (tid == 0) {
+            sh.tau = 0xffffffffu;
+            sh.take_equal = k;
+        }
+        __syncthreads();
+    } else if (in_bin <= kCandidates) {
         for_each_quad(a4, quads, [&](int i0, const float (&x)[4]) {
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
@@ -581,8 +473,6 @@ sparf_select_kernel(const SparfParams p)
         exact_threshold(sh, S, k - above, [&](int i) { return bin_of(i, a[i]) == bin; },
                         [&](int i) { return ordered_key(a[i]); });
     }
-    }
-    __syncthreads();
     const unsigned tau = sh.tau;                 // key of the k-th largest
     const int take_equal = sh.take_equal;        // how many keys equal to tau belong to the top k
 
