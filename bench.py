@@ -243,9 +243,11 @@ class Layer:
         """The same step as a caller with host-resident q,k,v sees it: the three new vectors
         go up from pinned memory, the attention output comes back (the KV cache stays on the
         device, which is the point of the method: Sec. IV-D)."""
-        self.qkv.copy_(self.host_qkv, non_blocking=True)
-        self.run(flags)
-        self.host_out.copy_(self.out, non_blocking=True)
+        from paper_2409_04992_b200 import binding
+        c = self.case
+        binding.decode_step_host(self.host_out, self.host_qkv, self.qkv, self.out, self.lse, c.k_cache,
+                                 c.v_cache, c.seq_lens, c.block_table, self.max_len, c.scale,
+                                 self.workspace, flags)
 
     @property
     def h2d_bytes(self) -> int:

@@ -173,6 +173,30 @@ int instinfer_decode_attention_static(void *out, float *lse, const void *q,
                                       int32_t *status_flags, void *cuda_stream);
 
 /*
+ * One whole decode step for a caller whose new vectors live in host memory (the paper's
+ * decode flow, Sec. IV-D: only q, k, v travel to the device that owns the KV cache and only
+ * the attention output travels back; the cache never moves).
+ *   qkv_host  HOST (pinned for an asynchronous copy) fp16 [3, batch, heads, head_dim]:
+ *             q, k_new, v_new packed in this order
+ *   out_host  HOST fp16 [batch, heads, head_dim]
+ *   qkv_dev, out_dev  DEVICE staging buffers of the same shapes, owned by the caller
+ *   lse       DEVICE fp32 [batch, heads], nullable
+ * Enqueued on the stream, in order: copy qkv_host -> qkv_dev, instinfer_kv_append,
+ * instinfer_decode_attention (block_table == NULL) or instinfer_decode_attention_paged,
+ * copy out_dev -> out_host.  out_host holds the result once the stream has reached that
+ * point; the call itself does not synchronise.  Other arguments and errors as in the calls
+ * it is made of.
+ */
+int instinfer_decode_step_host(void *out_host, const void *qkv_host, void *qkv_dev, void *out_dev,
+                               float *lse, void *k_cache, void *v_cache, const int32_t *seq_lens,
+                               const int32_t *block_table, int32_t max_blocks_per_seq,
+                               int32_t block_tokens, int64_t num_phys_blocks,
+                               int32_t batch, int32_t heads, int32_t head_dim, int32_t s_max,
+                               int32_t max_seq_len, float scale,
+                               void *workspace, size_t workspace_bytes,
+                               int32_t *status_flags, void *cuda_stream);
+
+/*
  * ---- Sparse decode attention (the paper's Algorithm 1, SparF; SparQ's arithmetic) ----
  * Paged layout only.  Besides the K and V pools the cache keeps
  *   kt_pool  fp16 [num_phys_blocks, heads, head_dim, block_tokens]: K a second time,

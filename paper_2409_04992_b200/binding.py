@@ -54,6 +54,10 @@ def load() -> ctypes.CDLL:
         lib.instinfer_decode_attention_static.argtypes = [ptr, ptr, ptr, ptr, ptr, ptr, ptr,
                                                           i32, i32, i32, i32, i32, i32, i64, i32,
                                                           f32, ptr, ptr]
+        lib.instinfer_decode_step_host.restype = ctypes.c_int
+        lib.instinfer_decode_step_host.argtypes = [ptr, ptr, ptr, ptr, ptr, ptr, ptr, ptr, ptr,
+                                                   i32, i32, i64, i32, i32, i32, i32, i32, f32,
+                                                   ptr, sz, ptr, ptr]
         lib.instinfer_sparf_append.restype = ctypes.c_int
         lib.instinfer_sparf_append.argtypes = [ptr, ptr, ptr, ptr, ptr, ptr, ptr, ptr, i32, i32, i64,
                                                i32, i32, i32, ptr, ptr]
@@ -204,6 +208,27 @@ def decode_attention_static(out: torch.Tensor, lse: Optional[torch.Tensor], q: t
         _ptr(out), _ptr(lse), _ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(block_table),
         _ptr(seq_lens), batch, heads, head_dim, s_max, block_tokens, max_blocks, phys,
         int(max_seq_len), float(scale), _ptr(status_flags), _stream(stream)))
+
+
+def decode_step_host(out_host: torch.Tensor, qkv_host: torch.Tensor, qkv_dev: torch.Tensor,
+                     out_dev: torch.Tensor, lse: Optional[torch.Tensor], k_cache: torch.Tensor,
+                     v_cache: torch.Tensor, seq_lens: torch.Tensor,
+                     block_table: Optional[torch.Tensor], max_seq_len: int, scale: float,
+                     workspace: torch.Tensor, status_flags: Optional[torch.Tensor] = None,
+                     stream: Optional[torch.cuda.Stream] = None) -> None:
+    """instinfer_decode_step_host: qkv_host [3,B,H,D] and out_host [B,H,D] are (pinned) host
+    tensors, qkv_dev / out_dev device staging buffers of the same shapes."""
+    _, batch, heads, head_dim = qkv_host.shape
+    if block_table is None:
+        max_blocks, block_tokens, phys, s_max = 0, 0, 0, k_cache.shape[2]
+    else:
+        max_blocks, block_tokens, phys, s_max = (block_table.shape[1], k_cache.shape[2],
+                                                 k_cache.shape[0], 0)
+    _check(load().instinfer_decode_step_host(
+        _ptr(out_host), _ptr(qkv_host), _ptr(qkv_dev), _ptr(out_dev), _ptr(lse), _ptr(k_cache),
+        _ptr(v_cache), _ptr(seq_lens), _ptr(block_table), max_blocks, block_tokens, phys, batch,
+        heads, head_dim, s_max, int(max_seq_len), float(scale), _ptr(workspace),
+        workspace.numel() * workspace.element_size(), _ptr(status_flags), _stream(stream)))
 
 
 def sparf_append(k_pool: torch.Tensor, v_pool: torch.Tensor, kt_pool: torch.Tensor,

@@ -404,6 +404,48 @@ int instinfer_decode_attention_static(void *out, float *lse, const void *q, cons
                                             cuda_stream);
 }
 
+int instinfer_decode_step_host(void *out_host, const void *qkv_host, void *qkv_dev, void *out_dev,
+                               float *lse, void *k_cache, void *v_cache, const int32_t *seq_lens,
+                               const int32_t *block_table, int32_t max_blocks_per_seq,
+                               int32_t block_tokens, int64_t num_phys_blocks, int32_t batch,
+                               int32_t heads, int32_t head_dim, int32_t s_max, int32_t max_seq_len,
+                               float scale, void *workspace, size_t workspace_bytes,
+                               int32_t *status_flags, void *cuda_stream)
+{
+    if (batch < 0 || heads <= 0 || head_dim <= 0) return INSTINFER_ERR_INVALID_ARG;
+    if (head_dim != kHeadDim) return INSTINFER_ERR_UNSUPPORTED;
+    if (batch == 0) return INSTINFER_OK;
+    if (out_host == nullptr || qkv_host == nullptr || !usable(qkv_dev) || !usable(out_dev))
+        return INSTINFER_ERR_INVALID_ARG;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const size_t one = (size_t)batch * heads * head_dim * sizeof(__half);
+    if (cudaMemcpyAsync(qkv_dev, qkv_host, 3 * one, cudaMemcpyHostToDevice, stream) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return INSTINFER_ERR_CUDA;
+    }
+    const unsigned char *staged = static_cast<const unsigned char *>(qkv_dev);
+    int rc = instinfer_kv_append(k_cache, v_cache, staged + one, staged + 2 * one, seq_lens, block_table,
+                                 max_blocks_per_seq, block_tokens, num_phys_blocks, batch, heads,
+                                 head_dim, s_max, status_flags, cuda_stream);
+    if (rc != INSTINFER_OK) return rc;
+    if (block_table == nullptr)
+        rc = instinfer_decode_attention(out_dev, lse, staged, k_cache, v_cache, seq_lens, batch, heads,
+                                        head_dim, s_max, max_seq_len, scale, workspace,
+                                        workspace_bytes, status_flags, cuda_stream);
+    else
+        rc = instinfer_decode_attention_paged(out_dev, lse, staged, k_cache, v_cache, block_table,
+                                              seq_lens, batch, heads, head_dim, block_tokens,
+                                              max_blocks_per_seq, num_phys_blocks, max_seq_len,
+                                              scale, workspace, workspace_bytes, status_flags,
+                                              cuda_stream);
+    if (rc != INSTINFER_OK) return rc;
+    if (cudaMemcpyAsync(out_host, out_dev, one, cudaMemcpyDeviceToHost, stream) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return INSTINFER_ERR_CUDA;
+    }
+    return INSTINFER_OK;
+}
+
 namespace {
 
 struct SparfLayout {
