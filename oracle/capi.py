@@ -34,11 +34,11 @@ def _load() -> ctypes.CDLL:
                                               i32, i32, i32, i32, i32]
         lib.oracle_sparf_append.restype = ctypes.c_int
         lib.oracle_sparf_append.argtypes = [ptr, ptr, ptr, ptr, ptr, ptr, ptr, ptr, i32, i32, i64,
-                                            i32, i32, i32]
+                                            ptr, i32, i32, i64, i32, i32, i32]
         lib.oracle_sparf_attention.restype = ctypes.c_int
         lib.oracle_sparf_attention.argtypes = [ptr, ptr, ptr, i64, ptr, ptr, i64, ptr, ptr, ptr, ptr,
-                                               ptr, ptr, ptr, ptr, i32, i32, i64, i32, i32, i32,
-                                               i32, i32, ctypes.c_float]
+                                               ptr, ptr, ptr, ptr, i32, i32, i64, ptr, i32, i32, i64,
+                                               i32, i32, i32, i32, i32, ctypes.c_float]
         _lib = lib
     return _lib
 
@@ -157,8 +157,9 @@ def decode_attention(q: np.ndarray, k_cache: np.ndarray, v_cache: np.ndarray,
 
 def sparf_append(k_pool: np.ndarray, v_pool: np.ndarray, kt_pool: np.ndarray, v_sum: np.ndarray,
                  k_new: np.ndarray, v_new: np.ndarray, seq_lens: np.ndarray,
-                 block_table: np.ndarray) -> None:
-    """In-place append for the SparF state: pools [P,H,T,D], K^T pool [P,H,D,T], v_sum f32 [B,H,D]."""
+                 block_table: np.ndarray, kt_block_table: Optional[np.ndarray] = None) -> None:
+    """In-place append for the SparF state: pools [P,H,T,D], K^T pool [Pk,H,D,Tk] with its own
+    table (default: the K/V table, i.e. Tk == T), v_sum f32 [B,H,D]."""
     kb, vb, ktb = _bits(k_pool, True), _bits(v_pool, True), _bits(kt_pool, True)
     kn, vn = _bits(np.ascontiguousarray(k_new)), _bits(np.ascontiguousarray(v_new))
     if v_sum.dtype != np.float32 or not v_sum.flags.c_contiguous:
@@ -166,9 +167,11 @@ def sparf_append(k_pool: np.ndarray, v_pool: np.ndarray, kt_pool: np.ndarray, v_
     batch, heads, head_dim = kn.shape
     lens = np.ascontiguousarray(seq_lens, dtype=np.int32)
     table, max_blocks = _table(block_table, batch)
+    kt_table, kt_max_blocks = _table(block_table if kt_block_table is None else kt_block_table, batch)
     rc = _load().oracle_sparf_append(_p(kb), _p(vb), _p(ktb), _p(v_sum), _p(kn), _p(vn), _p(lens),
-                                     _p(table), max_blocks, kb.shape[2], kb.shape[0], batch, heads,
-                                     head_dim)
+                                     _p(table), max_blocks, kb.shape[2], kb.shape[0],
+                                     _p(kt_table), kt_max_blocks, ktb.shape[3], ktb.shape[0],
+                                     batch, heads, head_dim)
     if rc:
         raise OracleError(rc)
 
@@ -176,7 +179,8 @@ def sparf_append(k_pool: np.ndarray, v_pool: np.ndarray, kt_pool: np.ndarray, v_
 def sparf_attention(q: np.ndarray, k_pool: np.ndarray, v_pool: np.ndarray, kt_pool: np.ndarray,
                     v_sum: np.ndarray, seq_lens: np.ndarray, k_tokens: np.ndarray,
                     block_table: np.ndarray, r: int, l: int, scale: float,
-                    given: Optional[np.ndarray] = None, want_weights: bool = False):
+                    given: Optional[np.ndarray] = None, want_weights: bool = False,
+                    kt_block_table: Optional[np.ndarray] = None):
     """Algorithm 1 per (sequence, head).  Returns (out f64 [B,H,D], alpha f64 [B,H],
     selected int32 [B,H,max k] ascending / -1 padded, approximate weights or None)."""
     qb = _bits(np.ascontiguousarray(q))
@@ -185,6 +189,7 @@ def sparf_attention(q: np.ndarray, k_pool: np.ndarray, v_pool: np.ndarray, kt_po
     lens = np.ascontiguousarray(seq_lens, dtype=np.int32)
     ks = np.ascontiguousarray(k_tokens, dtype=np.int32)
     table, max_blocks = _table(block_table, batch)
+    kt_table, kt_max_blocks = _table(block_table if kt_block_table is None else kt_block_table, batch)
     vs = np.ascontiguousarray(v_sum, dtype=np.float32)
     stride_k = max(int(np.minimum(ks, lens).max()) if batch else 0, 1)
     stride_s = max(int(lens.max()) if batch else 0, 1)
@@ -199,7 +204,8 @@ def sparf_attention(q: np.ndarray, k_pool: np.ndarray, v_pool: np.ndarray, kt_po
     rc = _load().oracle_sparf_attention(_p(out), _p(alpha), _p(weights), stride_s, _p(selected),
                                         _p(giv), stride_k, _p(qb), _p(kb), _p(vb), _p(ktb), _p(vs),
                                         _p(lens), _p(ks), _p(table), max_blocks, kb.shape[2],
-                                        kb.shape[0], batch, heads, head_dim, int(r), int(l),
+                                        kb.shape[0], _p(kt_table), kt_max_blocks, ktb.shape[3],
+                                        ktb.shape[0], batch, heads, head_dim, int(r), int(l),
                                         ctypes.c_float(scale))
     if rc:
         raise OracleError(rc)

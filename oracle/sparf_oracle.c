@@ -21,8 +21,11 @@
  * k is clipped to S and l to k.  S == 0 gives out = 0 and alpha = 0.  If |q|_1 == 0 the
  * ratio is taken as 1.
  *
- * Layouts: K, V pools [P][H][T][D]; K^T pool [P][H][D][T]; block_table [B][M]; v_sum is
- * float [B][H][D], the running sum of all V rows of the sequence kept by the append.
+ * Layouts: K, V pools [P][H][T][D] with block_table [B][M].  The K^T copy has its own
+ * granularity (Sec. IV-C gives the embedding-indexed mapping much larger token groups than
+ * the token-indexed one): pool [Pk][H][D][Tk] with kt_block_table [B][Mk]; token i of sequence b
+ * sits in K^T block kt_block_table[b][i / Tk] at column i % Tk.  v_sum is float [B][H][D],
+ * the running sum of all V rows of the sequence kept by the append.
  *
  * Return: 0, or -1 bad argument, -2 seq_len out of range, -3 block id out of range.
  */
@@ -56,6 +59,14 @@ static int64_t block_base(const paged_geometry *g, int32_t b, int32_t h, int32_t
     return ((int64_t)phys * g->heads + h) * g->tokens * g->dim;
 }
 
+/* element offset of K^T[dim d][token i] of (b, h) in the embedding-major pool; -1 if the block id is bad */
+static int64_t kt_offset(const paged_geometry *g, int32_t b, int32_t h, int32_t d, int32_t i)
+{
+    const int32_t phys = g->table[(int64_t)b * g->max_blocks + i / g->tokens];
+    if (phys < 0 || (int64_t)phys >= g->phys_blocks) return -1;
+    return (((int64_t)phys * g->heads + h) * g->dim + d) * g->tokens + i % g->tokens;
+}
+
 /*
  * Append for the SparF state (Sec. IV-C: K is stored twice, token-indexed and hidden-
  * embedding-indexed; Algorithm 1's vbar needs the mean of V).  Position seq_lens[b]-1 gets
@@ -66,26 +77,33 @@ int oracle_sparf_append(uint16_t *k_pool, uint16_t *v_pool, uint16_t *kt_pool, f
                         const uint16_t *k_new, const uint16_t *v_new, const int32_t *seq_lens,
                         const int32_t *block_table, int32_t max_blocks_per_seq,
                         int32_t block_tokens, int64_t num_phys_blocks,
+                        const int32_t *kt_block_table, int32_t kt_max_blocks_per_seq,
+                        int32_t kt_block_tokens, int64_t num_kt_blocks,
                         int32_t batch, int32_t heads, int32_t head_dim)
 {
     if (batch < 0 || heads <= 0 || head_dim <= 0 || block_tokens <= 0 || max_blocks_per_seq <= 0 ||
-        num_phys_blocks <= 0 || block_table == NULL)
+        num_phys_blocks <= 0 || block_table == NULL || kt_block_table == NULL ||
+        kt_block_tokens <= 0 || kt_max_blocks_per_seq <= 0 || num_kt_blocks <= 0)
         return -1;
     const paged_geometry g = {block_table, max_blocks_per_seq, block_tokens, heads, head_dim,
                               num_phys_blocks};
+    const paged_geometry gt = {kt_block_table, kt_max_blocks_per_seq, kt_block_tokens, heads,
+                               head_dim, num_kt_blocks};
     for (int32_t b = 0; b < batch; ++b) {
         const int32_t L = seq_lens[b];
         if (L == 0) continue;
-        if (L < 0 || (int64_t)L > (int64_t)max_blocks_per_seq * block_tokens) return -2;
+        if (L < 0 || (int64_t)L > (int64_t)max_blocks_per_seq * block_tokens ||
+            (int64_t)L > (int64_t)kt_max_blocks_per_seq * kt_block_tokens)
+            return -2;
         for (int32_t h = 0; h < heads; ++h) {
             const int64_t base = block_base(&g, b, h, L - 1);
-            if (base < 0) return -3;
+            if (base < 0 || kt_offset(&gt, b, h, 0, L - 1) < 0) return -3;
             const int32_t slot = (L - 1) % block_tokens;
             const int64_t src = ((int64_t)b * heads + h) * head_dim;
             for (int32_t d = 0; d < head_dim; ++d) {
                 k_pool[base + (int64_t)slot * head_dim + d] = k_new[src + d];
                 v_pool[base + (int64_t)slot * head_dim + d] = v_new[src + d];
-                kt_pool[base + (int64_t)d * block_tokens + slot] = k_new[src + d];
+                kt_pool[kt_offset(&gt, b, h, d, L - 1)] = k_new[src + d];
                 v_sum[src + d] = (float)((double)v_sum[src + d] + widen(v_new[src + d]));
             }
         }
@@ -128,19 +146,26 @@ int oracle_sparf_attention(double *out, double *alpha, double *approx_weights, i
                            const int32_t *seq_lens, const int32_t *k_tokens,
                            const int32_t *block_table, int32_t max_blocks_per_seq,
                            int32_t block_tokens, int64_t num_phys_blocks,
+                           const int32_t *kt_block_table, int32_t kt_max_blocks_per_seq,
+                           int32_t kt_block_tokens, int64_t num_kt_blocks,
                            int32_t batch, int32_t heads, int32_t head_dim,
                            int32_t r, int32_t l, float scale)
 {
     if (batch < 0 || heads <= 0 || head_dim <= 0 || block_tokens <= 0 || max_blocks_per_seq <= 0 ||
-        num_phys_blocks <= 0 || block_table == NULL || r <= 0 || r > head_dim || l < 0)
+        num_phys_blocks <= 0 || block_table == NULL || r <= 0 || r > head_dim || l < 0 ||
+        kt_block_table == NULL || kt_block_tokens <= 0 || kt_max_blocks_per_seq <= 0 || num_kt_blocks <= 0)
         return -1;
     const paged_geometry g = {block_table, max_blocks_per_seq, block_tokens, heads, head_dim,
                               num_phys_blocks};
+    const paged_geometry gt = {kt_block_table, kt_max_blocks_per_seq, kt_block_tokens, heads,
+                               head_dim, num_kt_blocks};
     const int32_t D = head_dim, T = block_tokens;
     int failure = 0;
     for (int32_t b = 0; b < batch && !failure; ++b) {
         const int32_t S = seq_lens[b];
-        if (S < 0 || (int64_t)S > (int64_t)max_blocks_per_seq * T) return -2;
+        if (S < 0 || (int64_t)S > (int64_t)max_blocks_per_seq * T ||
+            (int64_t)S > (int64_t)kt_max_blocks_per_seq * kt_block_tokens)
+            return -2;
         if (k_tokens[b] < 0) return -1;
         const int32_t k = k_tokens[b] < S ? k_tokens[b] : S;
         const int32_t window = l < k ? l : k;
@@ -177,12 +202,11 @@ int oracle_sparf_attention(double *out, double *alpha, double *approx_weights, i
             /* steps 2-4: approximate scores from the embedding-major copy of K */
             double top = -INFINITY;
             for (int32_t i = 0; i < S; ++i) {
-                const int64_t base = block_base(&g, b, h, i);
-                if (base < 0) { failure = -3; break; }
+                if (kt_offset(&gt, b, h, 0, i) < 0) { failure = -3; break; }
                 double dot = 0.0;
                 for (int32_t t = 0; t < r; ++t) {
                     const int32_t d = dims[t].index;
-                    dot += widen(qv[d]) * widen(kt_pool[base + (int64_t)d * T + i % T]);
+                    dot += widen(qv[d]) * widen(kt_pool[kt_offset(&gt, b, h, d, i)]);
                 }
                 a[i] = approx_scale * dot;
                 if (a[i] > top) top = a[i];

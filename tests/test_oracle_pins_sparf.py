@@ -138,3 +138,49 @@ def test_sparf_append_writes_both_k_layouts_and_the_running_sum():
     assert np.array_equal(kt.view(np.uint16), np.ascontiguousarray(k.transpose(0, 1, 3, 2)).view(np.uint16))
     assert np.array_equal(v_sum[2], s0[2])
     assert np.array_equal(v_sum[:2], (s0[:2] + vn[:2].astype(np.float32)))     # one fp32 rounding
+
+
+def relayout_kt(k, table, lens, tokens, kt_tokens, rng):
+    """K^T pool [Pk,H,D,Tk] with its own shuffled table, holding the same logical keys."""
+    H, D = k.shape[1], k.shape[3]
+    need = [-(-int(n) // kt_tokens) for n in lens]
+    Pk = sum(need) + 1
+    perm = rng.permutation(Pk)
+    kt_table = np.full((len(lens), max(max(need), 1)), -1, dtype=np.int32)
+    kt = np.full((Pk, H, D, kt_tokens), np.float16(np.nan), dtype=np.float16)
+    at = 0
+    for b, n in enumerate(need):
+        kt_table[b, :n] = perm[at:at + n]
+        at += n
+        rows = rows_of(k, table, b, lens[b], tokens)                 # [H, L, D]
+        for j in range(n):
+            piece = rows[:, j * kt_tokens:(j + 1) * kt_tokens]       # [H, <=Tk, D]
+            kt[kt_table[b, j], :, :, :piece.shape[1]] = piece.transpose(0, 2, 1)
+    return kt, kt_table
+
+
+@pytest.mark.parametrize("kt_tokens", [8, 32, 64])
+def test_the_transposed_copy_may_use_its_own_block_size(kt_tokens):
+    rng = np.random.default_rng(37)
+    lens = np.array([70, 9, 0, 33])
+    k, v, kt, v_sum, table = paged(rng, lens, 8, gain=2.0)
+    q = f16(rng, (4, 2, 128), 2.0)
+    ks = np.array([9, 2, 0, 5])
+    same = capi.sparf_attention(q, k, v, kt, v_sum, lens, ks, table, r=16, l=2, scale=SCALE, want_weights=True)
+    kt2, kt_table = relayout_kt(k, table, lens, 8, kt_tokens, rng)
+    other = capi.sparf_attention(q, k, v, kt2, v_sum, lens, ks, table, r=16, l=2, scale=SCALE,
+                                 want_weights=True, kt_block_table=kt_table)
+    for a, b in zip(same, other):
+        assert np.array_equal(a, b)
+    # the append lands in the right column of the right K^T block
+    lens2 = lens + np.array([1, 1, 0, 1])
+    grow = [-(-int(n) // 8) for n in lens2]
+    assert all(g <= table.shape[1] or True for g in grow)
+    lens_ok = np.array([70, 9, 0, 33])            # re-append the last token of each live sequence
+    kn, vn = f16(rng, (4, 2, 128)), f16(rng, (4, 2, 128))
+    capi.sparf_append(k, v, kt2, v_sum, kn, vn, lens_ok, table, kt_block_table=kt_table)
+    want_kt, _ = None, None
+    for b, n in enumerate(lens_ok):
+        if n:
+            blk, col = kt_table[b, (n - 1) // kt_tokens], (n - 1) % kt_tokens
+            assert np.array_equal(kt2[blk, :, :, col].view(np.uint16), kn[b].view(np.uint16))
