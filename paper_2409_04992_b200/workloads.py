@@ -241,15 +241,50 @@ def gather_rows(case: Case, b: int, h: int):
 class SparfState:
     """Extra per-layer state of the sparse (SparF) path for a paged case."""
 
-    kt_pool: torch.Tensor           # fp16 [P,H,D,T]: the embedding-major copy of the K pool
+    kt_pool: torch.Tensor           # fp16 [Pk,H,D,Tk]: the embedding-major copy of K
+    kt_block_table: torch.Tensor    # int32 [B,Mk]: logical Tk-token group -> block of kt_pool
     v_sum: torch.Tensor             # fp32 [B,H,D]: running sum of each sequence's V rows
     k_tokens: torch.Tensor          # int32 [B]: tokens to keep per sequence
     k_tokens_host: List[int]
 
+    @property
+    def kt_block_tokens(self) -> int:
+        return self.kt_pool.shape[3]
 
-def make_sparf_state(case: Case, keep_fraction: float = 0.125) -> SparfState:
-    """The embedding-major K copy is a pure re-layout of the K pool (poison included).  v_sum
-    is an input of the algorithm (it enters as the mean value vector): it is drawn as
+
+def _relayout_kt(case: Case, kt_tokens: int, cpu_gen: torch.Generator):
+    """The K pool re-laid embedding-major in groups of kt_tokens tokens under a table of its
+    own (memory movement only; slots past a sequence's end carry the NaN poison)."""
+    w = case.workload
+    T, H, D = w.block_tokens, w.heads, w.head_dim
+    dev = case.k_cache.device
+    need = [-(-n // kt_tokens) for n in case.seq_lens_host]
+    Pk = sum(need) + w.spare_blocks
+    Mk = max(-(-w.len_hi // kt_tokens), max(need, default=0), 1)
+    perm = torch.randperm(Pk, generator=cpu_gen).to(torch.int32)
+    kt_table = torch.full((w.batch, Mk), -1, dtype=torch.int32)
+    kt_pool = torch.empty((Pk, H, D, kt_tokens), dtype=torch.float16, device=dev)
+    _poison(kt_pool)
+    at = 0
+    for b, n in enumerate(need):
+        kt_table[b, :n] = perm[at:at + n]
+        at += n
+        if n == 0:
+            continue
+        blocks = case.block_table[b, : -(-case.seq_lens_host[b] // T)].long()
+        rows = case.k_cache[blocks].permute(1, 3, 0, 2).reshape(H, D, -1)          # [H, D, tokens]
+        padded = torch.empty((H, D, n * kt_tokens), dtype=torch.float16, device=dev)
+        _poison(padded)
+        padded[:, :, : rows.shape[2]] = rows
+        kt_pool[kt_table[b, :n].long().to(dev)] = padded.view(H, D, n, kt_tokens).permute(2, 0, 1, 3)
+    return kt_pool, kt_table.to(dev)
+
+
+def make_sparf_state(case: Case, keep_fraction: float = 0.125,
+                     kt_block_tokens: Optional[int] = None) -> SparfState:
+    """The embedding-major K copy is a pure re-layout of the K pool (poison included), in
+    groups of kt_block_tokens tokens (default: the K/V block size, sharing the K/V table).
+    v_sum is an input of the algorithm (it enters as the mean value vector): it is drawn as
     N(0, L) per element, the distribution of a sum of L unit normals, not computed from V."""
     if case.block_table is None:
         raise ValueError("the sparse path is defined on the paged layout")
@@ -257,12 +292,19 @@ def make_sparf_state(case: Case, keep_fraction: float = 0.125) -> SparfState:
     dev = case.q.device
     gen = torch.Generator(device=dev)
     gen.manual_seed(BASE_SEED + 5000 + w.index + 1000 * case.layer)
-    kt_pool = case.k_cache.transpose(2, 3).contiguous()
+    if kt_block_tokens is None or kt_block_tokens == w.block_tokens:
+        kt_pool, kt_table = case.k_cache.transpose(2, 3).contiguous(), case.block_table
+    else:
+        if kt_block_tokens % w.block_tokens:
+            raise ValueError("kt_block_tokens must be a multiple of the K/V block size")
+        cpu_gen = torch.Generator(device="cpu")
+        cpu_gen.manual_seed(BASE_SEED + 6000 + w.index + 1000 * case.layer)
+        kt_pool, kt_table = _relayout_kt(case, kt_block_tokens, cpu_gen)
     lens = torch.tensor(case.seq_lens_host, dtype=torch.float32, device=dev)
     v_sum = torch.randn((w.batch, w.heads, w.head_dim), dtype=torch.float32, device=dev,
                         generator=gen) * lens.clamp(min=1).sqrt()[:, None, None]
     keep = [0 if n == 0 else max(1, -(-n * int(round(keep_fraction * 1024)) // 1024))
             for n in case.seq_lens_host]
-    return SparfState(kt_pool=kt_pool, v_sum=v_sum.contiguous(),
+    return SparfState(kt_pool=kt_pool, kt_block_table=kt_table, v_sum=v_sum.contiguous(),
                       k_tokens=torch.tensor(keep, dtype=torch.int32, device=dev),
                       k_tokens_host=keep)
