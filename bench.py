@@ -495,12 +495,12 @@ def measure_workload(w: wl.Workload, ranks: Ranks, device, steps: int, warmup: i
 
 
 def measure_sparse(w: wl.Workload, device, steps: int, r: int = 16, keep: float = 0.125,
-                   window: int = 16) -> dict:
+                   window: int = 16, kt_block_tokens: int = 256) -> dict:
     """One layer of `w` through the sparse (Algorithm 1) entry points next to the dense ones on
     the same data: append + attention per step, CUDA events, inputs far larger than L2."""
     from paper_2409_04992_b200 import binding
     case = wl.generate(w.replace(layers=1), device=str(device), poison=False)
-    state = wl.make_sparf_state(case, keep)
+    state = wl.make_sparf_state(case, keep, kt_block_tokens)
     B, H, D = case.q.shape
     max_len, max_k = case.max_seq_len, max(state.k_tokens_host)
     out = torch.empty((B, H, D), dtype=torch.float16, device=device)
@@ -518,11 +518,11 @@ def measure_sparse(w: wl.Workload, device, steps: int, r: int = 16, keep: float 
 
     def sparse():
         binding.sparf_append(case.k_cache, case.v_cache, state.kt_pool, state.v_sum, case.k_new,
-                             case.v_new, case.seq_lens, case.block_table, flags)
+                             case.v_new, case.seq_lens, case.block_table, state.kt_block_table, flags)
         binding.sparf_decode_attention(out, None, None, case.q, case.k_cache, case.v_cache,
-                                       state.kt_pool, state.v_sum, case.block_table, case.seq_lens,
-                                       state.k_tokens, max_len, max_k, r, window, case.scale,
-                                       ws_sparse, flags)
+                                       state.kt_pool, state.v_sum, case.block_table,
+                                       state.kt_block_table, case.seq_lens, state.k_tokens, max_len,
+                                       max_k, r, window, case.scale, ws_sparse, flags)
 
     def timed(fn):
         for _ in range(3):
@@ -538,7 +538,8 @@ def measure_sparse(w: wl.Workload, device, steps: int, r: int = 16, keep: float 
 
     t_dense, t_sparse = timed(dense), timed(sparse)
     moved = case.kv_tokens * H * r * 2 + sum(state.k_tokens_host) * H * 2 * D * 2
-    return {"r": r, "keep_fraction": keep, "local_window": window, "ms_per_step": t_sparse * 1e3,
+    return {"r": r, "keep_fraction": keep, "local_window": window,
+            "kt_block_tokens": kt_block_tokens, "ms_per_step": t_sparse * 1e3,
             "dense_ms_per_step": t_dense * 1e3, "speedup_over_dense": t_dense / t_sparse,
             "kv_tokens_per_s": case.kv_tokens / t_sparse,
             "algorithmic_bytes": moved, "algorithmic_gbs": moved / t_sparse / 1e9,

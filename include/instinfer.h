@@ -199,10 +199,16 @@ int instinfer_decode_step_host(void *out_host, const void *qkv_host, void *qkv_d
 /*
  * ---- Sparse decode attention (the paper's Algorithm 1, SparF; SparQ's arithmetic) ----
  * Paged layout only.  Besides the K and V pools the cache keeps
- *   kt_pool  fp16 [num_phys_blocks, heads, head_dim, block_tokens]: K a second time,
- *            embedding-major inside each block (Sec. IV-C, hidden-embedding-indexed copy);
- *            slots past a sequence's end inside its last block may be read (in groups of 8
- *            tokens) but never influence a result;
+ *   kt_pool  fp16 [num_kt_blocks, heads, head_dim, kt_block_tokens]: K a second time,
+ *            embedding-major inside each block (Sec. IV-C, hidden-embedding-indexed copy).
+ *            It has its own block size and its own table kt_block_table
+ *            [batch, kt_max_blocks_per_seq]: token i of sequence b is column
+ *            i % kt_block_tokens of block kt_block_table[b][i / kt_block_tokens].  As in the
+ *            paper, where this mapping uses far larger token groups than the 16-token pages
+ *            of K and V, a larger kt_block_tokens (a positive multiple of 8; 128-512 is a good
+ *            choice) makes the r selected rows of a block long contiguous runs.  Slots past a
+ *            sequence's end inside its last block may be read (in groups of 8 tokens) but
+ *            never influence a result;
  *   v_sum    fp32 [batch, heads, head_dim]: the sum of all cached V rows of each sequence;
  *            Algorithm 1's mean value vector is v_sum / seq_lens[b].
  *
@@ -213,6 +219,8 @@ int instinfer_sparf_append(void *k_pool, void *v_pool, void *kt_pool, float *v_s
                            const void *k_new, const void *v_new, const int32_t *seq_lens,
                            const int32_t *block_table, int32_t max_blocks_per_seq,
                            int32_t block_tokens, int64_t num_phys_blocks,
+                           const int32_t *kt_block_table, int32_t kt_max_blocks_per_seq,
+                           int32_t kt_block_tokens, int64_t num_kt_blocks,
                            int32_t batch, int32_t heads, int32_t head_dim,
                            int32_t *status_flags, void *cuda_stream);
 
@@ -245,7 +253,10 @@ int instinfer_sparf_decode_attention(void *out, float *alpha, int32_t *selected,
                                      const int32_t *seq_lens, const int32_t *k_tokens,
                                      int32_t batch, int32_t heads, int32_t head_dim,
                                      int32_t block_tokens, int32_t max_blocks_per_seq,
-                                     int64_t num_phys_blocks, int32_t max_seq_len, int32_t max_k,
+                                     int64_t num_phys_blocks,
+                                     const int32_t *kt_block_table, int32_t kt_max_blocks_per_seq,
+                                     int32_t kt_block_tokens, int64_t num_kt_blocks,
+                                     int32_t max_seq_len, int32_t max_k,
                                      int32_t r, int32_t local_window, float scale,
                                      void *workspace, size_t workspace_bytes,
                                      int32_t *status_flags, void *cuda_stream);

@@ -60,10 +60,11 @@ def load() -> ctypes.CDLL:
                                                    ptr, sz, ptr, ptr]
         lib.instinfer_sparf_append.restype = ctypes.c_int
         lib.instinfer_sparf_append.argtypes = [ptr, ptr, ptr, ptr, ptr, ptr, ptr, ptr, i32, i32, i64,
-                                               i32, i32, i32, ptr, ptr]
+                                               ptr, i32, i32, i64, i32, i32, i32, ptr, ptr]
         lib.instinfer_sparf_decode_attention.restype = ctypes.c_int
         lib.instinfer_sparf_decode_attention.argtypes = [ptr, ptr, ptr, ptr, ptr, ptr, ptr, ptr, ptr,
                                                          ptr, ptr, i32, i32, i32, i32, i32, i64,
+                                                         ptr, i32, i32, i64,
                                                          i32, i32, i32, i32, f32, ptr, sz, ptr, ptr]
         lib.instinfer_sparf_workspace_bytes.restype = sz
         lib.instinfer_sparf_workspace_bytes.argtypes = [i32, i32, i32, i32, i32]
@@ -233,14 +234,16 @@ def decode_step_host(out_host: torch.Tensor, qkv_host: torch.Tensor, qkv_dev: to
 
 def sparf_append(k_pool: torch.Tensor, v_pool: torch.Tensor, kt_pool: torch.Tensor,
                  v_sum: torch.Tensor, k_new: torch.Tensor, v_new: torch.Tensor,
-                 seq_lens: torch.Tensor, block_table: torch.Tensor,
+                 seq_lens: torch.Tensor, block_table: torch.Tensor, kt_block_table: torch.Tensor,
                  status_flags: Optional[torch.Tensor] = None,
                  stream: Optional[torch.cuda.Stream] = None) -> None:
-    """instinfer_sparf_append: pools [P,H,T,D], kt_pool [P,H,D,T], v_sum fp32 [B,H,D]."""
+    """instinfer_sparf_append: pools [P,H,T,D], kt_pool [Pk,H,D,Tk] with kt_block_table [B,Mk],
+    v_sum fp32 [B,H,D]."""
     batch, heads, head_dim = k_new.shape
     _check(load().instinfer_sparf_append(
         _ptr(k_pool), _ptr(v_pool), _ptr(kt_pool), _ptr(v_sum), _ptr(k_new), _ptr(v_new),
         _ptr(seq_lens), _ptr(block_table), block_table.shape[1], k_pool.shape[2], k_pool.shape[0],
+        _ptr(kt_block_table), kt_block_table.shape[1], kt_pool.shape[3], kt_pool.shape[0],
         batch, heads, head_dim, _ptr(status_flags), _stream(stream)))
 
 
@@ -251,7 +254,8 @@ def sparf_workspace_bytes(batch: int, heads: int, head_dim: int, max_seq_len: in
 def sparf_decode_attention(out: torch.Tensor, alpha: Optional[torch.Tensor],
                            selected: Optional[torch.Tensor], q: torch.Tensor,
                            k_pool: torch.Tensor, v_pool: torch.Tensor, kt_pool: torch.Tensor,
-                           v_sum: torch.Tensor, block_table: torch.Tensor, seq_lens: torch.Tensor,
+                           v_sum: torch.Tensor, block_table: torch.Tensor,
+                           kt_block_table: torch.Tensor, seq_lens: torch.Tensor,
                            k_tokens: torch.Tensor, max_seq_len: int, max_k: int, r: int,
                            local_window: int, scale: float, workspace: torch.Tensor,
                            status_flags: Optional[torch.Tensor] = None,
@@ -261,8 +265,9 @@ def sparf_decode_attention(out: torch.Tensor, alpha: Optional[torch.Tensor],
     _check(load().instinfer_sparf_decode_attention(
         _ptr(out), _ptr(alpha), _ptr(selected), _ptr(q), _ptr(k_pool), _ptr(v_pool), _ptr(kt_pool),
         _ptr(v_sum), _ptr(block_table), _ptr(seq_lens), _ptr(k_tokens), batch, heads, head_dim,
-        k_pool.shape[2], block_table.shape[1], k_pool.shape[0], int(max_seq_len), int(max_k),
-        int(r), int(local_window), float(scale), _ptr(workspace),
+        k_pool.shape[2], block_table.shape[1], k_pool.shape[0],
+        _ptr(kt_block_table), kt_block_table.shape[1], kt_pool.shape[3], kt_pool.shape[0],
+        int(max_seq_len), int(max_k), int(r), int(local_window), float(scale), _ptr(workspace),
         workspace.numel() * workspace.element_size(), _ptr(status_flags), _stream(stream)))
 
 

@@ -483,16 +483,20 @@ bool sparf_sizes_ok(int32_t batch, int32_t heads, int32_t head_dim, int32_t bloc
 int instinfer_sparf_append(void *k_pool, void *v_pool, void *kt_pool, float *v_sum,
                            const void *k_new, const void *v_new, const int32_t *seq_lens,
                            const int32_t *block_table, int32_t max_blocks_per_seq,
-                           int32_t block_tokens, int64_t num_phys_blocks, int32_t batch,
+                           int32_t block_tokens, int64_t num_phys_blocks,
+                           const int32_t *kt_block_table, int32_t kt_max_blocks_per_seq,
+                           int32_t kt_block_tokens, int64_t num_kt_blocks, int32_t batch,
                            int32_t heads, int32_t head_dim, int32_t *status_flags,
                            void *cuda_stream)
 {
-    if (!sparf_sizes_ok(batch, heads, head_dim, block_tokens, max_blocks_per_seq, num_phys_blocks))
+    if (!sparf_sizes_ok(batch, heads, head_dim, block_tokens, max_blocks_per_seq, num_phys_blocks) ||
+        kt_block_tokens <= 0 || kt_max_blocks_per_seq <= 0 || num_kt_blocks <= 0)
         return INSTINFER_ERR_INVALID_ARG;
-    if (head_dim != kHeadDim || block_tokens % 8 != 0) return INSTINFER_ERR_UNSUPPORTED;
+    if (head_dim != kHeadDim || block_tokens % 8 != 0 || kt_block_tokens % 8 != 0)
+        return INSTINFER_ERR_UNSUPPORTED;
     if (batch == 0) return INSTINFER_OK;
     if (!usable(k_pool) || !usable(v_pool) || !usable(kt_pool) || !usable(v_sum) || !usable(k_new) ||
-        !usable(v_new) || seq_lens == nullptr || block_table == nullptr)
+        !usable(v_new) || seq_lens == nullptr || block_table == nullptr || kt_block_table == nullptr)
         return INSTINFER_ERR_INVALID_ARG;
     SparfParams p = {};
     p.k_pool = static_cast<__half *>(k_pool);
@@ -509,6 +513,10 @@ int instinfer_sparf_append(void *k_pool, void *v_pool, void *kt_pool, float *v_s
     p.heads = heads;
     p.block_tokens = block_tokens;
     p.max_blocks_per_seq = max_blocks_per_seq;
+    p.kt_block_table = kt_block_table;
+    p.kt_block_tokens = kt_block_tokens;
+    p.kt_max_blocks_per_seq = kt_max_blocks_per_seq;
+    p.num_kt_blocks = num_kt_blocks;
     sparf_append_kernel<<<(unsigned)((int64_t)batch * heads), kSparfThreads, 0,
                           static_cast<cudaStream_t>(cuda_stream)>>>(p);
     return cudaGetLastError() == cudaSuccess ? INSTINFER_OK : INSTINFER_ERR_CUDA;
@@ -530,21 +538,28 @@ int instinfer_sparf_decode_attention(void *out, float *alpha, int32_t *selected,
                                      const int32_t *seq_lens, const int32_t *k_tokens,
                                      int32_t batch, int32_t heads, int32_t head_dim,
                                      int32_t block_tokens, int32_t max_blocks_per_seq,
-                                     int64_t num_phys_blocks, int32_t max_seq_len, int32_t max_k,
+                                     int64_t num_phys_blocks,
+                                     const int32_t *kt_block_table, int32_t kt_max_blocks_per_seq,
+                                     int32_t kt_block_tokens, int64_t num_kt_blocks,
+                                     int32_t max_seq_len, int32_t max_k,
                                      int32_t r, int32_t local_window, float scale,
                                      void *workspace, size_t workspace_bytes,
                                      int32_t *status_flags, void *cuda_stream)
 {
     if (!sparf_sizes_ok(batch, heads, head_dim, block_tokens, max_blocks_per_seq, num_phys_blocks) ||
+        kt_block_tokens <= 0 || kt_max_blocks_per_seq <= 0 || num_kt_blocks <= 0 ||
         max_seq_len <= 0 || (int64_t)max_seq_len > (int64_t)max_blocks_per_seq * block_tokens ||
+        (int64_t)max_seq_len > (int64_t)kt_max_blocks_per_seq * kt_block_tokens ||
         max_k <= 0 || max_k > max_seq_len || local_window < 0 || !std::isfinite(scale))
         return INSTINFER_ERR_INVALID_ARG;
-    if (head_dim != kHeadDim || block_tokens % 8 != 0) return INSTINFER_ERR_UNSUPPORTED;
+    if (head_dim != kHeadDim || block_tokens % 8 != 0 || kt_block_tokens % 8 != 0)
+        return INSTINFER_ERR_UNSUPPORTED;
     if (r <= 0 || r > head_dim) return INSTINFER_ERR_INVALID_ARG;
     if (num_phys_blocks * heads * block_tokens >= (int64_t)1 << 31) return INSTINFER_ERR_UNSUPPORTED;
     if (batch == 0) return INSTINFER_OK;
     if (!usable(out) || !usable(q) || !usable(k_pool) || !usable(v_pool) || !usable(kt_pool) ||
-        !usable(v_sum) || block_table == nullptr || seq_lens == nullptr || k_tokens == nullptr)
+        !usable(v_sum) || block_table == nullptr || kt_block_table == nullptr || seq_lens == nullptr ||
+        k_tokens == nullptr)
         return INSTINFER_ERR_INVALID_ARG;
     const int64_t pairs = (int64_t)batch * heads;
     const SparfLayout w = sparf_layout(pairs, max_seq_len, max_k);
@@ -576,6 +591,10 @@ int instinfer_sparf_decode_attention(void *out, float *alpha, int32_t *selected,
     sp.heads = heads;
     sp.block_tokens = block_tokens;
     sp.max_blocks_per_seq = max_blocks_per_seq;
+    sp.kt_block_table = kt_block_table;
+    sp.kt_block_tokens = kt_block_tokens;
+    sp.kt_max_blocks_per_seq = kt_max_blocks_per_seq;
+    sp.num_kt_blocks = num_kt_blocks;
     sp.max_seq_len = max_seq_len;
     sp.max_k = max_k;
     sp.score_stride = w.score_stride;

@@ -28,7 +28,7 @@ struct SparfParams {
     // cache
     __half *k_pool;
     __half *v_pool;
-    __half *kt_pool;           // [P, H, D, T]
+    __half *kt_pool;           // [Pk, H, D, Tk]: its own block size and table
     float *v_sum;              // [B, H, D]
     const __half *q;
     const __half *k_new;
@@ -36,6 +36,7 @@ struct SparfParams {
     const int32_t *seq_lens;
     const int32_t *k_tokens;
     const int32_t *block_table;
+    const int32_t *kt_block_table;   // [batch, kt_max_blocks_per_seq]
     int32_t *status;
     // scratch
     float *scores;             // [pairs, score_stride] approximate logits, base-2 domain
@@ -45,7 +46,9 @@ struct SparfParams {
     float *alpha_out;          // nullable [pairs]
     int32_t *selected;         // nullable [pairs, max_k] logical token index, ascending, -1 padded
     int64_t num_phys_blocks;
+    int64_t num_kt_blocks;
     int32_t batch, heads, block_tokens, max_blocks_per_seq;
+    int32_t kt_block_tokens, kt_max_blocks_per_seq;
     int32_t max_seq_len, max_k, score_stride, score_chunks, r, window;
     float scale_log2e;
 };
@@ -81,13 +84,19 @@ sparf_append_kernel(const SparfParams p)
         if (d == 0 && h == 0 && p.status) atomicOr(p.status, kFlagBlockRange);
         return;
     }
+    const int Tk = p.kt_block_tokens;
+    const int kt_phys = p.kt_block_table[(int64_t)b * p.kt_max_blocks_per_seq + pos / Tk];
+    if (kt_phys < 0 || (int64_t)kt_phys >= p.num_kt_blocks || (int64_t)len > (int64_t)p.kt_max_blocks_per_seq * Tk) {
+        if (d == 0 && h == 0 && p.status) atomicOr(p.status, kFlagBlockRange);
+        return;
+    }
     const int slot = pos % T;
     const int64_t base = ((int64_t)phys * p.heads + h) * T * kHeadDim;      // elements
     const __half k = p.k_new[(int64_t)pair * kHeadDim + d];
     const __half v = p.v_new[(int64_t)pair * kHeadDim + d];
     p.k_pool[base + (int64_t)slot * kHeadDim + d] = k;
     p.v_pool[base + (int64_t)slot * kHeadDim + d] = v;
-    p.kt_pool[base + (int64_t)d * T + slot] = k;
+    p.kt_pool[(((int64_t)kt_phys * p.heads + h) * kHeadDim + d) * Tk + pos % Tk] = k;
     p.v_sum[(int64_t)pair * kHeadDim + d] += __half2float(v);
 }
 
@@ -138,10 +147,10 @@ sparf_scores_kernel(const SparfParams p)
     const float approx_scale = p.scale_log2e * rsqrtf(ratio);
 
     // Steps 2-4: one thread per group of 8 consecutive tokens (one 16-byte load per selected
-    // dim; block_tokens is a multiple of 8, so a group never straddles a block).  The loads
+    // dim; kt_block_tokens is a multiple of 8, so a group never straddles a block).  The loads
     // of 8 dims are issued together to keep enough bytes in flight.
-    const int T = p.block_tokens;
-    const int32_t *table_row = p.block_table + (int64_t)b * p.max_blocks_per_seq;
+    const int T = p.kt_block_tokens;
+    const int32_t *table_row = p.kt_block_table + (int64_t)b * p.kt_max_blocks_per_seq;
     float *dst = p.scores + (int64_t)pair * p.score_stride;
     for (int i = begin + d * 8; i < end; i += kSparfThreads * 8) {
         const int blk = i / T, slot = i - blk * T;
@@ -149,7 +158,7 @@ sparf_scores_kernel(const SparfParams p)
         float dot[8];
 #pragma unroll
         for (int e = 0; e < 8; ++e) dot[e] = 0.f;
-        if (phys >= 0 && (int64_t)phys < p.num_phys_blocks) {
+        if (phys >= 0 && (int64_t)phys < p.num_kt_blocks) {
             const __half *kt = p.kt_pool + ((int64_t)phys * p.heads + h) * T * kHeadDim + slot;
             for (int t0 = 0; t0 < p.r; t0 += 8) {
                 uint4 raw[8];

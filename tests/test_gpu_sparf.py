@@ -21,15 +21,16 @@ SCORE_RTOL = 1e-4          # relative slack on an approximate weight at the sele
 ALPHA_ATOL = 2e-5
 
 
-def make(lens, tokens=16, heads=3, index=2, peaked=0.0, keep=0.125):
+def make(lens, tokens=16, heads=3, index=2, peaked=0.0, keep=0.125, kt_tokens=None):
     w = wl.Workload("sparf", index, batch=len(lens), len_lo=min(lens), len_hi=max(lens),
                     layout="paged", block_tokens=tokens, heads=heads, peaked_fraction=peaked)
     cpu = wl.generate(w, seq_lens=list(lens))
-    return cpu, wl.make_sparf_state(cpu, keep)
+    return cpu, wl.make_sparf_state(cpu, keep, kt_tokens)
 
 
 def dev_state(state):
-    return wl.SparfState(state.kt_pool.cuda(), state.v_sum.cuda(), state.k_tokens.cuda(), state.k_tokens_host)
+    return wl.SparfState(state.kt_pool.cuda(), state.kt_block_table.cuda(), state.v_sum.cuda(),
+                         state.k_tokens.cuda(), state.k_tokens_host)
 
 
 def gpu_sparf(case, state, r, l, do_append=True, max_k=None):
@@ -43,10 +44,11 @@ def gpu_sparf(case, state, r, l, do_append=True, max_k=None):
     flags = torch.zeros(1, dtype=torch.int32, device="cuda")
     if do_append:
         binding.sparf_append(case.k_cache, case.v_cache, state.kt_pool, state.v_sum, case.k_new,
-                             case.v_new, case.seq_lens, case.block_table, flags)
+                             case.v_new, case.seq_lens, case.block_table, state.kt_block_table, flags)
     binding.sparf_decode_attention(out.view, alpha.view, sel.view, case.q, case.k_cache, case.v_cache,
-                                   state.kt_pool, state.v_sum, case.block_table, case.seq_lens,
-                                   state.k_tokens, max_len, max_k, r, l, case.scale, ws.view, flags)
+                                   state.kt_pool, state.v_sum, case.block_table, state.kt_block_table,
+                                   case.seq_lens, state.k_tokens, max_len, max_k, r, l, case.scale,
+                                   ws.view, flags)
     torch.cuda.synchronize()
     assert out.intact() and alpha.intact() and sel.intact() and ws.intact()
     return out.view.cpu(), alpha.view.cpu().numpy(), sel.view.cpu().numpy(), int(flags.item())
@@ -56,11 +58,13 @@ def oracle_sparf(cpu, state, r, l, do_append=True, given=None, want_weights=Fals
     k, v, kt = cpu.k_cache.numpy(), cpu.v_cache.numpy(), state.kt_pool.numpy()
     v_sum = state.v_sum.numpy()
     lens = np.array(cpu.seq_lens_host, dtype=np.int32)
-    table = cpu.block_table.numpy()
+    table, kt_table = cpu.block_table.numpy(), state.kt_block_table.numpy()
     if do_append:
-        capi.sparf_append(k, v, kt, v_sum, cpu.k_new.numpy(), cpu.v_new.numpy(), lens, table)
+        capi.sparf_append(k, v, kt, v_sum, cpu.k_new.numpy(), cpu.v_new.numpy(), lens, table,
+                          kt_block_table=kt_table)
     return capi.sparf_attention(cpu.q.numpy(), k, v, kt, v_sum, lens, np.array(state.k_tokens_host),
-                                table, r, l, cpu.scale, given=given, want_weights=want_weights)
+                                table, r, l, cpu.scale, given=given, want_weights=want_weights,
+                                kt_block_table=kt_table)
 
 
 def check_selection(sel_gpu, weights, lens, ks, l):
@@ -113,6 +117,13 @@ def test_sparse_attention_matches_the_oracle(tokens, r, l):
     run_and_check(cpu, state, r, l, f"T={tokens} r={r} l={l}")
 
 
+@pytest.mark.parametrize("tokens,kt_tokens", [(8, 64), (16, 256), (32, 32), (16, 48)])
+def test_transposed_copy_with_its_own_block_size(tokens, kt_tokens):
+    cpu, state = make([1, 2, 9, 100, 257, 0, 640, 1500], tokens, kt_tokens=kt_tokens)
+    assert state.kt_block_tokens == kt_tokens
+    run_and_check(cpu, state, 16, 4, f"T={tokens} Tk={kt_tokens}")
+
+
 def test_long_peaked_sequences_and_forty_heads():
     cpu, state = make([5000, 3000], tokens=32, heads=40, index=3, peaked=0.02)
     out, alpha, sel, own = run_and_check(cpu, state, 16, 16, "long peaked")
@@ -159,7 +170,7 @@ def test_true_mean_makes_sparse_close_to_dense():
     table, S = cpu.block_table.numpy(), 2048
     v_rows = cpu.v_cache.numpy()[table[0, :S // 32]].transpose(1, 0, 2, 3).reshape(8, S, 128)
     state.v_sum = torch.from_numpy(v_rows.astype(np.float64).sum(axis=1).astype(np.float32))[None]
-    state.kt_pool = cpu.k_cache.transpose(2, 3).contiguous()
+    state.kt_pool, state.kt_block_table = cpu.k_cache.transpose(2, 3).contiguous(), cpu.block_table
     dev, dstate = gu.to_device(cpu), dev_state(state)
     out, alpha, _, _ = gpu_sparf(dev, dstate, 32, 32, do_append=False)
     dense, _ = gu.oracle_step(cpu, do_append=False)
