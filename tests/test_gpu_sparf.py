@@ -176,3 +176,24 @@ def test_true_mean_makes_sparse_close_to_dense():
     dense, _ = gu.oracle_step(cpu, do_append=False)
     err = np.abs(out.numpy().astype(np.float64) - dense)
     assert err.mean() < 0.05 and np.all(alpha > 0.3)
+
+
+def test_heavy_ties_are_cut_by_position():
+    # q = 0 makes every approximate score equal: the kept set must be the first positions
+    # plus the local window; duplicated key rows give large groups of equal scores.
+    cpu, state = make([3000, 500, 40000], tokens=16, heads=2, kt_tokens=64)
+    cpu.q[0].zero_()
+    cpu.q[2, 1].zero_()
+    table = cpu.block_table
+    first = cpu.k_cache[int(table[1, 0]), :, 0].clone()
+    for j in range(500 // 16):                                       # sequence 1: every key row the same
+        cpu.k_cache[int(table[1, j])] = first[:, None, :]
+    state.kt_pool, state.kt_block_table = wl.make_sparf_state(cpu, 0.125, 64).kt_pool, \
+        wl.make_sparf_state(cpu, 0.125, 64).kt_block_table
+    out, alpha, sel, own = run_and_check(cpu, state, 16, 8, "heavy ties")
+    k0 = state.k_tokens_host[0]
+    want = np.concatenate([np.arange(k0 - 8), np.arange(3000 - 8, 3000)])
+    assert np.array_equal(sel[0, 0, :k0], want) and np.array_equal(sel[0, 1, :k0], want)
+    ours, theirs = sel, own[2][:, :, :sel.shape[2]]                      # ties cut exactly as the oracle cuts them
+    assert np.array_equal(ours[0], theirs[0]) and np.array_equal(ours[1], theirs[1])
+    assert np.array_equal(ours[2, 1], theirs[2, 1])
