@@ -449,7 +449,8 @@ int instinfer_decode_step_host(void *out_host, const void *qkv_host, void *qkv_d
 namespace {
 
 struct SparfLayout {
-    size_t scores, row_ids, stats, partials, total;
+    size_t scores, row_ids, stats, rows_state, row_hist, row_cand, chunk_count, chunk_sums, partials, total;
+    size_t zeroed_bytes;      // rows_state and row_hist are adjacent and cleared before each call
     int32_t score_stride;
     SplitPlan plan;
 };
@@ -464,7 +465,14 @@ SparfLayout sparf_layout(int64_t pairs, int32_t max_seq_len, int32_t max_k)
     w.scores = 0;
     w.row_ids = w.scores + round256((size_t)pairs * w.score_stride * sizeof(float));
     w.stats = w.row_ids + round256((size_t)pairs * max_k * sizeof(int32_t));
-    w.partials = w.stats + round256((size_t)pairs * sizeof(float2));
+    const size_t chunks = (size_t)ceil_div(max_seq_len, kScoreChunk);
+    w.rows_state = w.stats + round256((size_t)pairs * sizeof(float2));
+    w.row_hist = w.rows_state + round256((size_t)pairs * sizeof(SelectRow));
+    w.row_cand = w.row_hist + round256((size_t)pairs * (kLinearBins + 1) * sizeof(unsigned));
+    w.zeroed_bytes = w.row_cand - w.rows_state;
+    w.chunk_count = w.row_cand + round256((size_t)pairs * kRowCandidates * sizeof(uint2));
+    w.chunk_sums = w.chunk_count + round256((size_t)pairs * chunks * sizeof(int32_t));
+    w.partials = w.chunk_sums + round256((size_t)pairs * chunks * sizeof(float2));
     w.total = w.partials + workspace_for(pairs, w.plan);
     return w;
 }
@@ -603,9 +611,27 @@ int instinfer_sparf_decode_attention(void *out, float *alpha, int32_t *selected,
     sp.window = local_window;
     sp.scale_log2e = scale * 1.44269504088896340736f;
 
-    sparf_scores_kernel<<<(unsigned)(pairs * score_chunks), kSparfThreads, 0, stream>>>(sp);
-    if (cudaGetLastError() != cudaSuccess) return INSTINFER_ERR_CUDA;
-    sparf_select_kernel<<<(unsigned)pairs, kSelectThreads, 0, stream>>>(sp);
+    sp.rows_state = reinterpret_cast<SelectRow *>(ws + w.rows_state);
+    sp.row_hist = reinterpret_cast<unsigned *>(ws + w.row_hist);
+    sp.row_cand = reinterpret_cast<uint2 *>(ws + w.row_cand);
+    sp.chunk_count = reinterpret_cast<int32_t *>(ws + w.chunk_count);
+    sp.chunk_sums = reinterpret_cast<float2 *>(ws + w.chunk_sums);
+
+    const unsigned chunk_grid = (unsigned)(pairs * score_chunks), row_grid = (unsigned)pairs;
+    if (cudaMemsetAsync(ws + w.rows_state, 0, w.zeroed_bytes, stream) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return INSTINFER_ERR_CUDA;
+    }
+    sparf_scores_kernel<<<chunk_grid, kSparfThreads, 0, stream>>>(sp);
+    // Steps 5-7, chunk-parallel; rows it cannot settle are redone by the single-block kernel.
+    sparf_range_kernel<<<chunk_grid, kChunkThreads, 0, stream>>>(sp);
+    sparf_hist_kernel<<<chunk_grid, kChunkThreads, 0, stream>>>(sp);
+    sparf_locate_kernel<<<row_grid, 32, 0, stream>>>(sp);
+    sparf_collect_kernel<<<chunk_grid, kChunkThreads, 0, stream>>>(sp);
+    sparf_threshold_kernel<<<row_grid, kChunkThreads, 0, stream>>>(sp);
+    sparf_compact_kernel<<<chunk_grid, kChunkThreads, 0, stream>>>(sp);
+    sparf_finish_kernel<<<row_grid, 64, 0, stream>>>(sp);
+    sparf_select_kernel<<<row_grid, kSelectThreads, 0, stream>>>(sp);
     if (cudaGetLastError() != cudaSuccess) return INSTINFER_ERR_CUDA;
 
     SparfMergeParams mp = {};

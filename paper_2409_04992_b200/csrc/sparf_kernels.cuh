@@ -24,6 +24,22 @@
 
 namespace instinfer {
 
+constexpr int kRowCandidates = 1024;     // chunk-parallel select: keys of the threshold bin kept per row
+
+// Per (sequence, head) state of the chunk-parallel selection.  Zero-initialised per call.
+struct SelectRow {
+    unsigned max_key;          // ordered key of the largest logit
+    unsigned neg_min_key;      // ~ordered key of the smallest logit (so both are atomicMax)
+    int bin;                   // linear bin holding the k-th largest
+    int above;                 // members of the bins above it
+    int n_cand;                // candidates collected from that bin
+    unsigned tau;              // exact ordered key of the k-th largest
+    int idx_cut;               // among keys equal to tau, positions <= idx_cut are taken
+    int solved;                // 0: the single-block kernel must redo this row
+    float z;                   // softmax denominator of the approximate logits
+    float top, low, bin_scale; // range of the linear bins
+};
+
 struct SparfParams {
     // cache
     __half *k_pool;
@@ -42,6 +58,12 @@ struct SparfParams {
     float *scores;             // [pairs, score_stride] approximate logits, base-2 domain
     int32_t *row_ids;          // [pairs, max_k]
     float2 *stats;             // [pairs] (alpha, number of selected rows)
+    // chunk-parallel selection (see SelectRow): all zeroed before each call
+    struct SelectRow *rows_state;   // [pairs]
+    unsigned *row_hist;        // [pairs, kLinearBins + 1]
+    uint2 *row_cand;           // [pairs, kRowCandidates] (ordered key, token index)
+    int32_t *chunk_count;      // [pairs, score_chunks] selected tokens per score chunk
+    float2 *chunk_sums;        // [pairs, score_chunks] (softmax denominator part, selected mass part)
     // outputs
     float *alpha_out;          // nullable [pairs]
     int32_t *selected;         // nullable [pairs, max_k] logical token index, ascending, -1 padded
@@ -343,6 +365,7 @@ sparf_select_kernel(const SparfParams p)
     const int pair = blockIdx.x, tid = threadIdx.x;
     const int lane = tid & 31, warp = tid >> 5;
     const int b = pair / p.heads, h = pair - b * p.heads;
+    if (p.rows_state && p.rows_state[pair].solved) return;      // done by the chunk-parallel kernels
     const int S = sparf_seq_len(p, b, tid == 0 && h == 0);
     const int k = min(S, min(max(p.k_tokens[b], 0), p.max_k));
     const int window = min(p.window, k);
@@ -553,6 +576,374 @@ sparf_select_kernel(const SparfParams p)
     mass = block_sum(mass, sh.red_f);
     if (tid == 0) {
         const float alpha = mass / z;
+        p.stats[pair] = make_float2(alpha, (float)k);
+        if (p.alpha_out) p.alpha_out[pair] = alpha;
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// Chunk-parallel selection.  The same steps as sparf_select_kernel, but every pass over the
+// scores runs as one block per (row, 2048-token chunk), so that long rows use the whole GPU:
+//   range   -> per-row min / max of the logits (two atomicMax per block)
+//   hist    -> per-row histogram over the monotone linear bins, softmax denominator parts
+//   locate  -> the bin holding the k-th largest (one warp per row)
+//   collect -> per chunk, how many tokens lie in higher bins (surely selected), and the
+//              (key, position) of the tokens inside the threshold bin
+//   thresh  -> exact threshold among those candidates, ties cut by position
+//   compact -> ordered compaction per chunk behind the prefix of the chunk counts
+//   finish  -> alpha, padding of the optional `selected` output
+// A row whose threshold bin holds more than kRowCandidates keys (many nearly equal scores)
+// is left unsolved and redone by sparf_select_kernel, which skips the solved rows.
+// One warp: among the linear bins (lane L owns bins [64 L, 64 L + 64)), the bin in which the
+// count from the top, started at `from_top`, reaches `target`; also the count above that bin.
+__device__ __forceinline__ void locate_linear_bin(const unsigned *hist, int from_top, int target, int *bin_out, int *above_out)
+{
+    const int lane = threadIdx.x & 31;
+    int mine = 0;
+    for (int j = 0; j < 64; ++j) mine += (int)hist[64 * lane + ((j + lane) & 63)];
+    int above = from_top;
+    for (int src = 31; src >= 0; --src) {
+        const int seg = __shfl_sync(0xffffffffu, mine, src);
+        if (src > lane) above += seg;
+    }
+    if (above < target && target <= above + mine) {
+        int bin = 64 * lane + 63;
+        for (; bin > 64 * lane; --bin) {
+            const int c = (int)hist[bin];
+            if (above + c >= target) break;
+            above += c;
+        }
+        *bin_out = bin;
+        *above_out = above;
+    }
+}
+
+constexpr int kChunkThreads = 256;       // 8 consecutive tokens per thread = one score chunk
+static_assert(kChunkThreads * 8 == kScoreChunk, "one thread block covers one score chunk");
+
+__device__ __forceinline__ float float_of_key(unsigned key)
+{
+    return __uint_as_float((key & 0x80000000u) ? (key & 0x7fffffffu) : ~key);
+}
+
+struct ChunkView {
+    int pair, chunk, b, h, S, k, window, i0;     // i0: first token of this thread
+    float x[8];
+};
+
+// Common prologue of the chunk kernels: indices, lengths and this thread's 8 logits.
+__device__ __forceinline__ bool load_chunk(const SparfParams &p, ChunkView &c)
+{
+    c.pair = blockIdx.x / p.score_chunks;
+    c.chunk = blockIdx.x - c.pair * p.score_chunks;
+    c.b = c.pair / p.heads;
+    c.h = c.pair - c.b * p.heads;
+    c.S = sparf_seq_len(p, c.b, false);
+    c.k = min(c.S, min(max(p.k_tokens[c.b], 0), p.max_k));
+    c.window = min(p.window, c.k);
+    c.i0 = c.chunk * kScoreChunk + threadIdx.x * 8;
+    if (c.chunk * kScoreChunk >= c.S) return false;
+#pragma unroll
+    for (int e = 0; e < 8; ++e) c.x[e] = 0.f;
+    if (c.i0 < c.S) {                              // rows are padded to whole groups of 8
+        const float4 *src = reinterpret_cast<const float4 *>(p.scores + (int64_t)c.pair * p.score_stride + c.i0);
+        const float4 a = src[0], b = src[1];
+        c.x[0] = a.x; c.x[1] = a.y; c.x[2] = a.z; c.x[3] = a.w;
+        c.x[4] = b.x; c.x[5] = b.y; c.x[6] = b.z; c.x[7] = b.w;
+    }
+    return true;
+}
+
+__device__ __forceinline__ int linear_bin(const SelectRow &row, int S, int window, int i, float x)
+{
+    return i >= S - window ? kLinearBins : min(kLinearBins - 1, (int)((x - row.low) * row.bin_scale));
+}
+
+__global__ void __launch_bounds__(kChunkThreads)
+sparf_range_kernel(const SparfParams p)
+{
+    __shared__ float sm[2][kChunkThreads / 32];
+    ChunkView c;
+    if (!load_chunk(p, c)) return;
+    float top = kMinusHuge, low = -kMinusHuge;
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+        if (c.i0 + e < c.S) {
+            top = fmaxf(top, c.x[e]);
+            low = fminf(low, c.x[e]);
+        }
+    }
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) {
+        top = fmaxf(top, __shfl_xor_sync(0xffffffffu, top, off));
+        low = fminf(low, __shfl_xor_sync(0xffffffffu, low, off));
+    }
+    if ((threadIdx.x & 31) == 0) {
+        sm[0][threadIdx.x >> 5] = top;
+        sm[1][threadIdx.x >> 5] = low;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (int w = 1; w < kChunkThreads / 32; ++w) {
+            top = fmaxf(top, sm[0][w]);
+            low = fminf(low, sm[1][w]);
+        }
+        atomicMax(&p.rows_state[c.pair].max_key, ordered_key(top));
+        atomicMax(&p.rows_state[c.pair].neg_min_key, ~ordered_key(low));
+    }
+}
+
+__global__ void __launch_bounds__(kChunkThreads)
+sparf_hist_kernel(const SparfParams p)
+{
+    __shared__ unsigned hist[kLinearBins + 1];
+    __shared__ float red[32];
+    ChunkView c;
+    if (!load_chunk(p, c)) return;
+    SelectRow row;
+    row.top = float_of_key(p.rows_state[c.pair].max_key);
+    row.low = float_of_key(~p.rows_state[c.pair].neg_min_key);
+    row.bin_scale = row.top > row.low ? (float)(kLinearBins - 1) / (row.top - row.low) : 0.f;
+    for (int t = threadIdx.x; t <= kLinearBins; t += kChunkThreads) hist[t] = 0u;
+    __syncthreads();
+    float z = 0.f;
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+        const int i = c.i0 + e;
+        if (i < c.S) {
+            z += fast_exp2(c.x[e] - row.top);
+            atomicAdd(&hist[linear_bin(row, c.S, c.window, i, c.x[e])], 1u);
+        }
+    }
+    z = block_sum(z, red);                       // its barriers also publish the histogram
+    unsigned *global_hist = p.row_hist + (int64_t)c.pair * (kLinearBins + 1);
+    for (int t = threadIdx.x; t <= kLinearBins; t += kChunkThreads)
+        if (hist[t]) atomicAdd(&global_hist[t], hist[t]);
+    if (threadIdx.x == 0) p.chunk_sums[blockIdx.x].x = z;
+}
+
+// One warp per row.
+__global__ void __launch_bounds__(32)
+sparf_locate_kernel(const SparfParams p)
+{
+    const int pair = blockIdx.x, lane = threadIdx.x;
+    const int b = pair / p.heads, h = pair - b * p.heads;
+    const int S = sparf_seq_len(p, b, lane == 0 && h == 0);
+    const int k = min(S, min(max(p.k_tokens[b], 0), p.max_k));
+    SelectRow *row = p.rows_state + pair;
+    if (k == 0) {                                // nothing is selected: no bin is "above" this one
+        if (lane == 0) {
+            row->bin = kLinearBins + 1;
+            row->solved = 1;
+        }
+        return;
+    }
+    const unsigned *hist = p.row_hist + (int64_t)pair * (kLinearBins + 1);
+    const int in_window = (int)hist[kLinearBins];
+    __shared__ int bin, above;
+    if (in_window >= k) {                        // the local window alone fills k
+        if (lane == 0) {
+            bin = kLinearBins;
+            above = 0;
+        }
+    } else {
+        locate_linear_bin(hist, in_window, k, &bin, &above);
+    }
+    __syncwarp();
+    if (lane == 0) {
+        const float top = float_of_key(row->max_key), low = float_of_key(~row->neg_min_key);
+        float z = 0.f;
+        const int chunks = (S + kScoreChunk - 1) / kScoreChunk;
+        for (int c = 0; c < chunks; ++c) z += p.chunk_sums[(int64_t)pair * p.score_chunks + c].x;   // fixed order
+        row->top = top;
+        row->low = low;
+        row->bin_scale = top > low ? (float)(kLinearBins - 1) / (top - low) : 0.f;
+        row->z = z;
+        row->bin = bin;
+        row->above = above;
+        if (bin == kLinearBins) {
+            row->tau = 0xffffffffu;
+            row->idx_cut = 0x7fffffff;
+            row->solved = 1;
+        }
+    }
+}
+
+__global__ void __launch_bounds__(kChunkThreads)
+sparf_collect_kernel(const SparfParams p)
+{
+    __shared__ int red[32];
+    ChunkView c;
+    if (!load_chunk(p, c)) return;
+    SelectRow *state = p.rows_state + c.pair;
+    const SelectRow row = *state;
+    int sure = 0;
+    if (row.bin <= kLinearBins) {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            const int i = c.i0 + e;
+            if (i < c.S) {
+                const int bin = linear_bin(row, c.S, c.window, i, c.x[e]);
+                if (bin > row.bin || (bin == kLinearBins && row.bin == kLinearBins)) {
+                    ++sure;
+                } else if (bin == row.bin) {
+                    const int at = atomicAdd(&state->n_cand, 1);
+                    if (at < kRowCandidates)
+                        p.row_cand[(int64_t)c.pair * kRowCandidates + at] = make_uint2(ordered_key(c.x[e]), (unsigned)i);
+                }
+            }
+        }
+    }
+    sure = block_sum(sure, red);
+    if (threadIdx.x == 0) p.chunk_count[blockIdx.x] = sure;
+}
+
+// One block per row: exact threshold among the collected candidates.
+__global__ void __launch_bounds__(kChunkThreads)
+sparf_threshold_kernel(const SparfParams p)
+{
+    __shared__ unsigned keys[kRowCandidates];
+    __shared__ int where[kRowCandidates];
+    __shared__ unsigned sh_tau;
+    __shared__ int sh_take, sh_cut;
+    const int pair = blockIdx.x, tid = threadIdx.x;
+    const int b = pair / p.heads;
+    SelectRow *state = p.rows_state + pair;
+    if (state->solved) return;
+    const int S = sparf_seq_len(p, b, false);
+    const int k = min(S, min(max(p.k_tokens[b], 0), p.max_k));
+    const int n = state->n_cand, need = k - state->above;
+    if (n > kRowCandidates || need < 1 || need > n) return;      // left to the single-block kernel
+    for (int t = tid; t < n; t += kChunkThreads) {
+        const uint2 c = p.row_cand[(int64_t)pair * kRowCandidates + t];
+        keys[t] = c.x;
+        where[t] = (int)c.y;
+    }
+    __syncthreads();
+    for (int t = tid; t < n; t += kChunkThreads) {
+        const unsigned mine = keys[t];
+        int greater = 0, equal = 0;
+        for (int j = 0; j < n; ++j) {
+            greater += keys[j] > mine;
+            equal += keys[j] == mine;
+        }
+        if (greater < need && need <= greater + equal) {         // all holders of this key agree
+            sh_tau = mine;
+            sh_take = need - greater;
+        }
+    }
+    __syncthreads();
+    const unsigned tau = sh_tau;
+    const int take = sh_take;
+    for (int t = tid; t < n; t += kChunkThreads) {               // the take-th smallest position among ties
+        if (keys[t] == tau) {
+            int before = 0;
+            for (int j = 0; j < n; ++j) before += keys[j] == tau && where[j] < where[t];
+            if (before == take - 1) sh_cut = where[t];
+        }
+    }
+    __syncthreads();
+    const int cut = sh_cut;
+    for (int t = tid; t < n; t += kChunkThreads) {
+        if (keys[t] > tau || (keys[t] == tau && where[t] <= cut))
+            atomicAdd(&p.chunk_count[(int64_t)pair * p.score_chunks + where[t] / kScoreChunk], 1);
+    }
+    if (tid == 0) {
+        state->tau = tau;
+        state->idx_cut = cut;
+        state->solved = 1;
+    }
+}
+
+__global__ void __launch_bounds__(kChunkThreads)
+sparf_compact_kernel(const SparfParams p)
+{
+    __shared__ int warp_total[kChunkThreads / 32];
+    __shared__ int sh_offset;
+    __shared__ float red[32];
+    ChunkView c;
+    if (!load_chunk(p, c)) return;
+    const SelectRow row = p.rows_state[c.pair];
+    if (!row.solved || row.bin > kLinearBins) return;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (warp == 0) {                             // tokens selected in the chunks before this one
+        int before = 0;
+        for (int j = lane; j < c.chunk; j += 32) before += p.chunk_count[(int64_t)c.pair * p.score_chunks + j];
+#pragma unroll
+        for (int off = 16; off >= 1; off >>= 1) before += __shfl_xor_sync(0xffffffffu, before, off);
+        if (lane == 0) sh_offset = before;
+    }
+    bool take[8];
+    int mine = 0;
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+        const int i = c.i0 + e;
+        take[e] = false;
+        if (i < c.S) {
+            const int bin = linear_bin(row, c.S, c.window, i, c.x[e]);
+            if (bin > row.bin || (bin == kLinearBins && row.bin == kLinearBins)) {
+                take[e] = true;
+            } else if (bin == row.bin) {
+                const unsigned key = ordered_key(c.x[e]);
+                take[e] = key > row.tau || (key == row.tau && i <= row.idx_cut);
+            }
+            mine += (int)take[e];
+        }
+    }
+    int incl = mine;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const int up = __shfl_up_sync(0xffffffffu, incl, off);
+        if (lane >= off) incl += up;
+    }
+    if (lane == 31) warp_total[warp] = incl;
+    __syncthreads();
+    int pos = sh_offset + incl - mine;
+    for (int w = 0; w < warp; ++w) pos += warp_total[w];
+    const int T = p.block_tokens;
+    const int32_t *table_row = p.block_table + (int64_t)c.b * p.max_blocks_per_seq;
+    int32_t *rows = p.row_ids + (int64_t)c.pair * p.max_k;
+    int32_t *sel = p.selected ? p.selected + (int64_t)c.pair * p.max_k : nullptr;
+    float mass = 0.f;
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+        if (take[e]) {
+            const int i = c.i0 + e;
+            const int blk = i / T, slot = i - blk * T;
+            const int phys = table_row[blk];
+            const bool ok = phys >= 0 && (int64_t)phys < p.num_phys_blocks;
+            if (!ok && p.status) atomicOr(p.status, kFlagBlockRange);
+            if (pos < p.max_k) {                 // always true for a consistent count; guards the buffer
+                rows[pos] = ok ? (phys * p.heads + c.h) * T + slot : 0;
+                if (sel) sel[pos] = i;
+            }
+            ++pos;
+            mass += fast_exp2(c.x[e] - row.top);
+        }
+    }
+    mass = block_sum(mass, red);
+    if (threadIdx.x == 0) p.chunk_sums[blockIdx.x].y = mass;
+}
+
+__global__ void __launch_bounds__(64)
+sparf_finish_kernel(const SparfParams p)
+{
+    const int pair = blockIdx.x, tid = threadIdx.x;
+    const int b = pair / p.heads;
+    const SelectRow row = p.rows_state[pair];
+    if (!row.solved) return;
+    const int S = sparf_seq_len(p, b, false);
+    const int k = min(S, min(max(p.k_tokens[b], 0), p.max_k));
+    if (p.selected)
+        for (int t = k + tid; t < p.max_k; t += 64) p.selected[(int64_t)pair * p.max_k + t] = -1;
+    if (tid == 0) {
+        float alpha = 0.f;
+        if (k > 0) {
+            float mass = 0.f;
+            const int chunks = (S + kScoreChunk - 1) / kScoreChunk;
+            for (int c = 0; c < chunks; ++c) mass += p.chunk_sums[(int64_t)pair * p.score_chunks + c].y;   // fixed order
+            alpha = mass / row.z;
+        }
         p.stats[pair] = make_float2(alpha, (float)k);
         if (p.alpha_out) p.alpha_out[pair] = alpha;
     }
