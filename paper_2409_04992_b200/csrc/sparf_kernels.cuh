@@ -861,6 +861,8 @@ sparf_compact_kernel(const SparfParams p)
     __shared__ int warp_total[kChunkThreads / 32];
     __shared__ int sh_offset;
     __shared__ float red[32];
+    __shared__ int list_pos[kScoreChunk];        // positions of this chunk's selected tokens, ascending
+    __shared__ float list_x[kScoreChunk];        // and their logits
     ChunkView c;
     if (!load_chunk(p, c)) return;
     const SelectRow row = p.rows_state[c.pair];
@@ -873,23 +875,18 @@ sparf_compact_kernel(const SparfParams p)
         for (int off = 16; off >= 1; off >>= 1) before += __shfl_xor_sync(0xffffffffu, before, off);
         if (lane == 0) sh_offset = before;
     }
-    bool take[8];
-    int mine = 0;
+    // Which of this thread's 8 tokens are selected (cheap, branch-free), as a bit mask.
+    unsigned take = 0u;
 #pragma unroll
     for (int e = 0; e < 8; ++e) {
         const int i = c.i0 + e;
-        take[e] = false;
-        if (i < c.S) {
-            const int bin = linear_bin(row, c.S, c.window, i, c.x[e]);
-            if (bin > row.bin || (bin == kLinearBins && row.bin == kLinearBins)) {
-                take[e] = true;
-            } else if (bin == row.bin) {
-                const unsigned key = ordered_key(c.x[e]);
-                take[e] = key > row.tau || (key == row.tau && i <= row.idx_cut);
-            }
-            mine += (int)take[e];
-        }
+        const int bin = linear_bin(row, c.S, c.window, i, c.x[e]);
+        const unsigned key = ordered_key(c.x[e]);
+        const bool sure = bin > row.bin || (bin == kLinearBins && row.bin == kLinearBins);
+        const bool tied = bin == row.bin && (key > row.tau || (key == row.tau && i <= row.idx_cut));
+        take |= (unsigned)(i < c.S && (sure || tied)) << e;
     }
+    const int mine = __popc(take);
     int incl = mine;
 #pragma unroll
     for (int off = 1; off < 32; off <<= 1) {
@@ -898,28 +895,38 @@ sparf_compact_kernel(const SparfParams p)
     }
     if (lane == 31) warp_total[warp] = incl;
     __syncthreads();
-    int pos = sh_offset + incl - mine;
-    for (int w = 0; w < warp; ++w) pos += warp_total[w];
+    int local = incl - mine, chunk_total = 0;
+    for (int w = 0; w < kChunkThreads / 32; ++w) {
+        if (w < warp) local += warp_total[w];
+        chunk_total += warp_total[w];
+    }
+    // Dense list of the selected tokens in shared memory: the costly part below then runs
+    // once per selected token instead of once per token slot of every warp.
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+        if (take >> e & 1u) {
+            list_pos[local] = c.i0 + e;
+            list_x[local] = c.x[e];
+            ++local;
+        }
+    }
+    __syncthreads();
     const int T = p.block_tokens;
     const int32_t *table_row = p.block_table + (int64_t)c.b * p.max_blocks_per_seq;
     int32_t *rows = p.row_ids + (int64_t)c.pair * p.max_k;
     int32_t *sel = p.selected ? p.selected + (int64_t)c.pair * p.max_k : nullptr;
     float mass = 0.f;
-#pragma unroll
-    for (int e = 0; e < 8; ++e) {
-        if (take[e]) {
-            const int i = c.i0 + e;
-            const int blk = i / T, slot = i - blk * T;
-            const int phys = table_row[blk];
-            const bool ok = phys >= 0 && (int64_t)phys < p.num_phys_blocks;
-            if (!ok && p.status) atomicOr(p.status, kFlagBlockRange);
-            if (pos < p.max_k) {                 // always true for a consistent count; guards the buffer
-                rows[pos] = ok ? (phys * p.heads + c.h) * T + slot : 0;
-                if (sel) sel[pos] = i;
-            }
-            ++pos;
-            mass += fast_exp2(c.x[e] - row.top);
+    for (int t = threadIdx.x; t < chunk_total; t += kChunkThreads) {
+        const int i = list_pos[t], pos = sh_offset + t;
+        const int blk = i / T, slot = i - blk * T;
+        const int phys = table_row[blk];
+        const bool ok = phys >= 0 && (int64_t)phys < p.num_phys_blocks;
+        if (!ok && p.status) atomicOr(p.status, kFlagBlockRange);
+        if (pos < p.max_k) {                     // always true for a consistent count; guards the buffer
+            rows[pos] = ok ? (phys * p.heads + c.h) * T + slot : 0;
+            if (sel) sel[pos] = i;
         }
+        mass += fast_exp2(list_x[t] - row.top);
     }
     mass = block_sum(mass, red);
     if (threadIdx.x == 0) p.chunk_sums[blockIdx.x].y = mass;
