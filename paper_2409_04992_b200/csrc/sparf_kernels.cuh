@@ -6,11 +6,14 @@
 //                         added to the running V sum that gives the mean value vector.
 //   sparf_scores_kernel   step 1 (the r largest |q_d|) and steps 2-4 without the softmax
 //                         normalisation: approximate logits from the embedding-major copy.
-//   sparf_select_kernel   softmax statistics of the approximate logits, steps 5-7: the k
-//                         largest scores with the last l tokens forced in (a monotone
-//                         linear histogram finds the threshold bin, its members are
-//                         resolved exactly; ties to the lower index), alpha, and the
-//                         ascending list of selected rows as physical row ids.
+//   steps 5-7             softmax statistics of the approximate logits, the k largest scores
+//                         with the last l tokens forced in (a monotone linear histogram finds
+//                         the threshold bin, its members are resolved exactly; ties to the
+//                         lower position), alpha, and the ascending list of selected rows as
+//                         physical row ids.  Run chunk-parallel by sparf_range / hist /
+//                         locate / collect / threshold / compact / finish kernels; rows with
+//                         too many nearly equal scores fall back to sparf_select_kernel,
+//                         which does the same steps with one block per row.
 //   (steps 8-10 run in decode_attn_split_kernel<Rows::kGathered>)
 //   sparf_merge_kernel    log-sum-exp merge of the chunk partials and step 11:
 //                         out = alpha * attended + (1 - alpha) * v_sum / S.
