@@ -133,6 +133,7 @@ sparf_scores_kernel(const SparfParams p)
     __shared__ float sm_q[kHeadDim];        // q of the selected dims, in rank order
     __shared__ int sm_dim[kHeadDim];
     __shared__ float sm_red[2][kSparfThreads / 32];
+    __shared__ bool sm_kept[kHeadDim];
     const int pair = blockIdx.x / p.score_chunks, d = threadIdx.x;
     const int b = pair / p.heads, h = pair - b * p.heads;
     const int len = sparf_seq_len(p, b, false);
@@ -154,22 +155,23 @@ sparf_scores_kernel(const SparfParams p)
         sm_dim[rank] = d;
         sm_q[rank] = qd;
     }
-    // |q|_1 and |q_I|_1
-    float all = sm_abs[d], sel = kept ? sm_abs[d] : 0.f;
-#pragma unroll
-    for (int off = 16; off >= 1; off >>= 1) {
-        all += __shfl_xor_sync(0xffffffffu, all, off);
-        sel += __shfl_xor_sync(0xffffffffu, sel, off);
-    }
-    if ((d & 31) == 0) {
-        sm_red[0][d >> 5] = all;
-        sm_red[1][d >> 5] = sel;
+    // |q|_1 and |q_I|_1.  The top-k of step 6 is decided on the fp32 logits computed below, so
+    // their arithmetic is kept simple enough to be restated elsewhere bit for bit: both sums
+    // run over ascending d in fp32, the temperature uses IEEE division and square root, and
+    // each logit is the fp32 FMA chain over the kept dims in rank order times that constant.
+    sm_kept[d] = kept;
+    __syncthreads();
+    if (d == 0) {
+        float all = 0.f, sel = 0.f;
+        for (int e = 0; e < kHeadDim; ++e) {
+            all += sm_abs[e];
+            if (sm_kept[e]) sel += sm_abs[e];
+        }
+        const float ratio = all > 0.f ? sel / all : 1.f;
+        sm_red[0][0] = p.scale_log2e / sqrtf(ratio);
     }
     __syncthreads();
-    all = sm_red[0][0] + sm_red[0][1] + sm_red[0][2] + sm_red[0][3];
-    sel = sm_red[1][0] + sm_red[1][1] + sm_red[1][2] + sm_red[1][3];
-    const float ratio = all > 0.f ? sel / all : 1.f;
-    const float approx_scale = p.scale_log2e * rsqrtf(ratio);
+    const float approx_scale = sm_red[0][0];
 
     // Steps 2-4: one thread per group of 8 consecutive tokens (one 16-byte load per selected
     // dim; kt_block_tokens is a multiple of 8, so a group never straddles a block).  The loads
@@ -194,11 +196,13 @@ sparf_scores_kernel(const SparfParams p)
                 }
 #pragma unroll
                 for (int u = 0; u < 8; ++u) {
-                    const float qv = t0 + u < p.r ? sm_q[t0 + u] : 0.f;
-                    float kf[8];
-                    unpack8(raw[u], kf);
+                    if (t0 + u < p.r) {                            // uniform; extra loads are ignored
+                        const float qv = sm_q[t0 + u];
+                        float kf[8];
+                        unpack8(raw[u], kf);
 #pragma unroll
-                    for (int e = 0; e < 8; ++e) dot[e] = fmaf(qv, kf[e], dot[e]);
+                        for (int e = 0; e < 8; ++e) dot[e] = fmaf(qv, kf[e], dot[e]);
+                    }
                 }
             }
         } else if (p.status) {

@@ -1,10 +1,10 @@
 """GPU parity of the sparse (SparF, Algorithm 1) path against its CPU oracle.
 
-Floating point decides two integer sets here (the kept query dims and the kept tokens).  The
-dims are decided on exact fp16 magnitudes on both sides, so they must agree exactly.  The
-token scores are fp32 on the GPU and fp64 in the oracle, so near-ties may be cut differently:
-the GPU's set is checked to be a valid top-k of the oracle's scores up to that rounding, and
-the oracle then recomputes the output for the GPU's set, which is compared element-wise."""
+Floating point decides two integer sets here (the kept query dims and the kept tokens).  Both
+sides take each decision in the same precision: the dims on exact fp16 magnitudes, the tokens
+on binary32 logits computed by the rule stated in the oracle's header (ties to the lower
+position).  The kept sets must therefore agree exactly; outputs and alpha are then compared
+with the usual tolerances against the oracle's fp64 arithmetic."""
 import math
 
 import numpy as np
@@ -17,7 +17,6 @@ from tests import gpu_util as gu
 
 pytestmark = pytest.mark.gpu
 
-SCORE_RTOL = 1e-4          # relative slack on an approximate weight at the selection threshold
 ALPHA_ATOL = 2e-5
 
 
@@ -54,7 +53,7 @@ def gpu_sparf(case, state, r, l, do_append=True, max_k=None):
     return out.view.cpu(), alpha.view.cpu().numpy(), sel.view.cpu().numpy(), int(flags.item())
 
 
-def oracle_sparf(cpu, state, r, l, do_append=True, given=None, want_weights=False):
+def oracle_sparf(cpu, state, r, l, do_append=True, want_weights=False):
     k, v, kt = cpu.k_cache.numpy(), cpu.v_cache.numpy(), state.kt_pool.numpy()
     v_sum = state.v_sum.numpy()
     lens = np.array(cpu.seq_lens_host, dtype=np.int32)
@@ -63,13 +62,12 @@ def oracle_sparf(cpu, state, r, l, do_append=True, given=None, want_weights=Fals
         capi.sparf_append(k, v, kt, v_sum, cpu.k_new.numpy(), cpu.v_new.numpy(), lens, table,
                           kt_block_table=kt_table)
     return capi.sparf_attention(cpu.q.numpy(), k, v, kt, v_sum, lens, np.array(state.k_tokens_host),
-                                table, r, l, cpu.scale, given=given, want_weights=want_weights,
+                                table, r, l, cpu.scale, want_weights=want_weights,
                                 kt_block_table=kt_table)
 
 
-def check_selection(sel_gpu, weights, lens, ks, l):
-    """The GPU's J must be a valid top-k of the oracle's approximate weights (up to rounding)."""
-    differing = 0
+def check_structure(sel_gpu, lens, ks, l):
+    """Shape of the kept sets: size, order, range, window membership, -1 padding."""
     for b, S in enumerate(lens):
         k = min(ks[b], S)
         window = min(l, k)
@@ -78,36 +76,26 @@ def check_selection(sel_gpu, weights, lens, ks, l):
             assert np.all(sel_gpu[b, h, k:] == -1)
             assert np.all(np.diff(J) > 0) and (k == 0 or (J[0] >= 0 and J[-1] < S))
             assert np.all(np.isin(np.arange(S - window, S), J))
-            w = weights[b, h, :S].copy()
-            w[S - window:] = np.inf
-            chosen = np.zeros(S, dtype=bool)
-            chosen[J] = True
-            if k == 0 or k == S:
-                continue
-            lowest_in, highest_out = w[chosen].min(), w[~chosen].max()
-            assert lowest_in >= highest_out * (1 - SCORE_RTOL), (b, h, lowest_in, highest_out)
-            differing += lowest_in < highest_out
-    return differing
 
 
 def run_and_check(cpu, state, r, l, what):
     dev, dstate = gu.to_device(cpu), dev_state(state)
     out, alpha, sel, flags = gpu_sparf(dev, dstate, r, l)
     assert flags == 0
-    own = oracle_sparf(cpu, state, r, l, want_weights=True)          # appends into the CPU copies
+    want, want_alpha, want_sel, weights = oracle_sparf(cpu, state, r, l, want_weights=True)   # appends into the CPU copies
     # the append: both K layouts, V and the running sum, bit for bit
     assert np.array_equal(gu.bits(dev.k_cache), gu.bits(cpu.k_cache))
     assert np.array_equal(gu.bits(dev.v_cache), gu.bits(cpu.v_cache))
     assert np.array_equal(gu.bits(dstate.kt_pool), gu.bits(state.kt_pool))
     assert np.array_equal(dstate.v_sum.cpu().numpy().view(np.uint32), state.v_sum.numpy().view(np.uint32))
     lens, ks = cpu.seq_lens_host, state.k_tokens_host
-    cut_differently = check_selection(sel, own[3], lens, ks, l)
-    pairs = len(lens) * sel.shape[1]
-    assert cut_differently <= max(1, pairs // 20), f"{what}: {cut_differently} of {pairs} selections differ"
-    want, want_alpha, _, _ = oracle_sparf(cpu, state, r, l, do_append=False, given=sel)
+    check_structure(sel, lens, ks, l)
+    width = want_sel.shape[2]
+    assert np.array_equal(sel[:, :, :width], want_sel), f"{what}: kept sets differ"
+    assert np.all(sel[:, :, width:] == -1)
     gu.assert_close(out, want, what=what)
     assert np.abs(alpha - want_alpha).max() <= ALPHA_ATOL
-    return out, alpha, sel, own
+    return out, alpha, sel, (want, want_alpha, want_sel, weights)
 
 
 @pytest.mark.parametrize("tokens", [8, 16, 64])
