@@ -35,6 +35,9 @@ def _load() -> ctypes.CDLL:
         lib.oracle_sparf_append.restype = ctypes.c_int
         lib.oracle_sparf_append.argtypes = [ptr, ptr, ptr, ptr, ptr, ptr, ptr, ptr, i32, i32, i64,
                                             ptr, i32, i32, i64, i32, i32, i32]
+        lib.oracle_sparf_append_bulk.restype = ctypes.c_int
+        lib.oracle_sparf_append_bulk.argtypes = [ptr, ptr, ptr, ptr, ptr, ptr, ptr, ptr, ptr, i32, i32,
+                                                 i64, ptr, i32, i32, i64, i32, i32, i32, i32]
         lib.oracle_sparf_attention.restype = ctypes.c_int
         lib.oracle_sparf_attention.argtypes = [ptr, ptr, ptr, i64, ptr, ptr, i64, ptr, ptr, ptr, ptr,
                                                ptr, ptr, ptr, ptr, i32, i32, i64, ptr, i32, i32, i64,
@@ -172,6 +175,27 @@ def sparf_append(k_pool: np.ndarray, v_pool: np.ndarray, kt_pool: np.ndarray, v_
                                      _p(table), max_blocks, kb.shape[2], kb.shape[0],
                                      _p(kt_table), kt_max_blocks, ktb.shape[3], ktb.shape[0],
                                      batch, heads, head_dim)
+    if rc:
+        raise OracleError(rc)
+
+
+def sparf_append_bulk(k_pool: np.ndarray, v_pool: np.ndarray, kt_pool: np.ndarray, v_sum: np.ndarray,
+                      k_new: np.ndarray, v_new: np.ndarray, seq_lens: np.ndarray, new_lens: np.ndarray,
+                      block_table: np.ndarray, kt_block_table: Optional[np.ndarray] = None) -> None:
+    """In-place bulk append for the SparF state; k_new, v_new are [B,N,H,D]."""
+    kb, vb, ktb = _bits(k_pool, True), _bits(v_pool, True), _bits(kt_pool, True)
+    kn, vn = _bits(np.ascontiguousarray(k_new)), _bits(np.ascontiguousarray(v_new))
+    if v_sum.dtype != np.float32 or not v_sum.flags.c_contiguous:
+        raise TypeError("v_sum must be contiguous float32")
+    batch, max_new, heads, head_dim = kn.shape
+    lens = np.ascontiguousarray(seq_lens, dtype=np.int32)
+    news = np.ascontiguousarray(new_lens, dtype=np.int32)
+    table, max_blocks = _table(block_table, batch)
+    kt_table, kt_max_blocks = _table(block_table if kt_block_table is None else kt_block_table, batch)
+    rc = _load().oracle_sparf_append_bulk(_p(kb), _p(vb), _p(ktb), _p(v_sum), _p(kn), _p(vn), _p(lens),
+                                          _p(news), _p(table), max_blocks, kb.shape[2], kb.shape[0],
+                                          _p(kt_table), kt_max_blocks, ktb.shape[3], ktb.shape[0],
+                                          batch, max_new, heads, head_dim)
     if rc:
         raise OracleError(rc)
 

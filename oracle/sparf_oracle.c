@@ -120,6 +120,53 @@ int oracle_sparf_append(uint16_t *k_pool, uint16_t *v_pool, uint16_t *kt_pool, f
     return 0;
 }
 
+/*
+ * Bulk append for the SparF state (prefill, Sec. IV-D): new_lens[b] tokens per sequence from
+ * token-major k_new / v_new [batch][max_new][heads][head_dim] go to logical positions
+ * seq_lens[b]-new_lens[b] .. seq_lens[b]-1 of K, V and the embedding-major copy, and each is
+ * added to v_sum in token order with one fp32 rounding per addition.
+ */
+int oracle_sparf_append_bulk(uint16_t *k_pool, uint16_t *v_pool, uint16_t *kt_pool, float *v_sum,
+                             const uint16_t *k_new, const uint16_t *v_new,
+                             const int32_t *seq_lens, const int32_t *new_lens,
+                             const int32_t *block_table, int32_t max_blocks_per_seq,
+                             int32_t block_tokens, int64_t num_phys_blocks,
+                             const int32_t *kt_block_table, int32_t kt_max_blocks_per_seq,
+                             int32_t kt_block_tokens, int64_t num_kt_blocks,
+                             int32_t batch, int32_t max_new, int32_t heads, int32_t head_dim)
+{
+    if (batch < 0 || heads <= 0 || head_dim <= 0 || block_tokens <= 0 || max_blocks_per_seq <= 0 ||
+        num_phys_blocks <= 0 || block_table == NULL || kt_block_table == NULL || max_new < 0 ||
+        kt_block_tokens <= 0 || kt_max_blocks_per_seq <= 0 || num_kt_blocks <= 0)
+        return -1;
+    const paged_geometry g = {block_table, max_blocks_per_seq, block_tokens, heads, head_dim,
+                              num_phys_blocks};
+    const paged_geometry gt = {kt_block_table, kt_max_blocks_per_seq, kt_block_tokens, heads,
+                               head_dim, num_kt_blocks};
+    for (int32_t b = 0; b < batch; ++b) {
+        const int32_t L = seq_lens[b], n = new_lens[b];
+        if (L < 0 || (int64_t)L > (int64_t)max_blocks_per_seq * block_tokens ||
+            (int64_t)L > (int64_t)kt_max_blocks_per_seq * kt_block_tokens || n < 0 || n > max_new || n > L)
+            return -2;
+        for (int32_t t = 0; t < n; ++t) {
+            const int32_t pos = L - n + t;
+            for (int32_t h = 0; h < heads; ++h) {
+                const int64_t base = block_base(&g, b, h, pos);
+                if (base < 0 || kt_offset(&gt, b, h, 0, pos) < 0) return -3;
+                const int64_t src = ((((int64_t)b * max_new + t) * heads) + h) * head_dim;
+                const int64_t sum = ((int64_t)b * heads + h) * head_dim;
+                for (int32_t d = 0; d < head_dim; ++d) {
+                    k_pool[base + (int64_t)(pos % block_tokens) * head_dim + d] = k_new[src + d];
+                    v_pool[base + (int64_t)(pos % block_tokens) * head_dim + d] = v_new[src + d];
+                    kt_pool[kt_offset(&gt, b, h, d, pos)] = k_new[src + d];
+                    v_sum[sum + d] = (float)((double)v_sum[sum + d] + widen(v_new[src + d]));
+                }
+            }
+        }
+    }
+    return 0;
+}
+
 typedef struct {
     double key;
     int32_t index;
