@@ -225,6 +225,22 @@ int instinfer_sparf_append(void *k_pool, void *v_pool, void *kt_pool, float *v_s
                            int32_t *status_flags, void *cuda_stream);
 
 /*
+ * Bulk form of instinfer_sparf_append for the prefill phase (Sec. IV-D): new_lens[b] tokens
+ * per sequence from token-major k_new / v_new [batch, max_new, heads, head_dim], as in
+ * instinfer_kv_append_bulk; v_sum receives the tokens in order, one fp32 rounding each, so
+ * the result equals that of appending them one by one.
+ */
+int instinfer_sparf_append_bulk(void *k_pool, void *v_pool, void *kt_pool, float *v_sum,
+                                const void *k_new, const void *v_new, const int32_t *seq_lens,
+                                const int32_t *new_lens,
+                                const int32_t *block_table, int32_t max_blocks_per_seq,
+                                int32_t block_tokens, int64_t num_phys_blocks,
+                                const int32_t *kt_block_table, int32_t kt_max_blocks_per_seq,
+                                int32_t kt_block_tokens, int64_t num_kt_blocks,
+                                int32_t batch, int32_t max_new, int32_t heads, int32_t head_dim,
+                                int32_t *status_flags, void *cuda_stream);
+
+/*
  * Algorithm 1 per (sequence, head), S = seq_lens[b]:
  *   1     I = the r dims of largest |q_d| (ties: lower d)
  *   2-4   approximate weights s^ = softmax_i(q_I . K^T[I, i] * scale / sqrt(|q_I|_1 / |q|_1)),

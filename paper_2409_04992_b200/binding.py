@@ -61,6 +61,9 @@ def load() -> ctypes.CDLL:
         lib.instinfer_sparf_append.restype = ctypes.c_int
         lib.instinfer_sparf_append.argtypes = [ptr, ptr, ptr, ptr, ptr, ptr, ptr, ptr, i32, i32, i64,
                                                ptr, i32, i32, i64, i32, i32, i32, ptr, ptr]
+        lib.instinfer_sparf_append_bulk.restype = ctypes.c_int
+        lib.instinfer_sparf_append_bulk.argtypes = [ptr, ptr, ptr, ptr, ptr, ptr, ptr, ptr, ptr, i32, i32,
+                                                    i64, ptr, i32, i32, i64, i32, i32, i32, i32, ptr, ptr]
         lib.instinfer_sparf_decode_attention.restype = ctypes.c_int
         lib.instinfer_sparf_decode_attention.argtypes = [ptr, ptr, ptr, ptr, ptr, ptr, ptr, ptr, ptr,
                                                          ptr, ptr, i32, i32, i32, i32, i32, i64,
@@ -245,6 +248,20 @@ def sparf_append(k_pool: torch.Tensor, v_pool: torch.Tensor, kt_pool: torch.Tens
         _ptr(seq_lens), _ptr(block_table), block_table.shape[1], k_pool.shape[2], k_pool.shape[0],
         _ptr(kt_block_table), kt_block_table.shape[1], kt_pool.shape[3], kt_pool.shape[0],
         batch, heads, head_dim, _ptr(status_flags), _stream(stream)))
+
+
+def sparf_append_bulk(k_pool: torch.Tensor, v_pool: torch.Tensor, kt_pool: torch.Tensor,
+                      v_sum: torch.Tensor, k_new: torch.Tensor, v_new: torch.Tensor,
+                      seq_lens: torch.Tensor, new_lens: torch.Tensor, block_table: torch.Tensor,
+                      kt_block_table: torch.Tensor, status_flags: Optional[torch.Tensor] = None,
+                      stream: Optional[torch.cuda.Stream] = None) -> None:
+    """instinfer_sparf_append_bulk: k_new, v_new are [B, max_new, H, D] (token-major)."""
+    batch, max_new, heads, head_dim = k_new.shape
+    _check(load().instinfer_sparf_append_bulk(
+        _ptr(k_pool), _ptr(v_pool), _ptr(kt_pool), _ptr(v_sum), _ptr(k_new), _ptr(v_new),
+        _ptr(seq_lens), _ptr(new_lens), _ptr(block_table), block_table.shape[1], k_pool.shape[2],
+        k_pool.shape[0], _ptr(kt_block_table), kt_block_table.shape[1], kt_pool.shape[3],
+        kt_pool.shape[0], batch, max_new, heads, head_dim, _ptr(status_flags), _stream(stream)))
 
 
 def sparf_workspace_bytes(batch: int, heads: int, head_dim: int, max_seq_len: int, max_k: int) -> int:

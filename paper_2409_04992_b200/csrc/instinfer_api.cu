@@ -530,6 +530,54 @@ int instinfer_sparf_append(void *k_pool, void *v_pool, void *kt_pool, float *v_s
     return cudaGetLastError() == cudaSuccess ? INSTINFER_OK : INSTINFER_ERR_CUDA;
 }
 
+int instinfer_sparf_append_bulk(void *k_pool, void *v_pool, void *kt_pool, float *v_sum,
+                                const void *k_new, const void *v_new, const int32_t *seq_lens,
+                                const int32_t *new_lens, const int32_t *block_table,
+                                int32_t max_blocks_per_seq, int32_t block_tokens,
+                                int64_t num_phys_blocks, const int32_t *kt_block_table,
+                                int32_t kt_max_blocks_per_seq, int32_t kt_block_tokens,
+                                int64_t num_kt_blocks, int32_t batch, int32_t max_new,
+                                int32_t heads, int32_t head_dim, int32_t *status_flags,
+                                void *cuda_stream)
+{
+    if (!sparf_sizes_ok(batch, heads, head_dim, block_tokens, max_blocks_per_seq, num_phys_blocks) ||
+        kt_block_tokens <= 0 || kt_max_blocks_per_seq <= 0 || num_kt_blocks <= 0 || max_new < 0)
+        return INSTINFER_ERR_INVALID_ARG;
+    if (head_dim != kHeadDim || block_tokens % 8 != 0 || kt_block_tokens % 8 != 0)
+        return INSTINFER_ERR_UNSUPPORTED;
+    if (batch == 0 || max_new == 0) return INSTINFER_OK;
+    if (!usable(kt_pool) || !usable(v_sum) || block_table == nullptr || kt_block_table == nullptr)
+        return INSTINFER_ERR_INVALID_ARG;
+    // K and V rows: the ordinary bulk append on the paged pools.
+    const int rc = instinfer_kv_append_bulk(k_pool, v_pool, k_new, v_new, seq_lens, new_lens, block_table,
+                                            max_blocks_per_seq, block_tokens, num_phys_blocks, batch,
+                                            max_new, heads, head_dim, 0, status_flags, cuda_stream);
+    if (rc != INSTINFER_OK) return rc;
+    SparfBulkParams q = {};
+    SparfParams &p = q.base;
+    p.kt_pool = static_cast<__half *>(kt_pool);
+    p.v_sum = v_sum;
+    p.k_new = static_cast<const __half *>(k_new);
+    p.v_new = static_cast<const __half *>(v_new);
+    p.seq_lens = seq_lens;
+    p.block_table = block_table;
+    p.kt_block_table = kt_block_table;
+    p.status = status_flags;
+    p.num_phys_blocks = num_phys_blocks;
+    p.num_kt_blocks = num_kt_blocks;
+    p.batch = batch;
+    p.heads = heads;
+    p.block_tokens = block_tokens;
+    p.max_blocks_per_seq = max_blocks_per_seq;
+    p.kt_block_tokens = kt_block_tokens;
+    p.kt_max_blocks_per_seq = kt_max_blocks_per_seq;
+    q.new_lens = new_lens;
+    q.max_new = max_new;
+    sparf_append_bulk_kernel<<<(unsigned)((int64_t)batch * heads), kSparfThreads, 0,
+                               static_cast<cudaStream_t>(cuda_stream)>>>(q);
+    return cudaGetLastError() == cudaSuccess ? INSTINFER_OK : INSTINFER_ERR_CUDA;
+}
+
 size_t instinfer_sparf_workspace_bytes(int32_t batch, int32_t heads, int32_t head_dim,
                                        int32_t max_seq_len, int32_t max_k)
 {

@@ -125,6 +125,63 @@ sparf_append_kernel(const SparfParams p)
     p.v_sum[(int64_t)pair * kHeadDim + d] += __half2float(v);
 }
 
+// Bulk append, the part specific to the sparse state (K and V rows go through
+// kv_append_bulk_kernel): one block per (sequence, head), one thread per dim.  The thread
+// walks the new tokens in order, adds v to the running sum (fp32, one rounding per token, the
+// order a token-by-token append would use) and writes k into the embedding-major copy, 8
+// tokens (16 bytes) at a time where a whole aligned group is new.
+struct SparfBulkParams {
+    SparfParams base;             // k_new / v_new point at [batch, max_new, heads, 128]
+    const int32_t *new_lens;
+    int32_t max_new;
+};
+
+__global__ void __launch_bounds__(kSparfThreads)
+sparf_append_bulk_kernel(const SparfBulkParams q)
+{
+    const SparfParams &p = q.base;
+    const int pair = blockIdx.x, d = threadIdx.x;
+    const int b = pair / p.heads, h = pair - b * p.heads;
+    const int len = p.seq_lens[b], fresh = q.new_lens[b];
+    const int Tk = p.kt_block_tokens;
+    if (len < 0 || (int64_t)len > (int64_t)p.max_blocks_per_seq * p.block_tokens ||
+        (int64_t)len > (int64_t)p.kt_max_blocks_per_seq * Tk || fresh < 0 || fresh > q.max_new || fresh > len) {
+        if (d == 0 && h == 0 && p.status) atomicOr(p.status, kFlagSeqLenRange);
+        return;
+    }
+    const int first = len - fresh;
+    const int32_t *kt_table = p.kt_block_table + (int64_t)b * p.kt_max_blocks_per_seq;
+    const int64_t token_stride = (int64_t)p.heads * kHeadDim;                 // elements between tokens
+    const __half *k_src = p.k_new + ((int64_t)b * q.max_new * p.heads + h) * kHeadDim + d;
+    const __half *v_src = p.v_new + ((int64_t)b * q.max_new * p.heads + h) * kHeadDim + d;
+    float sum = p.v_sum[(int64_t)pair * kHeadDim + d];
+    int t = 0;
+    while (t < fresh) {
+        const int pos = first + t;
+        const int phys = kt_table[pos / Tk];
+        if (phys < 0 || (int64_t)phys >= p.num_kt_blocks) {
+            if (d == 0 && p.status) atomicOr(p.status, kFlagBlockRange);
+            return;                                                            // uniform: the rest is skipped
+        }
+        __half *dst = p.kt_pool + (((int64_t)phys * p.heads + h) * kHeadDim + d) * Tk + pos % Tk;
+        if ((pos & 7) == 0 && t + 8 <= fresh) {                                // a whole aligned group
+            __align__(16) __half group[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                group[e] = k_src[(int64_t)(t + e) * token_stride];
+                sum += __half2float(v_src[(int64_t)(t + e) * token_stride]);
+            }
+            *reinterpret_cast<uint4 *>(dst) = *reinterpret_cast<const uint4 *>(group);
+            t += 8;
+        } else {
+            *dst = k_src[(int64_t)t * token_stride];
+            sum += __half2float(v_src[(int64_t)t * token_stride]);
+            t += 1;
+        }
+    }
+    p.v_sum[(int64_t)pair * kHeadDim + d] = sum;
+}
+
 // grid pairs * score_chunks: approximate logits of the tokens of one chunk of one (sequence, head).
 __global__ void __launch_bounds__(kSparfThreads)
 sparf_scores_kernel(const SparfParams p)

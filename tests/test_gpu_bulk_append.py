@@ -61,3 +61,29 @@ def test_bad_lengths_are_flagged_and_skipped():
     assert np.array_equal(gu.bits(dev.k_cache[first]), gu.bits(before[first]))          # sequence 0 untouched
     blk = int(table[1, 2])
     assert torch.all(dev.k_cache[blk, :, 4:8] == 0)                                     # sequence 1 written (positions 36..39)
+
+
+@pytest.mark.parametrize("tokens,kt_tokens", [(8, 8), (16, 64), (32, 256)])
+def test_sparse_bulk_append_is_bit_exact(tokens, kt_tokens):
+    lens = [300, 17, 64, 0, 129]
+    news = [300, 5, 61, 0, 1]
+    cpu = case_for("paged", tokens, lens)
+    state = wl.make_sparf_state(cpu, 0.125, kt_tokens)
+    g = torch.Generator().manual_seed(8)
+    kn = torch.randn(5, 300, 5, 128, generator=g).half()
+    vn = torch.randn(5, 300, 5, 128, generator=g).half()
+    dev = gu.to_device(cpu)
+    kt_dev, sum_dev, kt_table_dev = state.kt_pool.cuda(), state.v_sum.cuda(), state.kt_block_table.cuda()
+    flags = torch.zeros(1, dtype=torch.int32, device="cuda")
+    binding.sparf_append_bulk(dev.k_cache, dev.v_cache, kt_dev, sum_dev, kn.cuda(), vn.cuda(), dev.seq_lens,
+                              torch.tensor(news, dtype=torch.int32, device="cuda"), dev.block_table,
+                              kt_table_dev, flags)
+    torch.cuda.synchronize()
+    k, v, kt, v_sum = cpu.k_cache.numpy(), cpu.v_cache.numpy(), state.kt_pool.numpy(), state.v_sum.numpy()
+    capi.sparf_append_bulk(k, v, kt, v_sum, kn.numpy(), vn.numpy(), np.array(lens), np.array(news),
+                           cpu.block_table.numpy(), kt_block_table=state.kt_block_table.numpy())
+    assert int(flags.item()) == 0
+    assert np.array_equal(gu.bits(dev.k_cache), k.view(np.uint16))
+    assert np.array_equal(gu.bits(dev.v_cache), v.view(np.uint16))
+    assert np.array_equal(gu.bits(kt_dev), kt.view(np.uint16))
+    assert np.array_equal(sum_dev.cpu().numpy().view(np.uint32), v_sum.view(np.uint32))
