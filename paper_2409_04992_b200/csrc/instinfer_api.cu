@@ -655,6 +655,7 @@ int instinfer_sparf_decode_attention(void *out, float *alpha, int32_t *selected,
     sp.max_k = max_k;
     sp.score_stride = w.score_stride;
     sp.score_chunks = (int32_t)score_chunks;
+    sp.score_blocks = (int32_t)ceil_div(max_seq_len, kScoreBlockTokens);
     sp.r = r;
     sp.window = local_window;
     sp.scale_log2e = scale * 1.44269504088896340736f;
@@ -670,7 +671,7 @@ int instinfer_sparf_decode_attention(void *out, float *alpha, int32_t *selected,
         (void)cudaGetLastError();
         return INSTINFER_ERR_CUDA;
     }
-    sparf_scores_kernel<<<chunk_grid, kSparfThreads, 0, stream>>>(sp);
+    sparf_scores_kernel<<<(unsigned)(pairs * sp.score_blocks), kSparfThreads, 0, stream>>>(sp);
     // Steps 5-7, chunk-parallel; rows it cannot settle are redone by the single-block kernel.
     sparf_range_kernel<<<chunk_grid, kChunkThreads, 0, stream>>>(sp);
     sparf_hist_kernel<<<chunk_grid, kChunkThreads, 0, stream>>>(sp);

@@ -74,12 +74,13 @@ struct SparfParams {
     int64_t num_kt_blocks;
     int32_t batch, heads, block_tokens, max_blocks_per_seq;
     int32_t kt_block_tokens, kt_max_blocks_per_seq;
-    int32_t max_seq_len, max_k, score_stride, score_chunks, r, window;
+    int32_t max_seq_len, max_k, score_stride, score_chunks, score_blocks, r, window;
     float scale_log2e;
 };
 
 constexpr int kSparfThreads = 128;       // append and scores: one thread per head dim
-constexpr int kScoreChunk = 2048;        // tokens per scores block
+constexpr int kScoreChunk = 2048;        // tokens per block of the selection kernels
+constexpr int kScoreBlockTokens = 8192;  // tokens per block of the score kernel (amortises its prologue)
 constexpr int kSelectThreads = 1024;
 
 __device__ __forceinline__ int sparf_seq_len(const SparfParams &p, int b, bool report)
@@ -182,7 +183,7 @@ sparf_append_bulk_kernel(const SparfBulkParams q)
     p.v_sum[(int64_t)pair * kHeadDim + d] = sum;
 }
 
-// grid pairs * score_chunks: approximate logits of the tokens of one chunk of one (sequence, head).
+// grid pairs * score_blocks: approximate logits of kScoreBlockTokens tokens of one (sequence, head).
 __global__ void __launch_bounds__(kSparfThreads)
 sparf_scores_kernel(const SparfParams p)
 {
@@ -191,12 +192,12 @@ sparf_scores_kernel(const SparfParams p)
     __shared__ int sm_dim[kHeadDim];
     __shared__ float sm_red[2][kSparfThreads / 32];
     __shared__ bool sm_kept[kHeadDim];
-    const int pair = blockIdx.x / p.score_chunks, d = threadIdx.x;
+    const int pair = blockIdx.x / p.score_blocks, d = threadIdx.x;
     const int b = pair / p.heads, h = pair - b * p.heads;
     const int len = sparf_seq_len(p, b, false);
-    const int begin = (blockIdx.x - pair * p.score_chunks) * kScoreChunk;
+    const int begin = (blockIdx.x - pair * p.score_blocks) * kScoreBlockTokens;
     if (begin >= len) return;
-    const int end = min(begin + kScoreChunk, len);
+    const int end = min(begin + kScoreBlockTokens, len);
 
     // Step 1: rank of |q_d| (exact comparisons of fp16 magnitudes, ties to the lower index).
     const float qd = __half2float(p.q[(int64_t)pair * kHeadDim + d]);
