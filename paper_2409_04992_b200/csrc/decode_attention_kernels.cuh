@@ -10,11 +10,14 @@
 //   * each warp streams its own 8-token tiles of K and V through a private ring of shared
 //     memory stages filled by 16-byte cp.async copies (coalesced 512 B per warp instruction),
 //     with no block-wide barrier and no spin-wait anywhere in the main loop;
-//   * logits: 4 lanes share a key row (32 dims each, fp32 FMA, 2 xor-shuffles), so a warp
-//     scores the 8 rows of a tile at once; the running maximum is uniform over the warp and
-//     each row's exponential (base 2, fp32) is computed once;
+//   * logits: 4 lanes share a key row (32 dims each, mixed-precision FMA: fp16 x fp16
+//     products are exact in the fp32 accumulator; 2 xor-shuffles), so a warp scores the 8
+//     rows of a tile at once; the softmax reference is uniform over the warp, follows the
+//     true maximum lazily, and each row's exponential (base 2, fp32) is computed once;
 //   * weighted sum: 16 lanes share a value row (8 dims each), the half-warps take alternate
-//     rows and fetch the row's weight with one shuffle;
+//     rows and fetch the row's weight (split into two fp16 parts) with one shuffle;
+//   * rows come from a contiguous cache, from paged pools through the block table, or from
+//     a list of selected rows (the sparse path);
 //   * the 4 warp states of a block are merged once at the end of the chunk; chunk partials
 //     go to the workspace and a small second kernel merges them.
 #pragma once
