@@ -634,7 +634,7 @@ def main(argv=None) -> int:
             line["cpu_baseline"] = cpu_baseline(w, args.cpu_seconds)
         if not args.no_others and ranks.world == 1:
             others = {}
-            for idx in (1, 2, 3):
+            for idx in (0, 1, 2, 3):
                 if idx == w.index:
                     continue
                 o = wl.STANDARD[idx]
@@ -645,7 +645,8 @@ def main(argv=None) -> int:
                     "pct_of_nominal_8TBs": 100.0 * r["gbs"] / NOMINAL_HBM_GBS,
                     "pct_of_measured_copy": 100.0 * r["gbs"] / peak,
                     "split_kernel_gbs": r["split_bytes"] / r["split_seconds"] / 1e9,
-                    "chunk_tokens": r["chunk_tokens"], "sm_mhz": r["clocks"]["sm_mhz"],
+                    "chunk_tokens": r["chunk_tokens"], "l2_flushed_between_steps": r["flush"],
+                    "sm_mhz": r["clocks"]["sm_mhz"],
                     "reasons": r["clocks"]["reasons"]}
             line["other_workloads"] = others
             line["bulk_append"] = measure_bulk_append(device)
