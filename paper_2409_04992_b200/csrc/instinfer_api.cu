@@ -99,7 +99,10 @@ SplitPlan make_plan(int64_t pairs, int32_t max_seq_len)
     }
     const int64_t slots = (int64_t)sm_count() * kCtasPerSm;
     const int64_t fewest = ceil_div(max_seq_len, kChunkCeiling);
-    const int64_t most = ceil_div(max_seq_len, kChunkFloor);
+    // Small problems that cannot fill the GPU with kChunkFloor-token chunks are latency-bound:
+    // cut them down to the granule so that more blocks share the work.
+    const int64_t floor_tokens = pairs * ceil_div(max_seq_len, kChunkFloor) < slots ? kChunkGranule : kChunkFloor;
+    const int64_t most = ceil_div(max_seq_len, floor_tokens);
     int64_t n = ceil_div(slots * kTargetWaves, pairs);
     if (n > most) n = most;
     if (n < fewest) n = fewest;
