@@ -173,6 +173,42 @@ int instinfer_decode_attention_static(void *out, float *lse, const void *q,
                                       int32_t *status_flags, void *cuda_stream);
 
 /*
+ * Decode attention on one head shard of a multi-GPU deployment, with the all-gather of the
+ * outputs fused into the last kernel (Sec. IV-D, "Scale to CSD array": heads are independent,
+ * each device keeps the KV cache of its own heads and computes them locally; only the small
+ * output vectors are exchanged).  This GPU holds `heads` consecutive heads, global heads
+ * head_offset .. head_offset + heads - 1 of total_heads, in caches shaped as for the two
+ * single-GPU entry points with H = heads (block_table == NULL: contiguous, else paged).  The
+ * kernel that finishes a (sequence, head) writes its output row into EVERY rank's full
+ * output buffer at [b, head_offset + h, :], with plain 16-byte stores:
+ *   out_all   HOST array of n_ranks DEVICE pointers; entry r is rank r's fp16
+ *             [batch, total_heads, head_dim] buffer as addressable from THIS GPU (its own
+ *             allocation, or a peer mapping: CUDA IPC, symmetric memory).  The array is read
+ *             during the call only.  1 <= n_ranks <= INSTINFER_MAX_RANKS.
+ *   lse       nullable, this shard's own [batch, heads] (not exchanged).
+ *   workspace at least instinfer_allgather_workspace_bytes(batch, heads, head_dim, max_seq_len).
+ * Every other argument as in instinfer_decode_attention / instinfer_decode_attention_paged.
+ * No rank waits for another inside the kernels and nothing here synchronises GPUs: when every
+ * rank's call has completed, every buffer holds all heads.  Ordering a reader on rank r after
+ * the other ranks' calls is the caller's job (an event exchange, or a barrier collective
+ * enqueued after the call on each rank's stream).  Errors as for the single-GPU entry points;
+ * head_offset < 0 or head_offset + heads > total_heads: INSTINFER_ERR_INVALID_ARG.
+ */
+#define INSTINFER_MAX_RANKS 16
+int instinfer_decode_attention_allgather(void *const *out_all, int32_t n_ranks, float *lse,
+                                         const void *q, const void *k_cache, const void *v_cache,
+                                         const int32_t *block_table, const int32_t *seq_lens,
+                                         int32_t batch, int32_t heads, int32_t head_offset,
+                                         int32_t total_heads, int32_t head_dim, int32_t s_max,
+                                         int32_t block_tokens, int32_t max_blocks_per_seq,
+                                         int64_t num_phys_blocks, int32_t max_seq_len, float scale,
+                                         void *workspace, size_t workspace_bytes,
+                                         int32_t *status_flags, void *cuda_stream);
+
+size_t instinfer_allgather_workspace_bytes(int32_t batch, int32_t heads, int32_t head_dim,
+                                           int32_t max_seq_len);
+
+/*
  * One whole decode step for a caller whose new vectors live in host memory (the paper's
  * decode flow, Sec. IV-D: only q, k, v travel to the device that owns the KV cache and only
  * the attention output travels back; the cache never moves).

@@ -8,7 +8,7 @@ from __future__ import annotations
 
 import ctypes
 from pathlib import Path
-from typing import Optional
+from typing import Optional, Sequence, Union
 
 import torch
 
@@ -54,6 +54,12 @@ def load() -> ctypes.CDLL:
         lib.instinfer_decode_attention_static.argtypes = [ptr, ptr, ptr, ptr, ptr, ptr, ptr,
                                                           i32, i32, i32, i32, i32, i32, i64, i32,
                                                           f32, ptr, ptr]
+        lib.instinfer_decode_attention_allgather.restype = ctypes.c_int
+        lib.instinfer_decode_attention_allgather.argtypes = [ptr, i32, ptr, ptr, ptr, ptr, ptr, ptr,
+                                                             i32, i32, i32, i32, i32, i32, i32, i32,
+                                                             i64, i32, f32, ptr, sz, ptr, ptr]
+        lib.instinfer_allgather_workspace_bytes.restype = sz
+        lib.instinfer_allgather_workspace_bytes.argtypes = [i32, i32, i32, i32]
         lib.instinfer_decode_step_host.restype = ctypes.c_int
         lib.instinfer_decode_step_host.argtypes = [ptr, ptr, ptr, ptr, ptr, ptr, ptr, ptr, ptr,
                                                    i32, i32, i64, i32, i32, i32, i32, i32, f32,
@@ -212,6 +218,36 @@ def decode_attention_static(out: torch.Tensor, lse: Optional[torch.Tensor], q: t
         _ptr(out), _ptr(lse), _ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(block_table),
         _ptr(seq_lens), batch, heads, head_dim, s_max, block_tokens, max_blocks, phys,
         int(max_seq_len), float(scale), _ptr(status_flags), _stream(stream)))
+
+
+def allgather_workspace_bytes(batch: int, heads: int, head_dim: int, max_seq_len: int) -> int:
+    return int(load().instinfer_allgather_workspace_bytes(batch, heads, head_dim, max_seq_len))
+
+
+def decode_attention_allgather(out_all: Sequence[Union[torch.Tensor, int]], lse: Optional[torch.Tensor],
+                               q: torch.Tensor, k_cache: torch.Tensor, v_cache: torch.Tensor,
+                               block_table: Optional[torch.Tensor], seq_lens: torch.Tensor,
+                               head_offset: int, total_heads: int, max_seq_len: int, scale: float,
+                               workspace: torch.Tensor,
+                               status_flags: Optional[torch.Tensor] = None,
+                               stream: Optional[torch.cuda.Stream] = None) -> None:
+    """instinfer_decode_attention_allgather: this rank's head shard (q [B, heads, D]), output
+    rows stored into every rank's [B, total_heads, D] buffer.  out_all holds one entry per
+    rank, a tensor or a raw device address of a peer mapping."""
+    batch, heads, head_dim = q.shape
+    if block_table is None:
+        s_max, block_tokens, max_blocks, phys = k_cache.shape[2], 0, 0, 0
+    else:
+        s_max, block_tokens, max_blocks, phys = (0, k_cache.shape[2], block_table.shape[1],
+                                                 k_cache.shape[0])
+    addresses = [t.data_ptr() if isinstance(t, torch.Tensor) else int(t) for t in out_all]
+    table = (ctypes.c_void_p * len(addresses))(*addresses)
+    _check(load().instinfer_decode_attention_allgather(
+        table, len(addresses), _ptr(lse), _ptr(q), _ptr(k_cache), _ptr(v_cache),
+        _ptr(block_table), _ptr(seq_lens), batch, heads, int(head_offset), int(total_heads),
+        head_dim, s_max, block_tokens, max_blocks, phys, int(max_seq_len), float(scale),
+        _ptr(workspace), workspace.numel() * workspace.element_size(), _ptr(status_flags),
+        _stream(stream)))
 
 
 def decode_step_host(out_host: torch.Tensor, qkv_host: torch.Tensor, qkv_dev: torch.Tensor,

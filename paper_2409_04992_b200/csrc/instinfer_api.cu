@@ -5,6 +5,7 @@
 
 #include <cmath>
 
+#include "allgather_merge_kernel.cuh"
 #include "decode_attention_kernels.cuh"
 #include "kv_append_kernel.cuh"
 #include "sparf_kernels.cuh"
@@ -53,9 +54,9 @@ int sm_count()
 // Launch with programmatic stream serialization: the kernel may be scheduled while the
 // previous kernel in the stream drains; it orders itself with griddepcontrol.wait.  Falls
 // back to an ordinary launch if the runtime refuses the attribute.
-template <typename Params>
-cudaError_t launch_overlapped(void (*kernel)(Params), unsigned grid, unsigned block, size_t smem,
-                              cudaStream_t stream, const Params &params)
+template <typename... Params>
+cudaError_t launch_overlapped(void (*kernel)(Params...), unsigned grid, unsigned block, size_t smem,
+                              cudaStream_t stream, const Params &...params)
 {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid);
@@ -67,11 +68,11 @@ cudaError_t launch_overlapped(void (*kernel)(Params), unsigned grid, unsigned bl
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    cudaError_t err = cudaLaunchKernelEx(&cfg, kernel, params);
+    cudaError_t err = cudaLaunchKernelEx(&cfg, kernel, params...);
     if (err != cudaSuccess) {
         (void)cudaGetLastError();
         cfg.numAttrs = 0;
-        err = cudaLaunchKernelEx(&cfg, kernel, params);
+        err = cudaLaunchKernelEx(&cfg, kernel, params...);
     }
     return err;
 }
@@ -156,12 +157,21 @@ int ensure_split_smem(bool paged)
     return INSTINFER_OK;
 }
 
+// Bytes of finished fp16 rows parked in the workspace, behind the partials, by the
+// head-sharded path when the plan has a single chunk.
+size_t staging_for(int64_t pairs) { return ((size_t)pairs * kHeadDim * sizeof(__half) + 255) / 256 * 256; }
+
+// gather == nullptr: outputs go to p.out.  Otherwise p.out is unused and every finished row
+// is stored into all of gather->out (the fused all-gather of the head-sharded path).
 int launch_attention(AttnParams p, bool paged, int32_t batch, void *workspace,
-                     size_t workspace_bytes, cudaStream_t stream)
+                     size_t workspace_bytes, cudaStream_t stream,
+                     const GatherTargets *gather = nullptr)
 {
     const int64_t pairs = (int64_t)batch * p.heads;
     const SplitPlan plan = make_plan(pairs, p.max_seq_len);
-    if (workspace == nullptr || !aligned16(workspace) || workspace_bytes < workspace_for(pairs, plan))
+    const size_t partial_bytes = workspace_for(pairs, plan);
+    if (workspace == nullptr || !aligned16(workspace) ||
+        workspace_bytes < partial_bytes + (gather ? staging_for(pairs) : 0))
         return INSTINFER_ERR_WORKSPACE;
     if (pairs * plan.n_splits >= (int64_t)1 << 31) return INSTINFER_ERR_INVALID_ARG;
     p.chunk_tokens = plan.chunk_tokens;
@@ -171,6 +181,12 @@ int launch_attention(AttnParams p, bool paged, int32_t batch, void *workspace,
     p.pairs = (int32_t)pairs;
     p.part_o = static_cast<float *>(workspace);
     p.part_lse = p.part_o + (size_t)pairs * plan.n_splits * kHeadDim;
+    GatherTargets targets = {};
+    if (gather) {
+        targets = *gather;
+        p.out = reinterpret_cast<__half *>(static_cast<unsigned char *>(workspace) + partial_bytes);
+        targets.staged = p.out;
+    }
 
     const int rc = ensure_split_smem(paged);
     if (rc != INSTINFER_OK) return rc;
@@ -184,7 +200,10 @@ int launch_attention(AttnParams p, bool paged, int32_t batch, void *workspace,
         err = launch_overlapped(decode_attn_split_kernel<Rows::kContiguous>, grid, kThreads, kSplitSmemBytes, stream, p);
     if (timed) cudaEventRecord(g_after_split, stream);
     if (err != cudaSuccess || cudaGetLastError() != cudaSuccess) return INSTINFER_ERR_CUDA;
-    if (plan.n_splits > 1) {
+    if (gather) {
+        err = launch_overlapped(lse_merge_allgather_kernel, (unsigned)pairs, kHeadDim, 0, stream, p, targets);
+        if (err != cudaSuccess || cudaGetLastError() != cudaSuccess) return INSTINFER_ERR_CUDA;
+    } else if (plan.n_splits > 1) {
         err = launch_overlapped(lse_merge_kernel, (unsigned)pairs, kHeadDim, 0, stream, p);
         if (err != cudaSuccess || cudaGetLastError() != cudaSuccess) return INSTINFER_ERR_CUDA;
     }
@@ -405,6 +424,70 @@ int instinfer_decode_attention_static(void *out, float *lse, const void *q, cons
                                             max_blocks_per_seq, num_phys_blocks, max_seq_len,
                                             scale, scratch, kStaticWorkspaceBytes, status_flags,
                                             cuda_stream);
+}
+
+int instinfer_decode_attention_allgather(void *const *out_all, int32_t n_ranks, float *lse,
+                                         const void *q, const void *k_cache, const void *v_cache,
+                                         const int32_t *block_table, const int32_t *seq_lens,
+                                         int32_t batch, int32_t heads, int32_t head_offset,
+                                         int32_t total_heads, int32_t head_dim, int32_t s_max,
+                                         int32_t block_tokens, int32_t max_blocks_per_seq,
+                                         int64_t num_phys_blocks, int32_t max_seq_len, float scale,
+                                         void *workspace, size_t workspace_bytes,
+                                         int32_t *status_flags, void *cuda_stream)
+{
+    const bool paged = block_table != nullptr;
+    if (head_dim <= 0 || !sizes_ok(batch, heads, max_seq_len) || out_all == nullptr ||
+        n_ranks < 1 || n_ranks > kMaxRanks || head_offset < 0 || total_heads <= 0 ||
+        (int64_t)head_offset + heads > total_heads || !std::isfinite(scale))
+        return INSTINFER_ERR_INVALID_ARG;
+    if (paged) {
+        if (block_tokens <= 0 || max_blocks_per_seq <= 0 || num_phys_blocks <= 0 ||
+            (int64_t)max_seq_len > (int64_t)max_blocks_per_seq * block_tokens)
+            return INSTINFER_ERR_INVALID_ARG;
+    } else if (s_max <= 0 || max_seq_len > s_max) {
+        return INSTINFER_ERR_INVALID_ARG;
+    }
+    if (head_dim != kHeadDim || (paged && block_tokens % 8 != 0)) return INSTINFER_ERR_UNSUPPORTED;
+    if (batch == 0) return INSTINFER_OK;
+    if (!usable(q) || !usable(k_cache) || !usable(v_cache) || seq_lens == nullptr)
+        return INSTINFER_ERR_INVALID_ARG;
+
+    GatherTargets targets = {};
+    for (int r = 0; r < n_ranks; ++r) {
+        if (!usable(out_all[r])) return INSTINFER_ERR_INVALID_ARG;
+        targets.out[r] = static_cast<__half *>(out_all[r]);
+    }
+    targets.n_ranks = n_ranks;
+    targets.head_offset = head_offset;
+    targets.total_heads = total_heads;
+
+    AttnParams p = {};
+    p.q = static_cast<const __half *>(q);
+    p.k = static_cast<const __half *>(k_cache);
+    p.v = static_cast<const __half *>(v_cache);
+    p.seq_lens = seq_lens;
+    p.block_table = block_table;
+    p.lse = lse;
+    p.status = status_flags;
+    p.num_phys_blocks = paged ? num_phys_blocks : 0;
+    p.heads = heads;
+    p.s_max = paged ? 0 : s_max;
+    p.block_tokens = paged ? block_tokens : 0;
+    p.max_blocks_per_seq = paged ? max_blocks_per_seq : 0;
+    p.max_seq_len = max_seq_len;
+    p.scale_log2e = scale * 1.44269504088896340736f;
+    return launch_attention(p, paged, batch, workspace, workspace_bytes,
+                            static_cast<cudaStream_t>(cuda_stream), &targets);
+}
+
+size_t instinfer_allgather_workspace_bytes(int32_t batch, int32_t heads, int32_t head_dim,
+                                           int32_t max_seq_len)
+{
+    if (head_dim != kHeadDim || !sizes_ok(batch, heads, max_seq_len)) return 0;
+    const int64_t pairs = (int64_t)batch * heads;
+    if (pairs == 0) return 256;
+    return workspace_for(pairs, make_plan(pairs, max_seq_len)) + staging_for(pairs);
 }
 
 int instinfer_decode_step_host(void *out_host, const void *qkv_host, void *qkv_dev, void *out_dev,
