@@ -1,8 +1,9 @@
 """Head-sharded decode attention with the fused all-gather, on one GPU: the ranks' calls run
 one after another on the same device, each on its own head shard of the same case, each
 storing into all ranks' output buffers (here ordinary buffers of this GPU).  No call waits
-for another.  Afterwards every buffer must hold, bit for bit, what the single-GPU entry
-point gives on the whole case, and that must agree with the CPU oracle."""
+for another.  Afterwards all buffers must be identical, each shard's rows must be, bit for
+bit, what the single-GPU entry point gives on that shard (same number of (sequence, head)
+pairs, hence the same chunking), and the whole must agree with the CPU oracle."""
 import numpy as np
 import pytest
 import torch
@@ -56,11 +57,18 @@ def run_sharded(dev: wl.Case, world: int, chunk_tokens=0):
 def test_every_rank_ends_with_all_heads(layout, tokens, world, heads):
     cpu = make_case(layout, tokens, heads)
     dev = gu.to_device(cpu)
-    whole, whole_lse, _ = gu.gpu_step(dev)                      # appends, then single-GPU attention
-    outs, lse = run_sharded(dev, world)                         # same (already appended) caches
+    gu.gpu_step(dev)                                            # the step's append
+    outs, lse = run_sharded(dev, world)
     for r, out in enumerate(outs):
-        assert np.array_equal(gu.bits(out), gu.bits(whole)), f"rank {r}'s buffer differs"
-    assert np.array_equal(lse.numpy(), whole_lse.numpy())
+        assert np.array_equal(gu.bits(out), gu.bits(outs[0])), f"rank {r}'s buffer differs"
+    for rank in range(world):
+        off, cnt = sharding.head_shard(heads, world, rank)
+        shard = wl.Case(**{**dev.__dict__, "q": sharding.take_heads(dev.q, off, cnt),
+                           "k_cache": sharding.take_heads(dev.k_cache, off, cnt),
+                           "v_cache": sharding.take_heads(dev.v_cache, off, cnt)})
+        alone, alone_lse, _ = gu.gpu_step(shard, do_append=False)
+        assert np.array_equal(gu.bits(outs[0][:, off:off + cnt]), gu.bits(alone)), f"shard {rank}"
+        assert np.array_equal(lse[:, off:off + cnt].numpy(), alone_lse.numpy())
     want, want_lse = gu.oracle_step(cpu)
     gu.assert_close(outs[0], want, lse, want_lse, f"{layout} world={world}")
 
