@@ -29,6 +29,10 @@ def _load() -> ctypes.CDLL:
         lib.oracle_decode_attention.argtypes = [ptr, ptr, ptr, i64, ptr, ptr, ptr, ptr, ptr,
                                                 i32, i32, i64, i32, i32, i32, i32,
                                                 ctypes.c_float]
+        lib.oracle_decode_attention_grouped.restype = ctypes.c_int
+        lib.oracle_decode_attention_grouped.argtypes = [ptr, ptr, ptr, ptr, ptr, ptr, ptr, i32, i32,
+                                                        i64, i32, i32, i32, i32, i32, i32,
+                                                        ctypes.c_float]
         lib.oracle_kv_append_bulk.restype = ctypes.c_int
         lib.oracle_kv_append_bulk.argtypes = [ptr, ptr, ptr, ptr, ptr, ptr, ptr, i32, i32, i64,
                                               i32, i32, i32, i32, i32]
@@ -156,6 +160,35 @@ def decode_attention(q: np.ndarray, k_cache: np.ndarray, v_cache: np.ndarray,
     if rc:
         raise OracleError(rc)
     return out, lse, weights
+
+
+def decode_attention_grouped(q: np.ndarray, k_cache: np.ndarray, v_cache: np.ndarray,
+                             seq_lens: np.ndarray, scale: float,
+                             block_table: Optional[np.ndarray] = None):
+    """Grouped-head, multi-token decode attention in fp64: q [B,Tq,Hq,D], caches with Hkv heads
+    (Hq a multiple of Hkv); new token t sees positions [0, seq_lens[b] - (Tq-1-t)).
+
+    Returns (out [B,Tq,Hq,D] float64, lse [B,Tq,Hq] float64).
+    """
+    qb = _bits(np.ascontiguousarray(q))
+    kb, vb = _bits(k_cache), _bits(v_cache)
+    batch, q_tokens, q_heads, head_dim = qb.shape
+    kv_heads = kb.shape[1]
+    lens = np.ascontiguousarray(seq_lens, dtype=np.int32)
+    table, max_blocks = _table(block_table, batch)
+    if table is None:
+        s_max, block_tokens, phys = kb.shape[2], 0, 0
+    else:
+        s_max, block_tokens, phys = 0, kb.shape[2], kb.shape[0]
+    out = np.zeros((batch, q_tokens, q_heads, head_dim), dtype=np.float64)
+    lse = np.zeros((batch, q_tokens, q_heads), dtype=np.float64)
+    rc = _load().oracle_decode_attention_grouped(_p(out), _p(lse), _p(qb), _p(kb), _p(vb), _p(lens),
+                                                 _p(table), max_blocks, block_tokens, phys, batch,
+                                                 q_tokens, q_heads, kv_heads, head_dim, s_max,
+                                                 ctypes.c_float(scale))
+    if rc:
+        raise OracleError(rc)
+    return out, lse
 
 
 def sparf_append(k_pool: np.ndarray, v_pool: np.ndarray, kt_pool: np.ndarray, v_sum: np.ndarray,

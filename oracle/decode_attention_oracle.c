@@ -269,3 +269,65 @@ int oracle_decode_attention(double *out, double *lse, double *weights, int64_t w
     }
     return failure;
 }
+
+/*
+ * Grouped / multi-token variant.  The paper's models use one KV head per query head and one
+ * new token per step (Sec. II-A, II-B); it only notes that other configurations exist
+ * (Sec. IV-C).  This is the same definition applied row by row to the two common ones:
+ *   - grouped heads: query head hq reads the cache of KV head hq / group, group = q_heads /
+ *     kv_heads (group == 1 is the paper's case);
+ *   - several new tokens per sequence in one step: the cache already holds all q_tokens new
+ *     tokens, seq_lens[b] counts them, and new token t (0 = oldest) attends causally to
+ *     positions [0, seq_lens[b] - (q_tokens - 1 - t)), i.e. to itself and everything before.
+ *     A token whose range is empty (sequence shorter than q_tokens) gives zero output, lse -inf.
+ *   q, out  [batch][q_tokens][q_heads][head_dim]   (fp16 bits / fp64)
+ *   lse     [batch][q_tokens][q_heads]             (nullable)
+ *   caches  as above with kv_heads heads.
+ */
+int oracle_decode_attention_grouped(double *out, double *lse, const uint16_t *q,
+                                    const uint16_t *k_cache, const uint16_t *v_cache,
+                                    const int32_t *seq_lens,
+                                    const int32_t *block_table, int32_t max_blocks_per_seq,
+                                    int32_t block_tokens, int64_t num_phys_blocks,
+                                    int32_t batch, int32_t q_tokens, int32_t q_heads,
+                                    int32_t kv_heads, int32_t head_dim, int32_t s_max, float scale)
+{
+    const cache_geometry g = {block_table, max_blocks_per_seq, block_tokens,
+                              num_phys_blocks, kv_heads, head_dim, s_max};
+    int rc = check_geometry(&g, batch);
+    if (rc) return rc;
+    if (q_tokens <= 0 || q_heads <= 0 || q_heads % kv_heads != 0) return -1;
+    const int32_t group = q_heads / kv_heads;
+    int32_t longest = 0;
+    for (int32_t b = 0; b < batch; ++b) {
+        if (seq_lens[b] < 0 || (int64_t)seq_lens[b] > capacity_tokens(&g)) return -2;
+        if (seq_lens[b] > longest) longest = seq_lens[b];
+    }
+    int failure = 0;
+    const int64_t rows = (int64_t)batch * q_tokens * q_heads;
+#pragma omp parallel
+    {
+        double scores_small[1];
+        double *scores = scores_small;
+        if (longest > 0) scores = (double *)malloc(sizeof(double) * (size_t)longest);
+#pragma omp for schedule(dynamic, 1)
+        for (int64_t row = 0; row < rows; ++row) {
+            const int32_t hq = (int32_t)(row % q_heads);
+            const int32_t t = (int32_t)((row / q_heads) % q_tokens);
+            const int32_t b = (int32_t)(row / ((int64_t)q_heads * q_tokens));
+            int32_t visible = seq_lens[b] - (q_tokens - 1 - t);
+            if (visible < 0) visible = 0;
+            double lse_val = 0.0;
+            const int err = attend_one(&g, b, hq / group, visible, q + row * head_dim,
+                                       k_cache, v_cache, (double)scale, scores,
+                                       out + row * head_dim, &lse_val, NULL);
+            if (lse) lse[row] = lse_val;
+            if (err) {
+#pragma omp atomic write
+                failure = err;
+            }
+        }
+        if (longest > 0) free(scores);
+    }
+    return failure;
+}

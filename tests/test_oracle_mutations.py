@@ -28,6 +28,12 @@ MUTANTS = {
     "append_off_by_one": ("const int64_t dst = row_offset(&g, b, h, L - 1);",
                           "const int64_t dst = row_offset(&g, b, h, L > 1 ? L - 2 : 0);"),
     "subnormal_exponent": ("mag = ldexp((double)frac, -24);", "mag = ldexp((double)frac, -25);"),
+    "grouped_head_map_interleaved": ("const int err = attend_one(&g, b, hq / group, visible,",
+                                     "const int err = attend_one(&g, b, hq % kv_heads, visible,"),
+    "grouped_causal_off_by_one": ("int32_t visible = seq_lens[b] - (q_tokens - 1 - t);",
+                                  "int32_t visible = seq_lens[b] - (q_tokens - t);"),
+    "grouped_token_order_reversed": ("int32_t visible = seq_lens[b] - (q_tokens - 1 - t);",
+                                     "int32_t visible = seq_lens[b] - t;"),
 }
 
 
@@ -95,6 +101,19 @@ def pins(monkey_lib):
     want = bits.view(np.float16).astype(np.float64).reshape(1, 512, 128)
     fin = ~np.isnan(want)
     check("half_widening", np.array_equal(out[fin], want[fin]))
+    # grouped heads and several new tokens: numpy softmax on the expanded, causally cut problem
+    L, Tq, Hq, Hkv = 9, 2, 4, 2
+    q, k, v = f16((1, Tq, Hq, 128)), f16((1, Hkv, L, 128)), f16((1, Hkv, L, 128))
+    out, _ = capi.decode_attention_grouped(q, k, v, np.array([L]), SCALE)
+    ok = True
+    for t in range(Tq):
+        n = L - (Tq - 1 - t)
+        for hq in range(Hq):
+            hk = hq // (Hq // Hkv)
+            s = k[0, hk, :n].astype(np.float64) @ q[0, t, hq].astype(np.float64) * float(np.float32(SCALE))
+            w = np.exp(s - s.max())
+            ok &= np.allclose(out[0, t, hq], (w / w.sum()) @ v[0, hk, :n].astype(np.float64), atol=1e-12, rtol=0)
+    check("grouped_definition", ok)
     return failed
 
 
@@ -107,7 +126,8 @@ def test_each_planted_mistake_is_caught(name, tmp_path, monkeypatch):
     lib_path = build_mutant(tmp_path, name)
     real = capi._load()
     mutant = ctypes.CDLL(lib_path)
-    for fn in ("oracle_num_threads", "oracle_kv_append", "oracle_decode_attention"):
+    for fn in ("oracle_num_threads", "oracle_kv_append", "oracle_decode_attention",
+               "oracle_decode_attention_grouped"):
         getattr(mutant, fn).restype = getattr(real, fn).restype
         getattr(mutant, fn).argtypes = getattr(real, fn).argtypes
     monkeypatch.setattr(capi, "_lib", mutant)
