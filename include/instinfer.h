@@ -17,7 +17,7 @@
  *   enqueued work has run.
  * - fp16 = IEEE binary16.  heads = number of attention heads (query heads == KV heads,
  *   multi-head attention, Sec. II-A).  head_dim must be 128 (the paper's head size,
- *   Sec. IV-C).
+ *   Sec. IV-C); the two appends and instinfer_decode_attention_grouped also take 64 and 256.
  * - seq_lens[b] (int32, device, [batch]) is the length of sequence b AFTER this step's
  *   append: the append writes logical position seq_lens[b]-1, attention covers positions
  *   [0, seq_lens[b]) -- the new token attends to itself (Sec. II-B).  seq_lens[b] == 0
@@ -59,7 +59,7 @@ extern "C" {
 typedef enum {
     INSTINFER_OK = 0,
     INSTINFER_ERR_INVALID_ARG = 1,   /* null / misaligned pointer, non-positive size, bad bound */
-    INSTINFER_ERR_UNSUPPORTED = 2,   /* head_dim != 128, block_tokens not a multiple of 8       */
+    INSTINFER_ERR_UNSUPPORTED = 2,   /* head_dim or block_tokens outside the supported set     */
     INSTINFER_ERR_WORKSPACE = 3,     /* workspace null or smaller than instinfer_workspace_bytes */
     INSTINFER_ERR_CUDA = 4           /* the CUDA runtime refused a launch                        */
 } instinfer_status;
@@ -207,6 +207,39 @@ int instinfer_decode_attention_allgather(void *const *out_all, int32_t n_ranks, 
 
 size_t instinfer_allgather_workspace_bytes(int32_t batch, int32_t heads, int32_t head_dim,
                                            int32_t max_seq_len);
+
+/*
+ * Decode attention for configurations other than the paper's one query head per KV head and
+ * one new token per step (Sec. II-A, II-B; Sec. IV-C only notes that other configurations
+ * exist): grouped heads, several new tokens per step, head sizes 64 / 128 / 256.
+ *   q, out   fp16 [batch, q_tokens, q_heads, head_dim]
+ *   lse      nullable fp32 [batch, q_tokens, q_heads]
+ *   caches   as for the entry points above with `kv_heads` heads (block_table == NULL:
+ *            contiguous [batch, kv_heads, s_max, head_dim], else paged pools
+ *            [num_phys_blocks, kv_heads, block_tokens, head_dim])
+ * Query head hq reads KV head hq / (q_heads / kv_heads); q_heads must be a multiple of
+ * kv_heads.  The caches already hold all q_tokens new tokens (append them with
+ * instinfer_kv_append, or instinfer_kv_append_bulk for q_tokens > 1) and seq_lens[b] counts
+ * them; new token t (0 = oldest) attends causally to positions
+ * [0, seq_lens[b] - (q_tokens - 1 - t)).  A token whose range is empty gives a zero row and
+ * lse = -inf.  With q_tokens = 1 and q_heads = kv_heads the result is that of the entry points
+ * above within the same tolerance (not bit for bit: the contractions run on the tensor cores).
+ * Limits (INSTINFER_ERR_UNSUPPORTED otherwise): (q_heads / kv_heads) * q_tokens <= 16;
+ * head_dim in {64, 128, 256}; paged block_tokens a multiple of 16.
+ *   workspace at least instinfer_grouped_workspace_bytes(...) bytes.
+ */
+int instinfer_decode_attention_grouped(void *out, float *lse, const void *q, const void *k_cache,
+                                       const void *v_cache, const int32_t *block_table,
+                                       const int32_t *seq_lens, int32_t batch, int32_t q_tokens,
+                                       int32_t q_heads, int32_t kv_heads, int32_t head_dim,
+                                       int32_t s_max, int32_t block_tokens,
+                                       int32_t max_blocks_per_seq, int64_t num_phys_blocks,
+                                       int32_t max_seq_len, float scale, void *workspace,
+                                       size_t workspace_bytes, int32_t *status_flags,
+                                       void *cuda_stream);
+
+size_t instinfer_grouped_workspace_bytes(int32_t batch, int32_t q_tokens, int32_t q_heads,
+                                         int32_t kv_heads, int32_t head_dim, int32_t max_seq_len);
 
 /*
  * One whole decode step for a caller whose new vectors live in host memory (the paper's

@@ -60,6 +60,12 @@ def load() -> ctypes.CDLL:
                                                              i64, i32, f32, ptr, sz, ptr, ptr]
         lib.instinfer_allgather_workspace_bytes.restype = sz
         lib.instinfer_allgather_workspace_bytes.argtypes = [i32, i32, i32, i32]
+        lib.instinfer_decode_attention_grouped.restype = ctypes.c_int
+        lib.instinfer_decode_attention_grouped.argtypes = [ptr, ptr, ptr, ptr, ptr, ptr, ptr,
+                                                           i32, i32, i32, i32, i32, i32, i32, i32,
+                                                           i64, i32, f32, ptr, sz, ptr, ptr]
+        lib.instinfer_grouped_workspace_bytes.restype = sz
+        lib.instinfer_grouped_workspace_bytes.argtypes = [i32, i32, i32, i32, i32, i32]
         lib.instinfer_decode_step_host.restype = ctypes.c_int
         lib.instinfer_decode_step_host.argtypes = [ptr, ptr, ptr, ptr, ptr, ptr, ptr, ptr, ptr,
                                                    i32, i32, i64, i32, i32, i32, i32, i32, f32,
@@ -248,6 +254,34 @@ def decode_attention_allgather(out_all: Sequence[Union[torch.Tensor, int]], lse:
         head_dim, s_max, block_tokens, max_blocks, phys, int(max_seq_len), float(scale),
         _ptr(workspace), workspace.numel() * workspace.element_size(), _ptr(status_flags),
         _stream(stream)))
+
+
+def grouped_workspace_bytes(batch: int, q_tokens: int, q_heads: int, kv_heads: int, head_dim: int,
+                            max_seq_len: int) -> int:
+    return int(load().instinfer_grouped_workspace_bytes(batch, q_tokens, q_heads, kv_heads,
+                                                        head_dim, max_seq_len))
+
+
+def decode_attention_grouped(out: torch.Tensor, lse: Optional[torch.Tensor], q: torch.Tensor,
+                             k_cache: torch.Tensor, v_cache: torch.Tensor,
+                             block_table: Optional[torch.Tensor], seq_lens: torch.Tensor,
+                             max_seq_len: int, scale: float, workspace: torch.Tensor,
+                             status_flags: Optional[torch.Tensor] = None,
+                             stream: Optional[torch.cuda.Stream] = None) -> None:
+    """instinfer_decode_attention_grouped: q, out [B, Tq, Hq, D]; caches with Hkv heads
+    ([B,Hkv,s_max,D], or pools [P,Hkv,T,D] with block_table)."""
+    batch, q_tokens, q_heads, head_dim = q.shape
+    kv_heads = k_cache.shape[1]
+    if block_table is None:
+        s_max, block_tokens, max_blocks, phys = k_cache.shape[2], 0, 0, 0
+    else:
+        s_max, block_tokens, max_blocks, phys = (0, k_cache.shape[2], block_table.shape[1],
+                                                 k_cache.shape[0])
+    _check(load().instinfer_decode_attention_grouped(
+        _ptr(out), _ptr(lse), _ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(block_table),
+        _ptr(seq_lens), batch, q_tokens, q_heads, kv_heads, head_dim, s_max, block_tokens,
+        max_blocks, phys, int(max_seq_len), float(scale), _ptr(workspace),
+        workspace.numel() * workspace.element_size(), _ptr(status_flags), _stream(stream)))
 
 
 def decode_step_host(out_host: torch.Tensor, qkv_host: torch.Tensor, qkv_dev: torch.Tensor,

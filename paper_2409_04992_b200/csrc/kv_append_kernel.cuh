@@ -1,6 +1,6 @@
 // KV append for sm_100a: the new token's k,v rows join the cache (Sec. II-B; the decode
 // phase's incremental writes of Sec. IV-C).  A pure bit copy: one thread moves one 16-byte
-// segment of K and one of V, 16 threads cover a (sequence, head) row pair.
+// segment of K and one of V; head_dim / 8 threads cover a (sequence, head) row pair.
 #pragma once
 
 #include <cuda_runtime.h>
@@ -11,7 +11,7 @@ namespace instinfer {
 struct AppendParams {
     uint4 *k_cache;
     uint4 *v_cache;
-    const uint4 *k_new;           // [batch, heads, 128] fp16 = 16 uint4 per row
+    const uint4 *k_new;           // [batch, heads, head_dim] fp16 = segs_per_row uint4 per row
     const uint4 *v_new;
     const int32_t *seq_lens;
     const int32_t *block_table;   // nullptr: contiguous
@@ -22,18 +22,18 @@ struct AppendParams {
     int32_t s_max;
     int32_t block_tokens;
     int32_t max_blocks_per_seq;
+    int32_t segs_per_row;         // 16-byte segments of one row: head_dim / 8 (16 at head_dim 128)
 };
 
 constexpr int kAppendThreads = 128;
-constexpr int kSegsPerRow = 16;   // 256 B / 16 B
 
 __global__ void __launch_bounds__(kAppendThreads)
 kv_append_kernel(const AppendParams p)
 {
     const int64_t idx = (int64_t)blockIdx.x * kAppendThreads + threadIdx.x;
-    const int64_t pair = idx / kSegsPerRow;
+    const int64_t pair = idx / p.segs_per_row;
     if (pair >= (int64_t)p.batch * p.heads) return;
-    const int seg = (int)(idx % kSegsPerRow);
+    const int seg = (int)(idx % p.segs_per_row);
     const int b = (int)(pair / p.heads), h = (int)(pair % p.heads);
     const bool reporter = seg == 0 && h == 0 && p.status != nullptr;
     asm volatile("griddepcontrol.launch_dependents;");      // the next kernel may start being scheduled
@@ -59,8 +59,8 @@ kv_append_kernel(const AppendParams p)
     } else {
         row = pair * p.s_max + pos;
     }
-    p.k_cache[row * kSegsPerRow + seg] = p.k_new[idx];
-    p.v_cache[row * kSegsPerRow + seg] = p.v_new[idx];
+    p.k_cache[row * p.segs_per_row + seg] = p.k_new[idx];
+    p.v_cache[row * p.segs_per_row + seg] = p.v_new[idx];
 }
 
 // Bulk append (prefill, Sec. IV-D): new_lens[b] tokens per sequence from token-major
@@ -78,9 +78,9 @@ kv_append_bulk_kernel(const BulkAppendParams q)
 {
     const AppendParams &p = q.base;
     const int64_t idx = (int64_t)blockIdx.x * kAppendThreads + threadIdx.x;
-    const int64_t row = idx / kSegsPerRow;                    // (b, t, h)
+    const int64_t row = idx / p.segs_per_row;                    // (b, t, h)
     if (row >= (int64_t)p.batch * q.max_new * p.heads) return;
-    const int seg = (int)(idx % kSegsPerRow);
+    const int seg = (int)(idx % p.segs_per_row);
     const int h = (int)(row % p.heads);
     const int64_t bt = row / p.heads;
     const int t = (int)(bt % q.max_new), b = (int)(bt / q.max_new);
@@ -106,8 +106,8 @@ kv_append_bulk_kernel(const BulkAppendParams q)
     } else {
         dst = ((int64_t)b * p.heads + h) * p.s_max + pos;
     }
-    p.k_cache[dst * kSegsPerRow + seg] = p.k_new[idx];
-    p.v_cache[dst * kSegsPerRow + seg] = p.v_new[idx];
+    p.k_cache[dst * p.segs_per_row + seg] = p.k_new[idx];
+    p.v_cache[dst * p.segs_per_row + seg] = p.v_new[idx];
 }
 
 }  // namespace instinfer

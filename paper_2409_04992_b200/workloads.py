@@ -224,6 +224,42 @@ def generate(w: Workload, layer: int = 0, device: str = "cpu", poison: bool = Tr
                 seq_lens_host=lens, scale=w.scale)
 
 
+@dataclasses.dataclass
+class GroupedCase:
+    """Inputs of the grouped-head / multi-token variant: `base` holds caches, lengths and the
+    block table for `base.workload.heads` KV heads (its own q, k_new, v_new are not used)."""
+
+    base: Case
+    q: torch.Tensor                 # fp16 [B,Tq,Hq,D]
+    k_new: torch.Tensor             # fp16 [B,Tq,Hkv,D], token-major as the bulk append takes it
+    v_new: torch.Tensor
+    new_lens: torch.Tensor          # int32 [B]: min(Tq, seq_len), the tokens this step appends
+
+    @property
+    def q_tokens(self) -> int:
+        return self.q.shape[1]
+
+
+def generate_grouped(w: Workload, q_tokens: int, q_heads: int, layer: int = 0, device: str = "cpu",
+                     seq_lens: Optional[List[int]] = None) -> GroupedCase:
+    """`w.heads` is the number of KV heads; q_heads must be a multiple of it.  Same arguments,
+    same bits."""
+    if q_heads % w.heads != 0:
+        raise ValueError("q_heads must be a multiple of the workload's (KV) heads")
+    base = generate(w, layer, device, seq_lens=seq_lens)
+    dev = torch.device(device)
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(BASE_SEED + w.index + 1000 * layer + 500)
+    q = torch.empty((w.batch, q_tokens, q_heads, w.head_dim), dtype=torch.float16, device=dev)
+    k_new = torch.empty((w.batch, q_tokens, w.heads, w.head_dim), dtype=torch.float16, device=dev)
+    v_new = torch.empty_like(k_new)
+    for t in (q, k_new, v_new):
+        if t.numel():
+            _fill_normal(t, gen)
+    new_lens = torch.tensor([min(q_tokens, n) for n in base.seq_lens_host], dtype=torch.int32, device=dev)
+    return GroupedCase(base=base, q=q, k_new=k_new, v_new=v_new, new_lens=new_lens)
+
+
 def gather_rows(case: Case, b: int, h: int):
     """The K and V rows of one (sequence, head) as contiguous [L,D] tensors (memory movement
     only: contiguous slice, or a walk of the block table)."""
