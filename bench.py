@@ -578,6 +578,56 @@ def measure_bulk_append(device, steps: int = 10, batch: int = 16, new_tokens: in
             "read_plus_write_gbs": moved / seconds / 1e9, "status_flags": int(flags.item())}
 
 
+GROUPED_SHAPES = [
+    # name, batch, context, block_tokens, kv_heads, q_heads, q_tokens, head_dim
+    ("gqa8_ctx16k_b64_paged16", 64, 16384, 16, 8, 64, 1, 128),
+    ("gqa4_ctx128k_b8_paged64", 8, 131072, 64, 8, 32, 1, 128),
+    ("mha_4new_tokens_ctx16k_b16_paged16", 16, 16384, 16, 40, 40, 4, 128),
+    ("mha_d64_ctx16k_b32_paged16", 32, 16384, 16, 32, 32, 1, 64),
+    ("mha_d256_ctx16k_b16_paged16", 16, 16384, 16, 16, 16, 1, 256),
+]
+
+
+def measure_grouped(device, steps: int = 10) -> dict:
+    """The grouped-head / multi-token / other-head-size entry point on a few long-context
+    shapes: fp16 K+V bytes read per second (each input several GB, far beyond L2)."""
+    from paper_2409_04992_b200 import binding
+    results = {}
+    for name, batch, ctx, tokens, kv_heads, q_heads, q_tokens, dim in GROUPED_SHAPES:
+        w = wl.Workload(name, 7, batch=batch, len_lo=ctx, len_hi=ctx, layout="paged",
+                        block_tokens=tokens, heads=kv_heads, head_dim=dim)
+        g = wl.generate_grouped(w, q_tokens, q_heads, device=str(device))
+        c = g.base
+        flags = torch.zeros(1, dtype=torch.int32, device=device)
+        out = torch.empty_like(g.q)
+        ws = torch.empty(binding.grouped_workspace_bytes(batch, q_tokens, q_heads, kv_heads, dim, ctx),
+                         dtype=torch.uint8, device=device)
+
+        def step():
+            binding.kv_append_bulk(c.k_cache, c.v_cache, g.k_new, g.v_new, c.seq_lens, g.new_lens,
+                                   c.block_table, flags)
+            binding.decode_attention_grouped(out, None, g.q, c.k_cache, c.v_cache, c.block_table,
+                                             c.seq_lens, ctx, c.scale, ws, flags)
+
+        for _ in range(3):
+            step()
+        a, z = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        a.record()
+        for _ in range(steps):
+            step()
+        z.record()
+        torch.cuda.synchronize()
+        seconds = a.elapsed_time(z) / 1e3 / steps
+        kv_bytes = batch * ctx * kv_heads * dim * 2 * 2
+        results[name] = {"value": kv_bytes / seconds / 1e9, "unit": UNIT, "ms_per_step": seconds * 1e3,
+                         "kv_bytes_per_step": kv_bytes, "query_rows_per_kv_head": q_heads // kv_heads * q_tokens,
+                         "status_flags": int(flags.item())}
+        del g, c, out, ws
+        torch.cuda.empty_cache()
+    return results
+
+
 def main(argv=None) -> int:
     args = parse_args(argv)
     if args.impl == "reference":          # CPU only: no process group; ranks other than 0 do nothing
@@ -650,6 +700,7 @@ def main(argv=None) -> int:
                     "reasons": r["clocks"]["reasons"]}
             line["other_workloads"] = others
             line["bulk_append"] = measure_bulk_append(device)
+            line["grouped_attention"] = measure_grouped(device)
             line["sparse_attention"] = {wl.STANDARD[i].name: measure_sparse(wl.STANDARD[i], device, 10)
                                         for i in (2, 3)}
         if ranks.rank == 0:
