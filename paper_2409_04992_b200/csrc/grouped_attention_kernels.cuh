@@ -29,6 +29,13 @@ namespace instinfer {
 constexpr int kGroupRows = 16;         // query rows one MMA tile holds
 constexpr int kGroupTile = 16;         // tokens per warp tile
 constexpr int kGroupStages = 3;
+// Softmax weights enter the second MMA as fp16 hi + lo of weight * 2^kGroupWeightLog2.  A
+// reference may lag its row's maximum by kGroupLag (base 2), so weights reach 2^kGroupLag and
+// the scaled ones 2^15 < 65504.  Small weights fall into fp16 subnormals, where hi and lo each
+// carry an absolute error below 2^-25 (scaled), i.e. below 2^-26 of the row's largest weight.
+constexpr float kGroupLag = 7.f;
+constexpr float kGroupWeightLog2 = 8.f;
+constexpr float kGroupWeightScale = 256.f;
 
 struct GroupedParams {
     // a.heads = KV heads, a.pairs = batch * KV heads; a.q and a.out are
@@ -68,7 +75,7 @@ __device__ __forceinline__ void ldmatrix_x4_trans(unsigned (&r)[4], unsigned add
 // c += a (16x16, row-major fragments) * b (16x8, column fragments); fp16 inputs, fp32 accumulate
 __device__ __forceinline__ void mma_16816(float (&c)[4], const unsigned (&a)[4], unsigned b0, unsigned b1)
 {
-    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0, %1, %2, %3}, "
+    asm("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0, %1, %2, %3}, "
                  "{%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
                  : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
                  : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
@@ -158,46 +165,78 @@ grouped_attn_split_kernel(const GroupedParams p)
     // ---- copy-issue side ----
     // A tile's 16 rows are contiguous in memory in both layouts (a paged block holds a
     // multiple of 16 tokens and chunks start on multiples of 64), so 16-byte segment s of the
-    // tile sits at tile base + 16 s; in shared memory its row is padded.
+    // tile sits at tile base + 16 s; in shared memory its row is padded.  Lane `lane` copies
+    // segments lane + 32 i: global offset 16 lane + 512 i, shared offset lane_dst + i kDstStep.
     const unsigned ring = smem_base + warp * (kGroupStages * G::kStageBytes);
-    constexpr int kTileRowSegs = D / 8;
-    const unsigned char *k_bytes = reinterpret_cast<const unsigned char *>(a.k);
-    const unsigned char *v_bytes = reinterpret_cast<const unsigned char *>(a.v);
-    const int32_t *table_row = kPaged ? a.block_table + (int64_t)b * a.max_blocks_per_seq : nullptr;
-    auto tile_token = [&](int j) { return begin + (warp + j * kWarps) * kGroupTile; };
-    auto table_entry = [&](int j) -> int {
-        return kPaged && j < my_tiles ? __ldg(table_row + tile_token(j) / a.block_tokens) : 0;
-    };
-    int next_phys = table_entry(0);            // looked up one tile ahead of its use
+    constexpr int kTileRowSegs = D / 8;                          // 16-byte segments per row
+    constexpr int kRowsPerPass = 32 / kTileRowSegs > 0 ? 32 / kTileRowSegs : 1;   // rows one warp copy covers
+    constexpr int kPassesPerRow = kTileRowSegs / 32 > 0 ? kTileRowSegs / 32 : 1;  // D = 512 and up only
+    static_assert(kPassesPerRow == 1, "rows longer than 512 bytes are not laid out here");
+    constexpr unsigned kDstStep = kRowsPerPass * G::kRowStride;
+    const int lane_row = lane / kTileRowSegs;
+    const unsigned lane_dst = lane_row * G::kRowStride + (lane - lane_row * kTileRowSegs) * 16;
+    const unsigned char *k_lane = reinterpret_cast<const unsigned char *>(a.k) + lane * 16;
+    const unsigned char *v_lane = reinterpret_cast<const unsigned char *>(a.v) + lane * 16;
+    constexpr int kStepTokens = kWarps * kGroupTile;             // a warp's next tile is this far ahead
+    const int first_token = begin + warp * kGroupTile;
+    // Walks this warp's tiles incrementally (no division per tile): contiguous byte offset,
+    // or paged (block index, slot inside the block) and the table entry one tile ahead.
+    int64_t src_off = 0, block_stride = 0, head_off = 0;
+    int blk = 0, rem = 0, step_blk = 0, step_rem = 0, next_phys = 0;
+    const int32_t *table_row = nullptr;
+    if (kPaged) {
+        const int tokens = a.block_tokens;
+        table_row = a.block_table + (int64_t)b * a.max_blocks_per_seq;
+        blk = first_token / tokens;
+        rem = first_token - blk * tokens;
+        step_blk = kStepTokens / tokens;
+        step_rem = kStepTokens - step_blk * tokens;
+        block_stride = (int64_t)a.heads * tokens * G::kRowBytes;
+        head_off = (int64_t)hk * tokens * G::kRowBytes;
+        next_phys = my_tiles > 0 ? __ldg(table_row + blk) : 0;
+    } else {
+        src_off = ((int64_t)pair * a.s_max + first_token) * G::kRowBytes;
+    }
 
     int issue_j = 0;
     unsigned issue_stage = 0;
     auto issue = [&]() {
         if (issue_j < my_tiles) {
-            const int tok0 = tile_token(issue_j);
-            const int rows_here = min(kGroupTile, end - tok0);
+            const int rows_here = end - (first_token + issue_j * kStepTokens);     // >= 1
             bool usable = true;
             int64_t off;
             if (kPaged) {
                 const int phys = next_phys;
-                next_phys = table_entry(issue_j + 1);
                 usable = phys >= 0 && (int64_t)phys < a.num_phys_blocks;
                 if (!usable && lane == 0 && a.status) atomicOr(a.status, kFlagBlockRange);
-                const int slot = tok0 % a.block_tokens;
-                off = usable ? (((int64_t)phys * a.heads + hk) * a.block_tokens + slot) * G::kRowBytes : 0;
+                off = usable ? (int64_t)phys * block_stride + head_off + rem * G::kRowBytes : 0;
+                blk += step_blk;
+                rem += step_rem;
+                if (rem >= a.block_tokens) {
+                    rem -= a.block_tokens;
+                    ++blk;
+                }
+                if (issue_j + 1 < my_tiles) next_phys = __ldg(table_row + blk);
             } else {
-                off = ((int64_t)pair * a.s_max + tok0) * G::kRowBytes;
+                off = src_off;
+                src_off += (int64_t)kStepTokens * G::kRowBytes;
             }
-            const unsigned dst = ring + issue_stage * G::kStageBytes;
+            const unsigned char *ks = k_lane + off, *vs = v_lane + off;
+            const unsigned dst = ring + issue_stage * G::kStageBytes + lane_dst;
+            if (usable && rows_here >= kGroupTile) {               // full tile: no predicates
 #pragma unroll
-            for (int i = 0; i < G::kSegsPerLane; ++i) {
-                const int s = i * 32 + lane;
-                const int row = s / kTileRowSegs, col = s - row * kTileRowSegs;
-                const bool valid = usable && row < rows_here;
-                const int64_t src = valid ? off + (int64_t)s * 16 : 0;
-                const unsigned d = dst + row * G::kRowStride + col * 16;
-                cp_async_16(d, k_bytes + src, valid ? 16 : 0);       // masked rows are zero-filled
-                cp_async_16(d + G::kTileBytes, v_bytes + src, valid ? 16 : 0);
+                for (int i = 0; i < G::kSegsPerLane; ++i) {
+                    cp_async_16(dst + i * kDstStep, ks + i * 512, 16);
+                    cp_async_16(dst + i * kDstStep + G::kTileBytes, vs + i * 512, 16);
+                }
+            } else {                                               // ragged tail: masked rows are zero-filled
+#pragma unroll
+                for (int i = 0; i < G::kSegsPerLane; ++i) {
+                    const bool valid = usable && lane_row + i * kRowsPerPass < rows_here;
+                    const int src = valid ? i * 512 : 0;
+                    cp_async_16(dst + i * kDstStep, ks + src, valid ? 16 : 0);
+                    cp_async_16(dst + i * kDstStep + G::kTileBytes, vs + src, valid ? 16 : 0);
+                }
             }
         }
         cp_async_commit();                     // empty groups keep the count uniform
@@ -215,11 +254,13 @@ grouped_attn_split_kernel(const GroupedParams p)
     const unsigned v_rd = G::kTileBytes + (mrow + (mat & 1) * 8) * G::kRowStride + (mat >> 1) * 16;
 
     // Running state of rows gid (lo) and gid + 8 (hi): reference m (base-2 logits), this
-    // lane's share of the sum l, and the output fragments, which carry kWeightScale.
+    // lane's share of the sum l, and the output fragments; l and o carry kGroupWeightScale.
     float m_lo = kMinusHuge, m_hi = kMinusHuge, l_lo = 0.f, l_hi = 0.f;
     float o[D / 8][4];
 #pragma unroll
     for (int i = 0; i < D / 8; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
+    // Tiles that end at or before this position need no causal or length mask for any row.
+    const int unmasked_end = len - (p.q_tokens - 1);
 
 #pragma unroll
     for (int j = 0; j < kGroupStages - 1; ++j) issue();
@@ -231,53 +272,63 @@ grouped_attn_split_kernel(const GroupedParams p)
         issue();                         // refills the slot tile j-1 used
         const unsigned base = ring + stage * G::kStageBytes;
         stage = stage + 1 == kGroupStages ? 0 : stage + 1;
-        const int tok0 = tile_token(j);
+        const int tok0 = first_token + j * kStepTokens;
 
         // Logits of 16 rows x 16 tokens: s[n][0..1] row gid, s[n][2..3] row gid + 8, tokens
-        // tok0 + 8 n + 2 quad + {0, 1}.
+        // tok0 + 8 n + 2 quad + {0, 1}.  Even and odd k-steps accumulate separately so that
+        // four independent MMA chains are in flight.
         float s[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+        float s_odd[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
 #pragma unroll
         for (int ks = 0; ks < G::kKSteps; ++ks) {
             unsigned kb[4];
             ldmatrix_x4(kb, base + k_rd + ks * 32);
+            float (&acc)[2][4] = (ks & 1) ? s_odd : s;
             if (G::kQInSmem) {
                 unsigned qf[4];
                 ldmatrix_x4(qf, q_rd + ks * 32);
-                mma_16816(s[0], qf, kb[0], kb[1]);
-                mma_16816(s[1], qf, kb[2], kb[3]);
+                mma_16816(acc[0], qf, kb[0], kb[1]);
+                mma_16816(acc[1], qf, kb[2], kb[3]);
             } else {
-                mma_16816(s[0], qa[ks], kb[0], kb[1]);
-                mma_16816(s[1], qa[ks], kb[2], kb[3]);
+                mma_16816(acc[0], qa[ks], kb[0], kb[1]);
+                mma_16816(acc[1], qa[ks], kb[2], kb[3]);
             }
         }
-        bool grows = false;
 #pragma unroll
         for (int n = 0; n < 2; ++n) {
 #pragma unroll
-            for (int e = 0; e < 2; ++e) {
-                const int tok = tok0 + n * 8 + quad * 2 + e;
-                s[n][e] = tok < vis_lo ? s[n][e] * a.scale_log2e : -INFINITY;
-                s[n][2 + e] = tok < vis_hi ? s[n][2 + e] * a.scale_log2e : -INFINITY;
-                grows |= s[n][e] > m_lo + kMaxLag || s[n][2 + e] > m_hi + kMaxLag;
+            for (int e = 0; e < 4; ++e) s[n][e] = (s[n][e] + s_odd[n][e]) * a.scale_log2e;
+        }
+        if (tok0 + kGroupTile > unmasked_end) {      // uniform: last tiles of the sequence only
+#pragma unroll
+            for (int n = 0; n < 2; ++n) {
+#pragma unroll
+                for (int e = 0; e < 2; ++e) {
+                    const int tok = tok0 + n * 8 + quad * 2 + e;
+                    if (tok >= vis_lo) s[n][e] = -INFINITY;
+                    if (tok >= vis_hi) s[n][2 + e] = -INFINITY;
+                }
             }
         }
         // Online softmax with per-row references that may lag the true maximum by up to
-        // kMaxLag (base-2 units): weights reach at most 2^kMaxLag, inside the range of the
+        // kGroupLag (base-2 units): weights reach at most 2^kGroupLag, inside the range of the
         // fp16 weight split.  References move, and accumulators are rescaled, only when some
-        // logit exceeds its row's reference by more than that.
-        if (__any_sync(0xffffffffu, grows)) {
-            float top_lo = fmaxf(fmaxf(s[0][0], s[0][1]), fmaxf(s[1][0], s[1][1]));
-            float top_hi = fmaxf(fmaxf(s[0][2], s[0][3]), fmaxf(s[1][2], s[1][3]));
+        // logit exceeds its row's reference by more than that: with 16 rows sharing the
+        // rescaling, a tight lag would rescale on most tiles of a short chunk.
+        const float top_lo_here = fmaxf(fmaxf(s[0][0], s[0][1]), fmaxf(s[1][0], s[1][1]));
+        const float top_hi_here = fmaxf(fmaxf(s[0][2], s[0][3]), fmaxf(s[1][2], s[1][3]));
+        if (__any_sync(0xffffffffu, top_lo_here > m_lo + kGroupLag || top_hi_here > m_hi + kGroupLag)) {
+            float top_lo = top_lo_here, top_hi = top_hi_here;
             top_lo = fmaxf(top_lo, __shfl_xor_sync(0xffffffffu, top_lo, 1));
             top_lo = fmaxf(top_lo, __shfl_xor_sync(0xffffffffu, top_lo, 2));
             top_hi = fmaxf(top_hi, __shfl_xor_sync(0xffffffffu, top_hi, 1));
             top_hi = fmaxf(top_hi, __shfl_xor_sync(0xffffffffu, top_hi, 2));
             float alpha_lo = 1.f, alpha_hi = 1.f;
-            if (top_lo > m_lo + kMaxLag) {
+            if (top_lo > m_lo + kGroupLag) {
                 alpha_lo = fast_exp2(m_lo - top_lo);
                 m_lo = top_lo;
             }
-            if (top_hi > m_hi + kMaxLag) {
+            if (top_hi > m_hi + kGroupLag) {
                 alpha_hi = fast_exp2(m_hi - top_hi);
                 m_hi = top_hi;
             }
@@ -291,37 +342,46 @@ grouped_attn_split_kernel(const GroupedParams p)
                 o[i][3] *= alpha_hi;
             }
         }
-        // Weights, their sums, and the A fragments of P V as fp16 hi + lo of weight * 2^14.
+        // Weights (scaled by kGroupWeightScale: the scale is folded into the exponent), their
+        // sums, and the A fragments of P V as an fp16 hi + lo pair.
+        const float e_lo = m_lo - kGroupWeightLog2, e_hi = m_hi - kGroupWeightLog2;
         unsigned p_hi[4], p_lo[4];
 #pragma unroll
         for (int n = 0; n < 2; ++n) {
-            float w[4], big[4];
+            float w[4];
 #pragma unroll
-            for (int e = 0; e < 4; ++e) w[e] = fast_exp2(s[n][e] - (e < 2 ? m_lo : m_hi)) * kWeightScale;
+            for (int e = 0; e < 4; ++e) w[e] = fast_exp2(s[n][e] - (e < 2 ? e_lo : e_hi));
             l_lo += w[0] + w[1];
             l_hi += w[2] + w[3];
             p_hi[2 * n] = pack_half2(w[0], w[1]);
             p_hi[2 * n + 1] = pack_half2(w[2], w[3]);
             const float2 f_lo = __half22float2(*reinterpret_cast<const __half2 *>(&p_hi[2 * n]));
             const float2 f_hi = __half22float2(*reinterpret_cast<const __half2 *>(&p_hi[2 * n + 1]));
-            big[0] = f_lo.x, big[1] = f_lo.y, big[2] = f_hi.x, big[3] = f_hi.y;
-            p_lo[2 * n] = pack_half2(w[0] - big[0], w[1] - big[1]);
-            p_lo[2 * n + 1] = pack_half2(w[2] - big[2], w[3] - big[3]);
+            p_lo[2 * n] = pack_half2(w[0] - f_lo.x, w[1] - f_lo.y);
+            p_lo[2 * n + 1] = pack_half2(w[2] - f_hi.x, w[3] - f_hi.y);
         }
-        // O += P V: two 8-dim output blocks per ldmatrix.
+        // O += P V: two 8-dim output blocks per ldmatrix, four ldmatrix per group so that
+        // eight independent accumulators separate the hi and the lo MMA of each block.
 #pragma unroll
-        for (int nb = 0; nb < D / 16; ++nb) {
-            unsigned vb[4];
-            ldmatrix_x4_trans(vb, base + v_rd + nb * 32);
-            mma_16816(o[2 * nb], p_hi, vb[0], vb[1]);
-            mma_16816(o[2 * nb + 1], p_hi, vb[2], vb[3]);
-            mma_16816(o[2 * nb], p_lo, vb[0], vb[1]);
-            mma_16816(o[2 * nb + 1], p_lo, vb[2], vb[3]);
+        for (int grp = 0; grp < D / 64; ++grp) {
+            unsigned vb[4][4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) ldmatrix_x4_trans(vb[i], base + v_rd + (grp * 4 + i) * 32);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                mma_16816(o[(grp * 4 + i) * 2], p_hi, vb[i][0], vb[i][1]);
+                mma_16816(o[(grp * 4 + i) * 2 + 1], p_hi, vb[i][2], vb[i][3]);
+            }
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                mma_16816(o[(grp * 4 + i) * 2], p_lo, vb[i][0], vb[i][1]);
+                mma_16816(o[(grp * 4 + i) * 2 + 1], p_lo, vb[i][2], vb[i][3]);
+            }
         }
     }
     cp_async_wait<0>();
 
-    // Row sums over the four lanes that share a row (both l and o carry kWeightScale).
+    // Row sums over the four lanes that share a row (both l and o carry kGroupWeightScale).
     l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 1);
     l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 2);
     l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 1);
@@ -360,7 +420,7 @@ grouped_attn_split_kernel(const GroupedParams p)
         // A row that sees no position of this chunk (causal limit before the chunk) has total 0.
         const bool empty = !(total > 0.f);
         const float value = empty ? 0.f : acc / total;
-        const float lse2 = empty ? kMinusHuge : top + log2f(total / kWeightScale);
+        const float lse2 = empty ? kMinusHuge : top + log2f(total) - kGroupWeightLog2;
         if (final_writer) {
             const int64_t row = grouped_row_index(p, b, hk, r);
             a.out[row * D + d] = __float2half_rn(value);
