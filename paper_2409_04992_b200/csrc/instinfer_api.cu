@@ -90,7 +90,16 @@ struct SplitPlan {
 // chunks at the end of the longest sequences run last: making those short keeps the tail of
 // a launch (SMs idling while the last blocks finish) short without paying the per-block
 // overhead of small chunks everywhere.
-SplitPlan make_plan(int64_t pairs, int32_t max_seq_len, int ctas_per_sm = kCtasPerSm)
+// What differs between the kernels that share the planner.
+struct PlanRules {
+    int ctas_per_sm;
+    int target_waves;
+    int chunk_ceiling;
+    bool short_tail_chunks;
+};
+constexpr PlanRules kOneRowRules = {kCtasPerSm, kTargetWaves, kChunkCeiling, true};
+
+SplitPlan make_plan(int64_t pairs, int32_t max_seq_len, const PlanRules &rules = kOneRowRules)
 {
     SplitPlan plan;
     if (g_forced_chunk > 0) {
@@ -99,13 +108,13 @@ SplitPlan make_plan(int64_t pairs, int32_t max_seq_len, int ctas_per_sm = kCtasP
         plan.n_splits = plan.n_big;
         return plan;
     }
-    const int64_t slots = (int64_t)sm_count() * ctas_per_sm;
-    const int64_t fewest = ceil_div(max_seq_len, kChunkCeiling);
+    const int64_t slots = (int64_t)sm_count() * rules.ctas_per_sm;
+    const int64_t fewest = ceil_div(max_seq_len, rules.chunk_ceiling);
     // Small problems that cannot fill the GPU with kChunkFloor-token chunks are latency-bound:
     // cut them down to the granule so that more blocks share the work.
     const int64_t floor_tokens = pairs * ceil_div(max_seq_len, kChunkFloor) < slots ? kChunkGranule : kChunkFloor;
     const int64_t most = ceil_div(max_seq_len, floor_tokens);
-    int64_t n = ceil_div(slots * kTargetWaves, pairs);
+    int64_t n = ceil_div(slots * rules.target_waves, pairs);
     if (n > most) n = most;
     if (n < fewest) n = fewest;
     int64_t chunk = ceil_div(ceil_div(max_seq_len, n), kChunkGranule) * kChunkGranule;
@@ -113,7 +122,7 @@ SplitPlan make_plan(int64_t pairs, int32_t max_seq_len, int ctas_per_sm = kCtasP
     // sequences, at most a quarter of the sequence; none when the chunks are that short anyway.
     int64_t tail_tokens = ceil_div(slots * kTailWaves, pairs) * kTailChunk;
     if (tail_tokens > max_seq_len / 4) tail_tokens = max_seq_len / 4 / kTailChunk * kTailChunk;
-    if (chunk <= 2 * kTailChunk || tail_tokens < kTailChunk) tail_tokens = 0;
+    if (chunk <= 2 * kTailChunk || tail_tokens < kTailChunk || !rules.short_tail_chunks) tail_tokens = 0;
     if (tail_tokens > 0)      // rounded down, so that at least tail_tokens are left for the tail
         chunk = (max_seq_len - tail_tokens) / n / kChunkGranule * kChunkGranule;
     int64_t big_span = n * chunk;
@@ -499,10 +508,14 @@ size_t instinfer_allgather_workspace_bytes(int32_t batch, int32_t heads, int32_t
 extern "C++" {
 namespace {
 
-int grouped_ctas_per_sm(int32_t head_dim)
+// The grouped kernel's blocks are heavier (query fragments to load, 16 rows to merge at the
+// end) and its warps are latency-bound, so it prefers long chunks over many waves: measured
+// best with about two waves of blocks, chunks up to 4096 tokens and no short tail chunks.
+PlanRules grouped_rules(int32_t head_dim)
 {
-    return head_dim == 64 ? GroupedGeometry<64>::kCtasPerSm
-         : head_dim == 128 ? GroupedGeometry<128>::kCtasPerSm : GroupedGeometry<256>::kCtasPerSm;
+    const int ctas = head_dim == 64 ? GroupedGeometry<64>::kCtasPerSm
+                   : head_dim == 128 ? GroupedGeometry<128>::kCtasPerSm : GroupedGeometry<256>::kCtasPerSm;
+    return PlanRules{ctas, 2, 4096, false};
 }
 
 size_t grouped_workspace_for(int64_t pairs, int32_t rows, int32_t head_dim, const SplitPlan &plan)
@@ -579,7 +592,7 @@ int instinfer_decode_attention_grouped(void *out, float *lse, const void *q, con
         return INSTINFER_ERR_INVALID_ARG;
 
     const int64_t pairs = (int64_t)batch * kv_heads;
-    const SplitPlan plan = make_plan(pairs, max_seq_len, grouped_ctas_per_sm(head_dim));
+    const SplitPlan plan = make_plan(pairs, max_seq_len, grouped_rules(head_dim));
     GroupedParams p = {};
     p.group = q_heads / kv_heads;
     p.q_tokens = q_tokens;
@@ -627,7 +640,7 @@ size_t instinfer_grouped_workspace_bytes(int32_t batch, int32_t q_tokens, int32_
     const int64_t pairs = (int64_t)batch * kv_heads;
     if (pairs == 0) return 256;
     return grouped_workspace_for(pairs, q_heads / kv_heads * q_tokens, head_dim,
-                                 make_plan(pairs, max_seq_len, grouped_ctas_per_sm(head_dim)));
+                                 make_plan(pairs, max_seq_len, grouped_rules(head_dim)));
 }
 
 int instinfer_decode_step_host(void *out_host, const void *qkv_host, void *qkv_dev, void *out_dev,
