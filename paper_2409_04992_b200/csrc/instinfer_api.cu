@@ -96,8 +96,9 @@ struct PlanRules {
     int target_waves;
     int chunk_ceiling;
     bool short_tail_chunks;
+    int block_overhead_tokens;   // > 0: choose the chunk count by modelled time (see make_plan)
 };
-constexpr PlanRules kOneRowRules = {kCtasPerSm, kTargetWaves, kChunkCeiling, true};
+constexpr PlanRules kOneRowRules = {kCtasPerSm, kTargetWaves, kChunkCeiling, true, 0};
 
 SplitPlan make_plan(int64_t pairs, int32_t max_seq_len, const PlanRules &rules = kOneRowRules)
 {
@@ -117,6 +118,22 @@ SplitPlan make_plan(int64_t pairs, int32_t max_seq_len, const PlanRules &rules =
     int64_t n = ceil_div(slots * rules.target_waves, pairs);
     if (n > most) n = most;
     if (n < fewest) n = fewest;
+    if (rules.block_overhead_tokens > 0) {
+        // Latency-bound blocks of equal length run in whole waves, so time goes as
+        // (waves of blocks) x (chunk length + a fixed per-block cost): take the chunk count
+        // that minimises it, assuming sequences of max_seq_len.
+        int64_t best = -1;
+        const int64_t last = most < fewest + 96 ? most : fewest + 96;
+        for (int64_t c = fewest; c <= last; ++c) {
+            const int64_t len = ceil_div(ceil_div(max_seq_len, c), kChunkGranule) * kChunkGranule;
+            const int64_t cost = ceil_div(pairs * ceil_div(max_seq_len, len), slots) *
+                                 (len + rules.block_overhead_tokens);
+            if (best < 0 || cost < best) {
+                best = cost;
+                n = c;
+            }
+        }
+    }
     int64_t chunk = ceil_div(ceil_div(max_seq_len, n), kChunkGranule) * kChunkGranule;
     // Tail region: about kTailWaves waves of kTailChunk-token blocks at the end of the longest
     // sequences, at most a quarter of the sequence; none when the chunks are that short anyway.
@@ -509,13 +526,14 @@ extern "C++" {
 namespace {
 
 // The grouped kernel's blocks are heavier (query fragments to load, 16 rows to merge at the
-// end) and its warps are latency-bound, so it prefers long chunks over many waves: measured
-// best with about two waves of blocks, chunks up to 4096 tokens and no short tail chunks.
+// end: about the cost of 20 tiles) and its warps are latency-bound, so a launch takes whole
+// waves of blocks: the chunk count is chosen by that model, chunks up to 4096 tokens, no
+// short tail chunks.
 PlanRules grouped_rules(int32_t head_dim)
 {
     const int ctas = head_dim == 64 ? GroupedGeometry<64>::kCtasPerSm
                    : head_dim == 128 ? GroupedGeometry<128>::kCtasPerSm : GroupedGeometry<256>::kCtasPerSm;
-    return PlanRules{ctas, 2, 4096, false};
+    return PlanRules{ctas, 2, 4096, false, 320};
 }
 
 size_t grouped_workspace_for(int64_t pairs, int32_t rows, int32_t head_dim, const SplitPlan &plan)
