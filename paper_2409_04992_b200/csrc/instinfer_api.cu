@@ -930,7 +930,6 @@ int instinfer_sparf_decode_attention(void *out, float *alpha, int32_t *selected,
     }
     sparf_scores_kernel<<<(unsigned)(pairs * sp.score_blocks), kSparfThreads, 0, stream>>>(sp);
     // Steps 5-7, chunk-parallel; rows it cannot settle are redone by the single-block kernel.
-    sparf_range_kernel<<<chunk_grid, kChunkThreads, 0, stream>>>(sp);
     sparf_hist_kernel<<<chunk_grid, kChunkThreads, 0, stream>>>(sp);
     sparf_locate_kernel<<<row_grid, 32, 0, stream>>>(sp);
     sparf_collect_kernel<<<chunk_grid, kChunkThreads, 0, stream>>>(sp);

@@ -10,7 +10,7 @@
 //                         with the last l tokens forced in (a monotone linear histogram finds
 //                         the threshold bin, its members are resolved exactly; ties to the
 //                         lower position), alpha, and the ascending list of selected rows as
-//                         physical row ids.  Run chunk-parallel by sparf_range / hist /
+//                         physical row ids.  Run chunk-parallel by sparf_hist /
 //                         locate / collect / threshold / compact / finish kernels; rows with
 //                         too many nearly equal scores fall back to sparf_select_kernel,
 //                         which does the same steps with one block per row.
@@ -183,6 +183,13 @@ sparf_append_bulk_kernel(const SparfBulkParams q)
     p.v_sum[(int64_t)pair * kHeadDim + d] = sum;
 }
 
+// Order-preserving map float -> uint32 (larger float, larger key).
+__device__ __forceinline__ unsigned ordered_key(float x)
+{
+    const unsigned u = __float_as_uint(x);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
 // grid pairs * score_blocks: approximate logits of kScoreBlockTokens tokens of one (sequence, head).
 __global__ void __launch_bounds__(kSparfThreads)
 sparf_scores_kernel(const SparfParams p)
@@ -237,6 +244,7 @@ sparf_scores_kernel(const SparfParams p)
     const int T = p.kt_block_tokens;
     const int32_t *table_row = p.kt_block_table + (int64_t)b * p.kt_max_blocks_per_seq;
     float *dst = p.scores + (int64_t)pair * p.score_stride;
+    float top = kMinusHuge, low = -kMinusHuge;          // range of this thread's logits
     for (int i = begin + d * 8; i < end; i += kSparfThreads * 8) {
         const int blk = i / T, slot = i - blk * T;
         const int phys = table_row[blk];
@@ -269,16 +277,41 @@ sparf_scores_kernel(const SparfParams p)
         // score_stride is a multiple of 8 and rows start 32-byte aligned; entries past `end`
         // inside the last group are scratch nobody reads.
         float4 *out4 = reinterpret_cast<float4 *>(dst + i);
-        out4[0] = make_float4(dot[0] * approx_scale, dot[1] * approx_scale, dot[2] * approx_scale, dot[3] * approx_scale);
-        out4[1] = make_float4(dot[4] * approx_scale, dot[5] * approx_scale, dot[6] * approx_scale, dot[7] * approx_scale);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) dot[e] *= approx_scale;
+        if (i + 8 <= end) {
+            top = fmaxf(top, fmaxf(fmaxf(fmaxf(dot[0], dot[1]), fmaxf(dot[2], dot[3])),
+                                   fmaxf(fmaxf(dot[4], dot[5]), fmaxf(dot[6], dot[7]))));
+            low = fminf(low, fminf(fminf(fminf(dot[0], dot[1]), fminf(dot[2], dot[3])),
+                                   fminf(fminf(dot[4], dot[5]), fminf(dot[6], dot[7]))));
+        } else {
+            for (int e = 0; i + e < end; ++e) {
+                top = fmaxf(top, dot[e]);
+                low = fminf(low, dot[e]);
+            }
+        }
+        out4[0] = make_float4(dot[0], dot[1], dot[2], dot[3]);
+        out4[1] = make_float4(dot[4], dot[5], dot[6], dot[7]);
     }
-}
-
-// Order-preserving map float -> uint32 (larger float, larger key).
-__device__ __forceinline__ unsigned ordered_key(float x)
-{
-    const unsigned u = __float_as_uint(x);
-    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+    // Range of the row's logits (what the linear bins of the selection span): two atomics per block.
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) {
+        top = fmaxf(top, __shfl_xor_sync(0xffffffffu, top, off));
+        low = fminf(low, __shfl_xor_sync(0xffffffffu, low, off));
+    }
+    if ((d & 31) == 0) {
+        sm_red[0][d >> 5] = top;
+        sm_red[1][d >> 5] = low;
+    }
+    __syncthreads();
+    if (d == 0) {
+        for (int w = 1; w < kSparfThreads / 32; ++w) {
+            top = fmaxf(top, sm_red[0][w]);
+            low = fminf(low, sm_red[1][w]);
+        }
+        atomicMax(&p.rows_state[pair].max_key, ordered_key(top));
+        atomicMax(&p.rows_state[pair].neg_min_key, ~ordered_key(low));
+    }
 }
 
 template <typename T>
@@ -649,7 +682,7 @@ sparf_select_kernel(const SparfParams p)
 // ---------------------------------------------------------------------------------------
 // Chunk-parallel selection.  The same steps as sparf_select_kernel, but every pass over the
 // scores runs as one block per (row, 2048-token chunk), so that long rows use the whole GPU:
-//   range   -> per-row min / max of the logits (two atomicMax per block)
+//   (the per-row min / max of the logits comes from the score kernel: two atomicMax per block)
 //   hist    -> per-row histogram over the monotone linear bins, softmax denominator parts
 //   locate  -> the bin holding the k-th largest (one warp per row)
 //   collect -> per chunk, how many tokens lie in higher bins (surely selected), and the
@@ -722,40 +755,6 @@ __device__ __forceinline__ bool load_chunk(const SparfParams &p, ChunkView &c)
 __device__ __forceinline__ int linear_bin(const SelectRow &row, int S, int window, int i, float x)
 {
     return i >= S - window ? kLinearBins : min(kLinearBins - 1, (int)((x - row.low) * row.bin_scale));
-}
-
-__global__ void __launch_bounds__(kChunkThreads)
-sparf_range_kernel(const SparfParams p)
-{
-    __shared__ float sm[2][kChunkThreads / 32];
-    ChunkView c;
-    if (!load_chunk(p, c)) return;
-    float top = kMinusHuge, low = -kMinusHuge;
-#pragma unroll
-    for (int e = 0; e < 8; ++e) {
-        if (c.i0 + e < c.S) {
-            top = fmaxf(top, c.x[e]);
-            low = fminf(low, c.x[e]);
-        }
-    }
-#pragma unroll
-    for (int off = 16; off >= 1; off >>= 1) {
-        top = fmaxf(top, __shfl_xor_sync(0xffffffffu, top, off));
-        low = fminf(low, __shfl_xor_sync(0xffffffffu, low, off));
-    }
-    if ((threadIdx.x & 31) == 0) {
-        sm[0][threadIdx.x >> 5] = top;
-        sm[1][threadIdx.x >> 5] = low;
-    }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        for (int w = 1; w < kChunkThreads / 32; ++w) {
-            top = fmaxf(top, sm[0][w]);
-            low = fminf(low, sm[1][w]);
-        }
-        atomicMax(&p.rows_state[c.pair].max_key, ordered_key(top));
-        atomicMax(&p.rows_state[c.pair].neg_min_key, ~ordered_key(low));
-    }
 }
 
 __global__ void __launch_bounds__(kChunkThreads)
