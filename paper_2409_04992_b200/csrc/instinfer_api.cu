@@ -928,15 +928,15 @@ int instinfer_sparf_decode_attention(void *out, float *alpha, int32_t *selected,
         (void)cudaGetLastError();
         return INSTINFER_ERR_CUDA;
     }
-    sparf_scores_kernel<<<(unsigned)(pairs * sp.score_blocks), kSparfThreads, 0, stream>>>(sp);
+    launch_overlapped(sparf_scores_kernel, (unsigned)(pairs * sp.score_blocks), kSparfThreads, 0, stream, sp);
     // Steps 5-7, chunk-parallel; rows it cannot settle are redone by the single-block kernel.
-    sparf_hist_kernel<<<chunk_grid, kChunkThreads, 0, stream>>>(sp);
-    sparf_locate_kernel<<<row_grid, 32, 0, stream>>>(sp);
-    sparf_collect_kernel<<<chunk_grid, kChunkThreads, 0, stream>>>(sp);
-    sparf_threshold_kernel<<<row_grid, kChunkThreads, 0, stream>>>(sp);
-    sparf_compact_kernel<<<chunk_grid, kChunkThreads, 0, stream>>>(sp);
-    sparf_finish_kernel<<<row_grid, 64, 0, stream>>>(sp);
-    sparf_select_kernel<<<row_grid, kSelectThreads, 0, stream>>>(sp);
+    launch_overlapped(sparf_hist_kernel, chunk_grid, kChunkThreads, 0, stream, sp);
+    launch_overlapped(sparf_locate_kernel, row_grid, 32, 0, stream, sp);
+    launch_overlapped(sparf_collect_kernel, chunk_grid, kChunkThreads, 0, stream, sp);
+    launch_overlapped(sparf_threshold_kernel, row_grid, kChunkThreads, 0, stream, sp);
+    launch_overlapped(sparf_compact_kernel, chunk_grid, kChunkThreads, 0, stream, sp);
+    launch_overlapped(sparf_finish_kernel, row_grid, 64, 0, stream, sp);
+    launch_overlapped(sparf_select_kernel, row_grid, kSelectThreads, 0, stream, sp);
     if (cudaGetLastError() != cudaSuccess) return INSTINFER_ERR_CUDA;
 
     SparfMergeParams mp = {};
@@ -974,11 +974,12 @@ int instinfer_sparf_decode_attention(void *out, float *alpha, int32_t *selected,
         }
         smem_set[dev] = true;
     }
-    decode_attn_split_kernel<Rows::kGathered>
-        <<<(unsigned)(pairs * w.plan.n_splits), kThreads, kSplitSmemBytes, stream>>>(ap);
-    if (cudaGetLastError() != cudaSuccess) return INSTINFER_ERR_CUDA;
-    sparf_merge_kernel<<<(unsigned)pairs, kHeadDim, 0, stream>>>(mp);
-    return cudaGetLastError() == cudaSuccess ? INSTINFER_OK : INSTINFER_ERR_CUDA;
+    if (launch_overlapped(decode_attn_split_kernel<Rows::kGathered>, (unsigned)(pairs * w.plan.n_splits),
+                          kThreads, kSplitSmemBytes, stream, ap) != cudaSuccess ||
+        cudaGetLastError() != cudaSuccess)
+        return INSTINFER_ERR_CUDA;
+    const cudaError_t err = launch_overlapped(sparf_merge_kernel, (unsigned)pairs, kHeadDim, 0, stream, mp);
+    return err == cudaSuccess && cudaGetLastError() == cudaSuccess ? INSTINFER_OK : INSTINFER_ERR_CUDA;
 }
 
 size_t instinfer_workspace_bytes(int32_t batch, int32_t heads, int32_t head_dim, int32_t max_seq_len)

@@ -190,10 +190,15 @@ __device__ __forceinline__ unsigned ordered_key(float x)
     return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
+// Every kernel of the attention call below starts with the programmatic-dependent-launch pair
+// (let the next kernel's blocks become resident, then wait for all earlier kernels), before
+// any return, so that the chain of short launches overlaps its launch latencies.
 // grid pairs * score_blocks: approximate logits of kScoreBlockTokens tokens of one (sequence, head).
 __global__ void __launch_bounds__(kSparfThreads)
 sparf_scores_kernel(const SparfParams p)
 {
+    allow_next_kernel();
+    wait_for_previous_kernels();
     __shared__ float sm_abs[kHeadDim];
     __shared__ float sm_q[kHeadDim];        // q of the selected dims, in rank order
     __shared__ int sm_dim[kHeadDim];
@@ -459,6 +464,8 @@ __device__ __forceinline__ void exact_threshold(SelectShared &sh, int n, int nee
 __global__ void __launch_bounds__(kSelectThreads)
 sparf_select_kernel(const SparfParams p)
 {
+    allow_next_kernel();
+    wait_for_previous_kernels();
     __shared__ SelectShared sh;
     const int pair = blockIdx.x, tid = threadIdx.x;
     const int lane = tid & 31, warp = tid >> 5;
@@ -760,6 +767,8 @@ __device__ __forceinline__ int linear_bin(const SelectRow &row, int S, int windo
 __global__ void __launch_bounds__(kChunkThreads)
 sparf_hist_kernel(const SparfParams p)
 {
+    allow_next_kernel();
+    wait_for_previous_kernels();
     __shared__ unsigned hist[kLinearBins + 1];
     __shared__ float red[32];
     ChunkView c;
@@ -790,6 +799,8 @@ sparf_hist_kernel(const SparfParams p)
 __global__ void __launch_bounds__(32)
 sparf_locate_kernel(const SparfParams p)
 {
+    allow_next_kernel();
+    wait_for_previous_kernels();
     const int pair = blockIdx.x, lane = threadIdx.x;
     const int b = pair / p.heads, h = pair - b * p.heads;
     const int S = sparf_seq_len(p, b, lane == 0 && h == 0);
@@ -836,6 +847,8 @@ sparf_locate_kernel(const SparfParams p)
 __global__ void __launch_bounds__(kChunkThreads)
 sparf_collect_kernel(const SparfParams p)
 {
+    allow_next_kernel();
+    wait_for_previous_kernels();
     __shared__ int red[32];
     ChunkView c;
     if (!load_chunk(p, c)) return;
@@ -866,6 +879,8 @@ sparf_collect_kernel(const SparfParams p)
 __global__ void __launch_bounds__(kChunkThreads)
 sparf_threshold_kernel(const SparfParams p)
 {
+    allow_next_kernel();
+    wait_for_previous_kernels();
     __shared__ unsigned keys[kRowCandidates];
     __shared__ int where[kRowCandidates];
     __shared__ unsigned sh_tau;
@@ -922,6 +937,8 @@ sparf_threshold_kernel(const SparfParams p)
 __global__ void __launch_bounds__(kChunkThreads)
 sparf_compact_kernel(const SparfParams p)
 {
+    allow_next_kernel();
+    wait_for_previous_kernels();
     __shared__ int warp_total[kChunkThreads / 32];
     __shared__ int sh_offset;
     __shared__ float red[32];
@@ -999,6 +1016,8 @@ sparf_compact_kernel(const SparfParams p)
 __global__ void __launch_bounds__(64)
 sparf_finish_kernel(const SparfParams p)
 {
+    allow_next_kernel();
+    wait_for_previous_kernels();
     const int pair = blockIdx.x, tid = threadIdx.x;
     const int b = pair / p.heads;
     const SelectRow row = p.rows_state[pair];
@@ -1030,6 +1049,8 @@ struct SparfMergeParams {
 __global__ void __launch_bounds__(kHeadDim)
 sparf_merge_kernel(const SparfMergeParams m)
 {
+    allow_next_kernel();
+    wait_for_previous_kernels();
     const AttnParams &p = m.attn;
     const int pair = blockIdx.x;
     const int b = pair / p.heads;
