@@ -923,7 +923,7 @@ int instinfer_sparf_decode_attention(void *out, float *alpha, int32_t *selected,
     sp.chunk_count = reinterpret_cast<int32_t *>(ws + w.chunk_count);
     sp.chunk_sums = reinterpret_cast<float2 *>(ws + w.chunk_sums);
 
-    const unsigned chunk_grid = (unsigned)(pairs * score_chunks), row_grid = (unsigned)pairs;
+    const unsigned chunk_grid = (unsigned)(pairs * ceil_div(score_chunks, kSubChunks)), row_grid = (unsigned)pairs;
     if (cudaMemsetAsync(ws + w.rows_state, 0, w.zeroed_bytes, stream) != cudaSuccess) {
         (void)cudaGetLastError();
         return INSTINFER_ERR_CUDA;

@@ -688,7 +688,8 @@ sparf_select_kernel(const SparfParams p)
 
 // ---------------------------------------------------------------------------------------
 // Chunk-parallel selection.  The same steps as sparf_select_kernel, but every pass over the
-// scores runs as one block per (row, 2048-token chunk), so that long rows use the whole GPU:
+// scores runs as one block per (row, group of four 2048-token chunks), so that long rows use
+// the whole GPU:
 //   (the per-row min / max of the logits comes from the score kernel: two atomicMax per block)
 //   hist    -> per-row histogram over the monotone linear bins, softmax denominator parts
 //   locate  -> the bin holding the k-th largest (one warp per row)
@@ -731,30 +732,44 @@ __device__ __forceinline__ float float_of_key(unsigned key)
     return __uint_as_float((key & 0x80000000u) ? (key & 0x7fffffffu) : ~key);
 }
 
+constexpr int kSubChunks = 4;             // score chunks handled by one block of the chunk kernels
+
 struct ChunkView {
-    int pair, chunk, b, h, S, k, window, i0;     // i0: first token of this thread
-    float x[8];
+    int pair, chunk0, n_sub, b, h, S, k, window;   // chunks chunk0 .. chunk0 + n_sub - 1 of the row
+    float x[kSubChunks][8];                        // this thread's 8 logits of each chunk
+    __device__ __forceinline__ int first_token(int sub) const
+    {
+        return (chunk0 + sub) * kScoreChunk + (int)threadIdx.x * 8;
+    }
 };
 
-// Common prologue of the chunk kernels: indices, lengths and this thread's 8 logits.
+// Common prologue of the chunk kernels: indices, lengths and this thread's logits.  A block
+// takes kSubChunks consecutive chunks of one row and issues all their loads together, so the
+// latency of one global round trip is paid once per 8192 tokens instead of once per 2048.
 __device__ __forceinline__ bool load_chunk(const SparfParams &p, ChunkView &c)
 {
-    c.pair = blockIdx.x / p.score_chunks;
-    c.chunk = blockIdx.x - c.pair * p.score_chunks;
+    const int groups = (p.score_chunks + kSubChunks - 1) / kSubChunks;
+    c.pair = blockIdx.x / groups;
+    c.chunk0 = (blockIdx.x - c.pair * groups) * kSubChunks;
     c.b = c.pair / p.heads;
     c.h = c.pair - c.b * p.heads;
     c.S = sparf_seq_len(p, c.b, false);
     c.k = min(c.S, min(max(p.k_tokens[c.b], 0), p.max_k));
     c.window = min(p.window, c.k);
-    c.i0 = c.chunk * kScoreChunk + threadIdx.x * 8;
-    if (c.chunk * kScoreChunk >= c.S) return false;
+    if (c.chunk0 * kScoreChunk >= c.S) return false;
+    c.n_sub = min(kSubChunks, (c.S - c.chunk0 * kScoreChunk + kScoreChunk - 1) / kScoreChunk);
+    const float *row_scores = p.scores + (int64_t)c.pair * p.score_stride;
 #pragma unroll
-    for (int e = 0; e < 8; ++e) c.x[e] = 0.f;
-    if (c.i0 < c.S) {                              // rows are padded to whole groups of 8
-        const float4 *src = reinterpret_cast<const float4 *>(p.scores + (int64_t)c.pair * p.score_stride + c.i0);
-        const float4 a = src[0], b = src[1];
-        c.x[0] = a.x; c.x[1] = a.y; c.x[2] = a.z; c.x[3] = a.w;
-        c.x[4] = b.x; c.x[5] = b.y; c.x[6] = b.z; c.x[7] = b.w;
+    for (int sub = 0; sub < kSubChunks; ++sub) {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) c.x[sub][e] = 0.f;
+        const int i0 = c.first_token(sub);
+        if (i0 < c.S) {                            // rows are padded to whole groups of 8
+            const float4 *src = reinterpret_cast<const float4 *>(row_scores + i0);
+            const float4 a = src[0], b = src[1];
+            c.x[sub][0] = a.x; c.x[sub][1] = a.y; c.x[sub][2] = a.z; c.x[sub][3] = a.w;
+            c.x[sub][4] = b.x; c.x[sub][5] = b.y; c.x[sub][6] = b.z; c.x[sub][7] = b.w;
+        }
     }
     return true;
 }
@@ -779,20 +794,31 @@ sparf_hist_kernel(const SparfParams p)
     row.bin_scale = row.top > row.low ? (float)(kLinearBins - 1) / (row.top - row.low) : 0.f;
     for (int t = threadIdx.x; t <= kLinearBins; t += kChunkThreads) hist[t] = 0u;
     __syncthreads();
-    float z = 0.f;
+    float z[kSubChunks];
 #pragma unroll
-    for (int e = 0; e < 8; ++e) {
-        const int i = c.i0 + e;
-        if (i < c.S) {
-            z += fast_exp2(c.x[e] - row.top);
-            atomicAdd(&hist[linear_bin(row, c.S, c.window, i, c.x[e])], 1u);
+    for (int sub = 0; sub < kSubChunks; ++sub) {
+        z[sub] = 0.f;
+        const int i0 = c.first_token(sub);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            const int i = i0 + e;
+            if (i < c.S) {
+                z[sub] += fast_exp2(c.x[sub][e] - row.top);
+                atomicAdd(&hist[linear_bin(row, c.S, c.window, i, c.x[sub][e])], 1u);
+            }
         }
     }
-    z = block_sum(z, red);                       // its barriers also publish the histogram
+#pragma unroll
+    for (int sub = 0; sub < kSubChunks; ++sub) z[sub] = block_sum(z[sub], red);   // barriers publish the histogram
     unsigned *global_hist = p.row_hist + (int64_t)c.pair * (kLinearBins + 1);
     for (int t = threadIdx.x; t <= kLinearBins; t += kChunkThreads)
         if (hist[t]) atomicAdd(&global_hist[t], hist[t]);
-    if (threadIdx.x == 0) p.chunk_sums[blockIdx.x].x = z;
+    if ((int)threadIdx.x < c.n_sub) {
+        float mine = z[0];
+#pragma unroll
+        for (int sub = 1; sub < kSubChunks; ++sub) if ((int)threadIdx.x == sub) mine = z[sub];
+        p.chunk_sums[(int64_t)c.pair * p.score_chunks + c.chunk0 + threadIdx.x].x = mine;
+    }
 }
 
 // One warp per row.
@@ -838,7 +864,7 @@ sparf_locate_kernel(const SparfParams p)
         row->above = above;
         if (bin == kLinearBins) {
             row->tau = 0xffffffffu;
-            row->idx_cut = 0x7fffffff;
+            row->idx_cut = -1;                 // nothing outside the window is taken
             row->solved = 1;
         }
     }
@@ -854,25 +880,35 @@ sparf_collect_kernel(const SparfParams p)
     if (!load_chunk(p, c)) return;
     SelectRow *state = p.rows_state + c.pair;
     const SelectRow row = *state;
-    int sure = 0;
-    if (row.bin <= kLinearBins) {
+    int sure[kSubChunks];
+#pragma unroll
+    for (int sub = 0; sub < kSubChunks; ++sub) {
+        sure[sub] = 0;
+        if (row.bin > kLinearBins) continue;
+        const int i0 = c.first_token(sub);
 #pragma unroll
         for (int e = 0; e < 8; ++e) {
-            const int i = c.i0 + e;
+            const int i = i0 + e;
             if (i < c.S) {
-                const int bin = linear_bin(row, c.S, c.window, i, c.x[e]);
+                const int bin = linear_bin(row, c.S, c.window, i, c.x[sub][e]);
                 if (bin > row.bin || (bin == kLinearBins && row.bin == kLinearBins)) {
-                    ++sure;
+                    ++sure[sub];
                 } else if (bin == row.bin) {
                     const int at = atomicAdd(&state->n_cand, 1);
                     if (at < kRowCandidates)
-                        p.row_cand[(int64_t)c.pair * kRowCandidates + at] = make_uint2(ordered_key(c.x[e]), (unsigned)i);
+                        p.row_cand[(int64_t)c.pair * kRowCandidates + at] = make_uint2(ordered_key(c.x[sub][e]), (unsigned)i);
                 }
             }
         }
     }
-    sure = block_sum(sure, red);
-    if (threadIdx.x == 0) p.chunk_count[blockIdx.x] = sure;
+#pragma unroll
+    for (int sub = 0; sub < kSubChunks; ++sub) sure[sub] = block_sum(sure[sub], red);
+    if ((int)threadIdx.x < c.n_sub) {
+        int mine = sure[0];
+#pragma unroll
+        for (int sub = 1; sub < kSubChunks; ++sub) if ((int)threadIdx.x == sub) mine = sure[sub];
+        p.chunk_count[(int64_t)c.pair * p.score_chunks + c.chunk0 + threadIdx.x] = mine;
+    }
 }
 
 // One block per row: exact threshold among the collected candidates.
@@ -942,75 +978,92 @@ sparf_compact_kernel(const SparfParams p)
     __shared__ int warp_total[kChunkThreads / 32];
     __shared__ int sh_offset;
     __shared__ float red[32];
-    __shared__ int list_pos[kScoreChunk];        // positions of this chunk's selected tokens, ascending
+    __shared__ int list_pos[kScoreChunk];        // positions of one chunk's selected tokens, ascending
     __shared__ float list_x[kScoreChunk];        // and their logits
     ChunkView c;
     if (!load_chunk(p, c)) return;
     const SelectRow row = p.rows_state[c.pair];
     if (!row.solved || row.bin > kLinearBins) return;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    if (warp == 0) {                             // tokens selected in the chunks before this one
+    if (warp == 0) {                             // tokens selected in the chunks before this block's
         int before = 0;
-        for (int j = lane; j < c.chunk; j += 32) before += p.chunk_count[(int64_t)c.pair * p.score_chunks + j];
+        for (int j = lane; j < c.chunk0; j += 32) before += p.chunk_count[(int64_t)c.pair * p.score_chunks + j];
 #pragma unroll
         for (int off = 16; off >= 1; off >>= 1) before += __shfl_xor_sync(0xffffffffu, before, off);
         if (lane == 0) sh_offset = before;
     }
-    // Which of this thread's 8 tokens are selected (cheap, branch-free), as a bit mask.
-    unsigned take = 0u;
-#pragma unroll
-    for (int e = 0; e < 8; ++e) {
-        const int i = c.i0 + e;
-        const int bin = linear_bin(row, c.S, c.window, i, c.x[e]);
-        const unsigned key = ordered_key(c.x[e]);
-        const bool sure = bin > row.bin || (bin == kLinearBins && row.bin == kLinearBins);
-        const bool tied = bin == row.bin && (key > row.tau || (key == row.tau && i <= row.idx_cut));
-        take |= (unsigned)(i < c.S && (sure || tied)) << e;
-    }
-    const int mine = __popc(take);
-    int incl = mine;
-#pragma unroll
-    for (int off = 1; off < 32; off <<= 1) {
-        const int up = __shfl_up_sync(0xffffffffu, incl, off);
-        if (lane >= off) incl += up;
-    }
-    if (lane == 31) warp_total[warp] = incl;
-    __syncthreads();
-    int local = incl - mine, chunk_total = 0;
-    for (int w = 0; w < kChunkThreads / 32; ++w) {
-        if (w < warp) local += warp_total[w];
-        chunk_total += warp_total[w];
-    }
-    // Dense list of the selected tokens in shared memory: the costly part below then runs
-    // once per selected token instead of once per token slot of every warp.
-#pragma unroll
-    for (int e = 0; e < 8; ++e) {
-        if (take >> e & 1u) {
-            list_pos[local] = c.i0 + e;
-            list_x[local] = c.x[e];
-            ++local;
-        }
-    }
-    __syncthreads();
     const int T = p.block_tokens;
     const int32_t *table_row = p.block_table + (int64_t)c.b * p.max_blocks_per_seq;
     int32_t *rows = p.row_ids + (int64_t)c.pair * p.max_k;
     int32_t *sel = p.selected ? p.selected + (int64_t)c.pair * p.max_k : nullptr;
-    float mass = 0.f;
-    for (int t = threadIdx.x; t < chunk_total; t += kChunkThreads) {
-        const int i = list_pos[t], pos = sh_offset + t;
-        const int blk = i / T, slot = i - blk * T;
-        const int phys = table_row[blk];
-        const bool ok = phys >= 0 && (int64_t)phys < p.num_phys_blocks;
-        if (!ok && p.status) atomicOr(p.status, kFlagBlockRange);
-        if (pos < p.max_k) {                     // always true for a consistent count; guards the buffer
-            rows[pos] = ok ? (phys * p.heads + c.h) * T + slot : 0;
-            if (sel) sel[pos] = i;
+    float mass[kSubChunks];
+    const int window_from = c.S - c.window;      // first position of the forced local window
+    int done = 0;                                // selected tokens of this block's earlier chunks
+#pragma unroll
+    for (int sub = 0; sub < kSubChunks; ++sub) {
+        mass[sub] = 0.f;
+        if (sub >= c.n_sub) continue;            // uniform
+        const int i0 = c.first_token(sub);
+        // Which of this thread's 8 tokens are selected, as a bit mask.  With the exact
+        // threshold known the bins are no longer needed: the bins are monotone in the logit, so
+        // a token is selected iff it lies in the local window, or its key exceeds the
+        // threshold key, or equals it at a position up to the cut.
+        unsigned take = 0u;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            const int i = i0 + e;
+            const unsigned key = ordered_key(c.x[sub][e]);
+            const bool chosen = i >= window_from || key > row.tau || (key == row.tau && i <= row.idx_cut);
+            take |= (unsigned)(i < c.S && chosen) << e;
         }
-        mass += fast_exp2(list_x[t] - row.top);
+        const int mine = __popc(take);
+        int incl = mine;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const int up = __shfl_up_sync(0xffffffffu, incl, off);
+            if (lane >= off) incl += up;
+        }
+        __syncthreads();                         // the previous chunk's list and totals are consumed
+        if (lane == 31) warp_total[warp] = incl;
+        __syncthreads();
+        int local = incl - mine, chunk_total = 0;
+        for (int w = 0; w < kChunkThreads / 32; ++w) {
+            if (w < warp) local += warp_total[w];
+            chunk_total += warp_total[w];
+        }
+        // Dense list of the selected tokens in shared memory: the costly part below then runs
+        // once per selected token instead of once per token slot of every warp.
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            if (take >> e & 1u) {
+                list_pos[local] = i0 + e;
+                list_x[local] = c.x[sub][e];
+                ++local;
+            }
+        }
+        __syncthreads();
+        for (int t = threadIdx.x; t < chunk_total; t += kChunkThreads) {
+            const int i = list_pos[t], pos = sh_offset + done + t;
+            const int blk = i / T, slot = i - blk * T;
+            const int phys = table_row[blk];
+            const bool ok = phys >= 0 && (int64_t)phys < p.num_phys_blocks;
+            if (!ok && p.status) atomicOr(p.status, kFlagBlockRange);
+            if (pos < p.max_k) {                 // always true for a consistent count; guards the buffer
+                rows[pos] = ok ? (phys * p.heads + c.h) * T + slot : 0;
+                if (sel) sel[pos] = i;
+            }
+            mass[sub] += fast_exp2(list_x[t] - row.top);
+        }
+        done += chunk_total;
     }
-    mass = block_sum(mass, red);
-    if (threadIdx.x == 0) p.chunk_sums[blockIdx.x].y = mass;
+#pragma unroll
+    for (int sub = 0; sub < kSubChunks; ++sub) mass[sub] = block_sum(mass[sub], red);
+    if ((int)threadIdx.x < c.n_sub) {
+        float mine = mass[0];
+#pragma unroll
+        for (int sub = 1; sub < kSubChunks; ++sub) if ((int)threadIdx.x == sub) mine = mass[sub];
+        p.chunk_sums[(int64_t)c.pair * p.score_chunks + c.chunk0 + threadIdx.x].y = mine;
+    }
 }
 
 __global__ void __launch_bounds__(64)
