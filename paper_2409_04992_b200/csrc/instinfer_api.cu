@@ -933,7 +933,7 @@ int instinfer_sparf_decode_attention(void *out, float *alpha, int32_t *selected,
     launch_overlapped(sparf_hist_kernel, chunk_grid, kChunkThreads, 0, stream, sp);
     launch_overlapped(sparf_locate_kernel, row_grid, 32, 0, stream, sp);
     launch_overlapped(sparf_collect_kernel, chunk_grid, kChunkThreads, 0, stream, sp);
-    launch_overlapped(sparf_threshold_kernel, row_grid, kChunkThreads, 0, stream, sp);
+    launch_overlapped(sparf_threshold_kernel, row_grid, kThresholdThreads, 0, stream, sp);
     launch_overlapped(sparf_compact_kernel, chunk_grid, kChunkThreads, 0, stream, sp);
     launch_overlapped(sparf_finish_kernel, row_grid, 64, 0, stream, sp);
     launch_overlapped(sparf_select_kernel, row_grid, kSelectThreads, 0, stream, sp);

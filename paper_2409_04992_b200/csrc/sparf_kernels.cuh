@@ -912,7 +912,9 @@ sparf_collect_kernel(const SparfParams p)
 }
 
 // One block per row: exact threshold among the collected candidates.
-__global__ void __launch_bounds__(kChunkThreads)
+constexpr int kThresholdThreads = kRowCandidates;    // one thread per candidate: ranking is O(n) per thread
+
+__global__ void __launch_bounds__(kThresholdThreads)
 sparf_threshold_kernel(const SparfParams p)
 {
     allow_next_kernel();
@@ -929,13 +931,13 @@ sparf_threshold_kernel(const SparfParams p)
     const int k = min(S, min(max(p.k_tokens[b], 0), p.max_k));
     const int n = state->n_cand, need = k - state->above;
     if (n > kRowCandidates || need < 1 || need > n) return;      // left to the single-block kernel
-    for (int t = tid; t < n; t += kChunkThreads) {
+    for (int t = tid; t < n; t += kThresholdThreads) {
         const uint2 c = p.row_cand[(int64_t)pair * kRowCandidates + t];
         keys[t] = c.x;
         where[t] = (int)c.y;
     }
     __syncthreads();
-    for (int t = tid; t < n; t += kChunkThreads) {
+    for (int t = tid; t < n; t += kThresholdThreads) {
         const unsigned mine = keys[t];
         int greater = 0, equal = 0;
         for (int j = 0; j < n; ++j) {
@@ -950,7 +952,7 @@ sparf_threshold_kernel(const SparfParams p)
     __syncthreads();
     const unsigned tau = sh_tau;
     const int take = sh_take;
-    for (int t = tid; t < n; t += kChunkThreads) {               // the take-th smallest position among ties
+    for (int t = tid; t < n; t += kThresholdThreads) {               // the take-th smallest position among ties
         if (keys[t] == tau) {
             int before = 0;
             for (int j = 0; j < n; ++j) before += keys[j] == tau && where[j] < where[t];
@@ -959,7 +961,7 @@ sparf_threshold_kernel(const SparfParams p)
     }
     __syncthreads();
     const int cut = sh_cut;
-    for (int t = tid; t < n; t += kChunkThreads) {
+    for (int t = tid; t < n; t += kThresholdThreads) {
         if (keys[t] > tau || (keys[t] == tau && where[t] <= cut))
             atomicAdd(&p.chunk_count[(int64_t)pair * p.score_chunks + where[t] / kScoreChunk], 1);
     }
