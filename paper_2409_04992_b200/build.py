@@ -10,7 +10,7 @@ _HERE = Path(__file__).resolve().parent
 CSRC = _HERE / "csrc"
 INCLUDE = _HERE.parent / "include"
 LIBRARY = _HERE / "libinstinfer.so"
-SOURCES = [CSRC / "instinfer_api.cu"]
+SOURCES = [CSRC / "instinfer_api.cu"]      # it includes the api_*.inl parts
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo",
               "-Xcompiler", "-fPIC", "-shared", "-cudart", "static", "-Xptxas", "-v"]
 
@@ -23,7 +23,8 @@ def _nvcc() -> str:
 
 
 def _inputs():
-    return list(CSRC.glob("*.cu")) + list(CSRC.glob("*.cuh")) + list(INCLUDE.glob("*.h"))
+    return (list(CSRC.glob("*.cu")) + list(CSRC.glob("*.cuh")) + list(CSRC.glob("*.inl")) +
+            list(INCLUDE.glob("*.h")))
 
 
 def is_current() -> bool:
