@@ -411,7 +411,8 @@ def oracle_pass(case: wl.Case):
     k, v = case.k_cache.numpy(), case.v_cache.numpy()
     t0 = time.perf_counter()
     capi.kv_append(k, v, case.k_new.numpy(), case.v_new.numpy(), lens, block_table=table)
-    capi.decode_attention(case.q.numpy(), k, v, lens, case.scale, block_table=table)
+    out, _, _ = capi.decode_attention(case.q.numpy(), k, v, lens, case.scale, block_table=table)
+    case.oracle_out = out                         # kept for the parity figure of cpu_baseline
     return time.perf_counter() - t0
 
 
@@ -422,8 +423,29 @@ def sample_text(case: wl.Case) -> str:
             f"{w.layout} layout, append + attention")
 
 
-def cpu_baseline(w: wl.Workload, seconds: float) -> dict:
+def device_output_of_sample(case: wl.Case, device) -> torch.Tensor:
+    """The CUDA path's output on the oracle's sample (its own copy of the same bits)."""
+    from paper_2409_04992_b200 import binding
+    moved = {k: (v.to(device) if isinstance(v, torch.Tensor) else v) for k, v in case.__dict__.items()
+             if k != "oracle_out"}
+    dev = wl.Case(**moved)
+    B, H, D = dev.q.shape
+    out = torch.empty((B, H, D), dtype=torch.float16, device=device)
+    ws = binding.alloc_workspace(B, H, D, dev.max_seq_len, device)
+    binding.kv_append(dev.k_cache, dev.v_cache, dev.k_new, dev.v_new, dev.seq_lens, dev.block_table)
+    if dev.block_table is None:
+        binding.decode_attention(out, None, dev.q, dev.k_cache, dev.v_cache, dev.seq_lens,
+                                 dev.max_seq_len, dev.scale, ws)
+    else:
+        binding.decode_attention_paged(out, None, dev.q, dev.k_cache, dev.v_cache, dev.block_table,
+                                       dev.seq_lens, dev.max_seq_len, dev.scale, ws)
+    torch.cuda.synchronize()
+    return out.cpu()
+
+
+def cpu_baseline(w: wl.Workload, seconds: float, device=None) -> dict:
     case, threads = oracle_sample(w, seconds)
+    got = device_output_of_sample(case, device) if device is not None else None
     first = oracle_pass(case)
     passes = 1 + max(0, min(30, int(seconds / max(first, 1e-3)) - 1))   # fill the budget, bounded
     elapsed = first + sum(oracle_pass(case) for _ in range(passes - 1))
@@ -431,7 +453,18 @@ def cpu_baseline(w: wl.Workload, seconds: float) -> dict:
     return {"value": case.kv_bytes_read * passes / elapsed / 1e9, "unit": UNIT, "cores": used,
             "kind": "oracle", "sample": f"{passes} passes over " + sample_text(case),
             "seconds": round(elapsed, 2),
-            "kv_tokens_per_s": case.kv_tokens * passes * case.workload.heads / wl.HEADS_13B / elapsed}
+            "kv_tokens_per_s": case.kv_tokens * passes * case.workload.heads / wl.HEADS_13B / elapsed,
+            **({} if got is None else {"gpu_vs_oracle_on_sample": parity_figures(got, case.oracle_out)})}
+
+
+def parity_figures(got_fp16: torch.Tensor, want) -> dict:
+    """Largest absolute error, and largest relative error over exact values that are normal fp16."""
+    import numpy as np
+    g = got_fp16.numpy().astype(np.float64)
+    diff = np.abs(g - want)
+    big = np.abs(want) >= 2.0 ** -14
+    return {"max_abs": float(diff.max()), "max_rel": float((diff[big] / np.abs(want[big])).max()),
+            "bounds": {"max_abs": 2e-3, "max_rel": 1e-2}, "elements": int(diff.size)}
 
 
 def reference_arm(args, world: int) -> None:
@@ -681,7 +714,7 @@ def main(argv=None) -> int:
                          "avg_launch_ms": main_res["split_seconds"] * 1e3},
         }
         if ranks.rank == 0 and ranks.world == 1 and args.cpu_seconds > 0:
-            line["cpu_baseline"] = cpu_baseline(w, args.cpu_seconds)
+            line["cpu_baseline"] = cpu_baseline(w, args.cpu_seconds, device)
         if not args.no_others and ranks.world == 1:
             others = {}
             for idx in (0, 1, 2, 3):
