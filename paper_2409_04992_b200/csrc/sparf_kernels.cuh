@@ -912,7 +912,8 @@ sparf_collect_kernel(const SparfParams p)
 }
 
 // One block per row: exact threshold among the collected candidates.
-constexpr int kThresholdThreads = kRowCandidates;    // one thread per candidate: ranking is O(n) per thread
+constexpr int kThresholdThreads = 256;    // more threads per row did not help: a row's O(n^2) ranking
+                                          // saturates its SM either way, and many-row launches lost occupancy
 
 __global__ void __launch_bounds__(kThresholdThreads)
 sparf_threshold_kernel(const SparfParams p)
