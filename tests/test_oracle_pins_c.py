@@ -119,3 +119,29 @@ def test_sizing_figures_printed_in_the_paper():
     # ... and batch 128 at 2K tokens is "up to 200 GB".
     gb = workloads.kv_cache_bytes(128, 2048, 40) / 1e9
     assert 0.9 * g["kv_bs128_ctx2k_13b_upto_GB"] < gb <= 1.1 * g["kv_bs128_ctx2k_13b_upto_GB"]
+
+
+def test_embedding_indexed_layout_and_transfer_figures_printed_in_the_paper():
+    import inspect
+
+    import bench
+    g = read_golden()
+    page = 4096
+    # one fp16 embedding per token: a 4 KB page holds 2K tokens; grouping 2-8 embeddings per
+    # page leaves 1K-256 tokens per group (the sizes the transposed K copy's blocks may take)
+    assert page // 2 == g["tokens_per_4KB_page_one_embedding"]
+    assert page // (2 * g["embeddings_per_page_max"]) == g["embedding_group_tokens_min"]
+    assert page // (2 * g["embeddings_per_page_min"]) == g["embedding_group_tokens_max"]
+    kt_default = inspect.signature(bench.measure_sparse).parameters["kt_block_tokens"].default
+    assert g["embedding_group_tokens_min"] <= kt_default <= g["embedding_group_tokens_max"]
+    keep_default = inspect.signature(bench.measure_sparse).parameters["keep"].default
+    assert keep_default * g["default_compression_ratio_inv"] == 1.0
+    # per (sequence, head) and step: the cache holds s rows of K and of V; the decode step moves
+    # q, k_new, v_new in and one output row back -- s/2 times less
+    row = workloads.HEAD_DIM_13B * 2
+    for s_len in (1024, 4096, 131072):
+        assert (2 * s_len * row) / (4 * row) == g["transfer_reduction_per_s"] * s_len
+    # and the benchmark's end-to-end byte accounting is exactly those four rows per (sequence, head)
+    w = workloads.STANDARD[4]
+    per_step = w.layers * w.batch * w.heads * row
+    assert 3 * per_step == 19660800 and per_step == 6553600
