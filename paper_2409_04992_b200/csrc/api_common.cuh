@@ -93,10 +93,10 @@ struct PlanRules {
     int ctas_per_sm;
     int target_waves;
     int chunk_ceiling;
-    bool short_tail_chunks;
+    int tail_chunk_tokens;       // 0: no short chunks at the end of long sequences
     int block_overhead_tokens;   // > 0: choose the chunk count by modelled time (see make_plan)
 };
-constexpr PlanRules kOneRowRules = {kCtasPerSm, kTargetWaves, kChunkCeiling, true, 0};
+constexpr PlanRules kOneRowRules = {kCtasPerSm, kTargetWaves, kChunkCeiling, kTailChunk, 0};
 
 inline SplitPlan make_plan(int64_t pairs, int32_t max_seq_len, const PlanRules &rules = kOneRowRules)
 {
@@ -135,16 +135,17 @@ inline SplitPlan make_plan(int64_t pairs, int32_t max_seq_len, const PlanRules &
     int64_t chunk = ceil_div(ceil_div(max_seq_len, n), kChunkGranule) * kChunkGranule;
     // Tail region: about kTailWaves waves of kTailChunk-token blocks at the end of the longest
     // sequences, at most a quarter of the sequence; none when the chunks are that short anyway.
-    int64_t tail_tokens = ceil_div(slots * kTailWaves, pairs) * kTailChunk;
-    if (tail_tokens > max_seq_len / 4) tail_tokens = max_seq_len / 4 / kTailChunk * kTailChunk;
-    if (chunk <= 2 * kTailChunk || tail_tokens < kTailChunk || !rules.short_tail_chunks) tail_tokens = 0;
+    const int64_t tail_chunk = rules.tail_chunk_tokens > 0 ? rules.tail_chunk_tokens : kTailChunk;
+    int64_t tail_tokens = ceil_div(slots * kTailWaves, pairs) * tail_chunk;
+    if (tail_tokens > max_seq_len / 4) tail_tokens = max_seq_len / 4 / tail_chunk * tail_chunk;
+    if (chunk <= 2 * tail_chunk || tail_tokens < tail_chunk || rules.tail_chunk_tokens <= 0) tail_tokens = 0;
     if (tail_tokens > 0)      // rounded down, so that at least tail_tokens are left for the tail
         chunk = (max_seq_len - tail_tokens) / n / kChunkGranule * kChunkGranule;
     int64_t big_span = n * chunk;
     while (big_span - chunk >= max_seq_len) big_span -= chunk;
     plan.chunk_tokens = (int32_t)chunk;
     plan.n_big = (int32_t)(big_span / chunk);
-    plan.tail_chunk = tail_tokens > 0 ? kTailChunk : (int32_t)chunk;
+    plan.tail_chunk = tail_tokens > 0 ? (int32_t)tail_chunk : (int32_t)chunk;
     plan.n_splits = plan.n_big + (big_span < max_seq_len
                                       ? (int32_t)ceil_div(max_seq_len - big_span, plan.tail_chunk) : 0);
     return plan;
