@@ -350,6 +350,17 @@ size_t instinfer_sparf_workspace_bytes(int32_t batch, int32_t heads, int32_t hea
                                        int32_t max_seq_len, int32_t max_k);
 
 /*
+ * Steps 1-7 of Algorithm 1 have two implementations with identical results: one thread block
+ * per (sequence, head) that keeps the row's approximate logits in shared memory (rows of at
+ * most 16384 tokens), and a chunk-parallel one that passes them through the workspace (any
+ * length).  The library picks by the sizes;
+ * instinfer_set_sparse_path forces the choice for later calls of this process: 0 automatic,
+ * 1 chunk-parallel, 2 one block per row where the rows fit (a tuning and test aid; returns
+ * INSTINFER_OK or INSTINFER_ERR_INVALID_ARG; not thread-safe against concurrent calls).
+ */
+int instinfer_set_sparse_path(int32_t path);
+
+/*
  * Workspace size (bytes, host computation only) for a call with these sizes under the
  * current split plan; 0 if an argument is invalid.
  */

@@ -81,6 +81,8 @@ def load() -> ctypes.CDLL:
                                                          ptr, ptr, i32, i32, i32, i32, i32, i64,
                                                          ptr, i32, i32, i64,
                                                          i32, i32, i32, i32, f32, ptr, sz, ptr, ptr]
+        lib.instinfer_set_sparse_path.restype = ctypes.c_int
+        lib.instinfer_set_sparse_path.argtypes = [i32]
         lib.instinfer_sparf_workspace_bytes.restype = sz
         lib.instinfer_sparf_workspace_bytes.argtypes = [i32, i32, i32, i32, i32]
         lib.instinfer_workspace_bytes.restype = sz
@@ -332,6 +334,11 @@ def sparf_append_bulk(k_pool: torch.Tensor, v_pool: torch.Tensor, kt_pool: torch
         _ptr(seq_lens), _ptr(new_lens), _ptr(block_table), block_table.shape[1], k_pool.shape[2],
         k_pool.shape[0], _ptr(kt_block_table), kt_block_table.shape[1], kt_pool.shape[3],
         kt_pool.shape[0], batch, max_new, heads, head_dim, _ptr(status_flags), _stream(stream)))
+
+
+def set_sparse_path(path: int) -> None:
+    """instinfer_set_sparse_path: 0 automatic, 1 chunk-parallel, 2 one block per row."""
+    _check(load().instinfer_set_sparse_path(int(path)))
 
 
 def sparf_workspace_bytes(batch: int, heads: int, head_dim: int, max_seq_len: int, max_k: int) -> int:

@@ -6,6 +6,8 @@
 
 namespace {
 
+int g_sparse_path = 0;      // 0 automatic, 1 chunk-parallel, 2 one block per row (see instinfer_set_sparse_path)
+
 struct SparfLayout {
     size_t scores, row_ids, stats, rows_state, row_hist, row_cand, chunk_count, chunk_sums, partials, total;
     size_t zeroed_bytes;      // rows_state and row_hist are adjacent and cleared before each call
@@ -227,6 +229,31 @@ int instinfer_sparf_decode_attention(void *out, float *alpha, int32_t *selected,
     sp.chunk_sums = reinterpret_cast<float2 *>(ws + w.chunk_sums);
 
     const unsigned chunk_grid = (unsigned)(pairs * ceil_div(score_chunks, kSubChunks)), row_grid = (unsigned)pairs;
+    // Two ways through steps 1-7.  For rows that fit in shared memory one block per row computes
+    // the logits there and selects from there (nothing goes through HBM); otherwise the logits
+    // go to the workspace and the selection runs chunk-parallel.
+    // Measured: the one-block-per-row form wins wherever the rows fit (by 4-45 %, most at
+    // small batches, where the chunk-parallel chain is all launch latency), except for very
+    // many rows of the largest size (2560 rows of 16384 tokens: 3-7 % slower).
+    const bool fits = max_seq_len <= kFusedMaxTokens;
+    const bool fused = g_sparse_path == 2 ? fits
+                     : g_sparse_path == 1 ? false
+                     : fits && (max_seq_len <= 12288 || pairs < 8 * (int64_t)sm_count());
+    if (fused) {
+        static bool fused_smem_set[kMaxDevices] = {};
+        int device = 0;
+        if (cudaGetDevice(&device) != cudaSuccess || device < 0 || device >= kMaxDevices) return INSTINFER_ERR_CUDA;
+        if (!fused_smem_set[device]) {
+            if (cudaFuncSetAttribute(sparf_fused_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     kFusedSmemBytes) != cudaSuccess) {
+                (void)cudaGetLastError();
+                return INSTINFER_ERR_CUDA;
+            }
+            fused_smem_set[device] = true;
+        }
+        launch_overlapped(sparf_fused_select_kernel, row_grid, kFusedThreads,
+                          (size_t)w.score_stride * sizeof(float), stream, sp);
+    } else {
     if (cudaMemsetAsync(ws + w.rows_state, 0, w.zeroed_bytes, stream) != cudaSuccess) {
         (void)cudaGetLastError();
         return INSTINFER_ERR_CUDA;
@@ -240,6 +267,7 @@ int instinfer_sparf_decode_attention(void *out, float *alpha, int32_t *selected,
     launch_overlapped(sparf_compact_kernel, chunk_grid, kChunkThreads, 0, stream, sp);
     launch_overlapped(sparf_finish_kernel, row_grid, 64, 0, stream, sp);
     launch_overlapped(sparf_select_kernel, row_grid, kSelectThreads, 0, stream, sp);
+    }
     if (cudaGetLastError() != cudaSuccess) return INSTINFER_ERR_CUDA;
 
     SparfMergeParams mp = {};
@@ -283,6 +311,13 @@ int instinfer_sparf_decode_attention(void *out, float *alpha, int32_t *selected,
         return INSTINFER_ERR_CUDA;
     const cudaError_t err = launch_overlapped(sparf_merge_kernel, (unsigned)pairs, kHeadDim, 0, stream, mp);
     return err == cudaSuccess && cudaGetLastError() == cudaSuccess ? INSTINFER_OK : INSTINFER_ERR_CUDA;
+}
+
+int instinfer_set_sparse_path(int32_t path)
+{
+    if (path < 0 || path > 2) return INSTINFER_ERR_INVALID_ARG;
+    g_sparse_path = path;
+    return INSTINFER_OK;
 }
 
 }  // extern "C"

@@ -190,6 +190,94 @@ __device__ __forceinline__ unsigned ordered_key(float x)
     return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
+// Step 1 and the temperature of steps 2-4, shared by the kernels that compute approximate
+// logits.  Threads d < 128 each own one head dim; every thread of the block must call it.
+struct ScoreShared {
+    float abs_q[kHeadDim];
+    float q[kHeadDim];          // q of the selected dims, in rank order
+    int dim[kHeadDim];          // the selected dims, in rank order
+    bool kept[kHeadDim];
+    float approx_scale;
+};
+
+__device__ __forceinline__ void score_setup(const SparfParams &p, int pair, ScoreShared &ss)
+{
+    const int d = threadIdx.x;
+    // Step 1: rank of |q_d| (exact comparisons of fp16 magnitudes, ties to the lower index).
+    float qd = 0.f;
+    if (d < kHeadDim) {
+        qd = __half2float(p.q[(int64_t)pair * kHeadDim + d]);
+        ss.abs_q[d] = fabsf(qd);
+    }
+    __syncthreads();
+    if (d < kHeadDim) {
+        int rank = 0;
+        for (int e = 0; e < kHeadDim; ++e) {
+            const float other = ss.abs_q[e];
+            rank += (other > ss.abs_q[d]) || (other == ss.abs_q[d] && e < d);
+        }
+        const bool kept = rank < p.r;
+        if (kept) {
+            ss.dim[rank] = d;
+            ss.q[rank] = qd;
+        }
+        ss.kept[d] = kept;
+    }
+    // |q|_1 and |q_I|_1.  The top-k of step 6 is decided on the fp32 logits computed below, so
+    // their arithmetic is kept simple enough to be restated elsewhere bit for bit: both sums
+    // run over ascending d in fp32, the temperature uses IEEE division and square root, and
+    // each logit is the fp32 FMA chain over the kept dims in rank order times that constant.
+    __syncthreads();
+    if (d == 0) {
+        float all = 0.f, sel = 0.f;
+        for (int e = 0; e < kHeadDim; ++e) {
+            all += ss.abs_q[e];
+            if (ss.kept[e]) sel += ss.abs_q[e];
+        }
+        const float ratio = all > 0.f ? sel / all : 1.f;
+        ss.approx_scale = p.scale_log2e / sqrtf(ratio);
+    }
+    __syncthreads();
+}
+
+// Steps 2-4 for the 8 consecutive tokens i .. i + 7 of (sequence b, head h): one 16-byte load
+// per selected dim from the transposed copy (kt_block_tokens is a multiple of 8, so a group
+// never straddles a block); the loads of 8 dims are issued together to keep bytes in flight.
+__device__ __forceinline__ void score_group(const SparfParams &p, const ScoreShared &ss,
+                                            const int32_t *table_row, int h, int i, float (&dot)[8])
+{
+    const int T = p.kt_block_tokens;
+    const int blk = i / T, slot = i - blk * T;
+    const int phys = table_row[blk];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) dot[e] = 0.f;
+    if (phys >= 0 && (int64_t)phys < p.num_kt_blocks) {
+        const __half *kt = p.kt_pool + ((int64_t)phys * p.heads + h) * T * kHeadDim + slot;
+        for (int t0 = 0; t0 < p.r; t0 += 8) {
+            uint4 raw[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int t = min(t0 + u, p.r - 1);            // clamped: extra loads repeat the last dim
+                raw[u] = __ldg(reinterpret_cast<const uint4 *>(kt + (int64_t)ss.dim[t] * T));
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                if (t0 + u < p.r) {                            // uniform; extra loads are ignored
+                    const float qv = ss.q[t0 + u];
+                    float kf[8];
+                    unpack8(raw[u], kf);
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) dot[e] = fmaf(qv, kf[e], dot[e]);
+                }
+            }
+        }
+    } else if (p.status) {
+        atomicOr(p.status, kFlagBlockRange);
+    }
+#pragma unroll
+    for (int e = 0; e < 8; ++e) dot[e] *= ss.approx_scale;
+}
+
 // Every kernel of the attention call below starts with the programmatic-dependent-launch pair
 // (let the next kernel's blocks become resident, then wait for all earlier kernels), before
 // any return, so that the chain of short launches overlaps its launch latencies.
@@ -199,91 +287,25 @@ sparf_scores_kernel(const SparfParams p)
 {
     allow_next_kernel();
     wait_for_previous_kernels();
-    __shared__ float sm_abs[kHeadDim];
-    __shared__ float sm_q[kHeadDim];        // q of the selected dims, in rank order
-    __shared__ int sm_dim[kHeadDim];
+    __shared__ ScoreShared ss;
     __shared__ float sm_red[2][kSparfThreads / 32];
-    __shared__ bool sm_kept[kHeadDim];
     const int pair = blockIdx.x / p.score_blocks, d = threadIdx.x;
     const int b = pair / p.heads, h = pair - b * p.heads;
     const int len = sparf_seq_len(p, b, false);
     const int begin = (blockIdx.x - pair * p.score_blocks) * kScoreBlockTokens;
     if (begin >= len) return;
     const int end = min(begin + kScoreBlockTokens, len);
+    score_setup(p, pair, ss);
 
-    // Step 1: rank of |q_d| (exact comparisons of fp16 magnitudes, ties to the lower index).
-    const float qd = __half2float(p.q[(int64_t)pair * kHeadDim + d]);
-    sm_abs[d] = fabsf(qd);
-    __syncthreads();
-    int rank = 0;
-    for (int e = 0; e < kHeadDim; ++e) {
-        const float other = sm_abs[e];
-        rank += (other > sm_abs[d]) || (other == sm_abs[d] && e < d);
-    }
-    const bool kept = rank < p.r;
-    if (kept) {
-        sm_dim[rank] = d;
-        sm_q[rank] = qd;
-    }
-    // |q|_1 and |q_I|_1.  The top-k of step 6 is decided on the fp32 logits computed below, so
-    // their arithmetic is kept simple enough to be restated elsewhere bit for bit: both sums
-    // run over ascending d in fp32, the temperature uses IEEE division and square root, and
-    // each logit is the fp32 FMA chain over the kept dims in rank order times that constant.
-    sm_kept[d] = kept;
-    __syncthreads();
-    if (d == 0) {
-        float all = 0.f, sel = 0.f;
-        for (int e = 0; e < kHeadDim; ++e) {
-            all += sm_abs[e];
-            if (sm_kept[e]) sel += sm_abs[e];
-        }
-        const float ratio = all > 0.f ? sel / all : 1.f;
-        sm_red[0][0] = p.scale_log2e / sqrtf(ratio);
-    }
-    __syncthreads();
-    const float approx_scale = sm_red[0][0];
-
-    // Steps 2-4: one thread per group of 8 consecutive tokens (one 16-byte load per selected
-    // dim; kt_block_tokens is a multiple of 8, so a group never straddles a block).  The loads
-    // of 8 dims are issued together to keep enough bytes in flight.
-    const int T = p.kt_block_tokens;
     const int32_t *table_row = p.kt_block_table + (int64_t)b * p.kt_max_blocks_per_seq;
     float *dst = p.scores + (int64_t)pair * p.score_stride;
     float top = kMinusHuge, low = -kMinusHuge;          // range of this thread's logits
     for (int i = begin + d * 8; i < end; i += kSparfThreads * 8) {
-        const int blk = i / T, slot = i - blk * T;
-        const int phys = table_row[blk];
         float dot[8];
-#pragma unroll
-        for (int e = 0; e < 8; ++e) dot[e] = 0.f;
-        if (phys >= 0 && (int64_t)phys < p.num_kt_blocks) {
-            const __half *kt = p.kt_pool + ((int64_t)phys * p.heads + h) * T * kHeadDim + slot;
-            for (int t0 = 0; t0 < p.r; t0 += 8) {
-                uint4 raw[8];
-#pragma unroll
-                for (int u = 0; u < 8; ++u) {
-                    const int t = min(t0 + u, p.r - 1);            // clamped: extra loads repeat the last dim
-                    raw[u] = __ldg(reinterpret_cast<const uint4 *>(kt + (int64_t)sm_dim[t] * T));
-                }
-#pragma unroll
-                for (int u = 0; u < 8; ++u) {
-                    if (t0 + u < p.r) {                            // uniform; extra loads are ignored
-                        const float qv = sm_q[t0 + u];
-                        float kf[8];
-                        unpack8(raw[u], kf);
-#pragma unroll
-                        for (int e = 0; e < 8; ++e) dot[e] = fmaf(qv, kf[e], dot[e]);
-                    }
-                }
-            }
-        } else if (p.status) {
-            atomicOr(p.status, kFlagBlockRange);
-        }
+        score_group(p, ss, table_row, h, i, dot);
         // score_stride is a multiple of 8 and rows start 32-byte aligned; entries past `end`
         // inside the last group are scratch nobody reads.
         float4 *out4 = reinterpret_cast<float4 *>(dst + i);
-#pragma unroll
-        for (int e = 0; e < 8; ++e) dot[e] *= approx_scale;
         if (i + 8 <= end) {
             top = fmaxf(top, fmaxf(fmaxf(fmaxf(dot[0], dot[1]), fmaxf(dot[2], dot[3])),
                                    fmaxf(fmaxf(dot[4], dot[5]), fmaxf(dot[6], dot[7]))));
@@ -346,19 +368,19 @@ struct SelectShared {
 };
 
 // Streams a score row as float4 with 4 loads in flight per thread; fn(first_index, values[4]).
-template <typename Fn>
+template <int NT, typename Fn>
 __device__ __forceinline__ void for_each_quad(const float4 *a4, int quads, Fn fn)
 {
-    for (int g0 = threadIdx.x; g0 < quads; g0 += 4 * kSelectThreads) {
+    for (int g0 = threadIdx.x; g0 < quads; g0 += 4 * NT) {
         float4 v[4];
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
-            const int g = g0 + u * kSelectThreads;
+            const int g = g0 + u * NT;
             v[u] = g < quads ? a4[g] : make_float4(0.f, 0.f, 0.f, 0.f);
         }
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
-            const int g = g0 + u * kSelectThreads;
+            const int g = g0 + u * NT;
             if (g < quads) {
                 const float x[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
                 fn(4 * g, x);
@@ -398,12 +420,12 @@ __device__ __forceinline__ void locate_bucket(const unsigned *hist, int remainin
 // per pass from the top.  Bytes on which all members agree are skipped without counting, so
 // a set of (nearly) equal keys costs nothing.  Returns through sh.tau / sh.take_equal the
 // threshold key and how many keys equal to it are among the `need` largest.
-template <typename Member, typename KeyAt>
+template <int NT, typename Member, typename KeyAt>
 __device__ __forceinline__ void exact_threshold(SelectShared &sh, int n, int need, Member member, KeyAt key_at)
 {
     const int tid = threadIdx.x;
     unsigned any = 0u, all = 0xffffffffu;
-    for (int i = tid; i < n; i += kSelectThreads) {
+    for (int i = tid; i < n; i += NT) {
         if (member(i)) {
             const unsigned key = key_at(i);
             any |= key;
@@ -423,7 +445,7 @@ __device__ __forceinline__ void exact_threshold(SelectShared &sh, int n, int nee
     __syncthreads();
     any = 0u;
     all = 0xffffffffu;
-    for (int w = 0; w < kSelectThreads / 32; ++w) {
+    for (int w = 0; w < NT / 32; ++w) {
         any |= sh.red_u[0][w];
         all &= sh.red_u[1][w];
     }
@@ -440,7 +462,7 @@ __device__ __forceinline__ void exact_threshold(SelectShared &sh, int n, int nee
         __syncthreads();
         if (tid < 256) sh.hist[tid] = 0u;
         __syncthreads();
-        for (int i = tid; i < n; i += kSelectThreads) {
+        for (int i = tid; i < n; i += NT) {
             if (member(i)) {
                 const unsigned key = key_at(i);
                 if ((key & done_mask) == prefix) atomicAdd(&sh.hist[(key >> shift) & 255u], 1u);
@@ -460,23 +482,17 @@ __device__ __forceinline__ void exact_threshold(SelectShared &sh, int n, int nee
     __syncthreads();
 }
 
-// One block per (sequence, head).
-__global__ void __launch_bounds__(kSelectThreads)
-sparf_select_kernel(const SparfParams p)
+// Steps 5-7 for one (sequence, head) by one block of NT threads (NT a multiple of 32, <= 1024): `a` is the row's
+// S approximate logits (global or shared memory; 32-byte aligned, padded to a multiple of 8
+// readable floats).  Writes the row-id list, the optional `selected` list, alpha and the count.
+template <int NT>
+__device__ __forceinline__ void select_row(const SparfParams &p, SelectShared &sh, const float *a,
+                                           int pair, int b, int h, int S, int k, int window)
 {
-    allow_next_kernel();
-    wait_for_previous_kernels();
-    __shared__ SelectShared sh;
-    const int pair = blockIdx.x, tid = threadIdx.x;
-    const int lane = tid & 31, warp = tid >> 5;
-    const int b = pair / p.heads, h = pair - b * p.heads;
-    if (p.rows_state && p.rows_state[pair].solved) return;      // done by the chunk-parallel kernels
-    const int S = sparf_seq_len(p, b, tid == 0 && h == 0);
-    const int k = min(S, min(max(p.k_tokens[b], 0), p.max_k));
-    const int window = min(p.window, k);
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     int32_t *rows = p.row_ids + (int64_t)pair * p.max_k;
     int32_t *sel = p.selected ? p.selected + (int64_t)pair * p.max_k : nullptr;
-    if (sel) for (int t = k + tid; t < p.max_k; t += kSelectThreads) sel[t] = -1;
+    if (sel) for (int t = k + tid; t < p.max_k; t += NT) sel[t] = -1;
     if (k == 0) {
         if (tid == 0) {
             p.stats[pair] = make_float2(0.f, 0.f);
@@ -484,8 +500,6 @@ sparf_select_kernel(const SparfParams p)
         }
         return;
     }
-    const float *a = p.scores + (int64_t)pair * p.score_stride;
-
     // The score row is 32-byte aligned and padded to a multiple of 8 floats (padding is
     // readable scratch), so every pass streams it as float4 and masks the tail by index.
     const float4 *a4 = reinterpret_cast<const float4 *>(a);
@@ -493,7 +507,7 @@ sparf_select_kernel(const SparfParams p)
 
     // Pass 1: largest and smallest approximate logit (base-2 domain).
     float top = kMinusHuge, low = -kMinusHuge;
-    for_each_quad(a4, quads, [&](int i0, const float (&x)[4]) {
+    for_each_quad<NT>(a4, quads, [&](int i0, const float (&x)[4]) {
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
             if (i0 + e < S) {
@@ -511,9 +525,10 @@ sparf_select_kernel(const SparfParams p)
         sh.red_f[warp] = top;
         sh.red_u[0][warp] = __float_as_uint(low);
     }
-    for (int t = tid; t <= kLinearBins; t += kSelectThreads) sh.hist[t] = 0u;
+    for (int t = tid; t <= kLinearBins; t += NT) sh.hist[t] = 0u;
+    if (tid < 32) sh.scan_gt[tid] = 0;           // warps that do not exist count nothing in the scans
     __syncthreads();
-    for (int w = 0; w < kSelectThreads / 32; ++w) {
+    for (int w = 0; w < NT / 32; ++w) {
         top = fmaxf(top, sh.red_f[w]);
         low = fminf(low, __uint_as_float(sh.red_u[0][w]));
     }
@@ -528,7 +543,7 @@ sparf_select_kernel(const SparfParams p)
 
     // Pass 2: histogram over the linear bins, and the softmax denominator.
     float z = 0.f;
-    for_each_quad(a4, quads, [&](int i0, const float (&x)[4]) {
+    for_each_quad<NT>(a4, quads, [&](int i0, const float (&x)[4]) {
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
             if (i0 + e < S) {
@@ -578,7 +593,7 @@ sparf_select_kernel(const SparfParams p)
         }
         __syncthreads();
     } else if (in_bin <= kCandidates) {
-        for_each_quad(a4, quads, [&](int i0, const float (&x)[4]) {
+        for_each_quad<NT>(a4, quads, [&](int i0, const float (&x)[4]) {
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
                 if (i0 + e < S && bin_of(i0 + e, x[e]) == bin)
@@ -586,7 +601,7 @@ sparf_select_kernel(const SparfParams p)
             }
         });
         __syncthreads();
-        if (in_bin <= kSelectThreads) {          // the usual case: rank every candidate directly
+        if (in_bin <= NT) {          // the usual case: rank every candidate directly
             const int need = k - above;
             if (tid < in_bin) {
                 const unsigned mine = sh.cand[tid];
@@ -603,11 +618,11 @@ sparf_select_kernel(const SparfParams p)
             }
             __syncthreads();
         } else {
-            exact_threshold(sh, in_bin, k - above, [](int) { return true; },
+            exact_threshold<NT>(sh, in_bin, k - above, [](int) { return true; },
                             [&](int i) { return sh.cand[i]; });
         }
     } else {                                     // very many near-equal logits: work from global memory
-        exact_threshold(sh, S, k - above, [&](int i) { return bin_of(i, a[i]) == bin; },
+        exact_threshold<NT>(sh, S, k - above, [&](int i) { return bin_of(i, a[i]) == bin; },
                         [&](int i) { return ordered_key(a[i]); });
     }
     const unsigned tau = sh.tau;                 // key of the k-th largest
@@ -620,10 +635,10 @@ sparf_select_kernel(const SparfParams p)
     float mass = 0.f;
     // Each thread takes 4 consecutive positions; counts travel packed (greater | equal << 16).
     float4 ahead = tid < quads ? a4[tid] : make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int start = 0; start < quads; start += kSelectThreads) {
+    for (int start = 0; start < quads; start += NT) {
         const int g = start + tid;
         const float4 v = ahead;
-        if (g + kSelectThreads < quads) ahead = a4[g + kSelectThreads];    // next tile's loads fly over the barriers
+        if (g + NT < quads) ahead = a4[g + NT];    // next tile's loads fly over the barriers
         float x[4] = {0.f, 0.f, 0.f, 0.f};
         bool gt[4] = {false, false, false, false}, eq[4] = {false, false, false, false};
         int mine = 0;
@@ -684,6 +699,57 @@ sparf_select_kernel(const SparfParams p)
         p.stats[pair] = make_float2(alpha, (float)k);
         if (p.alpha_out) p.alpha_out[pair] = alpha;
     }
+}
+
+// One block per (sequence, head), logits from the workspace: redoes the rows that the
+// chunk-parallel kernels left unsolved.
+__global__ void __launch_bounds__(kSelectThreads)
+sparf_select_kernel(const SparfParams p)
+{
+    allow_next_kernel();
+    wait_for_previous_kernels();
+    __shared__ SelectShared sh;
+    const int pair = blockIdx.x;
+    const int b = pair / p.heads, h = pair - b * p.heads;
+    if (p.rows_state && p.rows_state[pair].solved) return;      // done by the chunk-parallel kernels
+    const int S = sparf_seq_len(p, b, threadIdx.x == 0 && h == 0);
+    const int k = min(S, min(max(p.k_tokens[b], 0), p.max_k));
+    select_row<kSelectThreads>(p, sh, p.scores + (int64_t)pair * p.score_stride, pair, b, h, S, k, min(p.window, k));
+}
+
+// Steps 1-7 for one (sequence, head) by one block: the row's approximate logits are computed
+// straight into shared memory and selected from there, so they never travel through HBM.
+// For rows of at most kFusedMaxTokens tokens.  Two blocks share an SM, so one block's selection
+// (instruction-bound) overlaps the other's loads.
+constexpr int kFusedMaxTokens = 16384;
+constexpr int kFusedSmemBytes = kFusedMaxTokens * (int)sizeof(float);
+constexpr int kFusedThreads = 512;       // two blocks per SM: one selects while the other loads
+
+__global__ void __launch_bounds__(kFusedThreads, 2)
+sparf_fused_select_kernel(const SparfParams p)
+{
+    allow_next_kernel();
+    wait_for_previous_kernels();
+    extern __shared__ __align__(32) float row_scores[];
+    __shared__ SelectShared sh;
+    __shared__ ScoreShared ss;
+    const int pair = blockIdx.x;
+    const int b = pair / p.heads, h = pair - b * p.heads;
+    const int S = sparf_seq_len(p, b, threadIdx.x == 0 && h == 0);
+    const int k = min(S, min(max(p.k_tokens[b], 0), p.max_k));
+    if (k > 0) {                                 // uniform; with k == 0 no logit is needed
+        score_setup(p, pair, ss);
+        const int32_t *table_row = p.kt_block_table + (int64_t)b * p.kt_max_blocks_per_seq;
+        for (int i = threadIdx.x * 8; i < S; i += kFusedThreads * 8) {
+            float dot[8];
+            score_group(p, ss, table_row, h, i, dot);
+            float4 *out4 = reinterpret_cast<float4 *>(row_scores + i);    // S <= kFusedMaxTokens, whole groups
+            out4[0] = make_float4(dot[0], dot[1], dot[2], dot[3]);
+            out4[1] = make_float4(dot[4], dot[5], dot[6], dot[7]);
+        }
+        __syncthreads();
+    }
+    select_row<kFusedThreads>(p, sh, row_scores, pair, b, h, S, k, min(p.window, k));
 }
 
 // ---------------------------------------------------------------------------------------

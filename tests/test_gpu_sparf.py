@@ -20,6 +20,15 @@ pytestmark = pytest.mark.gpu
 ALPHA_ATOL = 2e-5
 
 
+@pytest.fixture(autouse=True, params=[1, 2], ids=["chunk-parallel", "block-per-row"])
+def sparse_path(request):
+    """Every test runs on both implementations of steps 1-7 (rows longer than 16384 tokens
+    always take the chunk-parallel one)."""
+    binding.set_sparse_path(request.param)
+    yield request.param
+    binding.set_sparse_path(0)
+
+
 def make(lens, tokens=16, heads=3, index=2, peaked=0.0, keep=0.125, kt_tokens=None):
     w = wl.Workload("sparf", index, batch=len(lens), len_lo=min(lens), len_hi=max(lens),
                     layout="paged", block_tokens=tokens, heads=heads, peaked_fraction=peaked)
