@@ -735,7 +735,7 @@ def main(argv=None) -> int:
             line["bulk_append"] = measure_bulk_append(device)
             line["grouped_attention"] = measure_grouped(device)
             line["sparse_attention"] = {wl.STANDARD[i].name: measure_sparse(wl.STANDARD[i], device, 10)
-                                        for i in (2, 3)}
+                                        for i in (2, 3, 4)}      # index 4: one of its layers
         if ranks.rank == 0:
             print(json.dumps(line), flush=True)
         return 0
