@@ -93,6 +93,123 @@ __device__ __forceinline__ int64_t grouped_row_index(const GroupedParams &p, int
     return ((int64_t)b * p.q_tokens + t) * ((int64_t)p.a.heads * p.group) + (int64_t)hk * p.group + g;
 }
 
+// One 16-token tile against the 16 query rows: logits, online softmax, and O += P V.  `base`
+// is the stage's shared-memory address; the running state (references, sums, output fragments)
+// is updated in place.
+template <int D>
+__device__ __forceinline__ void grouped_tile(unsigned base, unsigned k_rd, unsigned v_rd, unsigned q_rd,
+                                             const unsigned (&qa)[GroupedGeometry<D>::kQInSmem ? 1 : GroupedGeometry<D>::kKSteps][4],
+                                             int tok0, int unmasked_end, int vis_lo, int vis_hi,
+                                             float scale_log2e, int quad, float &m_lo, float &m_hi,
+                                             float &l_lo, float &l_hi, float (&o)[D / 8][4])
+{
+    using G = GroupedGeometry<D>;
+    // Logits of 16 rows x 16 tokens: s[n][0..1] row gid, s[n][2..3] row gid + 8, tokens
+    // tok0 + 8 n + 2 quad + {0, 1}.  Even and odd k-steps accumulate separately so that
+    // four independent MMA chains are in flight.
+    float s[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+    float s_odd[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+#pragma unroll
+    for (int ks = 0; ks < G::kKSteps; ++ks) {
+        unsigned kb[4];
+        ldmatrix_x4(kb, base + k_rd + ks * 32);
+        float (&acc)[2][4] = (ks & 1) ? s_odd : s;
+        if (G::kQInSmem) {
+            unsigned qf[4];
+            ldmatrix_x4(qf, q_rd + ks * 32);
+            mma_16816(acc[0], qf, kb[0], kb[1]);
+            mma_16816(acc[1], qf, kb[2], kb[3]);
+        } else {
+            mma_16816(acc[0], qa[ks], kb[0], kb[1]);
+            mma_16816(acc[1], qa[ks], kb[2], kb[3]);
+        }
+    }
+#pragma unroll
+    for (int n = 0; n < 2; ++n) {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) s[n][e] = (s[n][e] + s_odd[n][e]) * scale_log2e;
+    }
+    if (tok0 + kGroupTile > unmasked_end) {      // uniform: last tiles of the sequence only
+#pragma unroll
+        for (int n = 0; n < 2; ++n) {
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+                const int tok = tok0 + n * 8 + quad * 2 + e;
+                if (tok >= vis_lo) s[n][e] = -INFINITY;
+                if (tok >= vis_hi) s[n][2 + e] = -INFINITY;
+            }
+        }
+    }
+    // Online softmax with per-row references that may lag the true maximum by up to
+    // kGroupLag (base-2 units): weights reach at most 2^kGroupLag, inside the range of the
+    // fp16 weight split.  References move, and accumulators are rescaled, only when some
+    // logit exceeds its row's reference by more than that: with 16 rows sharing the
+    // rescaling, a tight lag would rescale on most tiles of a short chunk.
+    const float top_lo_here = fmaxf(fmaxf(s[0][0], s[0][1]), fmaxf(s[1][0], s[1][1]));
+    const float top_hi_here = fmaxf(fmaxf(s[0][2], s[0][3]), fmaxf(s[1][2], s[1][3]));
+    if (__any_sync(0xffffffffu, top_lo_here > m_lo + kGroupLag || top_hi_here > m_hi + kGroupLag)) {
+        float top_lo = top_lo_here, top_hi = top_hi_here;
+        top_lo = fmaxf(top_lo, __shfl_xor_sync(0xffffffffu, top_lo, 1));
+        top_lo = fmaxf(top_lo, __shfl_xor_sync(0xffffffffu, top_lo, 2));
+        top_hi = fmaxf(top_hi, __shfl_xor_sync(0xffffffffu, top_hi, 1));
+        top_hi = fmaxf(top_hi, __shfl_xor_sync(0xffffffffu, top_hi, 2));
+        float alpha_lo = 1.f, alpha_hi = 1.f;
+        if (top_lo > m_lo + kGroupLag) {
+            alpha_lo = fast_exp2(m_lo - top_lo);
+            m_lo = top_lo;
+        }
+        if (top_hi > m_hi + kGroupLag) {
+            alpha_hi = fast_exp2(m_hi - top_hi);
+            m_hi = top_hi;
+        }
+        l_lo *= alpha_lo;
+        l_hi *= alpha_hi;
+#pragma unroll
+        for (int i = 0; i < D / 8; ++i) {
+            o[i][0] *= alpha_lo;
+            o[i][1] *= alpha_lo;
+            o[i][2] *= alpha_hi;
+            o[i][3] *= alpha_hi;
+        }
+    }
+    // Weights (scaled by kGroupWeightScale: the scale is folded into the exponent), their
+    // sums, and the A fragments of P V as an fp16 hi + lo pair.
+    const float e_lo = m_lo - kGroupWeightLog2, e_hi = m_hi - kGroupWeightLog2;
+    unsigned p_hi[4], p_lo[4];
+#pragma unroll
+    for (int n = 0; n < 2; ++n) {
+        float w[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) w[e] = fast_exp2(s[n][e] - (e < 2 ? e_lo : e_hi));
+        l_lo += w[0] + w[1];
+        l_hi += w[2] + w[3];
+        p_hi[2 * n] = pack_half2(w[0], w[1]);
+        p_hi[2 * n + 1] = pack_half2(w[2], w[3]);
+        const float2 f_lo = __half22float2(*reinterpret_cast<const __half2 *>(&p_hi[2 * n]));
+        const float2 f_hi = __half22float2(*reinterpret_cast<const __half2 *>(&p_hi[2 * n + 1]));
+        p_lo[2 * n] = pack_half2(w[0] - f_lo.x, w[1] - f_lo.y);
+        p_lo[2 * n + 1] = pack_half2(w[2] - f_hi.x, w[3] - f_hi.y);
+    }
+    // O += P V: two 8-dim output blocks per ldmatrix, four ldmatrix per group so that
+    // eight independent accumulators separate the hi and the lo MMA of each block.
+#pragma unroll
+    for (int grp = 0; grp < D / 64; ++grp) {
+        unsigned vb[4][4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) ldmatrix_x4_trans(vb[i], base + v_rd + (grp * 4 + i) * 32);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            mma_16816(o[(grp * 4 + i) * 2], p_hi, vb[i][0], vb[i][1]);
+            mma_16816(o[(grp * 4 + i) * 2 + 1], p_hi, vb[i][2], vb[i][3]);
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            mma_16816(o[(grp * 4 + i) * 2], p_lo, vb[i][0], vb[i][1]);
+            mma_16816(o[(grp * 4 + i) * 2 + 1], p_lo, vb[i][2], vb[i][3]);
+        }
+    }
+}
+
 template <int D, bool kPaged>
 __global__ void __launch_bounds__(kThreads, GroupedGeometry<D>::kCtasPerSm)
 grouped_attn_split_kernel(const GroupedParams p)
@@ -274,110 +391,8 @@ grouped_attn_split_kernel(const GroupedParams p)
         stage = stage + 1 == kGroupStages ? 0 : stage + 1;
         const int tok0 = first_token + j * kStepTokens;
 
-        // Logits of 16 rows x 16 tokens: s[n][0..1] row gid, s[n][2..3] row gid + 8, tokens
-        // tok0 + 8 n + 2 quad + {0, 1}.  Even and odd k-steps accumulate separately so that
-        // four independent MMA chains are in flight.
-        float s[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
-        float s_odd[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
-#pragma unroll
-        for (int ks = 0; ks < G::kKSteps; ++ks) {
-            unsigned kb[4];
-            ldmatrix_x4(kb, base + k_rd + ks * 32);
-            float (&acc)[2][4] = (ks & 1) ? s_odd : s;
-            if (G::kQInSmem) {
-                unsigned qf[4];
-                ldmatrix_x4(qf, q_rd + ks * 32);
-                mma_16816(acc[0], qf, kb[0], kb[1]);
-                mma_16816(acc[1], qf, kb[2], kb[3]);
-            } else {
-                mma_16816(acc[0], qa[ks], kb[0], kb[1]);
-                mma_16816(acc[1], qa[ks], kb[2], kb[3]);
-            }
-        }
-#pragma unroll
-        for (int n = 0; n < 2; ++n) {
-#pragma unroll
-            for (int e = 0; e < 4; ++e) s[n][e] = (s[n][e] + s_odd[n][e]) * a.scale_log2e;
-        }
-        if (tok0 + kGroupTile > unmasked_end) {      // uniform: last tiles of the sequence only
-#pragma unroll
-            for (int n = 0; n < 2; ++n) {
-#pragma unroll
-                for (int e = 0; e < 2; ++e) {
-                    const int tok = tok0 + n * 8 + quad * 2 + e;
-                    if (tok >= vis_lo) s[n][e] = -INFINITY;
-                    if (tok >= vis_hi) s[n][2 + e] = -INFINITY;
-                }
-            }
-        }
-        // Online softmax with per-row references that may lag the true maximum by up to
-        // kGroupLag (base-2 units): weights reach at most 2^kGroupLag, inside the range of the
-        // fp16 weight split.  References move, and accumulators are rescaled, only when some
-        // logit exceeds its row's reference by more than that: with 16 rows sharing the
-        // rescaling, a tight lag would rescale on most tiles of a short chunk.
-        const float top_lo_here = fmaxf(fmaxf(s[0][0], s[0][1]), fmaxf(s[1][0], s[1][1]));
-        const float top_hi_here = fmaxf(fmaxf(s[0][2], s[0][3]), fmaxf(s[1][2], s[1][3]));
-        if (__any_sync(0xffffffffu, top_lo_here > m_lo + kGroupLag || top_hi_here > m_hi + kGroupLag)) {
-            float top_lo = top_lo_here, top_hi = top_hi_here;
-            top_lo = fmaxf(top_lo, __shfl_xor_sync(0xffffffffu, top_lo, 1));
-            top_lo = fmaxf(top_lo, __shfl_xor_sync(0xffffffffu, top_lo, 2));
-            top_hi = fmaxf(top_hi, __shfl_xor_sync(0xffffffffu, top_hi, 1));
-            top_hi = fmaxf(top_hi, __shfl_xor_sync(0xffffffffu, top_hi, 2));
-            float alpha_lo = 1.f, alpha_hi = 1.f;
-            if (top_lo > m_lo + kGroupLag) {
-                alpha_lo = fast_exp2(m_lo - top_lo);
-                m_lo = top_lo;
-            }
-            if (top_hi > m_hi + kGroupLag) {
-                alpha_hi = fast_exp2(m_hi - top_hi);
-                m_hi = top_hi;
-            }
-            l_lo *= alpha_lo;
-            l_hi *= alpha_hi;
-#pragma unroll
-            for (int i = 0; i < D / 8; ++i) {
-                o[i][0] *= alpha_lo;
-                o[i][1] *= alpha_lo;
-                o[i][2] *= alpha_hi;
-                o[i][3] *= alpha_hi;
-            }
-        }
-        // Weights (scaled by kGroupWeightScale: the scale is folded into the exponent), their
-        // sums, and the A fragments of P V as an fp16 hi + lo pair.
-        const float e_lo = m_lo - kGroupWeightLog2, e_hi = m_hi - kGroupWeightLog2;
-        unsigned p_hi[4], p_lo[4];
-#pragma unroll
-        for (int n = 0; n < 2; ++n) {
-            float w[4];
-#pragma unroll
-            for (int e = 0; e < 4; ++e) w[e] = fast_exp2(s[n][e] - (e < 2 ? e_lo : e_hi));
-            l_lo += w[0] + w[1];
-            l_hi += w[2] + w[3];
-            p_hi[2 * n] = pack_half2(w[0], w[1]);
-            p_hi[2 * n + 1] = pack_half2(w[2], w[3]);
-            const float2 f_lo = __half22float2(*reinterpret_cast<const __half2 *>(&p_hi[2 * n]));
-            const float2 f_hi = __half22float2(*reinterpret_cast<const __half2 *>(&p_hi[2 * n + 1]));
-            p_lo[2 * n] = pack_half2(w[0] - f_lo.x, w[1] - f_lo.y);
-            p_lo[2 * n + 1] = pack_half2(w[2] - f_hi.x, w[3] - f_hi.y);
-        }
-        // O += P V: two 8-dim output blocks per ldmatrix, four ldmatrix per group so that
-        // eight independent accumulators separate the hi and the lo MMA of each block.
-#pragma unroll
-        for (int grp = 0; grp < D / 64; ++grp) {
-            unsigned vb[4][4];
-#pragma unroll
-            for (int i = 0; i < 4; ++i) ldmatrix_x4_trans(vb[i], base + v_rd + (grp * 4 + i) * 32);
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                mma_16816(o[(grp * 4 + i) * 2], p_hi, vb[i][0], vb[i][1]);
-                mma_16816(o[(grp * 4 + i) * 2 + 1], p_hi, vb[i][2], vb[i][3]);
-            }
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                mma_16816(o[(grp * 4 + i) * 2], p_lo, vb[i][0], vb[i][1]);
-                mma_16816(o[(grp * 4 + i) * 2 + 1], p_lo, vb[i][2], vb[i][3]);
-            }
-        }
+        grouped_tile<D>(base, k_rd, v_rd, q_rd, qa, tok0, unmasked_end, vis_lo, vis_hi, a.scale_log2e, quad,
+                        m_lo, m_hi, l_lo, l_hi, o);
     }
     cp_async_wait<0>();
 
@@ -445,18 +460,18 @@ grouped_merge_kernel(const GroupedParams p)
     allow_next_kernel();
     wait_for_previous_kernels();
     const int len = checked_seq_len(a, b, threadIdx.x == 0 && hk == 0 && r == 0);
-    const int live = live_chunks(a, len);
+    const int parts = live_chunks(a, len);
     const int64_t row = grouped_row_index(p, b, hk, r);
     const int64_t first = (int64_t)pair * a.n_splits * p.rows + r;      // slot of chunk 0
     float top = kMinusHuge;
-    for (int s = 0; s < live; ++s) top = fmaxf(top, a.part_lse[first + (int64_t)s * p.rows]);
-    if (!(top > kMinusHuge)) {                 // no chunk holds a position this row may see
+    for (int s = 0; s < parts; ++s) top = fmaxf(top, a.part_lse[first + (int64_t)s * p.rows]);
+    if (!(top > kMinusHuge)) {                 // no part holds a position this row may see
         a.out[row * D + threadIdx.x] = __float2half_rn(0.f);
         if (a.lse && threadIdx.x == 0) a.lse[row] = -INFINITY;
         return;
     }
     float total = 0.f, acc = 0.f;
-    for (int s = 0; s < live; ++s) {
+    for (int s = 0; s < parts; ++s) {
         const int64_t slot = first + (int64_t)s * p.rows;
         const float w = fast_exp2(a.part_lse[slot] - top);
         total += w;
