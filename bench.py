@@ -621,7 +621,7 @@ GROUPED_SHAPES = [
 ]
 
 
-def measure_grouped(device, steps: int = 10) -> dict:
+def measure_grouped(device, steps: int = 20) -> dict:
     """The grouped-head / multi-token / other-head-size entry point on a few long-context
     shapes: fp16 K+V bytes read per second (each input several GB, far beyond L2)."""
     from paper_2409_04992_b200 import binding
@@ -642,7 +642,7 @@ def measure_grouped(device, steps: int = 10) -> dict:
             binding.decode_attention_grouped(out, None, g.q, c.k_cache, c.v_cache, c.block_table,
                                              c.seq_lens, ctx, c.scale, ws, flags)
 
-        for _ in range(3):
+        for _ in range(5):
             step()
         a, z = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         torch.cuda.synchronize()
