@@ -135,6 +135,65 @@ def test_append_rejects_bad_arguments(lib):
     assert append(lib, batch=0) == E.OK
 
 
+def grouped(lib, **kw):
+    a = dict(out=FAKE, q=FAKE, k=FAKE, v=FAKE, table=None, lens=FAKE, batch=2, tq=1, hq=8, hkv=2,
+             dim=128, s_max=256, T=0, M=0, P=0, max_len=256, scale=0.1, ws=FAKE, ws_bytes=1 << 30)
+    a.update(kw)
+    return lib.instinfer_decode_attention_grouped(a["out"], None, a["q"], a["k"], a["v"], a["table"],
+                                                  a["lens"], a["batch"], a["tq"], a["hq"], a["hkv"],
+                                                  a["dim"], a["s_max"], a["T"], a["M"], a["P"],
+                                                  a["max_len"], a["scale"], a["ws"], a["ws_bytes"],
+                                                  None, None)
+
+
+def test_grouped_attention_rejects_bad_arguments(lib):
+    E = binding
+    assert grouped(lib, out=None) == E.ERR_INVALID_ARG
+    assert grouped(lib, hq=7) == E.ERR_INVALID_ARG               # 7 query heads over 2 KV heads
+    assert grouped(lib, tq=0) == E.ERR_INVALID_ARG
+    assert grouped(lib, max_len=257) == E.ERR_INVALID_ARG        # beyond s_max
+    assert grouped(lib, scale=float("inf")) == E.ERR_INVALID_ARG
+    assert grouped(lib, hq=34) == E.ERR_UNSUPPORTED              # 17 rows per KV head
+    assert grouped(lib, tq=9) == E.ERR_UNSUPPORTED               # 4 x 9 rows
+    assert grouped(lib, dim=96) == E.ERR_UNSUPPORTED
+    assert grouped(lib, table=FAKE, T=8, M=32, P=9) == E.ERR_UNSUPPORTED      # blocks of 8 tokens
+    assert grouped(lib, table=FAKE, T=16, M=4, P=9) == E.ERR_INVALID_ARG      # 256 tokens need 16 blocks
+    assert grouped(lib, ws_bytes=64) == E.ERR_WORKSPACE
+    assert grouped(lib, batch=0, out=None) == E.OK
+    for dim in (64, 128, 256):
+        assert binding.grouped_workspace_bytes(2, 2, 8, 2, dim, 4096) > 0
+    assert binding.grouped_workspace_bytes(2, 1, 8, 3, 128, 4096) == 0
+
+
+def test_allgather_attention_rejects_bad_arguments(lib):
+    import ctypes
+    E = binding
+    one = (ctypes.c_void_p * 1)(FAKE)
+
+    def call(outs=one, n=1, heads=4, offset=0, total=8, batch=2, ws_bytes=1 << 30, q=FAKE):
+        return lib.instinfer_decode_attention_allgather(outs, n, None, q, FAKE, FAKE, None, FAKE, batch,
+                                                        heads, offset, total, 128, 256, 0, 0, 0, 256,
+                                                        0.1, FAKE, ws_bytes, None, None)
+
+    assert call(outs=None) == E.ERR_INVALID_ARG
+    assert call(n=0) == E.ERR_INVALID_ARG
+    assert call(n=17) == E.ERR_INVALID_ARG
+    assert call(offset=5) == E.ERR_INVALID_ARG                   # heads 5..8 of 8
+    assert call(offset=-1) == E.ERR_INVALID_ARG
+    assert call(outs=(ctypes.c_void_p * 1)(FAKE + 2)) == E.ERR_INVALID_ARG
+    assert call(q=None) == E.ERR_INVALID_ARG
+    assert call(ws_bytes=binding.workspace_bytes(2, 4, 128, 256)) == E.ERR_WORKSPACE   # no room for the staged rows
+    assert call(batch=0) == E.OK
+    assert binding.allgather_workspace_bytes(2, 4, 128, 256) > binding.workspace_bytes(2, 4, 128, 256)
+
+
+def test_sparse_path_knob(lib):
+    for path in (0, 1, 2, 0):
+        binding.set_sparse_path(path)
+    with pytest.raises(binding.InstInferError):
+        binding.set_sparse_path(3)
+
+
 def test_missing_library_fails_loudly(monkeypatch, tmp_path):
     monkeypatch.setattr(binding, "_lib", None)
     monkeypatch.setattr(binding, "LIBRARY", tmp_path / "libinstinfer.so")
