@@ -283,6 +283,11 @@ int instinfer_decode_step_host(void *out_host, const void *qkv_host, void *qkv_d
  *
  * instinfer_sparf_append does what instinfer_kv_append does on the paged pools and also
  * writes k_new into kt_pool and adds v_new to v_sum (one fp32 rounding per element).
+ * seq_lens[b] must fit both tables (max_blocks_per_seq * block_tokens and
+ * kt_max_blocks_per_seq * kt_block_tokens); a longer one is flagged and that sequence is left
+ * untouched, as is one whose block id in either table is out of range.
+ * Unlike the plain append this call is not idempotent: v_sum grows by v_new every time, so
+ * replaying a step (a retried request, a benchmark loop) adds the token's value again.
  */
 int instinfer_sparf_append(void *k_pool, void *v_pool, void *kt_pool, float *v_sum,
                            const void *k_new, const void *v_new, const int32_t *seq_lens,
@@ -297,7 +302,10 @@ int instinfer_sparf_append(void *k_pool, void *v_pool, void *kt_pool, float *v_s
  * Bulk form of instinfer_sparf_append for the prefill phase (Sec. IV-D): new_lens[b] tokens
  * per sequence from token-major k_new / v_new [batch, max_new, heads, head_dim], as in
  * instinfer_kv_append_bulk; v_sum receives the tokens in order, one fp32 rounding each, so
- * the result equals that of appending them one by one.
+ * the result equals that of appending them one by one.  A sequence with a block id out of
+ * range among the blocks its new tokens need keeps its transposed copy and its v_sum, but its
+ * K and V rows in valid blocks may already have been written: after a flagged call the cache
+ * state of the flagged sequence is undefined and the caller should rebuild or drop it.
  */
 int instinfer_sparf_append_bulk(void *k_pool, void *v_pool, void *kt_pool, float *v_sum,
                                 const void *k_new, const void *v_new, const int32_t *seq_lens,

@@ -21,14 +21,11 @@
  * k is clipped to S and l to k.  S == 0 gives out = 0 and alpha = 0.  If |q|_1 == 0 the
  * ratio is taken as 1.
  *
- * Precision of the decisions.  Step 1 compares fp16 magnitudes, which is exact.  Step 6 is a
- * decision taken on floating-point scores; the paper computes everything in FP16 and does
- * not fix how, so the decision is taken in the precision of the implementation under test,
- * binary32, by a rule simple enough to restate here: the |q| sums run over ascending d in
- * binary32; the approximate logit of token i is the binary32 FMA chain over the kept dims in
- * rank order, times the binary32 constant (scale * log2(e)) / sqrt(ratio); tokens are ranked
- * by that value in the usual total order of the bit patterns (so -0 < +0), ties to the lower
- * position.  The values s^ that enter alpha, and everything after step 6, are fp64.
+ * The two selections.  Step 1 compares fp16 magnitudes, which is exact.  Step 6 ranks the
+ * fp64 values s^_i + m_i.  Every s^_i is positive and they sum to 1, so in exact arithmetic
+ * s^_i + 1 exceeds every s^_j: the ranking of the sums is the ranking of the pairs
+ * (m_i, s^_i), and it is taken on the pairs so that rounding 1 + s^_i to 1 cannot push a
+ * window position below a dominant token.  Ties go to the lower position.
  *
  * Layouts: K, V pools [P][H][T][D] with block_table [B][M].  The K^T copy has its own
  * granularity (Sec. IV-C gives the embedding-indexed mapping much larger token groups than
@@ -170,19 +167,13 @@ int oracle_sparf_append_bulk(uint16_t *k_pool, uint16_t *v_pool, uint16_t *kt_po
 typedef struct {
     double key;
     int32_t index;
+    int32_t mask;      /* m_i of step 5; 0 where unused */
 } ranked;
-
-/* total order of binary32 bit patterns: larger float, larger key; -0 below +0 */
-static uint32_t order_key(float x)
-{
-    uint32_t u;
-    memcpy(&u, &x, sizeof u);
-    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
-}
 
 static int by_key_desc_then_index(const void *pa, const void *pb)
 {
     const ranked *a = (const ranked *)pa, *b = (const ranked *)pb;
+    if (a->mask != b->mask) return a->mask > b->mask ? -1 : 1;
     if (a->key > b->key) return -1;
     if (a->key < b->key) return 1;
     return (a->index > b->index) - (a->index < b->index);
@@ -255,6 +246,7 @@ int oracle_sparf_attention(double *out, double *alpha, double *approx_weights, i
             for (int32_t d = 0; d < D; ++d) {
                 dims[d].key = fabs(widen(qv[d]));
                 dims[d].index = d;
+                dims[d].mask = 0;
                 q_l1 += dims[d].key;
             }
             qsort(dims, (size_t)D, sizeof(ranked), by_key_desc_then_index);
@@ -281,29 +273,14 @@ int oracle_sparf_attention(double *out, double *alpha, double *approx_weights, i
             for (int32_t i = 0; i < S; ++i) a[i] /= z;                      /* s^ */
             if (approx_weights) memcpy(approx_weights + pair * stride_s, a, sizeof(double) * (size_t)S);
 
-            /* steps 5-6: top-k of s^ + m, the last `window` positions carry m = 1; the ranking
-               is done on the binary32 logits described in the header */
+            /* steps 5-6: J = the k largest of s^_i + m_i, where m_i = 1 on the last `window`
+               positions and 0 elsewhere, ranked as the pairs (m_i, s^_i) (see the header) */
             if (given) {
                 for (int32_t t = 0; t < k; ++t) J[t] = given[pair * stride_k + t];
             } else {
-                float all32 = 0.f, kept32 = 0.f;
-                for (int32_t d = 0; d < D; ++d) {
-                    const float mag = fabsf((float)widen(qv[d]));
-                    int kept = 0;
-                    for (int32_t t = 0; t < r; ++t) kept |= dims[t].index == d;
-                    all32 += mag;
-                    if (kept) kept32 += mag;
-                }
-                const float ratio32 = all32 > 0.f ? kept32 / all32 : 1.f;
-                const float scale32 = (scale * 1.44269504088896340736f) / sqrtf(ratio32);
                 for (int32_t i = 0; i < S; ++i) {
-                    float dot = 0.f;
-                    for (int32_t t = 0; t < r; ++t) {
-                        const int32_t d = dims[t].index;
-                        dot = fmaf((float)widen(qv[d]), (float)widen(kt_pool[kt_offset(&gt, b, h, d, i)]), dot);
-                    }
-                    const float logit = dot * scale32;
-                    order[i].key = i >= S - window ? 4294967296.0 : (double)order_key(logit);
+                    order[i].key = a[i];
+                    order[i].mask = i >= S - window ? 1 : 0;
                     order[i].index = i;
                 }
                 qsort(order, (size_t)S, sizeof(ranked), by_key_desc_then_index);

@@ -251,22 +251,27 @@ int instinfer_sparf_decode_attention(void *out, float *alpha, int32_t *selected,
             }
             fused_smem_set[device] = true;
         }
-        launch_overlapped(sparf_fused_select_kernel, row_grid, kFusedThreads,
-                          (size_t)w.score_stride * sizeof(float), stream, sp);
+        if (launch_overlapped(sparf_fused_select_kernel, row_grid, kFusedThreads,
+                              (size_t)w.score_stride * sizeof(float), stream, sp) != cudaSuccess)
+            return INSTINFER_ERR_CUDA;
     } else {
-    if (cudaMemsetAsync(ws + w.rows_state, 0, w.zeroed_bytes, stream) != cudaSuccess) {
-        (void)cudaGetLastError();
-        return INSTINFER_ERR_CUDA;
-    }
-    launch_overlapped(sparf_scores_kernel, (unsigned)(pairs * sp.score_blocks), kSparfThreads, 0, stream, sp);
-    // Steps 5-7, chunk-parallel; rows it cannot settle are redone by the single-block kernel.
-    launch_overlapped(sparf_hist_kernel, chunk_grid, kChunkThreads, 0, stream, sp);
-    launch_overlapped(sparf_locate_kernel, row_grid, 32, 0, stream, sp);
-    launch_overlapped(sparf_collect_kernel, chunk_grid, kChunkThreads, 0, stream, sp);
-    launch_overlapped(sparf_threshold_kernel, row_grid, kThresholdThreads, 0, stream, sp);
-    launch_overlapped(sparf_compact_kernel, chunk_grid, kChunkThreads, 0, stream, sp);
-    launch_overlapped(sparf_finish_kernel, row_grid, 64, 0, stream, sp);
-    launch_overlapped(sparf_select_kernel, row_grid, kSelectThreads, 0, stream, sp);
+        if (cudaMemsetAsync(ws + w.rows_state, 0, w.zeroed_bytes, stream) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return INSTINFER_ERR_CUDA;
+        }
+        // Steps 5-7, chunk-parallel; rows it cannot settle are redone by the single-block kernel.
+        bool ok = launch_overlapped(sparf_scores_kernel, (unsigned)(pairs * sp.score_blocks), kSparfThreads, 0, stream, sp) == cudaSuccess;
+        ok = ok && launch_overlapped(sparf_hist_kernel, chunk_grid, kChunkThreads, 0, stream, sp) == cudaSuccess;
+        ok = ok && launch_overlapped(sparf_locate_kernel, row_grid, 32, 0, stream, sp) == cudaSuccess;
+        ok = ok && launch_overlapped(sparf_collect_kernel, chunk_grid, kChunkThreads, 0, stream, sp) == cudaSuccess;
+        ok = ok && launch_overlapped(sparf_threshold_kernel, row_grid, kThresholdThreads, 0, stream, sp) == cudaSuccess;
+        ok = ok && launch_overlapped(sparf_compact_kernel, chunk_grid, kChunkThreads, 0, stream, sp) == cudaSuccess;
+        ok = ok && launch_overlapped(sparf_finish_kernel, row_grid, 64, 0, stream, sp) == cudaSuccess;
+        ok = ok && launch_overlapped(sparf_select_kernel, row_grid, kSelectThreads, 0, stream, sp) == cudaSuccess;
+        if (!ok) {
+            (void)cudaGetLastError();
+            return INSTINFER_ERR_CUDA;
+        }
     }
     if (cudaGetLastError() != cudaSuccess) return INSTINFER_ERR_CUDA;
 

@@ -374,11 +374,29 @@ int instinfer_decode_step_host(void *out_host, const void *qkv_host, void *qkv_d
                                float scale, void *workspace, size_t workspace_bytes,
                                int32_t *status_flags, void *cuda_stream)
 {
-    if (batch < 0 || heads <= 0 || head_dim <= 0) return INSTINFER_ERR_INVALID_ARG;
-    if (head_dim != kHeadDim) return INSTINFER_ERR_UNSUPPORTED;
-    if (batch == 0) return INSTINFER_OK;
-    if (out_host == nullptr || qkv_host == nullptr || !usable(qkv_dev) || !usable(out_dev))
+    // Everything the host can check is checked here, for all the calls this one is made of,
+    // so that a refused call has put nothing on the stream (not even the upload).
+    const bool paged = block_table != nullptr;
+    if (head_dim <= 0 || !sizes_ok(batch, heads, max_seq_len) || !std::isfinite(scale))
         return INSTINFER_ERR_INVALID_ARG;
+    if (paged) {
+        if (block_tokens <= 0 || max_blocks_per_seq <= 0 || num_phys_blocks <= 0 ||
+            (int64_t)max_seq_len > (int64_t)max_blocks_per_seq * block_tokens)
+            return INSTINFER_ERR_INVALID_ARG;
+    } else if (s_max <= 0 || max_seq_len > s_max) {
+        return INSTINFER_ERR_INVALID_ARG;
+    }
+    if (head_dim != kHeadDim || (paged && block_tokens % 8 != 0)) return INSTINFER_ERR_UNSUPPORTED;
+    if (batch == 0) return INSTINFER_OK;
+    if (out_host == nullptr || qkv_host == nullptr || !usable(qkv_dev) || !usable(out_dev) ||
+        !usable(k_cache) || !usable(v_cache) || seq_lens == nullptr)
+        return INSTINFER_ERR_INVALID_ARG;
+    {
+        const int64_t pairs = (int64_t)batch * heads;
+        if (workspace == nullptr || !aligned16(workspace) ||
+            workspace_bytes < workspace_for(pairs, make_plan(pairs, max_seq_len)))
+            return INSTINFER_ERR_WORKSPACE;
+    }
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     const size_t one = (size_t)batch * heads * head_dim * sizeof(__half);
     if (cudaMemcpyAsync(qkv_dev, qkv_host, 3 * one, cudaMemcpyHostToDevice, stream) != cudaSuccess) {

@@ -100,19 +100,18 @@ sparf_append_kernel(const SparfParams p)
     const int b = pair / p.heads, h = pair - b * p.heads;
     const int len = p.seq_lens[b];
     if (len == 0) return;
-    if (len < 0 || (int64_t)len > (int64_t)p.max_blocks_per_seq * p.block_tokens) {
+    // Both capacities are checked before either table is read: a length that fits the K/V
+    // table but not the transposed copy's must not index past that table's row.
+    const int T = p.block_tokens, Tk = p.kt_block_tokens;
+    if (len < 0 || (int64_t)len > (int64_t)p.max_blocks_per_seq * T ||
+        (int64_t)len > (int64_t)p.kt_max_blocks_per_seq * Tk) {
         if (d == 0 && h == 0 && p.status) atomicOr(p.status, kFlagSeqLenRange);
         return;
     }
-    const int pos = len - 1, T = p.block_tokens;
+    const int pos = len - 1;
     const int phys = p.block_table[(int64_t)b * p.max_blocks_per_seq + pos / T];
-    if (phys < 0 || (int64_t)phys >= p.num_phys_blocks) {
-        if (d == 0 && h == 0 && p.status) atomicOr(p.status, kFlagBlockRange);
-        return;
-    }
-    const int Tk = p.kt_block_tokens;
     const int kt_phys = p.kt_block_table[(int64_t)b * p.kt_max_blocks_per_seq + pos / Tk];
-    if (kt_phys < 0 || (int64_t)kt_phys >= p.num_kt_blocks || (int64_t)len > (int64_t)p.kt_max_blocks_per_seq * Tk) {
+    if (phys < 0 || (int64_t)phys >= p.num_phys_blocks || kt_phys < 0 || (int64_t)kt_phys >= p.num_kt_blocks) {
         if (d == 0 && h == 0 && p.status) atomicOr(p.status, kFlagBlockRange);
         return;
     }
@@ -150,8 +149,25 @@ sparf_append_bulk_kernel(const SparfBulkParams q)
         if (d == 0 && h == 0 && p.status) atomicOr(p.status, kFlagSeqLenRange);
         return;
     }
+    if (fresh == 0) return;
     const int first = len - fresh;
     const int32_t *kt_table = p.kt_block_table + (int64_t)b * p.kt_max_blocks_per_seq;
+    // Every block id the new tokens need, in both tables, is checked before anything is
+    // written, so that a flagged sequence keeps its transposed copy and its running sum as
+    // they were (its K and V rows go through kv_append_bulk_kernel, which skips the rows of
+    // bad blocks only: the header calls the state of a flagged sequence undefined).
+    {
+        const int32_t *kv_table = p.block_table + (int64_t)b * p.max_blocks_per_seq;
+        bool bad = false;
+        for (int blk = first / Tk; blk <= (len - 1) / Tk; ++blk)
+            bad |= kt_table[blk] < 0 || (int64_t)kt_table[blk] >= p.num_kt_blocks;
+        for (int blk = first / p.block_tokens; blk <= (len - 1) / p.block_tokens; ++blk)
+            bad |= kv_table[blk] < 0 || (int64_t)kv_table[blk] >= p.num_phys_blocks;
+        if (bad) {
+            if (d == 0 && h == 0 && p.status) atomicOr(p.status, kFlagBlockRange);
+            return;
+        }
+    }
     const int64_t token_stride = (int64_t)p.heads * kHeadDim;                 // elements between tokens
     const __half *k_src = p.k_new + ((int64_t)b * q.max_new * p.heads + h) * kHeadDim + d;
     const __half *v_src = p.v_new + ((int64_t)b * q.max_new * p.heads + h) * kHeadDim + d;
@@ -159,11 +175,7 @@ sparf_append_bulk_kernel(const SparfBulkParams q)
     int t = 0;
     while (t < fresh) {
         const int pos = first + t;
-        const int phys = kt_table[pos / Tk];
-        if (phys < 0 || (int64_t)phys >= p.num_kt_blocks) {
-            if (d == 0 && p.status) atomicOr(p.status, kFlagBlockRange);
-            return;                                                            // uniform: the rest is skipped
-        }
+        const int phys = kt_table[pos / Tk];                                   // checked above
         __half *dst = p.kt_pool + (((int64_t)phys * p.heads + h) * kHeadDim + d) * Tk + pos % Tk;
         if ((pos & 7) == 0 && t + 8 <= fresh) {                                // a whole aligned group
             __align__(16) __half group[8];
@@ -223,10 +235,9 @@ __device__ __forceinline__ void score_setup(const SparfParams &p, int pair, Scor
         }
         ss.kept[d] = kept;
     }
-    // |q|_1 and |q_I|_1.  The top-k of step 6 is decided on the fp32 logits computed below, so
-    // their arithmetic is kept simple enough to be restated elsewhere bit for bit: both sums
-    // run over ascending d in fp32, the temperature uses IEEE division and square root, and
-    // each logit is the fp32 FMA chain over the kept dims in rank order times that constant.
+    // |q|_1 and |q_I|_1 in fp32.  The temperature is one positive constant per row, so its
+    // rounding cannot change the ranking of step 6; each logit is an fp32 sum of r exact
+    // fp16 x fp16 products times that constant, i.e. within (r + 1) 2^-24 of sum |q_t k_t|.
     __syncthreads();
     if (d == 0) {
         float all = 0.f, sel = 0.f;

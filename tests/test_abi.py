@@ -1,9 +1,16 @@
 """The C-ABI library: it loads, exports what include/*.h declares, and rejects bad
-arguments on the host before anything is enqueued (no GPU needed, no compute calls)."""
+arguments on the host before anything is enqueued (no GPU needed, no compute calls).
+
+The rejection tests hand the library made-up device addresses.  They are only run in a
+process that sees no CUDA device, so that a slip in the order of validation could at worst
+end in a launch error, never in a kernel running on a bogus address: on a machine with a GPU
+this module re-runs itself in a child process with CUDA_VISIBLE_DEVICES emptied."""
 import ctypes
 import glob
 import os
 import re
+import subprocess
+import sys
 
 import pytest
 
@@ -11,6 +18,27 @@ from paper_2409_04992_b200 import binding, build
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 FAKE = 0x10000            # aligned, never dereferenced: every call below fails or no-ops first
+
+
+def _gpu_visible() -> bool:
+    try:
+        import torch
+        return torch.cuda.is_available()
+    except Exception:
+        return False
+
+
+fake_pointers = pytest.mark.skipif(_gpu_visible(), reason="made-up addresses: run in the GPU-less child instead")
+
+
+@pytest.mark.skipif(not _gpu_visible(), reason="no GPU here: the tests below run in this process")
+def test_rejection_tests_pass_in_a_child_that_sees_no_gpu():
+    env = dict(os.environ, CUDA_VISIBLE_DEVICES="")
+    done = subprocess.run([sys.executable, "-m", "pytest", os.path.abspath(__file__), "-q", "-x",
+                           "-p", "no:cacheprovider"], cwd=ROOT, env=env, capture_output=True, text=True,
+                          timeout=600)
+    assert done.returncode == 0, done.stdout[-3000:] + done.stderr[-2000:]
+    assert " passed" in done.stdout and "skipped" in done.stdout    # only this test is skipped there
 
 
 @pytest.fixture(scope="module")
@@ -92,6 +120,7 @@ def append(lib, **kw):
                                    None, None)
 
 
+@fake_pointers
 def test_contiguous_attention_rejects_bad_arguments(lib):
     E = binding
     assert attn(lib, out=None) == E.ERR_INVALID_ARG
@@ -110,6 +139,7 @@ def test_contiguous_attention_rejects_bad_arguments(lib):
     assert attn(lib, batch=0, out=None, q=None) == E.OK          # empty call: nothing enqueued
 
 
+@fake_pointers
 def test_paged_attention_rejects_bad_arguments(lib):
     E = binding
     assert paged(lib, table=None) == E.ERR_INVALID_ARG
@@ -123,6 +153,7 @@ def test_paged_attention_rejects_bad_arguments(lib):
     assert paged(lib, batch=0) == E.OK
 
 
+@fake_pointers
 def test_append_rejects_bad_arguments(lib):
     E = binding
     assert append(lib, kc=None) == E.ERR_INVALID_ARG
@@ -146,6 +177,7 @@ def grouped(lib, **kw):
                                                   None, None)
 
 
+@fake_pointers
 def test_grouped_attention_rejects_bad_arguments(lib):
     E = binding
     assert grouped(lib, out=None) == E.ERR_INVALID_ARG
@@ -165,6 +197,7 @@ def test_grouped_attention_rejects_bad_arguments(lib):
     assert binding.grouped_workspace_bytes(2, 1, 8, 3, 128, 4096) == 0
 
 
+@fake_pointers
 def test_allgather_attention_rejects_bad_arguments(lib):
     import ctypes
     E = binding

@@ -1,7 +1,10 @@
 """GPU parity at the full standard sizes, in the launch configuration the benchmark times
 (automatic split plan, device-generated inputs, NaN-poisoned padding).  Workloads 0 and 1 are
-compared element by element; for the 20 GiB ones the oracle recomputes sampled (sequence,
-head) pairs one by one from rows gathered off the device."""
+compared element by element; for the larger ones the oracle recomputes sampled (sequence,
+head) pairs one by one from rows gathered off the device: 64 pairs of each 20 GiB workload,
+8 pairs of every one of the 40 layers of the 13B-class step, and a batch of that step's shape
+whose lengths are placed on the edges of the split plan (last token in the first tile of a
+short end chunk, in a ragged last tile, on a chunk boundary)."""
 import numpy as np
 import pytest
 import torch
@@ -40,39 +43,53 @@ def device_step(case):
 
 
 def sampled_pairs(case, count, seed):
+    """The shortest and the longest sequence (first and last head), then random pairs."""
     lens = case.seq_lens_host
+    heads = case.workload.heads
     rng = np.random.default_rng(seed)
-    picks = {(int(np.argmin(lens)), 0), (int(np.argmax(lens)), case.workload.heads - 1)}
-    while len(picks) < count:
-        picks.add((int(rng.integers(len(lens))), int(rng.integers(case.workload.heads))))
+    lo, hi = int(np.argmin(lens)), int(np.argmax(lens))
+    picks = {(lo, 0), (lo, heads - 1), (hi, 0), (hi, heads - 1)}
+    while len(picks) < min(count, len(lens) * heads):
+        picks.add((int(rng.integers(len(lens))), int(rng.integers(heads))))
     return sorted(picks)
 
 
-def check_sampled(case, count=6, seed=0, what=""):
+def check_pairs(case, pairs, out, lse, before, what):
+    """Oracle on the given pairs, 16 at a time (bounds the host copy of the gathered rows)."""
+    worst = (0.0, 0.0)
+    for at in range(0, len(pairs), 16):
+        part = pairs[at:at + 16]
+        longest = max(case.seq_lens_host[b] for b, _ in part)
+        n = len(part)
+        k = np.zeros((n, 1, longest, 128), dtype=np.float16)
+        v = np.zeros((n, 1, longest, 128), dtype=np.float16)
+        q = np.zeros((n, 1, 128), dtype=np.float16)
+        lens = np.zeros(n, dtype=np.int32)
+        for i, (b, h) in enumerate(part):
+            kr, vr = wl.gather_rows(case, b, h)
+            L = case.seq_lens_host[b]
+            k[i, 0, :L], v[i, 0, :L] = kr.cpu().numpy(), vr.cpu().numpy()
+            q[i, 0], lens[i] = case.q[b, h].cpu().numpy(), L
+            # the append filled exactly the last row with k_new / v_new, bit for bit
+            assert np.array_equal(gu.bits(kr[L - 1]), gu.bits(case.k_new[b, h]))
+            assert np.array_equal(gu.bits(vr[L - 1]), gu.bits(case.v_new[b, h]))
+            if (b, h) in before:
+                assert np.array_equal(gu.bits(kr[:L - 1]), gu.bits(before[(b, h)][:L - 1]))
+                assert np.all(gu.bits(before[(b, h)][L - 1]) == wl.NAN_BITS)
+        want, want_lse, _ = capi.decode_attention(q, k, v, lens, case.scale)
+        got = torch.stack([out[b, h] for b, h in part])[:, None, :]
+        got_lse = torch.stack([lse[b, h] for b, h in part])[:, None]
+        errs = gu.assert_close(got, want, got_lse, want_lse, what)
+        worst = (max(worst[0], errs[0]), max(worst[1], errs[1]))
+    return worst
+
+
+def check_sampled(case, count=64, seed=0, what=""):
     pairs = sampled_pairs(case, count, seed)
-    before = {p: wl.gather_rows(case, *p)[0].cpu() for p in pairs}        # K rows before the append
+    before = {p: wl.gather_rows(case, *p)[0].cpu() for p in pairs[:8]}    # K rows before the append
     out, lse = device_step(case)
     assert torch.isfinite(out.float()).all(), "poison leaked into an output"
-    longest = max(case.seq_lens_host[b] for b, _ in pairs)
-    n = len(pairs)
-    k = np.zeros((n, 1, longest, 128), dtype=np.float16)
-    v = np.zeros((n, 1, longest, 128), dtype=np.float16)
-    q = np.zeros((n, 1, 128), dtype=np.float16)
-    lens = np.zeros(n, dtype=np.int32)
-    for i, (b, h) in enumerate(pairs):
-        kr, vr = wl.gather_rows(case, b, h)
-        L = case.seq_lens_host[b]
-        k[i, 0, :L], v[i, 0, :L] = kr.cpu().numpy(), vr.cpu().numpy()
-        q[i, 0], lens[i] = case.q[b, h].cpu().numpy(), L
-        # the append filled exactly the last row with k_new / v_new, bit for bit
-        assert np.array_equal(gu.bits(kr[L - 1]), gu.bits(case.k_new[b, h]))
-        assert np.array_equal(gu.bits(vr[L - 1]), gu.bits(case.v_new[b, h]))
-        assert np.array_equal(gu.bits(kr[:L - 1]), gu.bits(before[(b, h)][:L - 1]))
-        assert np.all(gu.bits(before[(b, h)][L - 1]) == wl.NAN_BITS)
-    want, want_lse, _ = capi.decode_attention(q, k, v, lens, case.scale)
-    got = torch.stack([out[b, h] for b, h in pairs])[:, None, :]
-    got_lse = torch.stack([lse[b, h] for b, h in pairs])[:, None]
-    return gu.assert_close(got, want, got_lse, want_lse, what)
+    return check_pairs(case, pairs, out, lse, before, what)
 
 
 def test_workload_0_every_element():
@@ -102,8 +119,33 @@ def test_workload_3_sampled_peaked_long_context():
     check_sampled(wl.generate(wl.STANDARD[3], device="cuda"), what="workload 3")
 
 
-@pytest.mark.parametrize("layer", [0, 17, 39])
-def test_workload_4_sampled_layers(layer):
+def test_workload_4_every_layer_sampled():
     need_memory(6)
-    check_sampled(wl.generate(wl.STANDARD[4], layer=layer, device="cuda"), seed=layer,
-                  what=f"workload 4 layer {layer}")
+    for layer in range(wl.STANDARD[4].layers):
+        case = wl.generate(wl.STANDARD[4], layer=layer, device="cuda")
+        check_sampled(case, count=8, seed=layer, what=f"workload 4 layer {layer}")
+        del case
+
+
+def test_workload_4_shape_with_lengths_on_the_edges_of_the_plan():
+    """The 13B-class step's shape (16 sequences x 40 heads, 32-token pages, lengths in
+    4096..8192) with lengths placed where the split plan has its seams."""
+    need_memory(6)
+    w = wl.STANDARD[4]
+    chunk = binding.plan_chunk_tokens(w.batch, w.heads, w.len_hi)
+    splits = binding.plan_num_splits(w.batch, w.heads, w.len_hi)
+    n_big = min(splits, w.len_hi // chunk)
+    span = n_big * chunk                         # where the short end chunks (256 tokens) begin, if any
+    tail = 256 if span < w.len_hi else chunk
+    edges = [w.len_hi, w.len_lo,
+             span + 1, span + 8, span + tail + 3, span + 2 * tail + 8,      # first tile of an end chunk
+             span, span - 1, span + tail,                                    # exactly on a seam, one before
+             5 * chunk + 1, 5 * chunk + 9,                                   # first tiles of a long chunk
+             w.len_hi - 1, w.len_hi - 3, w.len_lo + 5, 6001, 7777]           # ragged last tiles
+    lens = [int(min(max(n, w.len_lo), w.len_hi)) for n in edges][:w.batch]
+    assert len(lens) == w.batch
+    case = wl.generate(w, layer=3, device="cuda", seq_lens=lens)
+    pairs = [(b, h) for b in range(w.batch) for h in (0, 13, 26, 39)]
+    out, lse = device_step(case)
+    assert torch.isfinite(out.float()).all()
+    check_pairs(case, pairs, out, lse, {}, "workload 4 shape, lengths on plan edges")

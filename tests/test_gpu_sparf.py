@@ -1,10 +1,13 @@
 """GPU parity of the sparse (SparF, Algorithm 1) path against its CPU oracle.
 
-Floating point decides two integer sets here (the kept query dims and the kept tokens).  Both
-sides take each decision in the same precision: the dims on exact fp16 magnitudes, the tokens
-on binary32 logits computed by the rule stated in the oracle's header (ties to the lower
-position).  The kept sets must therefore agree exactly; outputs and alpha are then compared
-with the usual tolerances against the oracle's fp64 arithmetic."""
+Floating point decides two integer sets here (the kept query dims and the kept tokens).  The
+dims are ranked on fp16 magnitudes, which is exact on both sides.  The tokens are ranked in
+fp64 by the oracle, as Algorithm 1 prints step 6, and in fp32 by the CUDA path: the GPU's
+kept set must be a valid top-k of the oracle's fp64 scores up to the fp32 rounding band
+derived in tests/sparf_check.py (complete check: size, order, range, padding, window, every
+token above the band kept, every token below it dropped; exact ties cut by position).  The
+oracle then recomputes alpha and the output for the GPU's set, and those are compared with
+the usual tolerances."""
 import math
 
 import numpy as np
@@ -13,7 +16,7 @@ import torch
 
 from oracle import capi
 from paper_2409_04992_b200 import binding, workloads as wl
-from tests import gpu_util as gu
+from tests import gpu_util as gu, sparf_check
 
 pytestmark = pytest.mark.gpu
 
@@ -62,7 +65,7 @@ def gpu_sparf(case, state, r, l, do_append=True, max_k=None):
     return out.view.cpu(), alpha.view.cpu().numpy(), sel.view.cpu().numpy(), int(flags.item())
 
 
-def oracle_sparf(cpu, state, r, l, do_append=True, want_weights=False):
+def oracle_sparf(cpu, state, r, l, do_append=True, want_weights=False, given=None):
     k, v, kt = cpu.k_cache.numpy(), cpu.v_cache.numpy(), state.kt_pool.numpy()
     v_sum = state.v_sum.numpy()
     lens = np.array(cpu.seq_lens_host, dtype=np.int32)
@@ -71,40 +74,47 @@ def oracle_sparf(cpu, state, r, l, do_append=True, want_weights=False):
         capi.sparf_append(k, v, kt, v_sum, cpu.k_new.numpy(), cpu.v_new.numpy(), lens, table,
                           kt_block_table=kt_table)
     return capi.sparf_attention(cpu.q.numpy(), k, v, kt, v_sum, lens, np.array(state.k_tokens_host),
-                                table, r, l, cpu.scale, want_weights=want_weights,
+                                table, r, l, cpu.scale, want_weights=want_weights, given=given,
                                 kt_block_table=kt_table)
 
 
-def check_structure(sel_gpu, lens, ks, l):
-    """Shape of the kept sets: size, order, range, window membership, -1 padding."""
-    for b, S in enumerate(lens):
-        k = min(ks[b], S)
-        window = min(l, k)
+def check_kept_sets(cpu, sel_gpu, weights, ks, r, l, what):
+    """The GPU's kept sets against the oracle's fp64 scores (cpu holds the appended caches).
+    Returns the number of (token, row) decisions that fell inside the rounding band."""
+    in_band = 0
+    for b, S in enumerate(cpu.seq_lens_host):
         for h in range(sel_gpu.shape[1]):
-            J = sel_gpu[b, h, :k]
-            assert np.all(sel_gpu[b, h, k:] == -1)
-            assert np.all(np.diff(J) > 0) and (k == 0 or (J[0] >= 0 and J[-1] < S))
-            assert np.all(np.isin(np.arange(S - window, S), J))
+            k_rows, _ = wl.gather_rows(cpu, b, h)
+            k_abs_max = float(k_rows.float().abs().max()) if S else 0.0
+            delta = sparf_check.logit_band(cpu.q[b, h].numpy(), k_abs_max, r, cpu.scale)
+            in_band += sparf_check.check_kept_set(sel_gpu[b, h], weights[b, h], S, ks[b], l, delta,
+                                                  f"{what} pair {(b, h)}")
+    return in_band
 
 
-def run_and_check(cpu, state, r, l, what):
+def run_and_check(cpu, state, r, l, what, generic=True):
+    """generic: random data without planted ties, where only a handful of decisions may fall
+    inside the rounding band (guards against a band so wide that it checks nothing)."""
     dev, dstate = gu.to_device(cpu), dev_state(state)
     out, alpha, sel, flags = gpu_sparf(dev, dstate, r, l)
     assert flags == 0
-    want, want_alpha, want_sel, weights = oracle_sparf(cpu, state, r, l, want_weights=True)   # appends into the CPU copies
+    # the oracle's own selection and its fp64 scores (this call appends into the CPU copies)
+    _, _, own_sel, weights = oracle_sparf(cpu, state, r, l, want_weights=True)
     # the append: both K layouts, V and the running sum, bit for bit
     assert np.array_equal(gu.bits(dev.k_cache), gu.bits(cpu.k_cache))
     assert np.array_equal(gu.bits(dev.v_cache), gu.bits(cpu.v_cache))
     assert np.array_equal(gu.bits(dstate.kt_pool), gu.bits(state.kt_pool))
     assert np.array_equal(dstate.v_sum.cpu().numpy().view(np.uint32), state.v_sum.numpy().view(np.uint32))
     lens, ks = cpu.seq_lens_host, state.k_tokens_host
-    check_structure(sel, lens, ks, l)
-    width = want_sel.shape[2]
-    assert np.array_equal(sel[:, :, :width], want_sel), f"{what}: kept sets differ"
-    assert np.all(sel[:, :, width:] == -1)
+    in_band = check_kept_sets(cpu, sel, weights, ks, r, l, what)
+    decisions = sum(lens) * sel.shape[1]
+    if generic:
+        assert in_band <= max(16, decisions // 200), f"{what}: the band holds {in_band} of {decisions} decisions"
+    # alpha and the output for the GPU's set, in the oracle's fp64 arithmetic
+    want, want_alpha, _, _ = oracle_sparf(cpu, state, r, l, do_append=False, given=sel)
     gu.assert_close(out, want, what=what)
     assert np.abs(alpha - want_alpha).max() <= ALPHA_ATOL
-    return out, alpha, sel, (want, want_alpha, want_sel, weights)
+    return out, alpha, sel, (want, want_alpha, own_sel, weights)
 
 
 @pytest.mark.parametrize("tokens", [8, 16, 64])
@@ -187,10 +197,41 @@ def test_heavy_ties_are_cut_by_position():
         cpu.k_cache[int(table[1, j])] = first[:, None, :]
     state.kt_pool, state.kt_block_table = wl.make_sparf_state(cpu, 0.125, 64).kt_pool, \
         wl.make_sparf_state(cpu, 0.125, 64).kt_block_table
-    out, alpha, sel, own = run_and_check(cpu, state, 16, 8, "heavy ties")
+    out, alpha, sel, own = run_and_check(cpu, state, 16, 8, "heavy ties", generic=False)
     k0 = state.k_tokens_host[0]
     want = np.concatenate([np.arange(k0 - 8), np.arange(3000 - 8, 3000)])
     assert np.array_equal(sel[0, 0, :k0], want) and np.array_equal(sel[0, 1, :k0], want)
     ours, theirs = sel, own[2][:, :, :sel.shape[2]]                      # ties cut exactly as the oracle cuts them
     assert np.array_equal(ours[0], theirs[0]) and np.array_equal(ours[1], theirs[1])
     assert np.array_equal(ours[2, 1], theirs[2, 1])
+
+
+def test_length_beyond_the_transposed_copys_table_is_flagged_and_nothing_is_touched():
+    # The K/V table has room for 64 tokens per sequence (4 blocks of 16) but the transposed
+    # copy's table only for 32 (1 block of 32): a sequence of 40 tokens fits the first and not
+    # the second.  The append must flag it before reading either table and leave K, V, the
+    # transposed copy and the running sum exactly as they were; the other sequence proceeds.
+    cpu, state = make([40, 20], tokens=16, heads=3, kt_tokens=32)
+    dev, dstate = gu.to_device(cpu), dev_state(state)
+    assert dstate.kt_block_table.shape[1] == 2
+    short_table = dstate.kt_block_table[:, :1].contiguous()        # Mk = 1: capacity 32 tokens
+    before = [t.clone() for t in (dev.k_cache, dev.v_cache, dstate.kt_pool, dstate.v_sum)]
+    flags = torch.zeros(1, dtype=torch.int32, device="cuda")
+    binding.sparf_append(dev.k_cache, dev.v_cache, dstate.kt_pool, dstate.v_sum, dev.k_new, dev.v_new,
+                         dev.seq_lens, dev.block_table, short_table, flags)
+    torch.cuda.synchronize()
+    assert int(flags.item()) == binding.FLAG_SEQ_LEN_RANGE
+    # sequence 0: untouched everywhere
+    for b_table, pool, old, tokens in ((dev.block_table, dev.k_cache, before[0], 16),
+                                       (dev.block_table, dev.v_cache, before[1], 16)):
+        blk = int(b_table[0, 39 // tokens])
+        assert torch.equal(pool[blk].view(torch.int16), old[blk].view(torch.int16))
+    assert torch.equal(dstate.v_sum[0], before[3][0])
+    for blk in dstate.kt_block_table[0].tolist():
+        assert torch.equal(dstate.kt_pool[blk].view(torch.int16), before[2][blk].view(torch.int16))
+    # sequence 1 (20 tokens, fits both): appended as usual
+    blk, slot = int(dev.block_table[1, 19 // 16]), 19 % 16
+    assert torch.equal(dev.k_cache[blk, :, slot].view(torch.int16), dev.k_new[1].view(torch.int16))
+    kt_blk = int(short_table[1, 0])
+    assert torch.equal(dstate.kt_pool[kt_blk, :, :, 19].view(torch.int16), dev.k_new[1].view(torch.int16))
+    assert torch.equal(dstate.v_sum[1], before[3][1] + dev.v_new[1].float())

@@ -37,19 +37,51 @@ MUTANTS = {
 }
 
 
+# Planted mistakes in the sparse (Algorithm 1) oracle: lists of (old, new) replacements.
+SPARF_SOURCE = oracle_build.SOURCES[1]
+SPARF_MUTANTS = {
+    "window_mask_off_by_one": [("order[i].mask = i >= S - window ? 1 : 0;", "order[i].mask = i > S - window ? 1 : 0;")],
+    "temperature_ratio_inverted": [("(double)scale / sqrt(ratio);", "(double)scale * sqrt(ratio);")],
+    "alpha_summed_over_all_tokens": [("            if (alpha) alpha[pair] = mass;",
+                                      "            mass = 0.0; for (int32_t i = 0; i < S; ++i) mass += a[i];\n"
+                                      "            if (alpha) alpha[pair] = mass;")],
+    "one_minus_alpha_term_dropped": [("mass * attended + (1.0 - mass) * vbar;", "mass * attended;")],
+    "mean_value_divided_by_k": [("(double)v_sum[pair * D + d] / (double)S;",
+                                 "(double)v_sum[pair * D + d] / (double)(k > 0 ? k : 1);")],
+    "top_r_on_signed_q": [("dims[d].key = fabs(widen(qv[d]));", "dims[d].key = widen(qv[d]);"),
+                          ("q_l1 += dims[d].key;", "q_l1 += fabs(dims[d].key);"),
+                          ("qi_l1 += dims[t].key;", "qi_l1 += fabs(dims[t].key);")],
+    "ties_to_the_higher_position": [("return (a->index > b->index) - (a->index < b->index);",
+                                     "return (a->index < b->index) - (a->index > b->index);")],
+    "transposed_copy_stored_token_major": [("return (((int64_t)phys * g->heads + h) * g->dim + d) * g->tokens + i % g->tokens;",
+                                            "return (((int64_t)phys * g->heads + h) * g->tokens + i % g->tokens) * g->dim + d;")],
+    "exact_softmax_not_renormalised_over_J": [("const double attended = k > 0 ? o[d] / zs : 0.0;",
+                                               "const double attended = k > 0 ? o[d] : 0.0;")],
+    "approximate_scores_unscaled": [("a[i] = approx_scale * dot;", "a[i] = dot;")],
+}
+
+
 def build_mutant(tmp_path, name):
-    old, new = MUTANTS[name]
-    text = oracle_build.SOURCE.read_text()
-    assert old in text, f"mutation site for {name} not found"
-    src = tmp_path / f"{name}.c"
-    src.write_text(text.replace(old, new, 1))
+    sources = {src: src.read_text() for src in oracle_build.SOURCES}
+    if name in MUTANTS:
+        target, edits = oracle_build.SOURCE, [MUTANTS[name]]
+    else:
+        target, edits = SPARF_SOURCE, SPARF_MUTANTS[name]
+    for old, new in edits:
+        assert old in sources[target], f"mutation site for {name} not found"
+        sources[target] = sources[target].replace(old, new, 1)
+    paths = []
+    for src, text in sources.items():
+        path = tmp_path / f"{name}_{src.name}"
+        path.write_text(text)
+        paths.append(str(path))
     lib = tmp_path / f"{name}.so"
-    subprocess.run(["gcc", "-O1", "-std=c11", "-fopenmp", "-fPIC", "-shared", str(src), "-o", str(lib), "-lm"],
+    subprocess.run(["gcc", "-O1", "-std=c11", "-fopenmp", "-fPIC", "-shared", *paths, "-o", str(lib), "-lm"],
                    check=True, capture_output=True)
     return str(lib)
 
 
-def pins(monkey_lib):
+def pins(_unused=None):
     """A compact subset of the pins; returns the names of those that fail."""
     failed = []
     rng = np.random.default_rng(5)
@@ -117,19 +149,117 @@ def pins(monkey_lib):
     return failed
 
 
+def sparf_pins():
+    """A compact subset of the sparse oracle's pins; returns the names of those that fail."""
+    from tests.test_oracle_pins_sparf import paged, rows_of
+    from oracle import brute
+
+    failed = []
+    rng = np.random.default_rng(11)
+
+    def f16(shape, gain=1.0):
+        return (rng.standard_normal(shape) * gain).astype(np.float16)
+
+    def check(name, ok):
+        if not ok:
+            failed.append(name)
+
+    # every dim and every token kept: dense attention, alpha = 1
+    lens = np.array([1, 9, 40])
+    k, v, kt, v_sum, table = paged(rng, lens, 8)
+    q = f16((3, 2, 128), 2.0)
+    dense, _, _ = capi.decode_attention(q, k, v, lens, SCALE, block_table=table)
+    out, alpha, sel, _ = capi.sparf_attention(q, k, v, kt, v_sum, lens, lens, table, r=128, l=0, scale=SCALE)
+    check("dense_reduction", np.allclose(out, dense, rtol=0, atol=1e-13) and np.allclose(alpha, 1.0, atol=1e-13))
+    # every dim kept: the approximate weights are the dense weights, J their top-k, step 11 spelled out
+    lens = np.array([50])
+    k, v, kt, v_sum, table = paged(rng, lens, 16, gain=2.0)
+    q = f16((1, 2, 128), 2.0)
+    _, _, w = capi.decode_attention(q, k, v, lens, SCALE, block_table=table, want_weights=True)
+    out, alpha, sel, approx = capi.sparf_attention(q, k, v, kt, v_sum, lens, np.array([7]), table,
+                                                   r=128, l=0, scale=SCALE, want_weights=True)
+    ok = np.allclose(approx, w, rtol=0, atol=1e-14)
+    for h in range(2):
+        want = np.sort(np.argsort(-w[0, h], kind="stable")[:7])
+        ok &= np.array_equal(sel[0, h], want) and abs(alpha[0, h] - w[0, h, want].sum()) < 1e-14
+        vr = rows_of(v, table, 0, 50, 16)[h].astype(np.float64)
+        attn = (w[0, h, want] / w[0, h, want].sum()) @ vr[want]
+        vbar = v_sum[0, h].astype(np.float64) / 50
+        ok &= np.allclose(out[0, h], alpha[0, h] * attn + (1 - alpha[0, h]) * vbar, atol=1e-13)
+    check("all_dims_kept", bool(ok))
+    # window as large as k: local attention
+    lens = np.array([37])
+    k, v, kt, v_sum, table = paged(rng, lens, 8)
+    q = f16((1, 2, 128))
+    _, _, sel, _ = capi.sparf_attention(q, k, v, kt, v_sum, lens, np.array([10]), table, r=16, l=10, scale=SCALE)
+    check("local_window", np.array_equal(sel[0, 0], np.arange(27, 37)) and np.array_equal(sel[0, 1], np.arange(27, 37)))
+    # zero query: every score equal, the cut is by position
+    q0 = np.zeros((1, 2, 128), np.float16)
+    _, _, sel, _ = capi.sparf_attention(q0, k, v, kt, v_sum, lens, np.array([6]), table, r=16, l=2, scale=SCALE)
+    check("ties_by_position", np.array_equal(sel[0, 0], np.array([0, 1, 2, 3, 35, 36])))
+    # brute force on tiny shapes
+    ok = True
+    for r, kk, l in [(2, 3, 0), (4, 5, 2), (3, 6, 1)]:
+        lens = np.array([11, 6])
+        k, v, kt, v_sum, table = paged(rng, lens, 8, heads=2, dim=8, gain=2.0)
+        q = f16((2, 2, 8), 2.0)
+        scale = 1 / math.sqrt(8)
+        out, alpha, sel, _ = capi.sparf_attention(q, k, v, kt, v_sum, lens, np.full(2, kk), table, r=r, l=l, scale=scale)
+        for b, n in enumerate(lens):
+            kr, vr = rows_of(k, table, b, n, 8), rows_of(v, table, b, n, 8)
+            for h in range(2):
+                bo, ba, bj = brute.sparf_attention(q[b, h].view(np.uint16).tolist(), kr[h].view(np.uint16).tolist(),
+                                                   vr[h].view(np.uint16).tolist(), r, kk, l, scale)
+                ok &= sel[b, h, :len(bj)].tolist() == bj and abs(alpha[b, h] - ba) < 1e-13
+                ok &= np.allclose(out[b, h], np.array(bo), rtol=0, atol=1e-6)
+    check("brute_force", bool(ok))
+    # closed forms and the printed ranking (the pins of the sparse pin file itself)
+    from tests import test_oracle_pins_sparf as sparse_pins
+    for pin in (sparse_pins.test_the_temperature_is_the_printed_one_on_a_two_key_closed_form,
+                sparse_pins.test_step_six_is_the_ranking_of_the_printed_sum,
+                sparse_pins.test_the_window_survives_a_dominant_early_token):
+        try:
+            pin()
+        except AssertionError:
+            failed.append(pin.__name__)
+    # the append keeps the embedding-major copy the transpose of K
+    lens = np.array([9, 16])
+    k, v, kt, v_sum, table = paged(rng, lens, 8)
+    kn, vn = f16((2, 2, 128)), f16((2, 2, 128))
+    capi.sparf_append(k, v, kt, v_sum, kn, vn, lens, table)
+    check("append_transpose", np.array_equal(kt.view(np.uint16),
+                                             np.ascontiguousarray(k.transpose(0, 1, 3, 2)).view(np.uint16)))
+    return failed
+
+
 def test_the_real_oracle_passes_the_compact_pins():
     assert pins(None) == []
+    assert sparf_pins() == []
+
+
+ORACLE_FUNCTIONS = ("oracle_num_threads", "oracle_kv_append", "oracle_decode_attention",
+                    "oracle_decode_attention_grouped", "oracle_sparf_append", "oracle_sparf_attention")
+
+
+def load_mutant(lib_path, monkeypatch):
+    real = capi._load()
+    mutant = ctypes.CDLL(lib_path)
+    for fn in ORACLE_FUNCTIONS:
+        getattr(mutant, fn).restype = getattr(real, fn).restype
+        getattr(mutant, fn).argtypes = getattr(real, fn).argtypes
+    monkeypatch.setattr(capi, "_lib", mutant)
 
 
 @pytest.mark.parametrize("name", sorted(MUTANTS))
 def test_each_planted_mistake_is_caught(name, tmp_path, monkeypatch):
-    lib_path = build_mutant(tmp_path, name)
-    real = capi._load()
-    mutant = ctypes.CDLL(lib_path)
-    for fn in ("oracle_num_threads", "oracle_kv_append", "oracle_decode_attention",
-               "oracle_decode_attention_grouped"):
-        getattr(mutant, fn).restype = getattr(real, fn).restype
-        getattr(mutant, fn).argtypes = getattr(real, fn).argtypes
-    monkeypatch.setattr(capi, "_lib", mutant)
-    failed = pins(mutant)
+    load_mutant(build_mutant(tmp_path, name), monkeypatch)
+    failed = pins(None)
     assert failed, f"mutant {name} slipped through every pin"
+
+
+@pytest.mark.parametrize("name", sorted(SPARF_MUTANTS))
+def test_each_planted_mistake_in_the_sparse_oracle_is_caught(name, tmp_path, monkeypatch):
+    load_mutant(build_mutant(tmp_path, name), monkeypatch)
+    failed = sparf_pins()
+    assert failed, f"mutant {name} slipped through every pin"
+    print(name, "caught by", failed)

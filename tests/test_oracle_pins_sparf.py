@@ -184,3 +184,65 @@ def test_the_transposed_copy_may_use_its_own_block_size(kt_tokens):
         if n:
             blk, col = kt_table[b, (n - 1) // kt_tokens], (n - 1) % kt_tokens
             assert np.array_equal(kt2[blk, :, :, col].view(np.uint16), kn[b].view(np.uint16))
+
+
+def two_key_problem(q_vals, k0, k1):
+    """One sequence of two tokens, one head, 128 dims, one 8-token block; k0, k1 are dicts dim -> value."""
+    q = np.zeros((1, 1, 128), np.float16)
+    k = np.zeros((1, 1, 8, 128), np.float16)
+    for d, x in q_vals.items():
+        q[0, 0, d] = x
+    for d, x in k0.items():
+        k[0, 0, 0, d] = x
+    for d, x in k1.items():
+        k[0, 0, 1, d] = x
+    v = np.zeros((1, 1, 8, 128), np.float16)
+    v[0, 0, 0, 0], v[0, 0, 1, 0] = 1.0, -1.0
+    kt = np.ascontiguousarray(k.transpose(0, 1, 3, 2))
+    v_sum = np.zeros((1, 1, 128), np.float32)
+    return q, k, v, kt, v_sum, np.zeros((1, 1), np.int32)
+
+
+def test_the_temperature_is_the_printed_one_on_a_two_key_closed_form():
+    # |q| = 2 on dims 0-3 (negative: the ranking is on magnitudes), 1 on dims 4-15: with r = 4,
+    # |q_I|_1 / |q|_1 = 8 / 20, temperature sqrt(128 * 0.4); two keys give a logistic weight.
+    q_vals = {d: -2.0 for d in range(4)} | {d: 1.0 for d in range(4, 16)}
+    k0 = {0: 1.5, 1: -0.5, 5: 3.0}             # dims 5, 9 are outside I and must not count
+    k1 = {0: -1.0, 2: 0.5, 9: -3.0}
+    q, k, v, kt, v_sum, table = two_key_problem(q_vals, k0, k1)
+    _, alpha, sel, w = capi.sparf_attention(q, k, v, kt, v_sum, np.array([2]), np.array([1]), table,
+                                            r=4, l=0, scale=SCALE, want_weights=True)
+    dot0, dot1 = -2.0 * 1.5 + -2.0 * -0.5, -2.0 * -1.0 + -2.0 * 0.5
+    delta = (dot0 - dot1) / math.sqrt(128 * 0.4)
+    want0 = 1.0 / (1.0 + math.exp(-delta))
+    # the scale is rounded to binary32 on the way in: 6e-8 relative on delta
+    assert abs(w[0, 0, 0] - want0) < 1e-7 and abs(w[0, 0, 1] - (1 - want0)) < 1e-7
+    keep = 0 if want0 > 0.5 else 1
+    assert sel[0, 0, 0] == keep and abs(alpha[0, 0] - max(want0, 1 - want0)) < 1e-7
+
+
+def test_step_six_is_the_ranking_of_the_printed_sum():
+    # s^ + m ranked with numpy from the oracle's own s^ (generic data: no rounding corner)
+    rng = np.random.default_rng(38)
+    lens = np.array([200, 77])
+    k, v, kt, v_sum, table = paged(rng, lens, 8, gain=2.0)
+    q = f16(rng, (2, 2, 128), 2.0)
+    ks, l = np.array([25, 10]), 6
+    _, _, sel, w = capi.sparf_attention(q, k, v, kt, v_sum, lens, ks, table, r=16, l=l, scale=SCALE, want_weights=True)
+    for b, S in enumerate(lens):
+        m = (np.arange(S) >= S - l).astype(np.float64)
+        for h in range(2):
+            want = np.sort(np.argsort(-(w[b, h, :S] + m), kind="stable")[:ks[b]])
+            assert np.array_equal(sel[b, h, :ks[b]], want)
+
+
+def test_the_window_survives_a_dominant_early_token():
+    # token 0 takes all the approximate weight (s^ = 1 to fp64 rounding, the rest underflows
+    # against it); with k = l = 2 the kept set is still the last two positions
+    q_vals = {0: 60.0}
+    q, k, v, kt, v_sum, table = two_key_problem(q_vals, {0: 60.0}, {})
+    k[0, 0, 2, 0] = kt[0, 0, 0, 2] = -1.0
+    _, alpha, sel, w = capi.sparf_attention(q, k, v, kt, v_sum, np.array([3]), np.array([2]), table,
+                                            r=1, l=2, scale=SCALE, want_weights=True)
+    assert w[0, 0, 0] == 1.0 and 1.0 + w[0, 0, 1] == 1.0
+    assert sel[0, 0].tolist() == [1, 2] and alpha[0, 0] < 1e-100
