@@ -39,7 +39,9 @@
  *   inactive (nothing appended, zero output).  A block-table entry outside
  *   [0, num_phys_blocks) is not dereferenced: the append skips that sequence, attention
  *   reads that block's rows as zeros (the sequence's output is then meaningless but finite).
- *   No kernel traps, asserts or waits on another kernel.
+ *   No kernel traps, asserts or waits on another kernel; the only waits inside a kernel are
+ *   for its own asynchronous copies, and those give up after a time limit (see
+ *   INSTINFER_FLAG_COPY_TIMEOUT).
  * - Stream order is kept: each kernel sees everything enqueued before it on the stream as
  *   complete.  Internally the launches use programmatic dependent launch, so a kernel's
  *   blocks may already be resident while the previous kernel drains; they touch no memory
@@ -67,6 +69,9 @@ typedef enum {
 /* Bits OR-ed into *status_flags by the kernels. */
 #define INSTINFER_FLAG_SEQ_LEN_RANGE 1  /* seq_lens[b] < 0, beyond the cache capacity, or beyond max_seq_len */
 #define INSTINFER_FLAG_BLOCK_RANGE   2  /* a block_table entry that had to be read lies outside [0, num_phys_blocks) */
+#define INSTINFER_FLAG_COPY_TIMEOUT  4  /* an asynchronous copy inside a kernel did not complete within about two
+                                           seconds (a hardware problem, never a data problem); the kernel ended
+                                           instead of waiting on and the outputs of that call are undefined */
 
 /*
  * Append (Sec. II-B: the new token's k,v join the cache; Sec. IV-C, batch writing of the

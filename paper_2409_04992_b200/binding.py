@@ -15,7 +15,7 @@ import torch
 LIBRARY = Path(__file__).resolve().parent / "libinstinfer.so"
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA = range(5)
-FLAG_SEQ_LEN_RANGE, FLAG_BLOCK_RANGE = 1, 2
+FLAG_SEQ_LEN_RANGE, FLAG_BLOCK_RANGE, FLAG_COPY_TIMEOUT = 1, 2, 4
 STATIC_WORKSPACE_BYTES = 16 << 20
 
 _lib: Optional[ctypes.CDLL] = None

@@ -8,12 +8,18 @@
 // not around tensor cores:
 //   * a thread block owns one chunk of logical token positions of one (sequence, head);
 //   * each warp streams its own 8-token tiles of K and V through a private ring of shared
-//     memory stages filled by 16-byte cp.async copies (coalesced 512 B per warp instruction),
-//     with no block-wide barrier and no spin-wait anywhere in the main loop;
+//     memory stages with no block-wide barrier in the main loop.  A tile of a contiguous or
+//     paged cache is 2 KiB of K and 2 KiB of V, each one run of bytes in HBM: one lane moves
+//     each with a single bulk asynchronous copy (cp.async.bulk, 1-D, this GPU's memory only)
+//     that signals an mbarrier of the stage; the warp waits on it with a bounded try_wait.
+//     Rows picked from a list (the sparse path) come as 16-byte cp.async copies instead;
 //   * logits: 4 lanes share a key row (32 dims each, mixed-precision FMA: fp16 x fp16
 //     products are exact in the fp32 accumulator; 2 xor-shuffles), so a warp scores the 8
-//     rows of a tile at once; the softmax reference is uniform over the warp, follows the
-//     true maximum lazily, and each row's exponential (base 2, fp32) is computed once;
+//     rows of a tile at once.  Rows sit unpadded in shared memory; the 16-byte piece a lane
+//     reads in a step is rotated by its row (piece ^ row), which spreads the 8 rows of a
+//     quarter-warp over all banks, and the lane's query registers are loaded in that order.
+//     The softmax reference is uniform over the warp, follows the true maximum lazily, and
+//     each row's exponential (base 2, fp32) is computed once;
 //   * weighted sum: 16 lanes share a value row (8 dims each), the half-warps take alternate
 //     rows and fetch the row's weight (split into two fp16 parts) with one shuffle;
 //   * rows come from a contiguous cache, from paged pools through the block table, or from
@@ -34,18 +40,18 @@ constexpr int kWarps = 4;
 constexpr int kThreads = kWarps * 32;
 constexpr int kTileRows = 8;                       // tokens per warp tile
 constexpr int kStages = 3;                         // ring depth per warp
-constexpr int kKRowStride = kRowBytes + 16;        // K rows padded in shared memory: 4 lanes per
-                                                   // row read 8 rows at once without bank conflicts
-constexpr int kKTileBytes = kTileRows * kKRowStride;
+constexpr int kKTileBytes = kTileRows * kRowBytes;  // rows unpadded: a tile is one run of bytes
 constexpr int kVTileBytes = kTileRows * kRowBytes;
 constexpr int kStageBytes = kKTileBytes + kVTileBytes;
-constexpr int kSplitSmemBytes = kWarps * kStages * kStageBytes;   // 49.5 KiB
+constexpr int kRingBytes = kWarps * kStages * kStageBytes;        // 48 KiB
+constexpr int kSplitSmemBytes = kRingBytes + kWarps * kStages * 8; // + one mbarrier per stage
 constexpr int kCtasPerSm = 4;
 constexpr float kMinusHuge = -1.0e30f;             // finite stand-in for "no row seen yet"
 constexpr float kLn2 = 0.69314718055994530942f;
 
 constexpr int kFlagSeqLenRange = 1;
 constexpr int kFlagBlockRange = 2;
+constexpr int kFlagCopyTimeout = 4;
 
 struct AttnParams {
     const __half *q;
@@ -100,6 +106,48 @@ __device__ __forceinline__ void cp_async_16(unsigned dst, const void *gmem_src, 
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
 template <int kPending>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" :: "n"(kPending) : "memory"); }
+
+// Bulk asynchronous copies (global -> this block's shared memory) completing on an mbarrier.
+// Addresses are 16-byte aligned and sizes multiples of 16 bytes by construction (256-byte rows).
+__device__ __forceinline__ void mbarrier_init(unsigned bar, unsigned count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbarrier_init_fence()
+{
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void mbarrier_expect_bytes(unsigned bar, unsigned bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void bulk_copy(unsigned dst, const void *src, unsigned bytes, unsigned bar)
+{
+    asm volatile("cp.async.bulk.shared::cta.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 :: "r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbarrier_try_wait(unsigned bar, unsigned parity)
+{
+    unsigned done;
+    asm volatile("{\n\t.reg .pred p;\n\t"
+                 "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+                 "selp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+    return done != 0;
+}
+// Waits for phase `parity` of the barrier, giving up after about kWaitCycles clock cycles (a
+// copy of a few KiB completes in microseconds: running out means the hardware has a problem,
+// and the kernel must end rather than hang).
+constexpr long long kWaitCycles = 4000000000ll;
+__device__ __forceinline__ bool mbarrier_wait_bounded(unsigned bar, unsigned parity)
+{
+    if (mbarrier_try_wait(bar, parity)) return true;
+    const long long start = clock64();
+    for (;;) {
+        if (mbarrier_try_wait(bar, parity)) return true;
+        if (clock64() - start > kWaitCycles) return false;
+    }
+}
 
 // Sequence length as the kernels see it: out-of-range lengths make the slot inactive.
 __device__ __forceinline__ int checked_seq_len(const AttnParams &p, int b, bool report)
@@ -190,6 +238,7 @@ decode_attn_split_kernel(const AttnParams p)
 {
     constexpr bool kPaged = kRows == Rows::kPaged;
     constexpr bool kGathered = kRows == Rows::kGathered;
+    constexpr bool kBulk = !kGathered;                   // whole tiles by one bulk copy each
     extern __shared__ __align__(128) unsigned char smem[];
     constexpr int kStepTokens = kWarps * kTileRows;      // a warp's next tile is this far ahead
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -205,6 +254,13 @@ decode_attn_split_kernel(const AttnParams p)
     const int pair = blockIdx.x - split * p.pairs;
     const int b = pair / p.heads, h = pair - b * p.heads;
     const bool final_writer = !kGathered && p.n_splits == 1;
+    // one mbarrier per stage, behind the rings: a stage's bulk copies report their bytes to it
+    const unsigned bars = static_cast<unsigned>(__cvta_generic_to_shared(smem)) + kRingBytes + warp * (kStages * 8);
+    if (kBulk && lane == 0) {                            // each warp owns the barriers of its ring
+#pragma unroll
+        for (int s = 0; s < kStages; ++s) mbarrier_init(bars + s * 8, 1);
+        mbarrier_init_fence();
+    }
     allow_next_kernel();
     wait_for_previous_kernels();
 
@@ -228,26 +284,34 @@ decode_attn_split_kernel(const AttnParams p)
                                                          : kTileRows;
 
     // This lane's 32 query dims, kept in fp16 (16 registers): products with fp16 keys are
-    // exact in fp32 and the scale is applied to the finished dot product.
+    // exact in fp32 and the scale is applied to the finished dot product.  In step i the lane
+    // reads the 16-byte piece (4 quarter + i) ^ row of its key row (see k_rd below), so its
+    // query registers are loaded in that order.
     uint4 qh[4];
     {
-        const uint4 *src = reinterpret_cast<const uint4 *>(p.q + (int64_t)pair * kHeadDim + quarter * 32);
+        const uint4 *src = reinterpret_cast<const uint4 *>(p.q + (int64_t)pair * kHeadDim);
 #pragma unroll
-        for (int i = 0; i < 4; ++i) qh[i] = src[i];
+        for (int i = 0; i < 4; ++i) qh[i] = src[(quarter * 4 + i) ^ row];
     }
 
-    // Shared-memory addresses (shared window, 32 bit).  K rows are padded to kKRowStride.
+    // Shared-memory addresses (shared window, 32 bit).
     const unsigned ring = static_cast<unsigned>(__cvta_generic_to_shared(smem)) +
                           warp * (kStages * kStageBytes);
-    // copies: 16-byte segment lane + 32 i, i < 4, lies in row 2 i + half_warp at column segment col
-    const unsigned k_dst = half_warp * kKRowStride + col * 16;
+    // cp.async copies: 16-byte segment lane + 32 i, i < 4, lies in row 2 i + half_warp at column segment col
+    const unsigned k_dst = half_warp * kRowBytes + col * 16;
     const unsigned v_dst = kKTileBytes + lane * 16;
-    const unsigned k_rd = row * kKRowStride + quarter * 64;
+    // The 8 lanes of a quarter-warp read one piece each of rows 0..7 in the same step; rows are
+    // 256 bytes apart (the same banks), so the piece index is rotated by the row: 8 distinct
+    // 16-byte bank groups, no conflict.
+    const unsigned k_rd = row * kRowBytes;
+    unsigned k_piece[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) k_piece[i] = (((quarter * 4 + i) ^ row) & 15) * 16;
     const unsigned v_rd = kKTileBytes + lane * 16;
 
     // ---- copy-issue side: walks this warp's tiles incrementally (no division per tile) ----
-    const unsigned char *k_lane = reinterpret_cast<const unsigned char *>(p.k) + lane * 16;
-    const unsigned char *v_lane = reinterpret_cast<const unsigned char *>(p.v) + lane * 16;
+    const unsigned char *k_base = reinterpret_cast<const unsigned char *>(p.k);
+    const unsigned char *v_base = reinterpret_cast<const unsigned char *>(p.v);
     const int first_token = begin + warp * kTileRows;
     int64_t src_off = 0;                       // contiguous: byte offset of the next tile
     int blk = 0, rem = 0, win_base = 0;        // paged: block index, row inside it, window start
@@ -295,67 +359,75 @@ decode_attn_split_kernel(const AttnParams p)
     auto issue = [&]() {
         if (issue_j < my_tiles) {
             const int rows = issue_j == my_tiles - 1 ? last_rows : kTileRows;
-            bool usable = true;
-            int64_t off = 0;
+            const unsigned dst = ring + issue_stage * kStageBytes;
             if (kGathered) {
                 if ((issue_j & 3) == 0 && issue_j > 0) {       // uniform: next window of 4 tiles
                     rows_now = rows_next;
                     rows_next = load_rows(issue_j + 4);
                 }
-                const unsigned dst = ring + issue_stage * kStageBytes;
-                const unsigned char *k_col = reinterpret_cast<const unsigned char *>(p.k) + col * 16;
-                const unsigned char *v_col = reinterpret_cast<const unsigned char *>(p.v) + col * 16;
+                const unsigned char *k_col = k_base + col * 16;
+                const unsigned char *v_col = v_base + col * 16;
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
                     const int rid = __shfl_sync(0xffffffffu, rows_now, (issue_j & 3) * 8 + 2 * i + half_warp);
                     const bool valid = 2 * i + half_warp < rows;
                     const int64_t src = valid ? (int64_t)rid * kRowBytes : 0;
-                    cp_async_16(dst + k_dst + i * 2 * kKRowStride, k_col + src, valid ? 16 : 0);
+                    cp_async_16(dst + k_dst + i * 2 * kRowBytes, k_col + src, valid ? 16 : 0);
                     cp_async_16(dst + v_dst + i * 512, v_col + src, valid ? 16 : 0);
                 }
-            } else if (kPaged) {
-                int idx = blk - win_base;
-                if (idx >= 32) {               // uniform: slide the window of table entries
-                    idx -= 32;
-                    win_base += 32;
-                    window_now = window_next;
-                    window_next = load_window(win_base + 32);
-                }
-                const int phys = __shfl_sync(0xffffffffu, window_now, idx);
-                usable = phys >= 0 && (int64_t)phys < p.num_phys_blocks;
-                if (!usable && lane == 0 && p.status) atomicOr(p.status, kFlagBlockRange);
-                off = usable ? (int64_t)phys * block_stride + head_off + rem * kRowBytes : 0;
-                blk += step_blk;
-                rem += step_rem;
-                if (rem >= p.block_tokens) {
-                    rem -= p.block_tokens;
-                    ++blk;
-                }
             } else {
-                off = src_off;
-                src_off += kStepTokens * kRowBytes;
-            }
-            const unsigned char *ks = k_lane + off, *vs = v_lane + off;
-            const unsigned dst = ring + issue_stage * kStageBytes;
-            if (kGathered) {
-                // copies already issued above
-            } else if (usable && rows == kTileRows) {          // full tile: no predicates
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    cp_async_16(dst + k_dst + i * 2 * kKRowStride, ks + i * 512, 16);
-                    cp_async_16(dst + v_dst + i * 512, vs + i * 512, 16);
+                bool usable = true;
+                int64_t off;
+                if (kPaged) {
+                    int idx = blk - win_base;
+                    if (idx >= 32) {               // uniform: slide the window of table entries
+                        idx -= 32;
+                        win_base += 32;
+                        window_now = window_next;
+                        window_next = load_window(win_base + 32);
+                    }
+                    const int phys = __shfl_sync(0xffffffffu, window_now, idx);
+                    usable = phys >= 0 && (int64_t)phys < p.num_phys_blocks;
+                    if (!usable && lane == 0 && p.status) atomicOr(p.status, kFlagBlockRange);
+                    off = usable ? (int64_t)phys * block_stride + head_off + rem * kRowBytes : 0;
+                    blk += step_blk;
+                    rem += step_rem;
+                    if (rem >= p.block_tokens) {
+                        rem -= p.block_tokens;
+                        ++blk;
+                    }
+                } else {
+                    off = src_off;
+                    src_off += kStepTokens * kRowBytes;
                 }
-            } else {                                           // ragged tail: masked rows are zero-filled
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const bool valid = usable && (2 * i + half_warp < rows);
-                    const int src = valid ? i * 512 : 0;
-                    cp_async_16(dst + k_dst + i * 2 * kKRowStride, ks + src, valid ? 16 : 0);
-                    cp_async_16(dst + v_dst + i * 512, vs + src, valid ? 16 : 0);
+                // The tile's rows are one run of bytes in the cache (a tile never straddles a
+                // block: block_tokens is a multiple of the tile).  Rows past the chunk's end and
+                // the rows of a block with a bad id are not fetched; their value slots are
+                // zeroed (their weights are zero, but 0 x stale bits must not be NaN) and their
+                // logits are masked below.
+                const int fetch = usable ? rows : 0;
+                if (fetch < kTileRows) {
+                    const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
+                    for (int seg = fetch * 16 + lane; seg < kTileRows * 16; seg += 32) {
+                        asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};"
+                                     :: "r"(dst + kKTileBytes + seg * 16), "r"(zero.x), "r"(zero.y), "r"(zero.z), "r"(zero.w) : "memory");
+                        asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};"
+                                     :: "r"(dst + seg * 16), "r"(zero.x), "r"(zero.y), "r"(zero.z), "r"(zero.w) : "memory");
+                    }
+                    __syncwarp();
+                }
+                if (lane == 0) {
+                    const unsigned bar = bars + issue_stage * 8;
+                    const unsigned bytes = (unsigned)fetch * kRowBytes;
+                    mbarrier_expect_bytes(bar, 2 * bytes);
+                    if (fetch > 0) {
+                        bulk_copy(dst, k_base + off, bytes, bar);
+                        bulk_copy(dst + kKTileBytes, v_base + off, bytes, bar);
+                    }
                 }
             }
         }
-        cp_async_commit();                                     // empty groups keep the count uniform
+        if (kGathered) cp_async_commit();                      // empty groups keep the count uniform
         ++issue_j;
         issue_stage = issue_stage + 1 == kStages ? 0 : issue_stage + 1;
     };
@@ -366,22 +438,32 @@ decode_attn_split_kernel(const AttnParams p)
 #pragma unroll
     for (int i = 0; i < 8; ++i) acc[i] = 0.f;
 
+    if (kBulk) __syncwarp();             // the barriers are initialised before the first copy
 #pragma unroll
     for (int j = 0; j < kStages - 1; ++j) issue();
 
-    unsigned stage = 0;
+    unsigned stage = 0, phase = 0;
+    bool stalled = false;
     for (int j = 0; j < my_tiles; ++j) {
-        cp_async_wait<kStages - 2>();
+        if (kGathered) {
+            cp_async_wait<kStages - 2>();
+        } else if (!__all_sync(0xffffffffu, mbarrier_wait_bounded(bars + stage * 8, phase))) {
+            stalled = true;              // one decision for the whole warp
+            break;
+        }
         __syncwarp();                    // tile j visible to the warp; everyone is done with tile j-1
         issue();                         // refills the slot tile j-1 used
         const unsigned base = ring + stage * kStageBytes;
-        stage = stage + 1 == kStages ? 0 : stage + 1;
+        if (++stage == kStages) {
+            stage = 0;
+            phase ^= 1u;
+        }
 
         // Logit: this lane's quarter of row `row`, four independent fp32 chains.
         float part[4];
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-            const uint4 kr = lds128(base + k_rd + i * 16);
+            const uint4 kr = lds128(base + k_rd + k_piece[i]);
             const unsigned kw[4] = {kr.x, kr.y, kr.z, kr.w};
             const unsigned qw[4] = {qh[i].x, qh[i].y, qh[i].z, qh[i].w};
             float dot = 0.f;
@@ -439,7 +521,24 @@ decode_attn_split_kernel(const AttnParams p)
             }
         }
     }
-    cp_async_wait<0>();
+    if (kGathered) cp_async_wait<0>();
+    if (kBulk && stalled) {
+        // A copy did not arrive in time.  Report it, give the copies still in flight one more
+        // bounded chance to land (shared memory must not be handed on while they are pending)
+        // and leave; this block's partial result stays unwritten and the call's output is
+        // undefined, which the flag tells the caller.
+        if (lane == 0 && p.status) atomicOr(p.status, kFlagCopyTimeout);
+        const int issued = min(issue_j, my_tiles);
+        for (int t = issued - min(issued, kStages - 1); t < issued; ++t)
+            (void)mbarrier_wait_bounded(bars + (t % kStages) * 8, (t / kStages) & 1);
+    }
+    // (a block barrier follows: a stalled warp still joins it, then contributes an empty state)
+    if (kBulk && stalled) {
+        m = kMinusHuge;
+        l = 0.f;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) acc[i] = 0.f;
+    }
 
     // One state per warp: sum l over the 8 rows, fold the two half-warps' accumulators.
     l += __shfl_xor_sync(0xffffffffu, l, 1);
