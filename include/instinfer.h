@@ -382,13 +382,14 @@ size_t instinfer_workspace_bytes(int32_t batch, int32_t heads, int32_t head_dim,
 
 /*
  * Split plan.  A sequence is cut at fixed logical token positions, the same for every
- * sequence: first chunks of `chunk_tokens`, then, near the end of the longest admissible
- * sequence, shorter chunks (they are scheduled last and keep the tail of the launch short).
- * Each chunk of each (sequence, head) is reduced by one thread block and the partial results
- * are merged by log-sum-exp (no counterpart in the paper, whose engine streams token groups
- * through parallel GeMV units, Sec. IV-B).  instinfer_plan_chunk_tokens returns the first
- * chunk size the library would use for these sizes and instinfer_plan_num_splits the number
- * of chunks per sequence (0 if an argument is invalid).
+ * sequence: first a few short chunks (they are scheduled last: every sequence of a ragged
+ * batch has its first tokens, so every launch ends on short blocks and its tail stays short),
+ * then long chunks of `chunk_tokens`.  Each chunk of each (sequence, head) is reduced by one
+ * thread block and the partial results are merged by log-sum-exp in position order (no
+ * counterpart in the paper, whose engine streams token groups through parallel GeMV units,
+ * Sec. IV-B).  instinfer_plan_chunk_tokens returns the long chunk size the library would use
+ * for these sizes and instinfer_plan_num_splits the number of chunks per sequence, short ones
+ * included (0 if an argument is invalid).
  * instinfer_set_chunk_tokens(n) forces uniform chunks of n tokens for later calls of this
  * process (n > 0, a multiple of 64), n == 0 restores the automatic choice; it returns
  * INSTINFER_OK or INSTINFER_ERR_INVALID_ARG.  Not thread-safe against concurrent calls.

@@ -18,7 +18,7 @@ constexpr int kChunkGranule = 64;        // chunk_tokens is a multiple of this
 constexpr int kChunkCeiling = 2048;      // automatic plan: chunk never longer than this ...
 constexpr int kChunkFloor = 256;         // ... nor shorter than this, sequence permitting
 constexpr int kTargetWaves = 8;          // automatic plan: aim for this many waves of blocks
-constexpr int kTailChunk = 256;          // automatic plan: chunk size at the end of long sequences
+constexpr int kTailChunk = 256;          // automatic plan: size of the short chunks at the start of a sequence
 constexpr int kTailWaves = 2;            // ... covering about this many waves of blocks
 
 inline int g_forced_chunk = 0;
@@ -77,17 +77,18 @@ inline cudaError_t launch_overlapped(void (*kernel)(Params...), unsigned grid, u
 }
 
 struct SplitPlan {
-    int32_t chunk_tokens;   // size of the first n_big chunks
+    int32_t chunk_tokens;   // size of the n_big long chunks, which follow the short ones
     int32_t n_big;
-    int32_t tail_chunk;     // size of the chunks after them
+    int32_t tail_chunk;     // size of the n_splits - n_big short chunks at the start of a sequence
     int32_t n_splits;
 };
 
 // Cuts are at fixed logical token positions, the same for every sequence, so a result never
-// depends on the physical placement of blocks.  Blocks are scheduled chunk-major, so the
-// chunks at the end of the longest sequences run last: making those short keeps the tail of
-// a launch (SMs idling while the last blocks finish) short without paying the per-block
-// overhead of small chunks everywhere.
+// depends on the physical placement of blocks.  Blocks are scheduled chunk-major with the
+// short chunks last.  The short chunks cover the first tokens of a sequence, which every
+// sequence of a ragged batch has: a launch then ends on about kTailWaves waves of short
+// blocks whatever the lengths are (SMs idle only while the last short blocks finish),
+// without paying the per-block overhead of small chunks everywhere.
 // What differs between the kernels that share the planner.
 struct PlanRules {
     int ctas_per_sm;
@@ -101,7 +102,7 @@ constexpr PlanRules kOneRowRules = {kCtasPerSm, kTargetWaves, kChunkCeiling, kTa
 inline SplitPlan make_plan(int64_t pairs, int32_t max_seq_len, const PlanRules &rules = kOneRowRules)
 {
     SplitPlan plan;
-    if (g_forced_chunk > 0) {
+    if (g_forced_chunk > 0) {               // uniform chunks, no short ones
         plan.chunk_tokens = plan.tail_chunk = g_forced_chunk;
         plan.n_big = (int32_t)ceil_div(max_seq_len, g_forced_chunk);
         plan.n_splits = plan.n_big;
@@ -133,21 +134,19 @@ inline SplitPlan make_plan(int64_t pairs, int32_t max_seq_len, const PlanRules &
         }
     }
     int64_t chunk = ceil_div(ceil_div(max_seq_len, n), kChunkGranule) * kChunkGranule;
-    // Tail region: about kTailWaves waves of kTailChunk-token blocks at the end of the longest
-    // sequences, at most a quarter of the sequence; none when the chunks are that short anyway.
+    // Short region: about kTailWaves waves of tail_chunk-token blocks at the start of every
+    // sequence, at most a quarter of the longest; none when the chunks are that short anyway.
     const int64_t tail_chunk = rules.tail_chunk_tokens > 0 ? rules.tail_chunk_tokens : kTailChunk;
-    int64_t tail_tokens = ceil_div(slots * kTailWaves, pairs) * tail_chunk;
-    if (tail_tokens > max_seq_len / 4) tail_tokens = max_seq_len / 4 / tail_chunk * tail_chunk;
-    if (chunk <= 2 * tail_chunk || tail_tokens < tail_chunk || rules.tail_chunk_tokens <= 0) tail_tokens = 0;
-    if (tail_tokens > 0)      // rounded down, so that at least tail_tokens are left for the tail
-        chunk = (max_seq_len - tail_tokens) / n / kChunkGranule * kChunkGranule;
-    int64_t big_span = n * chunk;
-    while (big_span - chunk >= max_seq_len) big_span -= chunk;
+    int64_t short_tokens = ceil_div(slots * kTailWaves, pairs) * tail_chunk;
+    if (short_tokens > max_seq_len / 4) short_tokens = max_seq_len / 4 / tail_chunk * tail_chunk;
+    if (chunk <= 2 * tail_chunk || short_tokens < tail_chunk || rules.tail_chunk_tokens <= 0) short_tokens = 0;
+    if (short_tokens > 0)
+        chunk = ceil_div(ceil_div(max_seq_len - short_tokens, n), kChunkGranule) * kChunkGranule;
+    const int64_t n_short = short_tokens > 0 ? short_tokens / tail_chunk : 0;
     plan.chunk_tokens = (int32_t)chunk;
-    plan.n_big = (int32_t)(big_span / chunk);
-    plan.tail_chunk = tail_tokens > 0 ? (int32_t)tail_chunk : (int32_t)chunk;
-    plan.n_splits = plan.n_big + (big_span < max_seq_len
-                                      ? (int32_t)ceil_div(max_seq_len - big_span, plan.tail_chunk) : 0);
+    plan.n_big = (int32_t)ceil_div(max_seq_len - short_tokens, chunk);
+    plan.tail_chunk = short_tokens > 0 ? (int32_t)tail_chunk : (int32_t)chunk;
+    plan.n_splits = (int32_t)(n_short + plan.n_big);
     return plan;
 }
 

@@ -70,10 +70,11 @@ struct AttnParams {
     int32_t s_max;
     int32_t block_tokens;
     int32_t max_blocks_per_seq;
-    int32_t chunk_tokens; // tokens per chunk for the first n_big chunks of a sequence ...
-    int32_t n_big;
-    int32_t tail_chunk;   // ... and per chunk after that (scheduled last: short tail of the launch)
-    int32_t n_splits;     // n_big + number of tail chunks
+    int32_t chunk_tokens; // tokens per long chunk; the long chunks follow the short ones ...
+    int32_t n_big;        // number of long chunks
+    int32_t tail_chunk;   // ... tokens per short chunk: the first n_splits - n_big chunks of every
+                          // sequence (scheduled last, so that every launch ends on short blocks)
+    int32_t n_splits;     // short chunks + long chunks
     int32_t max_seq_len;
     float scale_log2e;    // scale * log2(e): logits are kept in the base-2 domain
     // gathered mode only (sparse attention over a list of selected rows):
@@ -166,24 +167,39 @@ __device__ __forceinline__ int gathered_count(const AttnParams &p, int b, int le
     return min(len, min(max(p.k_tokens[b], 0), p.row_stride));
 }
 
+// The split plan.  A sequence is cut at fixed logical positions, the same for every sequence:
+// first n_short = n_splits - n_big short chunks of tail_chunk tokens, then n_big long chunks of
+// chunk_tokens.  Chunks are numbered by position (that is also the order of the merge); the
+// grid runs the long chunks first and the short ones last.  Every sequence of a ragged batch
+// has its first tokens, so the last waves of a launch are made of many short blocks whatever
+// the lengths are, instead of a few long blocks at the ends of the longest sequences.
+
 // Logical token range [begin, begin + size) of chunk `split`.
 __device__ __forceinline__ void chunk_range(const AttnParams &p, int split, int &begin, int &size)
 {
-    if (split < p.n_big) {
-        begin = split * p.chunk_tokens;
-        size = p.chunk_tokens;
-    } else {
-        begin = p.n_big * p.chunk_tokens + (split - p.n_big) * p.tail_chunk;
+    const int n_short = p.n_splits - p.n_big;
+    if (split < n_short) {
+        begin = split * p.tail_chunk;
         size = p.tail_chunk;
+    } else {
+        begin = n_short * p.tail_chunk + (split - n_short) * p.chunk_tokens;
+        size = p.chunk_tokens;
     }
+}
+
+// The chunk that the `order`-th group of blocks of the grid works on: long chunks first.
+__device__ __forceinline__ int scheduled_chunk(const AttnParams &p, int order)
+{
+    return order < p.n_big ? p.n_splits - p.n_big + order : order - p.n_big;
 }
 
 // Number of chunks of a sequence of `len` tokens that hold at least one token.
 __device__ __forceinline__ int live_chunks(const AttnParams &p, int len)
 {
-    const int big_span = p.n_big * p.chunk_tokens;
-    if (len <= big_span) return (len + p.chunk_tokens - 1) / p.chunk_tokens;
-    return p.n_big + (len - big_span + p.tail_chunk - 1) / p.tail_chunk;
+    const int n_short = p.n_splits - p.n_big;
+    const int short_span = n_short * p.tail_chunk;
+    if (len <= short_span) return (len + p.tail_chunk - 1) / p.tail_chunk;
+    return n_short + (len - short_span + p.chunk_tokens - 1) / p.chunk_tokens;
 }
 
 // d = a * b + c with fp16 a, b and fp32 c, d: the product of two fp16 values is exact in
@@ -247,11 +263,12 @@ decode_attn_split_kernel(const AttnParams p)
     // take alternate rows.
     const int row = lane & 7, quarter = lane >> 3;
     const int col = lane & 15, half_warp = lane >> 4;
-    // Grid order: split slowest, then sequence, head fastest.  Blocks that run together then
-    // cover all heads of a few sequences (one paged block's heads are adjacent in memory),
-    // and the short last chunks of ragged sequences are scheduled last.
-    const int split = blockIdx.x / p.pairs;
-    const int pair = blockIdx.x - split * p.pairs;
+    // Grid order: chunk slowest (long chunks first, short ones last), then sequence, head
+    // fastest.  Blocks that run together then cover all heads of a few sequences (one paged
+    // block's heads are adjacent in memory).
+    const int order = blockIdx.x / p.pairs;
+    const int pair = blockIdx.x - order * p.pairs;
+    const int split = scheduled_chunk(p, order);
     const int b = pair / p.heads, h = pair - b * p.heads;
     const bool final_writer = !kGathered && p.n_splits == 1;
     // one mbarrier per stage, behind the rings: a stage's bulk copies report their bytes to it

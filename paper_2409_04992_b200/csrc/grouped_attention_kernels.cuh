@@ -219,8 +219,9 @@ grouped_attn_split_kernel(const GroupedParams p)
     const AttnParams &a = p.a;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int gid = lane >> 2, quad = lane & 3;          // MMA fragment coordinates
-    const int split = blockIdx.x / a.pairs;
-    const int pair = blockIdx.x - split * a.pairs;
+    const int order = blockIdx.x / a.pairs;
+    const int pair = blockIdx.x - order * a.pairs;
+    const int split = scheduled_chunk(a, order);
     const int b = pair / a.heads, hk = pair - b * a.heads;
     const bool final_writer = a.n_splits == 1;
     allow_next_kernel();

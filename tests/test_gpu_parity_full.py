@@ -4,7 +4,7 @@ compared element by element; for the larger ones the oracle recomputes sampled (
 head) pairs one by one from rows gathered off the device: 64 pairs of each 20 GiB workload,
 8 pairs of every one of the 40 layers of the 13B-class step, and a batch of that step's shape
 whose lengths are placed on the edges of the split plan (last token in the first tile of a
-short end chunk, in a ragged last tile, on a chunk boundary)."""
+chunk, in a ragged last tile, on a chunk boundary)."""
 import numpy as np
 import pytest
 import torch
@@ -134,14 +134,17 @@ def test_workload_4_shape_with_lengths_on_the_edges_of_the_plan():
     w = wl.STANDARD[4]
     chunk = binding.plan_chunk_tokens(w.batch, w.heads, w.len_hi)
     splits = binding.plan_num_splits(w.batch, w.heads, w.len_hi)
-    n_big = min(splits, w.len_hi // chunk)
-    span = n_big * chunk                         # where the short end chunks (256 tokens) begin, if any
-    tail = 256 if span < w.len_hi else chunk
+    # the plan: n_short chunks of 256 tokens, then long chunks; recover n_short from the counts
+    n_short = next(n for n in range(0, 64) if n + -(-(w.len_hi - 256 * n) // chunk) == splits)
+    first_long = 256 * n_short
+    seam = lambda j: first_long + j * chunk                      # start of long chunk j
+    mid = [j for j in range(1, splits) if w.len_lo < seam(j) < w.len_hi - 8]
+    assert len(mid) >= 3, (chunk, splits, n_short)
     edges = [w.len_hi, w.len_lo,
-             span + 1, span + 8, span + tail + 3, span + 2 * tail + 8,      # first tile of an end chunk
-             span, span - 1, span + tail,                                    # exactly on a seam, one before
-             5 * chunk + 1, 5 * chunk + 9,                                   # first tiles of a long chunk
-             w.len_hi - 1, w.len_hi - 3, w.len_lo + 5, 6001, 7777]           # ragged last tiles
+             seam(mid[0]) + 1, seam(mid[0]) + 8, seam(mid[1]) + 3, seam(mid[-1]) + 8,   # first tile of a chunk
+             seam(mid[0]), seam(mid[0]) - 1, seam(mid[1]), seam(mid[-1]) - 5,         # on a seam, just before one
+             seam(mid[1]) + 9, seam(mid[-1]) + 17,                                    # second and third tiles
+             w.len_hi - 1, w.len_hi - 3, w.len_lo + 5, 6001]                           # ragged last tiles
     lens = [int(min(max(n, w.len_lo), w.len_hi)) for n in edges][:w.batch]
     assert len(lens) == w.batch
     case = wl.generate(w, layer=3, device="cuda", seq_lens=lens)
