@@ -248,6 +248,78 @@ __device__ __forceinline__ uint4 lds128(unsigned shared_addr)
     return v;
 }
 
+// One 8-token tile of one warp: logits of the 8 key rows, online softmax update, weighted sum
+// of the 8 value rows.  k_row / v_seg are this lane's shared-memory addresses inside the tile
+// (row `row` of K; the lane's 16-byte segment of V rows 0 and 1), k_piece its four rotated
+// 16-byte pieces of the key row, qh the query dims that go with them.  m is the warp-uniform
+// softmax reference, l this lane's partial sum of weights, acc its 8 output dims (scaled by
+// kWeightScale); rows < 8 masks the rows past the end of the chunk.
+__device__ __forceinline__ void attend_tile(unsigned k_row, const unsigned (&k_piece)[4], unsigned v_seg,
+                                            const uint4 (&qh)[4], float scale_log2e, int rows, int row,
+                                            int half_warp, float &m, float &l, float (&acc)[8])
+{
+    // Logit: this lane's quarter of row `row`, four independent fp32 chains.
+    float part[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const uint4 kr = lds128(k_row + k_piece[i]);
+        const unsigned kw[4] = {kr.x, kr.y, kr.z, kr.w};
+        const unsigned qw[4] = {qh[i].x, qh[i].y, qh[i].z, qh[i].w};
+        float dot = 0.f;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            unsigned short k0, k1, q0, q1;
+            halves(kw[e], k0, k1);
+            halves(qw[e], q0, q1);
+            dot = fma_h(k0, q0, dot);
+            dot = fma_h(k1, q1, dot);
+        }
+        part[i] = dot;
+    }
+    float s = ((part[0] + part[1]) + (part[2] + part[3])) * scale_log2e;
+    s += __shfl_xor_sync(0xffffffffu, s, 8);
+    s += __shfl_xor_sync(0xffffffffu, s, 16);
+    if (row >= rows) s = -INFINITY;
+
+    // Online softmax with a warp-uniform reference m that may lag the true maximum by up to
+    // kMaxLag (base-2 units): weights then reach at most 2^kMaxLag, which is harmless in
+    // fp32 and inside the range of the fp16 weight split.  The reference only moves (and
+    // the accumulators are only rescaled) when some logit exceeds it by more than that,
+    // so the common tile pays one vote instead of a shuffle reduction.
+    if (__any_sync(0xffffffffu, s > m + kMaxLag)) {
+        float tile_max = s;
+        tile_max = fmaxf(tile_max, __shfl_xor_sync(0xffffffffu, tile_max, 1));
+        tile_max = fmaxf(tile_max, __shfl_xor_sync(0xffffffffu, tile_max, 2));
+        tile_max = fmaxf(tile_max, __shfl_xor_sync(0xffffffffu, tile_max, 4));
+        const float alpha = fast_exp2(m - tile_max);
+        l *= alpha;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) acc[i] *= alpha;
+        m = tile_max;
+    }
+    const float pw = fast_exp2(s - m);
+    l += pw;
+
+    // Attend: rows 2 r + half_warp, r < 4.
+    const unsigned packed = split_weight(pw);
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {
+        unsigned short w_lo, w_hi;
+        halves(__shfl_sync(0xffffffffu, packed, 2 * r + half_warp), w_lo, w_hi);
+        const uint4 vr = lds128(v_seg + r * 512);
+        const unsigned vw[4] = {vr.x, vr.y, vr.z, vr.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            unsigned short v0, v1;
+            halves(vw[e], v0, v1);
+            acc[2 * e] = fma_h(v0, w_hi, acc[2 * e]);
+            acc[2 * e + 1] = fma_h(v1, w_hi, acc[2 * e + 1]);
+            acc[2 * e] = fma_h(v0, w_lo, acc[2 * e]);
+            acc[2 * e + 1] = fma_h(v1, w_lo, acc[2 * e + 1]);
+        }
+    }
+}
+
 template <Rows kRows>
 __global__ void __launch_bounds__(kThreads, kCtasPerSm)
 decode_attn_split_kernel(const AttnParams p)
@@ -476,67 +548,8 @@ decode_attn_split_kernel(const AttnParams p)
             phase ^= 1u;
         }
 
-        // Logit: this lane's quarter of row `row`, four independent fp32 chains.
-        float part[4];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const uint4 kr = lds128(base + k_rd + k_piece[i]);
-            const unsigned kw[4] = {kr.x, kr.y, kr.z, kr.w};
-            const unsigned qw[4] = {qh[i].x, qh[i].y, qh[i].z, qh[i].w};
-            float dot = 0.f;
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                unsigned short k0, k1, q0, q1;
-                halves(kw[e], k0, k1);
-                halves(qw[e], q0, q1);
-                dot = fma_h(k0, q0, dot);
-                dot = fma_h(k1, q1, dot);
-            }
-            part[i] = dot;
-        }
-        float s = ((part[0] + part[1]) + (part[2] + part[3])) * p.scale_log2e;
-        s += __shfl_xor_sync(0xffffffffu, s, 8);
-        s += __shfl_xor_sync(0xffffffffu, s, 16);
         const int rows = j == my_tiles - 1 ? last_rows : kTileRows;
-        if (row >= rows) s = -INFINITY;
-
-        // Online softmax with a warp-uniform reference m that may lag the true maximum by up to
-        // kMaxLag (base-2 units): weights then reach at most 2^kMaxLag, which is harmless in
-        // fp32 and inside the range of the fp16 weight split.  The reference only moves (and
-        // the accumulators are only rescaled) when some logit exceeds it by more than that,
-        // so the common tile pays one vote instead of a shuffle reduction.
-        if (__any_sync(0xffffffffu, s > m + kMaxLag)) {
-            float tile_max = s;
-            tile_max = fmaxf(tile_max, __shfl_xor_sync(0xffffffffu, tile_max, 1));
-            tile_max = fmaxf(tile_max, __shfl_xor_sync(0xffffffffu, tile_max, 2));
-            tile_max = fmaxf(tile_max, __shfl_xor_sync(0xffffffffu, tile_max, 4));
-            const float alpha = fast_exp2(m - tile_max);
-            l *= alpha;
-#pragma unroll
-            for (int i = 0; i < 8; ++i) acc[i] *= alpha;
-            m = tile_max;
-        }
-        const float pw = fast_exp2(s - m);
-        l += pw;
-
-        // Attend: rows 2 r + half_warp, r < 4.
-        const unsigned packed = split_weight(pw);
-#pragma unroll
-        for (int r = 0; r < 4; ++r) {
-            unsigned short w_lo, w_hi;
-            halves(__shfl_sync(0xffffffffu, packed, 2 * r + half_warp), w_lo, w_hi);
-            const uint4 vr = lds128(base + v_rd + r * 512);
-            const unsigned vw[4] = {vr.x, vr.y, vr.z, vr.w};
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                unsigned short v0, v1;
-                halves(vw[e], v0, v1);
-                acc[2 * e] = fma_h(v0, w_hi, acc[2 * e]);
-                acc[2 * e + 1] = fma_h(v1, w_hi, acc[2 * e + 1]);
-                acc[2 * e] = fma_h(v0, w_lo, acc[2 * e]);
-                acc[2 * e + 1] = fma_h(v1, w_lo, acc[2 * e + 1]);
-            }
-        }
+        attend_tile(base + k_rd, k_piece, base + v_rd, qh, p.scale_log2e, rows, row, half_warp, m, l, acc);
     }
     if (kGathered) cp_async_wait<0>();
     if (kBulk && stalled) {
