@@ -127,13 +127,16 @@ __device__ __forceinline__ void bulk_copy(unsigned dst, const void *src, unsigne
     asm volatile("cp.async.bulk.shared::cta.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  :: "r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
+// One attempt: the thread may be parked by the hardware until the phase completes or a time
+// limit passes (the hint, in nanoseconds, asks for a long one, so that a warp that waits for
+// data sleeps instead of spinning through issue slots).
 __device__ __forceinline__ bool mbarrier_try_wait(unsigned bar, unsigned parity)
 {
     unsigned done;
     asm volatile("{\n\t.reg .pred p;\n\t"
-                 "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+                 "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
                  "selp.u32 %0, 1, 0, p;\n\t}"
-                 : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+                 : "=r"(done) : "r"(bar), "r"(parity), "r"(1000000u) : "memory");
     return done != 0;
 }
 // Waits for phase `parity` of the barrier, giving up after about kWaitCycles clock cycles (a
