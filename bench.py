@@ -37,6 +37,17 @@ DEFAULT_WORKLOAD = 4
 BAD_REASONS = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown")
 
 
+# Small long-context cases of the grouped-head entry point for profiling (about 1 GB of K and V each):
+# name: batch, context, block_tokens, kv_heads, q_heads, q_tokens, head_dim
+PROFILE_GROUPED = {
+    "mha": (4, 16384, 16, 32, 32, 1, 128),
+    "gqa8": (16, 16384, 16, 8, 64, 1, 128),
+    "gqa4_4new": (16, 16384, 16, 8, 32, 4, 128),
+    "d64": (8, 16384, 16, 32, 32, 1, 64),
+    "d256": (4, 16384, 16, 16, 16, 1, 256),
+}
+
+
 def parse_args(argv=None):
     ap = argparse.ArgumentParser(description=__doc__, formatter_class=argparse.RawDescriptionHelpFormatter)
     ap.add_argument("--gpus", type=int, default=1)
@@ -51,6 +62,11 @@ def parse_args(argv=None):
                     help="CPU budget of the oracle baseline (0 skips it)")
     ap.add_argument("--layers", type=int, default=0,
                     help="override the workload's layer count (profiling a small case)")
+    ap.add_argument("--case", default="",
+                    help="run one small profiling case instead of the benchmark and print its timing: "
+                         "sparse:<workload index>[:<batch>[:<kt block tokens>]] or grouped:<name> "
+                         "(names: " + ", ".join(n for n in PROFILE_GROUPED) + ")")
+    ap.add_argument("--launches", type=int, default=2, help="calls made by --case")
     return ap.parse_args(argv)
 
 
@@ -661,6 +677,61 @@ def measure_grouped(device, steps: int = 20) -> dict:
     return results
 
 
+def run_case(spec: str, launches: int, device) -> dict:
+    """One small case of the sparse or the grouped entry point, `launches` calls back to back
+    (what the ncu commands under profiles/ run)."""
+    from paper_2409_04992_b200 import binding
+    kind, _, rest = spec.partition(":")
+    flags = torch.zeros(1, dtype=torch.int32, device=device)
+    a, z = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    if kind == "sparse":
+        parts = rest.split(":")
+        w = wl.STANDARD[int(parts[0])].replace(layers=1)
+        if len(parts) > 1 and parts[1]:
+            w = w.replace(batch=int(parts[1]))
+        kt_tokens = int(parts[2]) if len(parts) > 2 else 256
+        case = wl.generate(w, device=str(device), poison=False)
+        state = wl.make_sparf_state(case, 0.125, kt_tokens)
+        B, H, D = case.q.shape
+        max_len, max_k = case.max_seq_len, max(state.k_tokens_host)
+        out = torch.empty((B, H, D), dtype=torch.float16, device=device)
+        ws = torch.empty(binding.sparf_workspace_bytes(B, H, D, max_len, max_k), dtype=torch.uint8, device=device)
+
+        def call():
+            binding.sparf_decode_attention(out, None, None, case.q, case.k_cache, case.v_cache, state.kt_pool,
+                                           state.v_sum, case.block_table, state.kt_block_table, case.seq_lens,
+                                           state.k_tokens, max_len, max_k, 16, 16, case.scale, ws, flags)
+        moved = case.kv_tokens * H * 16 * 2 + sum(state.k_tokens_host) * H * 2 * D * 2
+        name = f"sparse {w.name} batch {w.batch} kt block {kt_tokens}"
+    elif kind == "grouped":
+        batch, ctx, tokens, kv_heads, q_heads, q_tokens, dim = PROFILE_GROUPED[rest]
+        w = wl.Workload(rest, 7, batch=batch, len_lo=ctx, len_hi=ctx, layout="paged", block_tokens=tokens,
+                        heads=kv_heads, head_dim=dim)
+        g = wl.generate_grouped(w, q_tokens, q_heads, device=str(device))
+        c = g.base
+        out = torch.empty_like(g.q)
+        ws = torch.empty(binding.grouped_workspace_bytes(batch, q_tokens, q_heads, kv_heads, dim, ctx),
+                         dtype=torch.uint8, device=device)
+        binding.kv_append_bulk(c.k_cache, c.v_cache, g.k_new, g.v_new, c.seq_lens, g.new_lens, c.block_table, flags)
+
+        def call():
+            binding.decode_attention_grouped(out, None, g.q, c.k_cache, c.v_cache, c.block_table, c.seq_lens,
+                                             ctx, c.scale, ws, flags)
+        moved = batch * ctx * kv_heads * dim * 4
+        name = f"grouped {rest}"
+    else:
+        raise ValueError(f"unknown --case {spec!r}")
+    torch.cuda.synchronize()
+    a.record()
+    for _ in range(launches):
+        call()
+    z.record()
+    torch.cuda.synchronize()
+    ms = a.elapsed_time(z) / launches
+    return {"case": name, "launches": launches, "ms_per_call_first_calls_included": ms,
+            "algorithmic_bytes": moved, "algorithmic_gbs": moved / ms / 1e6, "status_flags": int(flags.item())}
+
+
 def main(argv=None) -> int:
     args = parse_args(argv)
     if args.impl == "reference":          # CPU only: no process group; ranks other than 0 do nothing
@@ -678,6 +749,10 @@ def main(argv=None) -> int:
             raise RuntimeError("bench.py needs a CUDA device: the path has no CPU fallback")
         device = torch.device("cuda", ranks.local_rank)
         torch.cuda.set_device(device)
+        if args.case:
+            if ranks.rank == 0:
+                print(json.dumps(run_case(args.case, args.launches, device)), flush=True)
+            return 0
         w = wl.by_name(args.workload)
         if args.layers > 0:
             w = w.replace(layers=args.layers)

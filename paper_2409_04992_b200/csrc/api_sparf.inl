@@ -2,16 +2,17 @@
 // running V sum, workspace layout, and the launch chain of the attention call.
 // Included by instinfer_api.cu (one translation unit: the kernels' headers define
 // non-template kernels, which must not be compiled twice).
-#include "sparf_kernels.cuh"
+#include "sparf_staged_select.cuh"
 
 namespace {
 
 int g_sparse_path = 0;      // 0 automatic, 1 chunk-parallel, 2 one block per row (see instinfer_set_sparse_path)
 
 struct SparfLayout {
-    size_t scores, row_ids, stats, rows_state, row_hist, row_cand, chunk_count, chunk_sums, partials, total;
-    size_t zeroed_bytes;      // rows_state and row_hist are adjacent and cleared before each call
-    int32_t score_stride;
+    size_t scores, stage_pos, row_ids, stats, rows_state, row_cand, seg_count, seg_final, blk_z, seg_mass,
+        partials, total;
+    size_t zeroed_bytes;      // rows_state is cleared before each call of the staged chain
+    int32_t score_stride, segments, score_blocks, cand_capacity;
     SplitPlan plan;
 };
 
@@ -21,18 +22,24 @@ SparfLayout sparf_layout(int64_t pairs, int32_t max_seq_len, int32_t max_k)
 {
     SparfLayout w;
     w.score_stride = (max_seq_len + 7) / 8 * 8;      // whole 8-token groups, 32-byte aligned rows
+    w.segments = (int32_t)ceil_div(max_seq_len, kSegmentTokens);
+    w.score_blocks = (int32_t)ceil_div(max_seq_len, kScoreBlockTokens);
+    // candidates per row: the bracket of the sampled pre-pass holds a few per cent of the row
+    int64_t cand = max_seq_len / 4;
+    w.cand_capacity = (int32_t)(cand < 1024 ? 1024 : cand > kCandidates ? kCandidates : cand);
     w.plan = make_plan(pairs, max_k);
     w.scores = 0;
-    w.row_ids = w.scores + round256((size_t)pairs * w.score_stride * sizeof(float));
+    w.stage_pos = w.scores + round256((size_t)pairs * w.score_stride * sizeof(float));
+    w.row_ids = w.stage_pos + round256((size_t)pairs * w.score_stride * sizeof(int32_t));
     w.stats = w.row_ids + round256((size_t)pairs * max_k * sizeof(int32_t));
-    const size_t chunks = (size_t)ceil_div(max_seq_len, kScoreChunk);
     w.rows_state = w.stats + round256((size_t)pairs * sizeof(float2));
-    w.row_hist = w.rows_state + round256((size_t)pairs * sizeof(SelectRow));
-    w.row_cand = w.row_hist + round256((size_t)pairs * (kLinearBins + 1) * sizeof(unsigned));
+    w.row_cand = w.rows_state + round256((size_t)pairs * sizeof(SelectRow));
     w.zeroed_bytes = w.row_cand - w.rows_state;
-    w.chunk_count = w.row_cand + round256((size_t)pairs * kRowCandidates * sizeof(uint2));
-    w.chunk_sums = w.chunk_count + round256((size_t)pairs * chunks * sizeof(int32_t));
-    w.partials = w.chunk_sums + round256((size_t)pairs * chunks * sizeof(float2));
+    w.seg_count = w.row_cand + round256((size_t)pairs * w.cand_capacity * sizeof(uint2));
+    w.seg_final = w.seg_count + round256((size_t)pairs * w.segments * sizeof(int32_t));
+    w.blk_z = w.seg_final + round256((size_t)pairs * w.segments * sizeof(int32_t));
+    w.seg_mass = w.blk_z + round256((size_t)pairs * w.score_blocks * sizeof(float));
+    w.partials = w.seg_mass + round256((size_t)pairs * w.segments * sizeof(float));
     w.total = w.partials + workspace_for(pairs, w.plan);
     return w;
 }
@@ -183,8 +190,7 @@ int instinfer_sparf_decode_attention(void *out, float *alpha, int32_t *selected,
     const SparfLayout w = sparf_layout(pairs, max_seq_len, max_k);
     if (workspace == nullptr || !aligned16(workspace) || workspace_bytes < w.total)
         return INSTINFER_ERR_WORKSPACE;
-    const int64_t score_chunks = ceil_div(max_seq_len, kScoreChunk);
-    if (pairs * score_chunks >= (int64_t)1 << 31 || pairs * w.plan.n_splits >= (int64_t)1 << 31)
+    if (pairs * w.score_blocks >= (int64_t)1 << 31 || pairs * w.plan.n_splits >= (int64_t)1 << 31)
         return INSTINFER_ERR_INVALID_ARG;
     unsigned char *ws = static_cast<unsigned char *>(workspace);
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
@@ -200,6 +206,7 @@ int instinfer_sparf_decode_attention(void *out, float *alpha, int32_t *selected,
     sp.block_table = block_table;
     sp.status = status_flags;
     sp.scores = reinterpret_cast<float *>(ws + w.scores);
+    sp.stage_pos = reinterpret_cast<int32_t *>(ws + w.stage_pos);
     sp.row_ids = reinterpret_cast<int32_t *>(ws + w.row_ids);
     sp.stats = reinterpret_cast<float2 *>(ws + w.stats);
     sp.alpha_out = alpha;
@@ -216,29 +223,27 @@ int instinfer_sparf_decode_attention(void *out, float *alpha, int32_t *selected,
     sp.max_seq_len = max_seq_len;
     sp.max_k = max_k;
     sp.score_stride = w.score_stride;
-    sp.score_chunks = (int32_t)score_chunks;
-    sp.score_blocks = (int32_t)ceil_div(max_seq_len, kScoreBlockTokens);
+    sp.segments = w.segments;
+    sp.score_blocks = w.score_blocks;
+    sp.cand_capacity = w.cand_capacity;
     sp.r = r;
     sp.window = local_window;
     sp.scale_log2e = scale * 1.44269504088896340736f;
 
     sp.rows_state = reinterpret_cast<SelectRow *>(ws + w.rows_state);
-    sp.row_hist = reinterpret_cast<unsigned *>(ws + w.row_hist);
     sp.row_cand = reinterpret_cast<uint2 *>(ws + w.row_cand);
-    sp.chunk_count = reinterpret_cast<int32_t *>(ws + w.chunk_count);
-    sp.chunk_sums = reinterpret_cast<float2 *>(ws + w.chunk_sums);
+    sp.seg_count = reinterpret_cast<int32_t *>(ws + w.seg_count);
+    sp.seg_final = reinterpret_cast<int32_t *>(ws + w.seg_final);
+    sp.blk_z = reinterpret_cast<float *>(ws + w.blk_z);
+    sp.seg_mass = reinterpret_cast<float *>(ws + w.seg_mass);
 
-    const unsigned chunk_grid = (unsigned)(pairs * ceil_div(score_chunks, kSubChunks)), row_grid = (unsigned)pairs;
+    const unsigned block_grid = (unsigned)(pairs * w.score_blocks), row_grid = (unsigned)pairs;
     // Two ways through steps 1-7.  For rows that fit in shared memory one block per row computes
-    // the logits there and selects from there (nothing goes through HBM); otherwise the logits
-    // go to the workspace and the selection runs chunk-parallel.
-    // Measured: the one-block-per-row form wins wherever the rows fit (by 4-45 %, most at
-    // small batches, where the chunk-parallel chain is all launch latency), except for very
-    // many rows of the largest size (2560 rows of 16384 tokens: 3-7 % slower).
+    // the logits there and selects from there; otherwise (and for very many rows of the largest
+    // size that fits) the staged chain: a sampled pre-pass brackets the threshold and the score
+    // pass keeps only the tokens that can still be selected.  Neither writes the logits to HBM.
     const bool fits = max_seq_len <= kFusedMaxTokens;
-    const bool fused = g_sparse_path == 2 ? fits
-                     : g_sparse_path == 1 ? false
-                     : fits && (max_seq_len <= 12288 || pairs < 8 * (int64_t)sm_count());
+    const bool fused = g_sparse_path == 1 ? false : fits;
     if (fused) {
         static bool fused_smem_set[kMaxDevices] = {};
         int device = 0;
@@ -255,18 +260,30 @@ int instinfer_sparf_decode_attention(void *out, float *alpha, int32_t *selected,
                               (size_t)w.score_stride * sizeof(float), stream, sp) != cudaSuccess)
             return INSTINFER_ERR_CUDA;
     } else {
+        static bool staged_smem_set[kMaxDevices] = {};
+        int device = 0;
+        if (cudaGetDevice(&device) != cudaSuccess || device < 0 || device >= kMaxDevices) return INSTINFER_ERR_CUDA;
+        if (!staged_smem_set[device]) {
+            if (cudaFuncSetAttribute(sparf_sample_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     kMaxSamples * (int)sizeof(float)) != cudaSuccess ||
+                cudaFuncSetAttribute(sparf_resolve_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     kCandidates * (int)sizeof(int)) != cudaSuccess) {
+                (void)cudaGetLastError();
+                return INSTINFER_ERR_CUDA;
+            }
+            staged_smem_set[device] = true;
+        }
         if (cudaMemsetAsync(ws + w.rows_state, 0, w.zeroed_bytes, stream) != cudaSuccess) {
             (void)cudaGetLastError();
             return INSTINFER_ERR_CUDA;
         }
-        // Steps 5-7, chunk-parallel; rows it cannot settle are redone by the single-block kernel.
-        bool ok = launch_overlapped(sparf_scores_kernel, (unsigned)(pairs * sp.score_blocks), kSparfThreads, 0, stream, sp) == cudaSuccess;
-        ok = ok && launch_overlapped(sparf_hist_kernel, chunk_grid, kChunkThreads, 0, stream, sp) == cudaSuccess;
-        ok = ok && launch_overlapped(sparf_locate_kernel, row_grid, 32, 0, stream, sp) == cudaSuccess;
-        ok = ok && launch_overlapped(sparf_collect_kernel, chunk_grid, kChunkThreads, 0, stream, sp) == cudaSuccess;
-        ok = ok && launch_overlapped(sparf_threshold_kernel, row_grid, kThresholdThreads, 0, stream, sp) == cudaSuccess;
-        ok = ok && launch_overlapped(sparf_compact_kernel, chunk_grid, kChunkThreads, 0, stream, sp) == cudaSuccess;
+        bool ok = launch_overlapped(sparf_sample_kernel, row_grid, kSampleThreads, kMaxSamples * sizeof(float), stream, sp) == cudaSuccess;
+        ok = ok && launch_overlapped(sparf_stage_kernel, block_grid, kSparfThreads, 0, stream, sp) == cudaSuccess;
+        ok = ok && launch_overlapped(sparf_resolve_kernel, row_grid, kResolveThreads, (size_t)w.cand_capacity * sizeof(int), stream, sp) == cudaSuccess;
+        ok = ok && launch_overlapped(sparf_emit_kernel, block_grid, kEmitThreads, 0, stream, sp) == cudaSuccess;
         ok = ok && launch_overlapped(sparf_finish_kernel, row_grid, 64, 0, stream, sp) == cudaSuccess;
+        // rows the chain could not settle: all their logits to the workspace, one block per row selects
+        ok = ok && launch_overlapped(sparf_scores_kernel, block_grid, kSparfThreads, 0, stream, sp) == cudaSuccess;
         ok = ok && launch_overlapped(sparf_select_kernel, row_grid, kSelectThreads, 0, stream, sp) == cudaSuccess;
         if (!ok) {
             (void)cudaGetLastError();
@@ -296,6 +313,7 @@ int instinfer_sparf_decode_attention(void *out, float *alpha, int32_t *selected,
     ap.row_ids = sp.row_ids;
     ap.k_tokens = k_tokens;
     ap.row_stride = max_k;
+    ap.row_limit = (int32_t)(num_phys_blocks * heads * block_tokens);      // below 2^31, checked above
     mp.stats = sp.stats;
     mp.v_sum = v_sum;
 

@@ -81,6 +81,7 @@ struct AttnParams {
     const int32_t *row_ids;    // [pairs, row_stride] physical row index (phys * H + h) * T + slot
     const int32_t *k_tokens;   // [batch] rows to attend per sequence (clipped to its length)
     int32_t row_stride;
+    int32_t row_limit;         // number of rows in the pools: a listed id outside [0, row_limit) reads as zeros
 };
 
 // Where a (sequence, head)'s rows come from.
@@ -462,7 +463,7 @@ decode_attn_split_kernel(const AttnParams p)
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
                     const int rid = __shfl_sync(0xffffffffu, rows_now, (issue_j & 3) * 8 + 2 * i + half_warp);
-                    const bool valid = 2 * i + half_warp < rows;
+                    const bool valid = 2 * i + half_warp < rows && (unsigned)rid < (unsigned)p.row_limit;
                     const int64_t src = valid ? (int64_t)rid * kRowBytes : 0;
                     cp_async_16(dst + k_dst + i * 2 * kRowBytes, k_col + src, valid ? 16 : 0);
                     cp_async_16(dst + v_dst + i * 512, v_col + src, valid ? 16 : 0);

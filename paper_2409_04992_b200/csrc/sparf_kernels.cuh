@@ -7,13 +7,15 @@
 //   sparf_scores_kernel   step 1 (the r largest |q_d|) and steps 2-4 without the softmax
 //                         normalisation: approximate logits from the embedding-major copy.
 //   steps 5-7             softmax statistics of the approximate logits, the k largest scores
-//                         with the last l tokens forced in (a monotone linear histogram finds
-//                         the threshold bin, its members are resolved exactly; ties to the
-//                         lower position), alpha, and the ascending list of selected rows as
-//                         physical row ids.  Run chunk-parallel by sparf_hist /
-//                         locate / collect / threshold / compact / finish kernels; rows with
-//                         too many nearly equal scores fall back to sparf_select_kernel,
-//                         which does the same steps with one block per row.
+//                         with the last l tokens forced in (ties to the lower position), alpha,
+//                         and the ascending list of selected rows as physical row ids.  Two
+//                         forms: one block per row with the row's logits in shared memory
+//                         (sparf_fused_select_kernel), and for long rows a chain that never
+//                         writes the logits out (sparf_staged_select.cuh: a sampled pre-pass
+//                         brackets the threshold, the score kernel stages only the tokens that
+//                         can still be selected, the rest is resolved on those).  Rows the
+//                         chain cannot settle fall back to sparf_scores_kernel +
+//                         sparf_select_kernel, the same steps with one block per row.
 //   (steps 8-10 run in decode_attn_split_kernel<Rows::kGathered>)
 //   sparf_merge_kernel    log-sum-exp merge of the chunk partials and step 11:
 //                         out = alpha * attended + (1 - alpha) * v_sum / S.
@@ -27,20 +29,16 @@
 
 namespace instinfer {
 
-constexpr int kRowCandidates = 1024;     // chunk-parallel select: keys of the threshold bin kept per row
-
-// Per (sequence, head) state of the chunk-parallel selection.  Zero-initialised per call.
+// Per (sequence, head) state of the staged selection.  Zero-initialised per call.
 struct SelectRow {
-    unsigned max_key;          // ordered key of the largest logit
-    unsigned neg_min_key;      // ~ordered key of the smallest logit (so both are atomicMax)
-    int bin;                   // linear bin holding the k-th largest
-    int above;                 // members of the bins above it
-    int n_cand;                // candidates collected from that bin
+    float lo;                  // tokens whose logit is below this cannot be selected
+    float hi;                  // tokens whose logit is above this are surely selected (never -0)
+    float ref;                 // reference of the softmax sums (the largest sampled logit)
+    int n_cand;                // candidates (lo <= logit <= hi, outside the window) collected so far
+    int overflow;              // a logit far above ref was seen: the sums are not trustworthy
     unsigned tau;              // exact ordered key of the k-th largest
     int idx_cut;               // among keys equal to tau, positions <= idx_cut are taken
-    int solved;                // 0: the single-block kernel must redo this row
-    float z;                   // softmax denominator of the approximate logits
-    float top, low, bin_scale; // range of the linear bins
+    int solved;                // 0: the single-block kernels must redo this row
 };
 
 struct SparfParams {
@@ -58,15 +56,17 @@ struct SparfParams {
     const int32_t *kt_block_table;   // [batch, kt_max_blocks_per_seq]
     int32_t *status;
     // scratch
-    float *scores;             // [pairs, score_stride] approximate logits, base-2 domain
+    float *scores;             // [pairs, score_stride]: logits of the staged tokens (staged chain), or
+                               // all approximate logits of a row (fallback); base-2 domain
+    int32_t *stage_pos;        // [pairs, score_stride]: positions of the staged tokens, per segment
     int32_t *row_ids;          // [pairs, max_k]
     float2 *stats;             // [pairs] (alpha, number of selected rows)
-    // chunk-parallel selection (see SelectRow): all zeroed before each call
-    struct SelectRow *rows_state;   // [pairs]
-    unsigned *row_hist;        // [pairs, kLinearBins + 1]
-    uint2 *row_cand;           // [pairs, kRowCandidates] (ordered key, token index)
-    int32_t *chunk_count;      // [pairs, score_chunks] selected tokens per score chunk
-    float2 *chunk_sums;        // [pairs, score_chunks] (softmax denominator part, selected mass part)
+    struct SelectRow *rows_state;   // [pairs], zeroed before each call
+    uint2 *row_cand;           // [pairs, cand_capacity] (ordered key, token index)
+    int32_t *seg_count;        // [pairs, segments] staged tokens per segment
+    int32_t *seg_final;        // [pairs, segments] selected tokens per segment
+    float *blk_z;              // [pairs, score_blocks] softmax denominator parts
+    float *seg_mass;           // [pairs, segments] selected mass parts
     // outputs
     float *alpha_out;          // nullable [pairs]
     int32_t *selected;         // nullable [pairs, max_k] logical token index, ascending, -1 padded
@@ -74,13 +74,13 @@ struct SparfParams {
     int64_t num_kt_blocks;
     int32_t batch, heads, block_tokens, max_blocks_per_seq;
     int32_t kt_block_tokens, kt_max_blocks_per_seq;
-    int32_t max_seq_len, max_k, score_stride, score_chunks, score_blocks, r, window;
+    int32_t max_seq_len, max_k, score_stride, segments, score_blocks, cand_capacity, r, window;
     float scale_log2e;
 };
 
 constexpr int kSparfThreads = 128;       // append and scores: one thread per head dim
-constexpr int kScoreChunk = 2048;        // tokens per block of the selection kernels
-constexpr int kScoreBlockTokens = 8192;  // tokens per block of the score kernel (amortises its prologue)
+constexpr int kSegmentTokens = 256;      // staged chain: tokens per staging segment (one pass of one warp)
+constexpr int kScoreBlockTokens = 8192;  // tokens per block of the score kernels (amortises their prologue)
 constexpr int kSelectThreads = 1024;
 
 __device__ __forceinline__ int sparf_seq_len(const SparfParams &p, int b, bool report)
@@ -206,7 +206,7 @@ __device__ __forceinline__ unsigned ordered_key(float x)
 // logits.  Threads d < 128 each own one head dim; every thread of the block must call it.
 struct ScoreShared {
     float abs_q[kHeadDim];
-    float q[kHeadDim];          // q of the selected dims, in rank order
+    unsigned short q_bits[kHeadDim];   // q of the selected dims as fp16 bit patterns, in rank order
     int dim[kHeadDim];          // the selected dims, in rank order
     bool kept[kHeadDim];
     float approx_scale;
@@ -231,7 +231,7 @@ __device__ __forceinline__ void score_setup(const SparfParams &p, int pair, Scor
         const bool kept = rank < p.r;
         if (kept) {
             ss.dim[rank] = d;
-            ss.q[rank] = qd;
+            ss.q_bits[rank] = __half_as_ushort(p.q[(int64_t)pair * kHeadDim + d]);
         }
         ss.kept[d] = kept;
     }
@@ -274,11 +274,17 @@ __device__ __forceinline__ void score_group(const SparfParams &p, const ScoreSha
 #pragma unroll
             for (int u = 0; u < 8; ++u) {
                 if (t0 + u < p.r) {                            // uniform; extra loads are ignored
-                    const float qv = ss.q[t0 + u];
-                    float kf[8];
-                    unpack8(raw[u], kf);
+                    // fp16 x fp16 products are exact in fp32: one rounding per addition, the
+                    // same values as converting first, without the conversions
+                    const unsigned short qv = ss.q_bits[t0 + u];
+                    const unsigned kw[4] = {raw[u].x, raw[u].y, raw[u].z, raw[u].w};
 #pragma unroll
-                    for (int e = 0; e < 8; ++e) dot[e] = fmaf(qv, kf[e], dot[e]);
+                    for (int e = 0; e < 4; ++e) {
+                        unsigned short k0, k1;
+                        halves(kw[e], k0, k1);
+                        dot[2 * e] = fma_h(k0, qv, dot[2 * e]);
+                        dot[2 * e + 1] = fma_h(k1, qv, dot[2 * e + 1]);
+                    }
                 }
             }
         }
@@ -292,16 +298,18 @@ __device__ __forceinline__ void score_group(const SparfParams &p, const ScoreSha
 // Every kernel of the attention call below starts with the programmatic-dependent-launch pair
 // (let the next kernel's blocks become resident, then wait for all earlier kernels), before
 // any return, so that the chain of short launches overlaps its launch latencies.
-// grid pairs * score_blocks: approximate logits of kScoreBlockTokens tokens of one (sequence, head).
+// grid pairs * score_blocks: all approximate logits of kScoreBlockTokens tokens of one
+// (sequence, head), written to the workspace.  Only for the rows the staged chain left
+// unsolved (its blocks leave at once on the others).
 __global__ void __launch_bounds__(kSparfThreads)
 sparf_scores_kernel(const SparfParams p)
 {
     allow_next_kernel();
     wait_for_previous_kernels();
     __shared__ ScoreShared ss;
-    __shared__ float sm_red[2][kSparfThreads / 32];
     const int pair = blockIdx.x / p.score_blocks, d = threadIdx.x;
     const int b = pair / p.heads, h = pair - b * p.heads;
+    if (p.rows_state[pair].solved) return;
     const int len = sparf_seq_len(p, b, false);
     const int begin = (blockIdx.x - pair * p.score_blocks) * kScoreBlockTokens;
     if (begin >= len) return;
@@ -310,45 +318,14 @@ sparf_scores_kernel(const SparfParams p)
 
     const int32_t *table_row = p.kt_block_table + (int64_t)b * p.kt_max_blocks_per_seq;
     float *dst = p.scores + (int64_t)pair * p.score_stride;
-    float top = kMinusHuge, low = -kMinusHuge;          // range of this thread's logits
     for (int i = begin + d * 8; i < end; i += kSparfThreads * 8) {
         float dot[8];
         score_group(p, ss, table_row, h, i, dot);
         // score_stride is a multiple of 8 and rows start 32-byte aligned; entries past `end`
         // inside the last group are scratch nobody reads.
         float4 *out4 = reinterpret_cast<float4 *>(dst + i);
-        if (i + 8 <= end) {
-            top = fmaxf(top, fmaxf(fmaxf(fmaxf(dot[0], dot[1]), fmaxf(dot[2], dot[3])),
-                                   fmaxf(fmaxf(dot[4], dot[5]), fmaxf(dot[6], dot[7]))));
-            low = fminf(low, fminf(fminf(fminf(dot[0], dot[1]), fminf(dot[2], dot[3])),
-                                   fminf(fminf(dot[4], dot[5]), fminf(dot[6], dot[7]))));
-        } else {
-            for (int e = 0; i + e < end; ++e) {
-                top = fmaxf(top, dot[e]);
-                low = fminf(low, dot[e]);
-            }
-        }
         out4[0] = make_float4(dot[0], dot[1], dot[2], dot[3]);
         out4[1] = make_float4(dot[4], dot[5], dot[6], dot[7]);
-    }
-    // Range of the row's logits (what the linear bins of the selection span): two atomics per block.
-#pragma unroll
-    for (int off = 16; off >= 1; off >>= 1) {
-        top = fmaxf(top, __shfl_xor_sync(0xffffffffu, top, off));
-        low = fminf(low, __shfl_xor_sync(0xffffffffu, low, off));
-    }
-    if ((d & 31) == 0) {
-        sm_red[0][d >> 5] = top;
-        sm_red[1][d >> 5] = low;
-    }
-    __syncthreads();
-    if (d == 0) {
-        for (int w = 1; w < kSparfThreads / 32; ++w) {
-            top = fmaxf(top, sm_red[0][w]);
-            low = fminf(low, sm_red[1][w]);
-        }
-        atomicMax(&p.rows_state[pair].max_key, ordered_key(top));
-        atomicMax(&p.rows_state[pair].neg_min_key, ~ordered_key(low));
     }
 }
 
@@ -722,7 +699,7 @@ sparf_select_kernel(const SparfParams p)
     __shared__ SelectShared sh;
     const int pair = blockIdx.x;
     const int b = pair / p.heads, h = pair - b * p.heads;
-    if (p.rows_state && p.rows_state[pair].solved) return;      // done by the chunk-parallel kernels
+    if (p.rows_state && p.rows_state[pair].solved) return;      // done by the staged chain
     const int S = sparf_seq_len(p, b, threadIdx.x == 0 && h == 0);
     const int k = min(S, min(max(p.k_tokens[b], 0), p.max_k));
     select_row<kSelectThreads>(p, sh, p.scores + (int64_t)pair * p.score_stride, pair, b, h, S, k, min(p.window, k));
@@ -761,415 +738,6 @@ sparf_fused_select_kernel(const SparfParams p)
         __syncthreads();
     }
     select_row<kFusedThreads>(p, sh, row_scores, pair, b, h, S, k, min(p.window, k));
-}
-
-// ---------------------------------------------------------------------------------------
-// Chunk-parallel selection.  The same steps as sparf_select_kernel, but every pass over the
-// scores runs as one block per (row, group of four 2048-token chunks), so that long rows use
-// the whole GPU:
-//   (the per-row min / max of the logits comes from the score kernel: two atomicMax per block)
-//   hist    -> per-row histogram over the monotone linear bins, softmax denominator parts
-//   locate  -> the bin holding the k-th largest (one warp per row)
-//   collect -> per chunk, how many tokens lie in higher bins (surely selected), and the
-//              (key, position) of the tokens inside the threshold bin
-//   thresh  -> exact threshold among those candidates, ties cut by position
-//   compact -> ordered compaction per chunk behind the prefix of the chunk counts
-//   finish  -> alpha, padding of the optional `selected` output
-// A row whose threshold bin holds more than kRowCandidates keys (many nearly equal scores)
-// is left unsolved and redone by sparf_select_kernel, which skips the solved rows.
-// One warp: among the linear bins (lane L owns bins [64 L, 64 L + 64)), the bin in which the
-// count from the top, started at `from_top`, reaches `target`; also the count above that bin.
-__device__ __forceinline__ void locate_linear_bin(const unsigned *hist, int from_top, int target, int *bin_out, int *above_out)
-{
-    const int lane = threadIdx.x & 31;
-    int mine = 0;
-    for (int j = 0; j < 64; ++j) mine += (int)hist[64 * lane + ((j + lane) & 63)];
-    int above = from_top;
-    for (int src = 31; src >= 0; --src) {
-        const int seg = __shfl_sync(0xffffffffu, mine, src);
-        if (src > lane) above += seg;
-    }
-    if (above < target && target <= above + mine) {
-        int bin = 64 * lane + 63;
-        for (; bin > 64 * lane; --bin) {
-            const int c = (int)hist[bin];
-            if (above + c >= target) break;
-            above += c;
-        }
-        *bin_out = bin;
-        *above_out = above;
-    }
-}
-
-constexpr int kChunkThreads = 256;       // 8 consecutive tokens per thread = one score chunk
-static_assert(kChunkThreads * 8 == kScoreChunk, "one thread block covers one score chunk");
-
-__device__ __forceinline__ float float_of_key(unsigned key)
-{
-    return __uint_as_float((key & 0x80000000u) ? (key & 0x7fffffffu) : ~key);
-}
-
-constexpr int kSubChunks = 4;             // score chunks handled by one block of the chunk kernels
-
-struct ChunkView {
-    int pair, chunk0, n_sub, b, h, S, k, window;   // chunks chunk0 .. chunk0 + n_sub - 1 of the row
-    float x[kSubChunks][8];                        // this thread's 8 logits of each chunk
-    __device__ __forceinline__ int first_token(int sub) const
-    {
-        return (chunk0 + sub) * kScoreChunk + (int)threadIdx.x * 8;
-    }
-};
-
-// Common prologue of the chunk kernels: indices, lengths and this thread's logits.  A block
-// takes kSubChunks consecutive chunks of one row and issues all their loads together, so the
-// latency of one global round trip is paid once per 8192 tokens instead of once per 2048.
-__device__ __forceinline__ bool load_chunk(const SparfParams &p, ChunkView &c)
-{
-    const int groups = (p.score_chunks + kSubChunks - 1) / kSubChunks;
-    c.pair = blockIdx.x / groups;
-    c.chunk0 = (blockIdx.x - c.pair * groups) * kSubChunks;
-    c.b = c.pair / p.heads;
-    c.h = c.pair - c.b * p.heads;
-    c.S = sparf_seq_len(p, c.b, false);
-    c.k = min(c.S, min(max(p.k_tokens[c.b], 0), p.max_k));
-    c.window = min(p.window, c.k);
-    if (c.chunk0 * kScoreChunk >= c.S) return false;
-    c.n_sub = min(kSubChunks, (c.S - c.chunk0 * kScoreChunk + kScoreChunk - 1) / kScoreChunk);
-    const float *row_scores = p.scores + (int64_t)c.pair * p.score_stride;
-#pragma unroll
-    for (int sub = 0; sub < kSubChunks; ++sub) {
-#pragma unroll
-        for (int e = 0; e < 8; ++e) c.x[sub][e] = 0.f;
-        const int i0 = c.first_token(sub);
-        if (i0 < c.S) {                            // rows are padded to whole groups of 8
-            const float4 *src = reinterpret_cast<const float4 *>(row_scores + i0);
-            const float4 a = src[0], b = src[1];
-            c.x[sub][0] = a.x; c.x[sub][1] = a.y; c.x[sub][2] = a.z; c.x[sub][3] = a.w;
-            c.x[sub][4] = b.x; c.x[sub][5] = b.y; c.x[sub][6] = b.z; c.x[sub][7] = b.w;
-        }
-    }
-    return true;
-}
-
-__device__ __forceinline__ int linear_bin(const SelectRow &row, int S, int window, int i, float x)
-{
-    return i >= S - window ? kLinearBins : min(kLinearBins - 1, (int)((x - row.low) * row.bin_scale));
-}
-
-__global__ void __launch_bounds__(kChunkThreads)
-sparf_hist_kernel(const SparfParams p)
-{
-    allow_next_kernel();
-    wait_for_previous_kernels();
-    __shared__ unsigned hist[kLinearBins + 1];
-    __shared__ float red[32];
-    ChunkView c;
-    if (!load_chunk(p, c)) return;
-    SelectRow row;
-    row.top = float_of_key(p.rows_state[c.pair].max_key);
-    row.low = float_of_key(~p.rows_state[c.pair].neg_min_key);
-    row.bin_scale = row.top > row.low ? (float)(kLinearBins - 1) / (row.top - row.low) : 0.f;
-    for (int t = threadIdx.x; t <= kLinearBins; t += kChunkThreads) hist[t] = 0u;
-    __syncthreads();
-    float z[kSubChunks];
-#pragma unroll
-    for (int sub = 0; sub < kSubChunks; ++sub) {
-        z[sub] = 0.f;
-        const int i0 = c.first_token(sub);
-#pragma unroll
-        for (int e = 0; e < 8; ++e) {
-            const int i = i0 + e;
-            if (i < c.S) {
-                z[sub] += fast_exp2(c.x[sub][e] - row.top);
-                atomicAdd(&hist[linear_bin(row, c.S, c.window, i, c.x[sub][e])], 1u);
-            }
-        }
-    }
-#pragma unroll
-    for (int sub = 0; sub < kSubChunks; ++sub) z[sub] = block_sum(z[sub], red);   // barriers publish the histogram
-    unsigned *global_hist = p.row_hist + (int64_t)c.pair * (kLinearBins + 1);
-    for (int t = threadIdx.x; t <= kLinearBins; t += kChunkThreads)
-        if (hist[t]) atomicAdd(&global_hist[t], hist[t]);
-    if ((int)threadIdx.x < c.n_sub) {
-        float mine = z[0];
-#pragma unroll
-        for (int sub = 1; sub < kSubChunks; ++sub) if ((int)threadIdx.x == sub) mine = z[sub];
-        p.chunk_sums[(int64_t)c.pair * p.score_chunks + c.chunk0 + threadIdx.x].x = mine;
-    }
-}
-
-// One warp per row.
-__global__ void __launch_bounds__(32)
-sparf_locate_kernel(const SparfParams p)
-{
-    allow_next_kernel();
-    wait_for_previous_kernels();
-    const int pair = blockIdx.x, lane = threadIdx.x;
-    const int b = pair / p.heads, h = pair - b * p.heads;
-    const int S = sparf_seq_len(p, b, lane == 0 && h == 0);
-    const int k = min(S, min(max(p.k_tokens[b], 0), p.max_k));
-    SelectRow *row = p.rows_state + pair;
-    if (k == 0) {                                // nothing is selected: no bin is "above" this one
-        if (lane == 0) {
-            row->bin = kLinearBins + 1;
-            row->solved = 1;
-        }
-        return;
-    }
-    const unsigned *hist = p.row_hist + (int64_t)pair * (kLinearBins + 1);
-    const int in_window = (int)hist[kLinearBins];
-    __shared__ int bin, above;
-    if (in_window >= k) {                        // the local window alone fills k
-        if (lane == 0) {
-            bin = kLinearBins;
-            above = 0;
-        }
-    } else {
-        locate_linear_bin(hist, in_window, k, &bin, &above);
-    }
-    __syncwarp();
-    if (lane == 0) {
-        const float top = float_of_key(row->max_key), low = float_of_key(~row->neg_min_key);
-        float z = 0.f;
-        const int chunks = (S + kScoreChunk - 1) / kScoreChunk;
-        for (int c = 0; c < chunks; ++c) z += p.chunk_sums[(int64_t)pair * p.score_chunks + c].x;   // fixed order
-        row->top = top;
-        row->low = low;
-        row->bin_scale = top > low ? (float)(kLinearBins - 1) / (top - low) : 0.f;
-        row->z = z;
-        row->bin = bin;
-        row->above = above;
-        if (bin == kLinearBins) {
-            row->tau = 0xffffffffu;
-            row->idx_cut = -1;                 // nothing outside the window is taken
-            row->solved = 1;
-        }
-    }
-}
-
-__global__ void __launch_bounds__(kChunkThreads)
-sparf_collect_kernel(const SparfParams p)
-{
-    allow_next_kernel();
-    wait_for_previous_kernels();
-    __shared__ int red[32];
-    ChunkView c;
-    if (!load_chunk(p, c)) return;
-    SelectRow *state = p.rows_state + c.pair;
-    const SelectRow row = *state;
-    int sure[kSubChunks];
-#pragma unroll
-    for (int sub = 0; sub < kSubChunks; ++sub) {
-        sure[sub] = 0;
-        if (row.bin > kLinearBins) continue;
-        const int i0 = c.first_token(sub);
-#pragma unroll
-        for (int e = 0; e < 8; ++e) {
-            const int i = i0 + e;
-            if (i < c.S) {
-                const int bin = linear_bin(row, c.S, c.window, i, c.x[sub][e]);
-                if (bin > row.bin || (bin == kLinearBins && row.bin == kLinearBins)) {
-                    ++sure[sub];
-                } else if (bin == row.bin) {
-                    const int at = atomicAdd(&state->n_cand, 1);
-                    if (at < kRowCandidates)
-                        p.row_cand[(int64_t)c.pair * kRowCandidates + at] = make_uint2(ordered_key(c.x[sub][e]), (unsigned)i);
-                }
-            }
-        }
-    }
-#pragma unroll
-    for (int sub = 0; sub < kSubChunks; ++sub) sure[sub] = block_sum(sure[sub], red);
-    if ((int)threadIdx.x < c.n_sub) {
-        int mine = sure[0];
-#pragma unroll
-        for (int sub = 1; sub < kSubChunks; ++sub) if ((int)threadIdx.x == sub) mine = sure[sub];
-        p.chunk_count[(int64_t)c.pair * p.score_chunks + c.chunk0 + threadIdx.x] = mine;
-    }
-}
-
-// One block per row: exact threshold among the collected candidates.
-constexpr int kThresholdThreads = 256;    // more threads per row did not help: a row's O(n^2) ranking
-                                          // saturates its SM either way, and many-row launches lost occupancy
-
-__global__ void __launch_bounds__(kThresholdThreads)
-sparf_threshold_kernel(const SparfParams p)
-{
-    allow_next_kernel();
-    wait_for_previous_kernels();
-    __shared__ unsigned keys[kRowCandidates];
-    __shared__ int where[kRowCandidates];
-    __shared__ unsigned sh_tau;
-    __shared__ int sh_take, sh_cut;
-    const int pair = blockIdx.x, tid = threadIdx.x;
-    const int b = pair / p.heads;
-    SelectRow *state = p.rows_state + pair;
-    if (state->solved) return;
-    const int S = sparf_seq_len(p, b, false);
-    const int k = min(S, min(max(p.k_tokens[b], 0), p.max_k));
-    const int n = state->n_cand, need = k - state->above;
-    if (n > kRowCandidates || need < 1 || need > n) return;      // left to the single-block kernel
-    for (int t = tid; t < n; t += kThresholdThreads) {
-        const uint2 c = p.row_cand[(int64_t)pair * kRowCandidates + t];
-        keys[t] = c.x;
-        where[t] = (int)c.y;
-    }
-    __syncthreads();
-    for (int t = tid; t < n; t += kThresholdThreads) {
-        const unsigned mine = keys[t];
-        int greater = 0, equal = 0;
-        for (int j = 0; j < n; ++j) {
-            greater += keys[j] > mine;
-            equal += keys[j] == mine;
-        }
-        if (greater < need && need <= greater + equal) {         // all holders of this key agree
-            sh_tau = mine;
-            sh_take = need - greater;
-        }
-    }
-    __syncthreads();
-    const unsigned tau = sh_tau;
-    const int take = sh_take;
-    for (int t = tid; t < n; t += kThresholdThreads) {               // the take-th smallest position among ties
-        if (keys[t] == tau) {
-            int before = 0;
-            for (int j = 0; j < n; ++j) before += keys[j] == tau && where[j] < where[t];
-            if (before == take - 1) sh_cut = where[t];
-        }
-    }
-    __syncthreads();
-    const int cut = sh_cut;
-    for (int t = tid; t < n; t += kThresholdThreads) {
-        if (keys[t] > tau || (keys[t] == tau && where[t] <= cut))
-            atomicAdd(&p.chunk_count[(int64_t)pair * p.score_chunks + where[t] / kScoreChunk], 1);
-    }
-    if (tid == 0) {
-        state->tau = tau;
-        state->idx_cut = cut;
-        state->solved = 1;
-    }
-}
-
-__global__ void __launch_bounds__(kChunkThreads)
-sparf_compact_kernel(const SparfParams p)
-{
-    allow_next_kernel();
-    wait_for_previous_kernels();
-    __shared__ int warp_total[kChunkThreads / 32];
-    __shared__ int sh_offset;
-    __shared__ float red[32];
-    __shared__ int list_pos[kScoreChunk];        // positions of one chunk's selected tokens, ascending
-    __shared__ float list_x[kScoreChunk];        // and their logits
-    ChunkView c;
-    if (!load_chunk(p, c)) return;
-    const SelectRow row = p.rows_state[c.pair];
-    if (!row.solved || row.bin > kLinearBins) return;
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    if (warp == 0) {                             // tokens selected in the chunks before this block's
-        int before = 0;
-        for (int j = lane; j < c.chunk0; j += 32) before += p.chunk_count[(int64_t)c.pair * p.score_chunks + j];
-#pragma unroll
-        for (int off = 16; off >= 1; off >>= 1) before += __shfl_xor_sync(0xffffffffu, before, off);
-        if (lane == 0) sh_offset = before;
-    }
-    const int T = p.block_tokens;
-    const int32_t *table_row = p.block_table + (int64_t)c.b * p.max_blocks_per_seq;
-    int32_t *rows = p.row_ids + (int64_t)c.pair * p.max_k;
-    int32_t *sel = p.selected ? p.selected + (int64_t)c.pair * p.max_k : nullptr;
-    float mass[kSubChunks];
-    const int window_from = c.S - c.window;      // first position of the forced local window
-    int done = 0;                                // selected tokens of this block's earlier chunks
-#pragma unroll
-    for (int sub = 0; sub < kSubChunks; ++sub) {
-        mass[sub] = 0.f;
-        if (sub >= c.n_sub) continue;            // uniform
-        const int i0 = c.first_token(sub);
-        // Which of this thread's 8 tokens are selected, as a bit mask.  With the exact
-        // threshold known the bins are no longer needed: the bins are monotone in the logit, so
-        // a token is selected iff it lies in the local window, or its key exceeds the
-        // threshold key, or equals it at a position up to the cut.
-        unsigned take = 0u;
-#pragma unroll
-        for (int e = 0; e < 8; ++e) {
-            const int i = i0 + e;
-            const unsigned key = ordered_key(c.x[sub][e]);
-            const bool chosen = i >= window_from || key > row.tau || (key == row.tau && i <= row.idx_cut);
-            take |= (unsigned)(i < c.S && chosen) << e;
-        }
-        const int mine = __popc(take);
-        int incl = mine;
-#pragma unroll
-        for (int off = 1; off < 32; off <<= 1) {
-            const int up = __shfl_up_sync(0xffffffffu, incl, off);
-            if (lane >= off) incl += up;
-        }
-        __syncthreads();                         // the previous chunk's list and totals are consumed
-        if (lane == 31) warp_total[warp] = incl;
-        __syncthreads();
-        int local = incl - mine, chunk_total = 0;
-        for (int w = 0; w < kChunkThreads / 32; ++w) {
-            if (w < warp) local += warp_total[w];
-            chunk_total += warp_total[w];
-        }
-        // Dense list of the selected tokens in shared memory: the costly part below then runs
-        // once per selected token instead of once per token slot of every warp.
-#pragma unroll
-        for (int e = 0; e < 8; ++e) {
-            if (take >> e & 1u) {
-                list_pos[local] = i0 + e;
-                list_x[local] = c.x[sub][e];
-                ++local;
-            }
-        }
-        __syncthreads();
-        for (int t = threadIdx.x; t < chunk_total; t += kChunkThreads) {
-            const int i = list_pos[t], pos = sh_offset + done + t;
-            const int blk = i / T, slot = i - blk * T;
-            const int phys = table_row[blk];
-            const bool ok = phys >= 0 && (int64_t)phys < p.num_phys_blocks;
-            if (!ok && p.status) atomicOr(p.status, kFlagBlockRange);
-            if (pos < p.max_k) {                 // always true for a consistent count; guards the buffer
-                rows[pos] = ok ? (phys * p.heads + c.h) * T + slot : 0;
-                if (sel) sel[pos] = i;
-            }
-            mass[sub] += fast_exp2(list_x[t] - row.top);
-        }
-        done += chunk_total;
-    }
-#pragma unroll
-    for (int sub = 0; sub < kSubChunks; ++sub) mass[sub] = block_sum(mass[sub], red);
-    if ((int)threadIdx.x < c.n_sub) {
-        float mine = mass[0];
-#pragma unroll
-        for (int sub = 1; sub < kSubChunks; ++sub) if ((int)threadIdx.x == sub) mine = mass[sub];
-        p.chunk_sums[(int64_t)c.pair * p.score_chunks + c.chunk0 + threadIdx.x].y = mine;
-    }
-}
-
-__global__ void __launch_bounds__(64)
-sparf_finish_kernel(const SparfParams p)
-{
-    allow_next_kernel();
-    wait_for_previous_kernels();
-    const int pair = blockIdx.x, tid = threadIdx.x;
-    const int b = pair / p.heads;
-    const SelectRow row = p.rows_state[pair];
-    if (!row.solved) return;
-    const int S = sparf_seq_len(p, b, false);
-    const int k = min(S, min(max(p.k_tokens[b], 0), p.max_k));
-    if (p.selected)
-        for (int t = k + tid; t < p.max_k; t += 64) p.selected[(int64_t)pair * p.max_k + t] = -1;
-    if (tid == 0) {
-        float alpha = 0.f;
-        if (k > 0) {
-            float mass = 0.f;
-            const int chunks = (S + kScoreChunk - 1) / kScoreChunk;
-            for (int c = 0; c < chunks; ++c) mass += p.chunk_sums[(int64_t)pair * p.score_chunks + c].y;   // fixed order
-            alpha = mass / row.z;
-        }
-        p.stats[pair] = make_float2(alpha, (float)k);
-        if (p.alpha_out) p.alpha_out[pair] = alpha;
-    }
 }
 
 // Merge of the gathered-attention partials and step 11.
