@@ -193,7 +193,7 @@ struct StageShared {
 // grid pairs * score_blocks, kSparfThreads threads: kScoreBlockTokens tokens of one row.  Each
 // warp takes whole segments of kSegmentTokens consecutive tokens (8 per lane), so the ordered
 // staging of a segment is a warp scan and the block never synchronises inside the loop.
-__global__ void __launch_bounds__(kSparfThreads)
+__global__ void __launch_bounds__(kSparfThreads, 8)
 sparf_stage_kernel(const SparfParams p)
 {
     allow_next_kernel();
