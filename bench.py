@@ -67,6 +67,8 @@ def parse_args(argv=None):
                          "sparse:<workload index>[:<batch>[:<kt block tokens>]] or grouped:<name> "
                          "(names: " + ", ".join(n for n in PROFILE_GROUPED) + ")")
     ap.add_argument("--launches", type=int, default=2, help="calls made by --case")
+    ap.add_argument("--sparse-path", type=int, default=0,
+                    help="--case sparse: 0 automatic, 1 staged chain, 2 one block per row")
     return ap.parse_args(argv)
 
 
@@ -677,11 +679,12 @@ def measure_grouped(device, steps: int = 20) -> dict:
     return results
 
 
-def run_case(spec: str, launches: int, device) -> dict:
+def run_case(spec: str, launches: int, device, sparse_path: int = 0) -> dict:
     """One small case of the sparse or the grouped entry point, `launches` calls back to back
     (what the ncu commands under profiles/ run)."""
     from paper_2409_04992_b200 import binding
     kind, _, rest = spec.partition(":")
+    binding.set_sparse_path(sparse_path)
     flags = torch.zeros(1, dtype=torch.int32, device=device)
     a, z = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     if kind == "sparse":
@@ -751,7 +754,7 @@ def main(argv=None) -> int:
         torch.cuda.set_device(device)
         if args.case:
             if ranks.rank == 0:
-                print(json.dumps(run_case(args.case, args.launches, device)), flush=True)
+                print(json.dumps(run_case(args.case, args.launches, device, args.sparse_path)), flush=True)
             return 0
         w = wl.by_name(args.workload)
         if args.layers > 0:

@@ -363,13 +363,16 @@ size_t instinfer_sparf_workspace_bytes(int32_t batch, int32_t heads, int32_t hea
                                        int32_t max_seq_len, int32_t max_k);
 
 /*
- * Steps 1-7 of Algorithm 1 have two implementations with identical results: one thread block
- * per (sequence, head) that keeps the row's approximate logits in shared memory (rows of at
- * most 16384 tokens), and a chunk-parallel one that passes them through the workspace (any
- * length).  The library picks by the sizes;
- * instinfer_set_sparse_path forces the choice for later calls of this process: 0 automatic,
- * 1 chunk-parallel, 2 one block per row where the rows fit (a tuning and test aid; returns
- * INSTINFER_OK or INSTINFER_ERR_INVALID_ARG; not thread-safe against concurrent calls).
+ * Steps 1-7 of Algorithm 1 have two implementations: one thread block per (sequence, head)
+ * that keeps the row's approximate logits in shared memory (rows of at most 16384 tokens), and
+ * a chain of kernels for long rows that first brackets the k-th largest score on a sample of
+ * the row and then keeps only the tokens that can still be selected (any length; rows it
+ * cannot settle, e.g. thousands of equal scores, are redone by one block per row).  Both
+ * compute the same fp32 scores and cut ties by position, so they select the same tokens.
+ * The library picks by the sizes; instinfer_set_sparse_path forces the choice for later calls
+ * of this process: 0 automatic, 1 the chain, 2 one block per row where the rows fit (a tuning
+ * and test aid; returns INSTINFER_OK or INSTINFER_ERR_INVALID_ARG; not thread-safe against
+ * concurrent calls).
  */
 int instinfer_set_sparse_path(int32_t path);
 

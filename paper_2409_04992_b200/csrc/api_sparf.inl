@@ -238,12 +238,17 @@ int instinfer_sparf_decode_attention(void *out, float *alpha, int32_t *selected,
     sp.seg_mass = reinterpret_cast<float *>(ws + w.seg_mass);
 
     const unsigned block_grid = (unsigned)(pairs * w.score_blocks), row_grid = (unsigned)pairs;
-    // Two ways through steps 1-7.  For rows that fit in shared memory one block per row computes
-    // the logits there and selects from there; otherwise (and for very many rows of the largest
-    // size that fits) the staged chain: a sampled pre-pass brackets the threshold and the score
-    // pass keeps only the tokens that can still be selected.  Neither writes the logits to HBM.
+    // Two ways through steps 1-7, neither of which writes the logits to HBM.  One block per row
+    // computes the row's logits into shared memory and selects from there (rows of at most
+    // kFusedMaxTokens tokens); the staged chain brackets the threshold on a sample and keeps
+    // only the tokens that can still be selected.  Measured on one B200: the chain wins for
+    // long rows with enough work to fill the GPU (2560 rows of 16k tokens: 0.86 against
+    // 0.97 ms a step; 320 rows of 128k only fit the chain), the single kernel for short rows,
+    // where the chain's nine launches are mostly latency (640 rows of 4k-8k tokens: 0.13
+    // against 0.17 ms).
     const bool fits = max_seq_len <= kFusedMaxTokens;
-    const bool fused = g_sparse_path == 1 ? false : fits;
+    const bool long_rows = max_seq_len > 8192 && pairs * (int64_t)max_seq_len >= (int64_t)1 << 24;
+    const bool fused = g_sparse_path == 1 ? false : g_sparse_path == 2 ? fits : fits && !long_rows;
     if (fused) {
         static bool fused_smem_set[kMaxDevices] = {};
         int device = 0;
@@ -264,9 +269,13 @@ int instinfer_sparf_decode_attention(void *out, float *alpha, int32_t *selected,
         int device = 0;
         if (cudaGetDevice(&device) != cudaSuccess || device < 0 || device >= kMaxDevices) return INSTINFER_ERR_CUDA;
         if (!staged_smem_set[device]) {
-            if (cudaFuncSetAttribute(sparf_sample_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+            if (cudaFuncSetAttribute(sparf_sample_kernel<512>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      kMaxSamples * (int)sizeof(float)) != cudaSuccess ||
-                cudaFuncSetAttribute(sparf_resolve_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                cudaFuncSetAttribute(sparf_sample_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     kMaxSamples * (int)sizeof(float)) != cudaSuccess ||
+                cudaFuncSetAttribute(sparf_resolve_kernel<512>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     kCandidates * (int)sizeof(int)) != cudaSuccess ||
+                cudaFuncSetAttribute(sparf_resolve_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      kCandidates * (int)sizeof(int)) != cudaSuccess) {
                 (void)cudaGetLastError();
                 return INSTINFER_ERR_CUDA;
@@ -277,14 +286,21 @@ int instinfer_sparf_decode_attention(void *out, float *alpha, int32_t *selected,
             (void)cudaGetLastError();
             return INSTINFER_ERR_CUDA;
         }
-        bool ok = launch_overlapped(sparf_sample_kernel, row_grid, kSampleThreads, kMaxSamples * sizeof(float), stream, sp) == cudaSuccess;
+        const size_t sample_bytes = (size_t)sample_capacity(max_seq_len) * sizeof(float);
+        bool ok = max_seq_len > 32768
+            ? launch_overlapped(sparf_sample_kernel<512>, row_grid, 512, sample_bytes, stream, sp) == cudaSuccess
+            : launch_overlapped(sparf_sample_kernel<256>, row_grid, 256, sample_bytes, stream, sp) == cudaSuccess;
         ok = ok && launch_overlapped(sparf_stage_kernel, block_grid, kSparfThreads, 0, stream, sp) == cudaSuccess;
-        ok = ok && launch_overlapped(sparf_resolve_kernel, row_grid, kResolveThreads, (size_t)w.cand_capacity * sizeof(int), stream, sp) == cudaSuccess;
+        const size_t where_bytes = (size_t)w.cand_capacity * sizeof(int);
+        ok = ok && (w.cand_capacity > 4096
+            ? launch_overlapped(sparf_resolve_kernel<512>, row_grid, 512, where_bytes, stream, sp)
+            : launch_overlapped(sparf_resolve_kernel<256>, row_grid, 256, where_bytes, stream, sp)) == cudaSuccess;
         ok = ok && launch_overlapped(sparf_emit_kernel, block_grid, kEmitThreads, 0, stream, sp) == cudaSuccess;
         ok = ok && launch_overlapped(sparf_finish_kernel, row_grid, 64, 0, stream, sp) == cudaSuccess;
         // rows the chain could not settle: all their logits to the workspace, one block per row selects
-        ok = ok && launch_overlapped(sparf_scores_kernel, block_grid, kSparfThreads, 0, stream, sp) == cudaSuccess;
-        ok = ok && launch_overlapped(sparf_select_kernel, row_grid, kSelectThreads, 0, stream, sp) == cudaSuccess;
+        const unsigned few = (unsigned)(2 * sm_count());
+        ok = ok && launch_overlapped(sparf_scores_kernel, block_grid < 4 * few ? block_grid : 4 * few, kSparfThreads, 0, stream, sp) == cudaSuccess;
+        ok = ok && launch_overlapped(sparf_select_kernel, row_grid < few ? row_grid : few, kSelectThreads, 0, stream, sp) == cudaSuccess;
         if (!ok) {
             (void)cudaGetLastError();
             return INSTINFER_ERR_CUDA;

@@ -298,34 +298,39 @@ __device__ __forceinline__ void score_group(const SparfParams &p, const ScoreSha
 // Every kernel of the attention call below starts with the programmatic-dependent-launch pair
 // (let the next kernel's blocks become resident, then wait for all earlier kernels), before
 // any return, so that the chain of short launches overlaps its launch latencies.
-// grid pairs * score_blocks: all approximate logits of kScoreBlockTokens tokens of one
-// (sequence, head), written to the workspace.  Only for the rows the staged chain left
-// unsolved (its blocks leave at once on the others).
+// All approximate logits of the rows the staged chain left unsolved, written to the workspace,
+// kScoreBlockTokens tokens of one (sequence, head) per step of a block; the grid is bounded
+// and its blocks walk over all (row, block) items, skipping those of solved rows.
 __global__ void __launch_bounds__(kSparfThreads)
 sparf_scores_kernel(const SparfParams p)
 {
     allow_next_kernel();
     wait_for_previous_kernels();
     __shared__ ScoreShared ss;
-    const int pair = blockIdx.x / p.score_blocks, d = threadIdx.x;
-    const int b = pair / p.heads, h = pair - b * p.heads;
-    if (p.rows_state[pair].solved) return;
-    const int len = sparf_seq_len(p, b, false);
-    const int begin = (blockIdx.x - pair * p.score_blocks) * kScoreBlockTokens;
-    if (begin >= len) return;
-    const int end = min(begin + kScoreBlockTokens, len);
-    score_setup(p, pair, ss);
+    const int d = threadIdx.x;
+    const int64_t items = (int64_t)p.batch * p.heads * p.score_blocks;
+    for (int64_t item = blockIdx.x; item < items; item += gridDim.x) {
+        const int pair = (int)(item / p.score_blocks);
+        if (p.rows_state[pair].solved) continue;
+        const int b = pair / p.heads, h = pair - b * p.heads;
+        const int len = sparf_seq_len(p, b, false);
+        const int begin = (int)(item - (int64_t)pair * p.score_blocks) * kScoreBlockTokens;
+        if (begin >= len) continue;
+        const int end = min(begin + kScoreBlockTokens, len);
+        __syncthreads();                                     // the previous item's set-up is no longer read
+        score_setup(p, pair, ss);
 
-    const int32_t *table_row = p.kt_block_table + (int64_t)b * p.kt_max_blocks_per_seq;
-    float *dst = p.scores + (int64_t)pair * p.score_stride;
-    for (int i = begin + d * 8; i < end; i += kSparfThreads * 8) {
-        float dot[8];
-        score_group(p, ss, table_row, h, i, dot);
-        // score_stride is a multiple of 8 and rows start 32-byte aligned; entries past `end`
-        // inside the last group are scratch nobody reads.
-        float4 *out4 = reinterpret_cast<float4 *>(dst + i);
-        out4[0] = make_float4(dot[0], dot[1], dot[2], dot[3]);
-        out4[1] = make_float4(dot[4], dot[5], dot[6], dot[7]);
+        const int32_t *table_row = p.kt_block_table + (int64_t)b * p.kt_max_blocks_per_seq;
+        float *dst = p.scores + (int64_t)pair * p.score_stride;
+        for (int i = begin + d * 8; i < end; i += kSparfThreads * 8) {
+            float dot[8];
+            score_group(p, ss, table_row, h, i, dot);
+            // score_stride is a multiple of 8 and rows start 32-byte aligned; entries past `end`
+            // inside the last group are scratch nobody reads.
+            float4 *out4 = reinterpret_cast<float4 *>(dst + i);
+            out4[0] = make_float4(dot[0], dot[1], dot[2], dot[3]);
+            out4[1] = make_float4(dot[4], dot[5], dot[6], dot[7]);
+        }
     }
 }
 
@@ -689,20 +694,25 @@ __device__ __forceinline__ void select_row(const SparfParams &p, SelectShared &s
     }
 }
 
-// One block per (sequence, head), logits from the workspace: redoes the rows that the
-// chunk-parallel kernels left unsolved.
+// One block per (sequence, head) at a time, logits from the workspace: redoes the rows that
+// the staged chain left unsolved.  Those are rare, so the grid is a few blocks per SM that walk
+// over all rows and skip the solved ones (a block per row would be thousands of blocks that
+// start only to leave).
 __global__ void __launch_bounds__(kSelectThreads)
 sparf_select_kernel(const SparfParams p)
 {
     allow_next_kernel();
     wait_for_previous_kernels();
     __shared__ SelectShared sh;
-    const int pair = blockIdx.x;
-    const int b = pair / p.heads, h = pair - b * p.heads;
-    if (p.rows_state && p.rows_state[pair].solved) return;      // done by the staged chain
-    const int S = sparf_seq_len(p, b, threadIdx.x == 0 && h == 0);
-    const int k = min(S, min(max(p.k_tokens[b], 0), p.max_k));
-    select_row<kSelectThreads>(p, sh, p.scores + (int64_t)pair * p.score_stride, pair, b, h, S, k, min(p.window, k));
+    const int pairs = p.batch * p.heads;
+    for (int pair = blockIdx.x; pair < pairs; pair += gridDim.x) {
+        if (p.rows_state[pair].solved) continue;             // done by the staged chain
+        const int b = pair / p.heads, h = pair - b * p.heads;
+        const int S = sparf_seq_len(p, b, threadIdx.x == 0 && h == 0);
+        const int k = min(S, min(max(p.k_tokens[b], 0), p.max_k));
+        __syncthreads();                                     // the scratch of the previous row is free
+        select_row<kSelectThreads>(p, sh, p.scores + (int64_t)pair * p.score_stride, pair, b, h, S, k, min(p.window, k));
+    }
 }
 
 // Steps 1-7 for one (sequence, head) by one block: the row's approximate logits are computed

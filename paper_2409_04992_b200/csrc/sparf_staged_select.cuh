@@ -35,10 +35,8 @@
 
 namespace instinfer {
 
-constexpr int kSampleThreads = 512;
 constexpr int kSampleRun = 256;          // consecutive tokens sampled per stride
 constexpr int kMaxSamples = 16384;       // per row (64 KiB of shared memory)
-constexpr int kResolveThreads = 512;
 constexpr int kEmitThreads = 256;
 constexpr float kRefSlack = 64.f;        // logits this far (base 2) above the sampled maximum void the sums
 
@@ -76,7 +74,18 @@ __device__ __forceinline__ void locate_linear_bin(const unsigned *hist, int from
     }
 }
 
-// grid pairs, dynamic shared memory kMaxSamples floats.
+// Shared memory (floats) that the samples of a row of at most max_seq_len tokens need.
+inline int sample_capacity(int max_seq_len)
+{
+    const int64_t most = max_seq_len >= 65536 ? (int64_t)max_seq_len / 16 + 4096 : (int64_t)max_seq_len / 8 + 2 * kSampleRun;
+    const int64_t floor = 8 * kSampleRun;                    // rows below 8k tokens are sampled more densely
+    const int64_t need = most > floor ? most : floor;
+    return (int)(need < kMaxSamples ? need : kMaxSamples);
+}
+
+// grid pairs, kSampleThreads threads (512 for long rows, 256 for rows whose sample is small,
+// so that more blocks share an SM), dynamic shared memory sample_capacity(max_seq_len) floats.
+template <int kSampleThreads>
 __global__ void __launch_bounds__(kSampleThreads)
 sparf_sample_kernel(const SparfParams p)
 {
@@ -279,8 +288,9 @@ sparf_stage_kernel(const SparfParams p)
     if (far_above) row->overflow = 1;
 }
 
-// grid pairs, kResolveThreads threads, dynamic shared memory cand_capacity * 4 bytes (positions;
+// grid pairs, kResolveThreads threads (512, or 256 when the candidate lists are short), dynamic shared memory cand_capacity * 4 bytes (positions;
 // the keys sit in the select scratch).  cand_capacity <= kCandidates.
+template <int kResolveThreads>
 __global__ void __launch_bounds__(kResolveThreads)
 sparf_resolve_kernel(const SparfParams p)
 {
@@ -326,9 +336,15 @@ sparf_resolve_kernel(const SparfParams p)
     // among the keys equal to tau the `take` lowest positions: the take-th smallest position,
     // found as the take-th largest of the complemented positions
     __syncthreads();
-    exact_threshold<kResolveThreads>(sh, n, take, [&](int i) { return keys[i] == tau; },
-                                     [&](int i) { return ~(unsigned)where[i]; });
-    const int cut = (int)~sh.tau;
+    int ties = 0;
+    for (int t = tid; t < n; t += kResolveThreads) ties += keys[t] == tau;
+    ties = block_sum(ties, reinterpret_cast<int *>(sh.red_f));
+    int cut = 0x7fffffff;                                    // every token that ties with tau is taken ...
+    if (take < ties) {                                       // ... unless the cut falls among them (uniform)
+        exact_threshold<kResolveThreads>(sh, n, take, [&](int i) { return keys[i] == tau; },
+                                         [&](int i) { return ~(unsigned)where[i]; });
+        cut = (int)~sh.tau;
+    }
     for (int t = tid; t < n; t += kResolveThreads) {
         if (keys[t] > tau || (keys[t] == tau && where[t] <= cut)) atomicAdd(&seg_final[where[t] / kSegmentTokens], 1);
     }
