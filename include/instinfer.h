@@ -69,6 +69,10 @@ typedef enum {
 /* Bits OR-ed into *status_flags by the kernels. */
 #define INSTINFER_FLAG_SEQ_LEN_RANGE 1  /* seq_lens[b] < 0, beyond the cache capacity, or beyond max_seq_len */
 #define INSTINFER_FLAG_BLOCK_RANGE   2  /* a block_table entry that had to be read lies outside [0, num_phys_blocks) */
+#define INSTINFER_FLAG_BOUNDS_CHECK  8  /* only in the bounds-checking build of the library (compiled with
+                                           -DINSTINFER_BOUNDS_CHECK): a kernel computed a global offset outside the
+                                           extent that the call's shapes imply and skipped that access; a defect of
+                                           the library, never of the caller's data */
 #define INSTINFER_FLAG_COPY_TIMEOUT  4  /* an asynchronous copy inside a kernel did not complete within about two
                                            seconds (a hardware problem, never a data problem); the kernel ended
                                            instead of waiting on and the outputs of that call are undefined */

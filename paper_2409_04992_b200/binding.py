@@ -7,15 +7,17 @@ library's kernels.  There is no fallback: if the library has not been built, loa
 from __future__ import annotations
 
 import ctypes
+import os
 from pathlib import Path
 from typing import Optional, Sequence, Union
 
 import torch
 
-LIBRARY = Path(__file__).resolve().parent / "libinstinfer.so"
+# INSTINFER_LIBRARY selects another build of the same library (the bounds-checking one, say).
+LIBRARY = Path(os.environ.get("INSTINFER_LIBRARY") or Path(__file__).resolve().parent / "libinstinfer.so")
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA = range(5)
-FLAG_SEQ_LEN_RANGE, FLAG_BLOCK_RANGE, FLAG_COPY_TIMEOUT = 1, 2, 4
+FLAG_SEQ_LEN_RANGE, FLAG_BLOCK_RANGE, FLAG_COPY_TIMEOUT, FLAG_BOUNDS_CHECK = 1, 2, 4, 8
 STATIC_WORKSPACE_BYTES = 16 << 20
 
 _lib: Optional[ctypes.CDLL] = None

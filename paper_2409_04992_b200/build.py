@@ -10,6 +10,7 @@ _HERE = Path(__file__).resolve().parent
 CSRC = _HERE / "csrc"
 INCLUDE = _HERE.parent / "include"
 LIBRARY = _HERE / "libinstinfer.so"
+CHECKED_LIBRARY = _HERE / "libinstinfer_checked.so"     # the bounds-checking build (-DINSTINFER_BOUNDS_CHECK)
 SOURCES = [CSRC / "instinfer_api.cu"]      # it includes the api_*.inl parts
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo",
               "-Xcompiler", "-fPIC", "-shared", "-cudart", "static", "-Xptxas", "-v"]
@@ -27,24 +28,30 @@ def _inputs():
             list(INCLUDE.glob("*.h")))
 
 
-def is_current() -> bool:
-    return LIBRARY.exists() and all(LIBRARY.stat().st_mtime >= f.stat().st_mtime for f in _inputs())
+def is_current(library: Path = LIBRARY) -> bool:
+    return library.exists() and all(library.stat().st_mtime >= f.stat().st_mtime for f in _inputs())
 
 
-def build(force: bool = False, verbose: bool = False) -> Path:
-    """nvcc -> libinstinfer.so; skipped when the library is newer than every source."""
-    if not force and is_current():
-        return LIBRARY
-    tmp = LIBRARY.with_suffix(f".{os.getpid()}.tmp.so")
-    cmd = [_nvcc(), *NVCC_FLAGS, "-I", str(INCLUDE), *map(str, SOURCES), "-o", str(tmp)]
+def build(force: bool = False, verbose: bool = False, checked: bool = False) -> Path:
+    """nvcc -> libinstinfer.so (or, with checked=True, the bounds-checking build
+    libinstinfer_checked.so, in which every data-dependent global offset is tested against the
+    extent the call's shapes imply and a violation sets status bit 8 instead of being used);
+    skipped when the library is newer than every source."""
+    library = CHECKED_LIBRARY if checked else LIBRARY
+    if not force and is_current(library):
+        return library
+    tmp = library.with_suffix(f".{os.getpid()}.tmp.so")
+    extra = ["-DINSTINFER_BOUNDS_CHECK"] if checked else []
+    cmd = [_nvcc(), *NVCC_FLAGS, *extra, "-I", str(INCLUDE), *map(str, SOURCES), "-o", str(tmp)]
     done = subprocess.run(cmd, capture_output=True, text=True)
     if verbose or done.returncode:
         print(done.stdout + done.stderr)
     if done.returncode:
         raise RuntimeError("nvcc failed")
-    os.replace(tmp, LIBRARY)
-    return LIBRARY
+    os.replace(tmp, library)
+    return library
 
 
 if __name__ == "__main__":
     print(build(force=True, verbose=True))
+    print(build(force=True, checked=True))

@@ -120,6 +120,7 @@ int instinfer_decode_attention_grouped(void *out, float *lse, const void *q, con
     p.a.tail_chunk = plan.tail_chunk;
     p.a.n_splits = plan.n_splits;
     p.a.max_seq_len = max_seq_len;
+    p.a.kv_bytes = (paged ? num_phys_blocks * kv_heads * block_tokens : (int64_t)batch * kv_heads * s_max) * head_dim * 2;
     p.a.scale_log2e = scale * 1.44269504088896340736f;
     p.a.part_o = static_cast<float *>(workspace);
     p.a.part_lse = p.a.part_o + (size_t)pairs * plan.n_splits * p.rows * head_dim;

@@ -220,6 +220,7 @@ int instinfer_sparf_decode_attention(void *out, float *alpha, int32_t *selected,
     sp.kt_block_tokens = kt_block_tokens;
     sp.kt_max_blocks_per_seq = kt_max_blocks_per_seq;
     sp.num_kt_blocks = num_kt_blocks;
+    sp.kt_elems = num_kt_blocks * heads * kHeadDim * kt_block_tokens;
     sp.max_seq_len = max_seq_len;
     sp.max_k = max_k;
     sp.score_stride = w.score_stride;
@@ -329,6 +330,7 @@ int instinfer_sparf_decode_attention(void *out, float *alpha, int32_t *selected,
     ap.row_ids = sp.row_ids;
     ap.k_tokens = k_tokens;
     ap.row_stride = max_k;
+    ap.kv_bytes = num_phys_blocks * heads * block_tokens * kRowBytes;
     ap.row_limit = (int32_t)(num_phys_blocks * heads * block_tokens);      // below 2^31, checked above
     mp.stats = sp.stats;
     mp.v_sum = v_sum;

@@ -52,6 +52,22 @@ constexpr float kLn2 = 0.69314718055994530942f;
 constexpr int kFlagSeqLenRange = 1;
 constexpr int kFlagBlockRange = 2;
 constexpr int kFlagCopyTimeout = 4;
+constexpr int kFlagBoundsCheck = 8;
+
+// Bounds-checking build (-DINSTINFER_BOUNDS_CHECK): every data-dependent global offset that a
+// kernel computes (from a block table, a length, a row list) is tested against the extent
+// that the call's shapes imply before it is used; a violation sets kFlagBoundsCheck in the
+// status word and the access is skipped.  It stands in for a memory checker: in a correct
+// library the bit never appears.  In the ordinary build the test compiles to nothing.
+#ifdef INSTINFER_BOUNDS_CHECK
+__device__ __forceinline__ bool bounds_ok(bool inside, int32_t *status)
+{
+    if (!inside && status) atomicOr(status, kFlagBoundsCheck);
+    return inside;
+}
+#else
+__device__ __forceinline__ bool bounds_ok(bool, int32_t *) { return true; }
+#endif
 
 struct AttnParams {
     const __half *q;
@@ -82,6 +98,7 @@ struct AttnParams {
     const int32_t *k_tokens;   // [batch] rows to attend per sequence (clipped to its length)
     int32_t row_stride;
     int32_t row_limit;         // number of rows in the pools: a listed id outside [0, row_limit) reads as zeros
+    int64_t kv_bytes;          // bytes of the K cache (= of the V cache) that the call's shapes imply
 };
 
 // Where a (sequence, head)'s rows come from.
@@ -440,7 +457,8 @@ decode_attn_split_kernel(const AttnParams p)
     }
     auto load_window = [&](int base) -> int {
         const int idx = base + lane;
-        return idx < blocks_needed ? __ldg(table_row + idx) : 0;
+        if (idx >= blocks_needed || !bounds_ok(idx < p.max_blocks_per_seq, p.status)) return 0;
+        return __ldg(table_row + idx);
     };
     if (kPaged && my_tiles > 0) {
         window_now = load_window(win_base);
@@ -498,6 +516,7 @@ decode_attn_split_kernel(const AttnParams p)
                 // the rows of a block with a bad id are not fetched; their value slots are
                 // zeroed (their weights are zero, but 0 x stale bits must not be NaN) and their
                 // logits are masked below.
+                usable = usable && bounds_ok(off >= 0 && off + rows * kRowBytes <= p.kv_bytes, p.status);
                 const int fetch = usable ? rows : 0;
                 if (fetch < kTileRows) {
                     const uint4 zero = make_uint4(0u, 0u, 0u, 0u);

@@ -311,7 +311,7 @@ grouped_attn_split_kernel(const GroupedParams p)
         step_rem = kStepTokens - step_blk * tokens;
         block_stride = (int64_t)a.heads * tokens * G::kRowBytes;
         head_off = (int64_t)hk * tokens * G::kRowBytes;
-        next_phys = my_tiles > 0 ? __ldg(table_row + blk) : 0;
+        next_phys = my_tiles > 0 && bounds_ok(blk < a.max_blocks_per_seq, a.status) ? __ldg(table_row + blk) : 0;
     } else {
         src_off = ((int64_t)pair * a.s_max + first_token) * G::kRowBytes;
     }
@@ -334,11 +334,14 @@ grouped_attn_split_kernel(const GroupedParams p)
                     rem -= a.block_tokens;
                     ++blk;
                 }
-                if (issue_j + 1 < my_tiles) next_phys = __ldg(table_row + blk);
+                if (issue_j + 1 < my_tiles)
+                    next_phys = bounds_ok(blk < a.max_blocks_per_seq, a.status) ? __ldg(table_row + blk) : -1;
             } else {
                 off = src_off;
                 src_off += (int64_t)kStepTokens * G::kRowBytes;
             }
+            usable = usable && bounds_ok(off >= 0 && off + (int64_t)min(rows_here, kGroupTile) * G::kRowBytes <= a.kv_bytes, a.status);
+            if (!usable) off = 0;
             const unsigned char *ks = k_lane + off, *vs = v_lane + off;
             const unsigned dst = ring + issue_stage * G::kStageBytes + lane_dst;
             if (usable && rows_here >= kGroupTile) {               // full tile: no predicates

@@ -151,6 +151,7 @@ int instinfer_kv_append(void *k_cache, void *v_cache, const void *k_new, const v
     p.block_tokens = block_tokens;
     p.max_blocks_per_seq = max_blocks_per_seq;
     p.segs_per_row = head_dim / 8;
+    p.cache_rows = block_table ? num_phys_blocks * heads * block_tokens : (int64_t)batch * heads * s_max;
     const int64_t threads = (int64_t)batch * heads * p.segs_per_row;
     const unsigned grid = (unsigned)ceil_div(threads, kAppendThreads);
     const cudaError_t err = launch_overlapped(kv_append_kernel, grid, kAppendThreads, 0,
@@ -179,7 +180,7 @@ int instinfer_kv_append_bulk(void *k_cache, void *v_cache, const void *k_new, co
     if (!usable(k_cache) || !usable(v_cache) || !usable(k_new) || !usable(v_new) ||
         seq_lens == nullptr || new_lens == nullptr)
         return INSTINFER_ERR_INVALID_ARG;
-    const int64_t threads = (int64_t)batch * max_new * heads * (head_dim / 8);
+    const int64_t threads = (int64_t)batch * ceil_div(max_new, kBulkTokens) * heads * (head_dim / 8);
     const int64_t grid = ceil_div(threads, kAppendThreads);
     if (grid >= (int64_t)1 << 31) return INSTINFER_ERR_INVALID_ARG;
 
@@ -199,6 +200,7 @@ int instinfer_kv_append_bulk(void *k_cache, void *v_cache, const void *k_new, co
     p.block_tokens = block_tokens;
     p.max_blocks_per_seq = max_blocks_per_seq;
     p.segs_per_row = head_dim / 8;
+    p.cache_rows = block_table ? num_phys_blocks * heads * block_tokens : (int64_t)batch * heads * s_max;
     q.new_lens = new_lens;
     q.max_new = max_new;
     kv_append_bulk_kernel<<<(unsigned)grid, kAppendThreads, 0, static_cast<cudaStream_t>(cuda_stream)>>>(q);
@@ -230,6 +232,7 @@ int instinfer_decode_attention(void *out, float *lse, const void *q, const void 
     p.heads = heads;
     p.s_max = s_max;
     p.max_seq_len = max_seq_len;
+    p.kv_bytes = (int64_t)batch * heads * s_max * kRowBytes;
     p.scale_log2e = scale * 1.44269504088896340736f;
     return launch_attention(p, false, batch, workspace, workspace_bytes,
                             static_cast<cudaStream_t>(cuda_stream));
@@ -269,6 +272,7 @@ int instinfer_decode_attention_paged(void *out, float *lse, const void *q, const
     p.block_tokens = block_tokens;
     p.max_blocks_per_seq = max_blocks_per_seq;
     p.max_seq_len = max_seq_len;
+    p.kv_bytes = num_phys_blocks * heads * block_tokens * kRowBytes;
     p.scale_log2e = scale * 1.44269504088896340736f;
     return launch_attention(p, true, batch, workspace, workspace_bytes,
                             static_cast<cudaStream_t>(cuda_stream));
@@ -353,6 +357,7 @@ int instinfer_decode_attention_allgather(void *const *out_all, int32_t n_ranks, 
     p.block_tokens = paged ? block_tokens : 0;
     p.max_blocks_per_seq = paged ? max_blocks_per_seq : 0;
     p.max_seq_len = max_seq_len;
+    p.kv_bytes = (paged ? num_phys_blocks * heads * block_tokens : (int64_t)batch * heads * s_max) * kRowBytes;
     p.scale_log2e = scale * 1.44269504088896340736f;
     return launch_attention(p, paged, batch, workspace, workspace_bytes,
                             static_cast<cudaStream_t>(cuda_stream), &targets);

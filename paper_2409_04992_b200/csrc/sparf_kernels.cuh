@@ -72,6 +72,7 @@ struct SparfParams {
     int32_t *selected;         // nullable [pairs, max_k] logical token index, ascending, -1 padded
     int64_t num_phys_blocks;
     int64_t num_kt_blocks;
+    int64_t kt_elems;          // elements of kt_pool that the call's shapes imply (attention call only)
     int32_t batch, heads, block_tokens, max_blocks_per_seq;
     int32_t kt_block_tokens, kt_max_blocks_per_seq;
     int32_t max_seq_len, max_k, score_stride, segments, score_blocks, cand_capacity, r, window;
@@ -259,11 +260,13 @@ __device__ __forceinline__ void score_group(const SparfParams &p, const ScoreSha
 {
     const int T = p.kt_block_tokens;
     const int blk = i / T, slot = i - blk * T;
-    const int phys = table_row[blk];
+    const int phys = bounds_ok(blk < p.kt_max_blocks_per_seq, p.status) ? table_row[blk] : -1;
 #pragma unroll
     for (int e = 0; e < 8; ++e) dot[e] = 0.f;
-    if (phys >= 0 && (int64_t)phys < p.num_kt_blocks) {
-        const __half *kt = p.kt_pool + ((int64_t)phys * p.heads + h) * T * kHeadDim + slot;
+    const int64_t area = ((int64_t)phys * p.heads + h) * T * kHeadDim;      // this (block, head): [D][T]
+    if (phys >= 0 && (int64_t)phys < p.num_kt_blocks &&
+        bounds_ok(area + (int64_t)(kHeadDim - 1) * T + slot + 8 <= p.kt_elems, p.status)) {
+        const __half *kt = p.kt_pool + area + slot;
         for (int t0 = 0; t0 < p.r; t0 += 8) {
             uint4 raw[8];
 #pragma unroll
@@ -672,7 +675,7 @@ __device__ __forceinline__ void select_row(const SparfParams &p, SelectShared &s
                 const int i = 4 * g + e;
                 const int pos = gt_before + min(eq_before, take_equal);
                 const int blk = i / T, slot = i - blk * T;
-                const int phys = table_row[blk];
+                const int phys = bounds_ok(blk < p.max_blocks_per_seq && pos < p.max_k, p.status) ? table_row[blk] : -1;
                 const bool ok = phys >= 0 && (int64_t)phys < p.num_phys_blocks;
                 if (!ok && p.status) atomicOr(p.status, kFlagBlockRange);
                 rows[pos] = ok ? (phys * p.heads + h) * T + slot : 0;

@@ -273,6 +273,7 @@ sparf_stage_kernel(const SparfParams p)
 #pragma unroll
         for (int e = 0; e < 8; ++e) {
             if (staged >> e & 1u) {
+                if (!bounds_ok(seg_begin + at < p.score_stride, p.status)) continue;
                 stage_x[seg_begin + at] = dot[e];
                 stage_pos[seg_begin + at] = i + e;
                 ++at;
@@ -445,7 +446,7 @@ sparf_emit_kernel(const SparfParams p)
             if (take >> e & 1u) {
                 const int i = pos[e];
                 const int blk = i / T, slot = i - blk * T;
-                const int phys = table_row[blk];
+                const int phys = bounds_ok(blk < p.max_blocks_per_seq && dst < p.max_k, p.status) ? table_row[blk] : -1;
                 const bool ok = phys >= 0 && (int64_t)phys < p.num_phys_blocks;
                 if (!ok && p.status) atomicOr(p.status, kFlagBlockRange);
                 if (dst < p.max_k) {         // always true for a consistent count; guards the buffer
