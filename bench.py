@@ -691,6 +691,75 @@ def measure_grouped(device, steps: int = 20) -> dict:
     return results
 
 
+def head_sharded_result(ranks: Ranks, units_this_rank: float, seconds_this_rank: float, heads_this_rank: int,
+                        total_heads: int, max_abs_error) -> dict:
+    """Whole-instance figures of the head-sharded section from per-rank measurements: bytes of
+    all ranks over the slowest rank's time (one model instance, strong scaling)."""
+    gbs, seconds = aggregate(ranks, units_this_rank, seconds_this_rank)
+    heads = ranks.sum(float(heads_this_rank))
+    return {"value": gbs, "unit": UNIT, "seconds": seconds, "scaling": "strong",
+            "heads_covered": int(round(heads)), "total_heads": total_heads,
+            "max_abs_vs_single_gpu": max_abs_error}
+
+
+def measure_head_sharded(ranks: Ranks, device, steps: int = 20) -> dict:
+    """One model instance spread over the ranks the way the paper spreads it over drives
+    (Sec. IV-D): one layer of the default workload, batch 16, the 40 heads split over the ranks,
+    every rank's KV cache holding only its heads, outputs exchanged by the fused all-gather
+    (peer stores of the last kernel into every rank's buffer in symmetric memory).  Only run
+    with more than one rank; any failure is returned as text instead of raised, so that it
+    cannot take the weak-scaling number down with it."""
+    try:
+        from paper_2409_04992_b200 import binding, sharding
+        w = wl.STANDARD[4].replace(layers=1)
+        case = wl.generate(w, device=str(device), poison=False)            # the same bits on every rank
+        B, H, D = case.q.shape
+        off, cnt = sharding.head_shard(H, ranks.world, ranks.rank)
+        q, k_new, v_new = (sharding.take_heads(t, off, cnt) for t in (case.q, case.k_new, case.v_new))
+        k_cache = sharding.take_heads(case.k_cache, off, cnt)
+        v_cache = sharding.take_heads(case.v_cache, off, cnt)
+        peers = sharding.PeerOutputs(B, H, D)
+        flags = torch.zeros(1, dtype=torch.int32, device=device)
+        max_len = case.max_seq_len
+        ws = torch.empty(binding.allgather_workspace_bytes(B, cnt, D, max_len), dtype=torch.uint8, device=device)
+
+        def step():
+            binding.kv_append(k_cache, v_cache, k_new, v_new, case.seq_lens, case.block_table, flags)
+            binding.decode_attention_allgather(peers.addresses, None, q, k_cache, v_cache, case.block_table,
+                                               case.seq_lens, off, H, max_len, case.scale, ws, flags)
+            peers.barrier()                        # every rank's rows have landed everywhere
+
+        for _ in range(5):
+            step()
+        torch.cuda.synchronize()
+        ranks.barrier()
+        a, z = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(steps):
+            step()
+        z.record()
+        torch.cuda.synchronize()
+        ranks.barrier()
+        seconds = a.elapsed_time(z) / 1e3
+        # rank 0 also runs all heads alone and compares its gathered buffer with that
+        error = None
+        if ranks.rank == 0:
+            out = torch.empty((B, H, D), dtype=torch.float16, device=device)
+            full_ws = binding.alloc_workspace(B, H, D, max_len, device)
+            binding.kv_append(case.k_cache, case.v_cache, case.k_new, case.v_new, case.seq_lens, case.block_table, flags)
+            binding.decode_attention_paged(out, None, case.q, case.k_cache, case.v_cache, case.block_table,
+                                           case.seq_lens, max_len, case.scale, full_ws, flags)
+            torch.cuda.synchronize()
+            error = float((out.float() - peers.local.float()).abs().max())
+        shard_bytes = case.kv_bytes_read * cnt / H
+        res = head_sharded_result(ranks, shard_bytes * steps / 1e9, seconds, cnt, H, error)
+        res["ms_per_step"] = res.pop("seconds") / steps * 1e3
+        res["status_flags"] = int(flags.item())
+        return res
+    except Exception as exc:                       # noqa: BLE001 - reported, never fatal
+        return {"error": f"{type(exc).__name__}: {exc}"[:400]}
+
+
 def run_case(spec: str, launches: int, device, sparse_path: int = 0) -> dict:
     """One small case of the sparse or the grouped entry point, `launches` calls back to back
     (what the ncu commands under profiles/ run)."""
@@ -805,6 +874,8 @@ def main(argv=None) -> int:
                          "algorithmic_bytes_per_launch": main_res["split_bytes"],
                          "avg_launch_ms": main_res["split_seconds"] * 1e3},
         }
+        if ranks.world > 1:
+            line["head_sharded"] = measure_head_sharded(ranks, device)
         if ranks.rank == 0 and ranks.world == 1 and args.cpu_seconds > 0:
             line["cpu_baseline"] = cpu_baseline(w, args.cpu_seconds, device)
         if not args.no_others and ranks.world == 1:

@@ -366,19 +366,6 @@ int instinfer_sparf_decode_attention(void *out, float *alpha, int32_t *selected,
 size_t instinfer_sparf_workspace_bytes(int32_t batch, int32_t heads, int32_t head_dim,
                                        int32_t max_seq_len, int32_t max_k);
 
-/*
- * Steps 1-7 of Algorithm 1 have two implementations: one thread block per (sequence, head)
- * that keeps the row's approximate logits in shared memory (rows of at most 16384 tokens), and
- * a chain of kernels for long rows that first brackets the k-th largest score on a sample of
- * the row and then keeps only the tokens that can still be selected (any length; rows it
- * cannot settle, e.g. thousands of equal scores, are redone by one block per row).  Both
- * compute the same fp32 scores and cut ties by position, so they select the same tokens.
- * The library picks by the sizes; instinfer_set_sparse_path forces the choice for later calls
- * of this process: 0 automatic, 1 the chain, 2 one block per row where the rows fit (a tuning
- * and test aid; returns INSTINFER_OK or INSTINFER_ERR_INVALID_ARG; not thread-safe against
- * concurrent calls).
- */
-int instinfer_set_sparse_path(int32_t path);
 
 /*
  * Workspace size (bytes, host computation only) for a call with these sizes under the
@@ -403,7 +390,31 @@ size_t instinfer_workspace_bytes(int32_t batch, int32_t heads, int32_t head_dim,
  */
 int32_t instinfer_plan_chunk_tokens(int32_t batch, int32_t heads, int32_t max_seq_len);
 int32_t instinfer_plan_num_splits(int32_t batch, int32_t heads, int32_t max_seq_len);
+
+/*
+ * ======================= Tuning, test and measurement aids =======================
+ * The three calls below set process-global state that later calls of the entry points above
+ * read.  They exist so that tests can drive every split plan and both forms of the sparse
+ * selection, and so that a benchmark can time one kernel where it runs; a serving process
+ * never needs them.  None is thread-safe against calls that run at the same time, and none
+ * changes a result beyond what its comment says.
+ */
 int instinfer_set_chunk_tokens(int32_t chunk_tokens);
+
+/*
+ * Steps 1-7 of Algorithm 1 have two implementations: one thread block per (sequence, head)
+ * that keeps the row's approximate logits in shared memory (rows of at most 16384 tokens), and
+ * a chain of kernels for long rows that first brackets the k-th largest score on a sample of
+ * the row and then keeps only the tokens that can still be selected (any length; rows it
+ * cannot settle, e.g. thousands of equal scores, are redone by one block per row).  Both
+ * compute the same fp32 scores and cut ties by position, so they select the same tokens.
+ * The library picks by the sizes; instinfer_set_sparse_path forces the choice for later calls
+ * of this process: 0 automatic, 1 the chain, 2 one block per row where the rows fit (a tuning
+ * and test aid; returns INSTINFER_OK or INSTINFER_ERR_INVALID_ARG; not thread-safe against
+ * concurrent calls).
+ */
+int instinfer_set_sparse_path(int32_t path);
+
 
 /*
  * Measurement aid (no counterpart in the paper).  Given two cudaEvent_t (as void*, owned by

@@ -16,8 +16,12 @@ ranks.barrier()
 units, seconds = (100.0, 2.0) if ranks.rank == 0 else (300.0, 4.0)     # rank 1 is the slow one
 value, job_seconds = bench.aggregate(ranks, units, seconds)
 total = ranks.sum(float(ranks.rank + 1))
+# the head-sharded section's aggregation: rank 0 owns 3 of 5 heads, rank 1 the other 2
+heads = 3 if ranks.rank == 0 else 2
+sharded = bench.head_sharded_result(ranks, 10.0 * heads, 1.0 + ranks.rank, heads, 5, 0.0 if ranks.rank == 0 else None)
 if ranks.rank == 0:
-    print(json.dumps({"value": value, "seconds": job_seconds, "world": ranks.world, "sum": total}))
+    print(json.dumps({"value": value, "seconds": job_seconds, "world": ranks.world, "sum": total,
+                      "sharded": sharded}))
 ranks.close()
 """
 
@@ -35,6 +39,9 @@ def test_two_gloo_ranks_aggregate_to_whole_job_throughput(tmp_path):
     assert got["world"] == 2 and got["sum"] == 3.0
     assert got["seconds"] == 4.0                       # the slowest rank sets the time
     assert got["value"] == (100.0 + 300.0) / 4.0       # all ranks' units over that time
+    sharded = got["sharded"]                           # one instance: all heads' bytes over the slowest rank
+    assert sharded["heads_covered"] == sharded["total_heads"] == 5 and sharded["scaling"] == "strong"
+    assert sharded["value"] == 50.0 / 2.0 and sharded["seconds"] == 2.0
 
 
 def test_reference_arm_only_rank_zero_prints(tmp_path):
