@@ -249,10 +249,13 @@ class Layer:
         self.host_out = torch.empty((B, H, D), dtype=torch.float16).pin_memory()
         self.chunk_tokens = binding.plan_chunk_tokens(B, H, self.max_len)
         self.n_splits = binding.plan_num_splits(B, H, self.max_len)
+        self.clustered = binding.plan_merges_in_cluster(B, H, self.max_len)
 
     @property
     def launches(self) -> int:
-        return 2 + (1 if self.n_splits > 1 else 0)
+        """append + split + merge; no merge kernel with a single chunk, nor for small problems,
+        where the chunks of a (sequence, head) merge inside the split kernel as a cluster."""
+        return 2 + (1 if self.n_splits > 1 and not self.clustered else 0)
 
     def run(self, flags):
         from paper_2409_04992_b200 import binding

@@ -390,6 +390,15 @@ size_t instinfer_workspace_bytes(int32_t batch, int32_t heads, int32_t head_dim,
  */
 int32_t instinfer_plan_chunk_tokens(int32_t batch, int32_t heads, int32_t max_seq_len);
 int32_t instinfer_plan_num_splits(int32_t batch, int32_t heads, int32_t max_seq_len);
+/*
+ * Small problems (at most 8 chunks of at most 512 tokens per sequence and about two waves of
+ * thread blocks in all) are bound by launch and memory latency: there the chunks of one
+ * (sequence, head) run as one thread-block cluster, leave their partials in shared memory and
+ * are merged inside the same kernel, so the call is one launch instead of two and the
+ * workspace is not touched.  Returns 1 if the single-GPU attention entry points would do
+ * that for these sizes under the current plan, else 0.
+ */
+int32_t instinfer_plan_merges_in_cluster(int32_t batch, int32_t heads, int32_t max_seq_len);
 
 /*
  * ======================= Tuning, test and measurement aids =======================

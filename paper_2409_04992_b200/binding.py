@@ -93,6 +93,8 @@ def load() -> ctypes.CDLL:
         lib.instinfer_plan_chunk_tokens.argtypes = [i32, i32, i32]
         lib.instinfer_plan_num_splits.restype = i32
         lib.instinfer_plan_num_splits.argtypes = [i32, i32, i32]
+        lib.instinfer_plan_merges_in_cluster.restype = i32
+        lib.instinfer_plan_merges_in_cluster.argtypes = [i32, i32, i32]
         lib.instinfer_set_chunk_tokens.restype = ctypes.c_int
         lib.instinfer_set_chunk_tokens.argtypes = [i32]
         lib.instinfer_set_timing_events.restype = ctypes.c_int
@@ -131,6 +133,10 @@ def plan_chunk_tokens(batch: int, heads: int, max_seq_len: int) -> int:
 
 def plan_num_splits(batch: int, heads: int, max_seq_len: int) -> int:
     return int(load().instinfer_plan_num_splits(batch, heads, max_seq_len))
+
+
+def plan_merges_in_cluster(batch: int, heads: int, max_seq_len: int) -> bool:
+    return bool(load().instinfer_plan_merges_in_cluster(batch, heads, max_seq_len))
 
 
 def set_chunk_tokens(chunk_tokens: int) -> None:

@@ -76,11 +76,42 @@ inline cudaError_t launch_overlapped(void (*kernel)(Params...), unsigned grid, u
     return err;
 }
 
+// The same with the grid cut into thread-block clusters of `cluster` consecutive blocks
+// (grid must be a multiple of it).  No fallback: a refused cluster launch is an error.
+template <typename... Params>
+inline cudaError_t launch_clustered(void (*kernel)(Params...), unsigned grid, unsigned cluster, unsigned block,
+                                    size_t smem, cudaStream_t stream, const Params &...params)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(block);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = cluster;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
+    cudaError_t err = cudaLaunchKernelEx(&cfg, kernel, params...);
+    if (err != cudaSuccess) {
+        (void)cudaGetLastError();
+        cfg.numAttrs = 1;                // without the programmatic overlap
+        err = cudaLaunchKernelEx(&cfg, kernel, params...);
+    }
+    return err;
+}
+
 struct SplitPlan {
     int32_t chunk_tokens;   // size of the n_big long chunks, which follow the short ones
     int32_t n_big;
     int32_t tail_chunk;     // size of the n_splits - n_big short chunks at the start of a sequence
     int32_t n_splits;
+    bool cluster;           // small problem: the chunks of a (sequence, head) form one thread-block
+                            // cluster that merges its partials itself (no merge kernel)
 };
 
 // Cuts are at fixed logical token positions, the same for every sequence, so a result never
@@ -96,12 +127,17 @@ struct PlanRules {
     int chunk_ceiling;
     int tail_chunk_tokens;       // 0: no short chunks at the end of long sequences
     int block_overhead_tokens;   // > 0: choose the chunk count by modelled time (see make_plan)
+    bool allow_cluster;          // the kernel has the cluster form for small problems
 };
-constexpr PlanRules kOneRowRules = {kCtasPerSm, kTargetWaves, kChunkCeiling, kTailChunk, 0};
+constexpr PlanRules kOneRowRules = {kCtasPerSm, kTargetWaves, kChunkCeiling, kTailChunk, 0, true};
+constexpr PlanRules kNoClusterRules = {kCtasPerSm, kTargetWaves, kChunkCeiling, kTailChunk, 0, false};
+constexpr int kClusterMaxChunks = 8;     // portable cluster size
+constexpr int kClusterMaxChunkTokens = 512;
 
 inline SplitPlan make_plan(int64_t pairs, int32_t max_seq_len, const PlanRules &rules = kOneRowRules)
 {
     SplitPlan plan;
+    plan.cluster = false;
     if (g_forced_chunk > 0) {               // uniform chunks, no short ones
         plan.chunk_tokens = plan.tail_chunk = g_forced_chunk;
         plan.n_big = (int32_t)ceil_div(max_seq_len, g_forced_chunk);
@@ -109,6 +145,18 @@ inline SplitPlan make_plan(int64_t pairs, int32_t max_seq_len, const PlanRules &
         return plan;
     }
     const int64_t slots = (int64_t)sm_count() * rules.ctas_per_sm;
+    if (rules.allow_cluster) {
+        // Small problems are bound by launch and memory latency, not by bandwidth: at most 8
+        // chunks per sequence, all resident at once, merged inside the kernel by a cluster.
+        const int64_t chunk = ceil_div(ceil_div(max_seq_len, kClusterMaxChunks), kChunkGranule) * kChunkGranule;
+        const int64_t n = ceil_div(max_seq_len, chunk);
+        if (n >= 2 && chunk <= kClusterMaxChunkTokens && pairs * n <= 2 * slots) {
+            plan.chunk_tokens = plan.tail_chunk = (int32_t)chunk;
+            plan.n_big = plan.n_splits = (int32_t)n;
+            plan.cluster = true;
+            return plan;
+        }
+    }
     const int64_t fewest = ceil_div(max_seq_len, rules.chunk_ceiling);
     // Small problems that cannot fill the GPU with kChunkFloor-token chunks are latency-bound:
     // cut them down to the granule so that more blocks share the work.

@@ -14,7 +14,7 @@ PlanRules grouped_rules(int32_t head_dim)
 {
     const int ctas = head_dim == 64 ? GroupedGeometry<64>::kCtasPerSm
                    : head_dim == 128 ? GroupedGeometry<128>::kCtasPerSm : GroupedGeometry<256>::kCtasPerSm;
-    return PlanRules{ctas, 2, 4096, 1024, 320};
+    return PlanRules{ctas, 2, 4096, 1024, 320, false};
 }
 
 size_t grouped_workspace_for(int64_t pairs, int32_t rows, int32_t head_dim, const SplitPlan &plan)

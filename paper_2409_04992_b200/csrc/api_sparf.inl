@@ -27,7 +27,7 @@ SparfLayout sparf_layout(int64_t pairs, int32_t max_seq_len, int32_t max_k)
     // candidates per row: the bracket of the sampled pre-pass holds a few per cent of the row
     int64_t cand = max_seq_len / 4;
     w.cand_capacity = (int32_t)(cand < 1024 ? 1024 : cand > kCandidates ? kCandidates : cand);
-    w.plan = make_plan(pairs, max_k);
+    w.plan = make_plan(pairs, max_k, kNoClusterRules);       // the row-list kernel has no cluster form
     w.scores = 0;
     w.stage_pos = w.scores + round256((size_t)pairs * w.score_stride * sizeof(float));
     w.row_ids = w.stage_pos + round256((size_t)pairs * w.score_stride * sizeof(int32_t));

@@ -25,9 +25,14 @@
 //   * rows come from a contiguous cache, from paged pools through the block table, or from
 //     a list of selected rows (the sparse path);
 //   * the 4 warp states of a block are merged once at the end of the chunk; chunk partials
-//     go to the workspace and a small second kernel merges them.
+//     go to the workspace and a small second kernel merges them.  Small problems (at most 8
+//     chunks per sequence, about one wave of blocks) skip both: the chunks of a (sequence,
+//     head) form one thread-block cluster, each block leaves its partial in its own shared
+//     memory, and after a cluster barrier the first block merges them through distributed
+//     shared memory and writes the row -- one launch less and no round trip through HBM.
 #pragma once
 
+#include <cooperative_groups.h>
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -341,10 +346,13 @@ __device__ __forceinline__ void attend_tile(unsigned k_row, const unsigned (&k_p
     }
 }
 
-template <Rows kRows>
+// kCluster: the grid is pair-major and launched with clusters of n_splits blocks (the chunks of
+// one (sequence, head)); the merge happens inside the kernel (see the file header).
+template <Rows kRows, bool kCluster = false>
 __global__ void __launch_bounds__(kThreads, kCtasPerSm)
 decode_attn_split_kernel(const AttnParams p)
 {
+    static_assert(!(kCluster && kRows == Rows::kGathered), "row lists use the two-kernel form");
     constexpr bool kPaged = kRows == Rows::kPaged;
     constexpr bool kGathered = kRows == Rows::kGathered;
     constexpr bool kBulk = !kGathered;                   // whole tiles by one bulk copy each
@@ -359,11 +367,11 @@ decode_attn_split_kernel(const AttnParams p)
     // Grid order: chunk slowest (long chunks first, short ones last), then sequence, head
     // fastest.  Blocks that run together then cover all heads of a few sequences (one paged
     // block's heads are adjacent in memory).
-    const int order = blockIdx.x / p.pairs;
-    const int pair = blockIdx.x - order * p.pairs;
-    const int split = scheduled_chunk(p, order);
+    const int order = kCluster ? (int)(blockIdx.x % p.n_splits) : (int)(blockIdx.x / p.pairs);
+    const int pair = kCluster ? (int)(blockIdx.x / p.n_splits) : (int)(blockIdx.x - order * p.pairs);
+    const int split = kCluster ? order : scheduled_chunk(p, order);      // cluster rank = chunk in position order
     const int b = pair / p.heads, h = pair - b * p.heads;
-    const bool final_writer = !kGathered && p.n_splits == 1;
+    const bool final_writer = !kGathered && !kCluster && p.n_splits == 1;
     // one mbarrier per stage, behind the rings: a stage's bulk copies report their bytes to it
     const unsigned bars = static_cast<unsigned>(__cvta_generic_to_shared(smem)) + kRingBytes + warp * (kStages * 8);
     if (kBulk && lane == 0) {                            // each warp owns the barriers of its ring
@@ -375,11 +383,13 @@ decode_attn_split_kernel(const AttnParams p)
     wait_for_previous_kernels();
 
     // With several splits the merge kernel reports a bad length; here only the lone writer does.
-    int len = checked_seq_len(p, b, threadIdx.x == 0 && h == 0 && final_writer);
+    // (the block that writes the final rows reports a bad length: the lone writer, or the
+    // first block of a cluster)
+    int len = checked_seq_len(p, b, threadIdx.x == 0 && h == 0 && (final_writer || (kCluster && split == 0)));
     if (kGathered) len = gathered_count(p, b, len);           // rows in this pair's list
     int begin, chunk_size;
     chunk_range(p, split, begin, chunk_size);
-    if (begin >= len) {
+    if (!kCluster && begin >= len) {
         if (final_writer) {            // inactive slot: zero output, lse = -inf
             p.out[(int64_t)pair * kHeadDim + threadIdx.x] = __float2half_rn(0.f);
             if (p.lse && threadIdx.x == 0) p.lse[pair] = -INFINITY;
@@ -387,11 +397,11 @@ decode_attn_split_kernel(const AttnParams p)
         return;
     }
     const int end = min(begin + chunk_size, len);
-    const int n_tiles = (end - begin + kTileRows - 1) / kTileRows;
+    const int n_tiles = end > begin ? (end - begin + kTileRows - 1) / kTileRows : 0;   // 0: an empty chunk of a cluster
     const int my_tiles = warp < n_tiles ? (n_tiles - warp + kWarps - 1) / kWarps : 0;
     // Only the chunk's very last tile can be ragged; it belongs to exactly one warp.
-    const int last_rows = warp == (n_tiles - 1) % kWarps ? (end - begin) - (n_tiles - 1) * kTileRows
-                                                         : kTileRows;
+    const int last_rows = n_tiles > 0 && warp == (n_tiles - 1) % kWarps ? (end - begin) - (n_tiles - 1) * kTileRows
+                                                                        : kTileRows;
 
     // This lane's 32 query dims, kept in fp16 (16 registers): products with fp16 keys are
     // exact in fp32 and the scale is applied to the finished dot product.  In step i the lane
@@ -625,7 +635,43 @@ decode_attn_split_kernel(const AttnParams p)
         o = fmaf(w, sm_acc[i * kHeadDim + threadIdx.x], o);
     }
     o /= total * kWeightScale;
-    const float lse2 = top + log2f(total);
+    float lse2 = top + log2f(total);
+    if (kCluster) {
+        // This chunk's partial stays in this block's shared memory (behind the fold's scratch);
+        // block 0 of the cluster merges all of them in position order, exactly as
+        // lse_merge_kernel would, and writes the row.  Every block stays until that is done.
+        namespace cg = cooperative_groups;
+        cg::cluster_group cluster = cg::this_cluster();
+        float *mine = reinterpret_cast<float *>(smem) + kWarps * (kHeadDim + 2);       // [kHeadDim] + lse
+        if (n_tiles == 0) {              // empty chunk: nothing to contribute (total is 0 here)
+            o = 0.f;
+            lse2 = -INFINITY;
+        }
+        mine[threadIdx.x] = o;
+        if (threadIdx.x == 0) mine[kHeadDim] = lse2;
+        cluster.sync();
+        if (split == 0) {
+            const int live = live_chunks(p, len);
+            if (live == 0) {
+                p.out[(int64_t)pair * kHeadDim + threadIdx.x] = __float2half_rn(0.f);
+                if (p.lse && threadIdx.x == 0) p.lse[pair] = -INFINITY;
+            } else {
+                float best = kMinusHuge;
+                for (int s = 0; s < live; ++s) best = fmaxf(best, cluster.map_shared_rank(mine, s)[kHeadDim]);
+                float weight_sum = 0.f, merged = 0.f;
+                for (int s = 0; s < live; ++s) {
+                    const float *theirs = cluster.map_shared_rank(mine, s);
+                    const float w = fast_exp2(theirs[kHeadDim] - best);
+                    weight_sum += w;
+                    merged = fmaf(w, theirs[threadIdx.x], merged);
+                }
+                p.out[(int64_t)pair * kHeadDim + threadIdx.x] = __float2half_rn(merged / weight_sum);
+                if (p.lse && threadIdx.x == 0) p.lse[pair] = (best + log2f(weight_sum)) * kLn2;
+            }
+        }
+        cluster.sync();                  // no block's shared memory goes away while block 0 reads it
+        return;
+    }
     if (final_writer) {
         p.out[(int64_t)pair * kHeadDim + threadIdx.x] = __float2half_rn(o);
         if (p.lse && threadIdx.x == 0) p.lse[pair] = lse2 * kLn2;

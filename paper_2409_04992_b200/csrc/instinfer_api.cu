@@ -12,22 +12,23 @@ namespace {
 using namespace instinfer;
 using namespace instinfer::api;
 
-int ensure_split_smem(bool paged)
+// Shared-memory opt-in of the split kernels, once per device: [paged][cluster form].
+int ensure_split_smem(bool paged, bool cluster)
 {
-    static bool done[kMaxDevices][2] = {};
+    static bool done[kMaxDevices][2][2] = {};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return INSTINFER_ERR_CUDA;
-    if (!done[dev][paged]) {
-        const cudaError_t err = paged
-            ? cudaFuncSetAttribute(decode_attn_split_kernel<Rows::kPaged>,
-                                   cudaFuncAttributeMaxDynamicSharedMemorySize, kSplitSmemBytes)
-            : cudaFuncSetAttribute(decode_attn_split_kernel<Rows::kContiguous>,
-                                   cudaFuncAttributeMaxDynamicSharedMemorySize, kSplitSmemBytes);
-        if (err != cudaSuccess) {
+    if (!done[dev][paged][cluster]) {
+        const void *kernel = cluster
+            ? (paged ? (const void *)decode_attn_split_kernel<Rows::kPaged, true>
+                     : (const void *)decode_attn_split_kernel<Rows::kContiguous, true>)
+            : (paged ? (const void *)decode_attn_split_kernel<Rows::kPaged, false>
+                     : (const void *)decode_attn_split_kernel<Rows::kContiguous, false>);
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSplitSmemBytes) != cudaSuccess) {
             (void)cudaGetLastError();
             return INSTINFER_ERR_CUDA;
         }
-        done[dev][paged] = true;
+        done[dev][paged][cluster] = true;
     }
     return INSTINFER_OK;
 }
@@ -43,7 +44,10 @@ int launch_attention(AttnParams p, bool paged, int32_t batch, void *workspace,
                      const GatherTargets *gather = nullptr)
 {
     const int64_t pairs = (int64_t)batch * p.heads;
-    const SplitPlan plan = make_plan(pairs, p.max_seq_len);
+    // The head-sharded path ends in its own merge-and-gather kernel: it takes the same chunks
+    // (so its rows equal the single-GPU ones bit for bit) but never the cluster form.
+    SplitPlan plan = make_plan(pairs, p.max_seq_len);
+    if (gather) plan.cluster = false;
     const size_t partial_bytes = workspace_for(pairs, plan);
     if (workspace == nullptr || !aligned16(workspace) ||
         workspace_bytes < partial_bytes + (gather ? staging_for(pairs) : 0))
@@ -63,22 +67,24 @@ int launch_attention(AttnParams p, bool paged, int32_t batch, void *workspace,
         targets.staged = p.out;
     }
 
-    const int rc = ensure_split_smem(paged);
+    const int rc = ensure_split_smem(paged, plan.cluster);
     if (rc != INSTINFER_OK) return rc;
     const unsigned grid = (unsigned)(pairs * plan.n_splits);
     if (g_before_split) cudaEventRecord(g_before_split, stream);
     const bool timed = g_before_split != nullptr;          // event records break the overlap anyway
     cudaError_t err;
-    if (paged)
-        err = launch_overlapped(decode_attn_split_kernel<Rows::kPaged>, grid, kThreads, kSplitSmemBytes, stream, p);
+    if (plan.cluster)                  // pair-major grid, the chunks of a pair form a cluster and merge themselves
+        err = paged ? launch_clustered(decode_attn_split_kernel<Rows::kPaged, true>, grid, (unsigned)plan.n_splits, kThreads, kSplitSmemBytes, stream, p)
+                    : launch_clustered(decode_attn_split_kernel<Rows::kContiguous, true>, grid, (unsigned)plan.n_splits, kThreads, kSplitSmemBytes, stream, p);
     else
-        err = launch_overlapped(decode_attn_split_kernel<Rows::kContiguous>, grid, kThreads, kSplitSmemBytes, stream, p);
+        err = paged ? launch_overlapped(decode_attn_split_kernel<Rows::kPaged, false>, grid, kThreads, kSplitSmemBytes, stream, p)
+                    : launch_overlapped(decode_attn_split_kernel<Rows::kContiguous, false>, grid, kThreads, kSplitSmemBytes, stream, p);
     if (timed) cudaEventRecord(g_after_split, stream);
     if (err != cudaSuccess || cudaGetLastError() != cudaSuccess) return INSTINFER_ERR_CUDA;
     if (gather) {
         err = launch_overlapped(lse_merge_allgather_kernel, (unsigned)pairs, kHeadDim, 0, stream, p, targets);
         if (err != cudaSuccess || cudaGetLastError() != cudaSuccess) return INSTINFER_ERR_CUDA;
-    } else if (plan.n_splits > 1) {
+    } else if (plan.n_splits > 1 && !plan.cluster) {
         err = launch_overlapped(lse_merge_kernel, (unsigned)pairs, kHeadDim, 0, stream, p);
         if (err != cudaSuccess || cudaGetLastError() != cudaSuccess) return INSTINFER_ERR_CUDA;
     }
@@ -448,6 +454,12 @@ int32_t instinfer_plan_num_splits(int32_t batch, int32_t heads, int32_t max_seq_
 {
     if (!sizes_ok(batch, heads, max_seq_len) || batch == 0) return 0;
     return make_plan((int64_t)batch * heads, max_seq_len).n_splits;
+}
+
+int32_t instinfer_plan_merges_in_cluster(int32_t batch, int32_t heads, int32_t max_seq_len)
+{
+    if (!sizes_ok(batch, heads, max_seq_len) || batch == 0) return 0;
+    return make_plan((int64_t)batch * heads, max_seq_len).cluster ? 1 : 0;
 }
 
 int instinfer_set_chunk_tokens(int32_t chunk_tokens)
