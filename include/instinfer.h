@@ -424,6 +424,19 @@ int instinfer_set_chunk_tokens(int32_t chunk_tokens);
  */
 int instinfer_set_sparse_path(int32_t path);
 
+/*
+ * instinfer_decode_attention_grouped has two implementations of the same arithmetic: warp-level
+ * tensor-core MMAs (every head size and block size the entry point takes) and, for head size
+ * 128 with a contiguous cache or 16, 32 or 64 tokens per block, asynchronous tcgen05 MMAs that
+ * take 128-token tiles as the long side, with accumulators in tensor memory and tiles moved by
+ * tensor-map copies.  The library picks the second where the shape allows;
+ * instinfer_set_grouped_path forces the choice for later calls of this process: 0 automatic,
+ * 1 warp-level, 2 tcgen05 where the shape allows (a tuning and test aid; returns INSTINFER_OK
+ * or INSTINFER_ERR_INVALID_ARG; not thread-safe against concurrent calls).  Both meet the
+ * entry point's tolerances; their results are not bit-identical to each other.
+ */
+int instinfer_set_grouped_path(int32_t path);
+
 
 /*
  * Measurement aid (no counterpart in the paper).  Given two cudaEvent_t (as void*, owned by

@@ -85,6 +85,8 @@ def load() -> ctypes.CDLL:
                                                          i32, i32, i32, i32, f32, ptr, sz, ptr, ptr]
         lib.instinfer_set_sparse_path.restype = ctypes.c_int
         lib.instinfer_set_sparse_path.argtypes = [i32]
+        lib.instinfer_set_grouped_path.restype = ctypes.c_int
+        lib.instinfer_set_grouped_path.argtypes = [i32]
         lib.instinfer_sparf_workspace_bytes.restype = sz
         lib.instinfer_sparf_workspace_bytes.argtypes = [i32, i32, i32, i32, i32]
         lib.instinfer_workspace_bytes.restype = sz
@@ -342,6 +344,11 @@ def sparf_append_bulk(k_pool: torch.Tensor, v_pool: torch.Tensor, kt_pool: torch
         _ptr(seq_lens), _ptr(new_lens), _ptr(block_table), block_table.shape[1], k_pool.shape[2],
         k_pool.shape[0], _ptr(kt_block_table), kt_block_table.shape[1], kt_pool.shape[3],
         kt_pool.shape[0], batch, max_new, heads, head_dim, _ptr(status_flags), _stream(stream)))
+
+
+def set_grouped_path(path: int) -> None:
+    """instinfer_set_grouped_path: 0 automatic, 1 warp-level MMAs, 2 tcgen05 where the shape allows."""
+    _check(load().instinfer_set_grouped_path(int(path)))
 
 
 def set_sparse_path(path: int) -> None:

@@ -1,9 +1,11 @@
 // C ABI, grouped-head / multi-token / other-head-size attention: checks, plan and launches.
 // Included by instinfer_api.cu (one translation unit: the kernels' headers define
 // non-template kernels, which must not be compiled twice).
-#include "grouped_attention_kernels.cuh"
+#include "grouped_umma_kernels.cuh"
 
 namespace {
+
+int g_grouped_path = 0;     // 0 automatic, 1 warp-level MMAs, 2 tcgen05 where the shape allows (see instinfer_set_grouped_path)
 
 // The grouped kernel's blocks are heavier (query fragments to load, 16 rows to merge at the
 // end: about the cost of 20 tiles) and its warps are latency-bound, so a launch takes whole
@@ -43,6 +45,73 @@ int launch_grouped(const GroupedParams &p, unsigned grid, cudaStream_t stream)
     if (err != cudaSuccess || cudaGetLastError() != cudaSuccess) return INSTINFER_ERR_CUDA;
     if (p.a.n_splits > 1) {
         err = launch_overlapped(grouped_merge_kernel<D>, (unsigned)(p.a.pairs * p.rows), D, 0, stream, p);
+        if (err != cudaSuccess || cudaGetLastError() != cudaSuccess) return INSTINFER_ERR_CUDA;
+    }
+    return INSTINFER_OK;
+}
+
+// ---- the tcgen05 form (head size 128; contiguous, or paged with 16, 32 or 64 tokens per block) ----
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// The driver's tensor-map encoder, looked up through the runtime (the library does not link libcuda).
+EncodeTiledFn tensor_map_encoder()
+{
+    static EncodeTiledFn fn = [] {
+        void *f = nullptr;
+        cudaDriverEntryPointQueryResult found = cudaDriverEntryPointSymbolNotFound;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &found) != cudaSuccess ||
+            found != cudaDriverEntryPointSuccess) {
+            (void)cudaGetLastError();
+            f = nullptr;
+        }
+        return reinterpret_cast<EncodeTiledFn>(f);
+    }();
+    return fn;
+}
+
+// A K or V cache as a 2-D fp16 tensor [rows][128] (a row is one token of one head, 256 bytes);
+// a box is 64 dims (128 bytes, the swizzle span) by `box_rows` tokens.
+bool make_cache_map(CUtensorMap *map, const void *cache, int64_t rows, int32_t box_rows)
+{
+    EncodeTiledFn encode = tensor_map_encoder();
+    if (encode == nullptr || rows <= 0 || rows >= ((int64_t)1 << 31)) return false;
+    const cuuint64_t dims[2] = {128, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {256};
+    const cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
+    const cuuint32_t elem[2] = {1, 1};
+    return encode(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void *>(cache), dims, strides, box, elem,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+bool umma_shape(int32_t head_dim, bool paged, int32_t block_tokens)
+{
+    return head_dim == 128 && (!paged || block_tokens == 16 || block_tokens == 32 || block_tokens == 64);
+}
+
+template <bool kPaged>
+int launch_grouped_umma(const GroupedParams &p, const CUtensorMap &map_k, const CUtensorMap &map_v, unsigned grid,
+                        cudaStream_t stream)
+{
+    static bool done[kMaxDevices] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return INSTINFER_ERR_CUDA;
+    if (!done[dev]) {
+        if (cudaFuncSetAttribute(grouped_attn_umma_kernel<kPaged>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 kUmmaSmemBytes) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return INSTINFER_ERR_CUDA;
+        }
+        done[dev] = true;
+    }
+    cudaError_t err = launch_overlapped(grouped_attn_umma_kernel<kPaged>, grid, kUmmaThreads, kUmmaSmemBytes, stream,
+                                        p, map_k, map_v);
+    if (err != cudaSuccess || cudaGetLastError() != cudaSuccess) return INSTINFER_ERR_CUDA;
+    if (p.a.n_splits > 1) {
+        err = launch_overlapped(grouped_merge_kernel<128>, (unsigned)(p.a.pairs * p.rows), 128, 0, stream, p);
         if (err != cudaSuccess || cudaGetLastError() != cudaSuccess) return INSTINFER_ERR_CUDA;
     }
     return INSTINFER_OK;
@@ -127,6 +196,16 @@ int instinfer_decode_attention_grouped(void *out, float *lse, const void *q, con
 
     const unsigned grid = (unsigned)(pairs * plan.n_splits);
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (g_grouped_path == 2 && umma_shape(head_dim, paged, block_tokens)) {     // automatic: warp-level, for now
+        // The cache as the copy engine sees it; a cache of 2^31 rows or more, or a driver
+        // without the encoder, takes the warp-level form below.
+        const int64_t rows = p.a.kv_bytes / (2 * 128);
+        CUtensorMap map_k, map_v;
+        if (make_cache_map(&map_k, k_cache, rows, paged ? block_tokens : kUmmaTile) &&
+            make_cache_map(&map_v, v_cache, rows, paged ? block_tokens : kUmmaTile))
+            return paged ? launch_grouped_umma<true>(p, map_k, map_v, grid, stream)
+                         : launch_grouped_umma<false>(p, map_k, map_v, grid, stream);
+    }
     switch (head_dim) {
     case 64: return paged ? launch_grouped<64, true>(p, grid, stream) : launch_grouped<64, false>(p, grid, stream);
     case 128: return paged ? launch_grouped<128, true>(p, grid, stream) : launch_grouped<128, false>(p, grid, stream);
@@ -142,6 +221,13 @@ size_t instinfer_grouped_workspace_bytes(int32_t batch, int32_t q_tokens, int32_
     if (pairs == 0) return 256;
     return grouped_workspace_for(pairs, q_heads / kv_heads * q_tokens, head_dim,
                                  make_plan(pairs, max_seq_len, grouped_rules(head_dim)));
+}
+
+int instinfer_set_grouped_path(int32_t path)
+{
+    if (path < 0 || path > 2) return INSTINFER_ERR_INVALID_ARG;
+    g_grouped_path = path;
+    return INSTINFER_OK;
 }
 
 }  // extern "C"

@@ -134,6 +134,8 @@ int main(void)
     /* knobs */
     expect("chunk override granule", instinfer_set_chunk_tokens(100), INSTINFER_ERR_INVALID_ARG);
     expect("sparse path range", instinfer_set_sparse_path(3), INSTINFER_ERR_INVALID_ARG);
+    expect("grouped path range", instinfer_set_grouped_path(3), INSTINFER_ERR_INVALID_ARG);
+    expect("grouped path automatic", instinfer_set_grouped_path(0), INSTINFER_OK);
     expect("timing events one null", instinfer_set_timing_events(fake, NULL), INSTINFER_ERR_INVALID_ARG);
     expect("timing events off", instinfer_set_timing_events(NULL, NULL), INSTINFER_OK);
     if (strcmp(instinfer_status_string(INSTINFER_OK), "ok") != 0) {

@@ -227,6 +227,13 @@ def test_sparse_path_knob(lib):
         binding.set_sparse_path(3)
 
 
+def test_grouped_path_knob(lib):
+    for path in (0, 1, 2, 0):
+        binding.set_grouped_path(path)
+    with pytest.raises(binding.InstInferError):
+        binding.set_grouped_path(3)
+
+
 def test_missing_library_fails_loudly(monkeypatch, tmp_path):
     monkeypatch.setattr(binding, "_lib", None)
     monkeypatch.setattr(binding, "LIBRARY", tmp_path / "libinstinfer.so")

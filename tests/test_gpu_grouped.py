@@ -15,6 +15,15 @@ pytestmark = pytest.mark.gpu
 RAGGED = [1, 2, 15, 16, 17, 31, 33, 64, 65, 100, 257, 0, 511, 640, 3, 1100]
 
 
+@pytest.fixture(autouse=True, params=[1, 2], ids=["warp-mma", "tcgen05"])
+def grouped_path(request):
+    """Every test runs on both implementations (shapes the tcgen05 form does not take fall back
+    to the warp-level one inside the library)."""
+    binding.set_grouped_path(request.param)
+    yield request.param
+    binding.set_grouped_path(0)
+
+
 def make(layout, tokens, kv_heads, q_tokens, q_heads, dim=128, lens=RAGGED, index=5):
     w = wl.Workload("grouped", index, batch=len(lens), len_lo=min(lens), len_hi=max(lens),
                     layout=layout, s_max=max(lens) if layout == "contiguous" else 0,
