@@ -69,6 +69,8 @@ def parse_args(argv=None):
     ap.add_argument("--launches", type=int, default=2, help="calls made by --case")
     ap.add_argument("--sparse-path", type=int, default=0,
                     help="--case sparse: 0 automatic, 1 staged chain, 2 one block per row")
+    ap.add_argument("--grouped-path", type=int, default=0,
+                    help="grouped entry point: 0 automatic, 1 warp-level MMAs, 2 tcgen05 where the shape allows")
     return ap.parse_args(argv)
 
 
@@ -763,12 +765,13 @@ def measure_head_sharded(ranks: Ranks, device, steps: int = 20) -> dict:
         return {"error": f"{type(exc).__name__}: {exc}"[:400]}
 
 
-def run_case(spec: str, launches: int, device, sparse_path: int = 0) -> dict:
+def run_case(spec: str, launches: int, device, sparse_path: int = 0, grouped_path: int = 0) -> dict:
     """One small case of the sparse or the grouped entry point, `launches` calls back to back
     (what the ncu commands under profiles/ run)."""
     from paper_2409_04992_b200 import binding
     kind, _, rest = spec.partition(":")
     binding.set_sparse_path(sparse_path)
+    binding.set_grouped_path(grouped_path)
     flags = torch.zeros(1, dtype=torch.int32, device=device)
     a, z = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     if kind == "sparse":
@@ -838,7 +841,7 @@ def main(argv=None) -> int:
         torch.cuda.set_device(device)
         if args.case:
             if ranks.rank == 0:
-                print(json.dumps(run_case(args.case, args.launches, device, args.sparse_path)), flush=True)
+                print(json.dumps(run_case(args.case, args.launches, device, args.sparse_path, args.grouped_path)), flush=True)
             return 0
         w = wl.by_name(args.workload)
         if args.layers > 0:

@@ -92,9 +92,24 @@ bool umma_shape(int32_t head_dim, bool paged, int32_t block_tokens)
     return head_dim == 128 && (!paged || block_tokens == 16 || block_tokens == 32 || block_tokens == 64);
 }
 
+// The query tensor [B, Tq, Hq, 128] as the copy engine sees it: a box is 64 dims of the `group`
+// heads of one KV head for all Tq new tokens, i.e. the chunk's rows t * group + g in order.
+bool make_query_map(CUtensorMap *map, const void *q, int32_t batch, int32_t q_tokens, int32_t q_heads, int32_t group)
+{
+    EncodeTiledFn encode = tensor_map_encoder();
+    if (encode == nullptr) return false;
+    const cuuint64_t dims[4] = {128, (cuuint64_t)q_heads, (cuuint64_t)q_tokens, (cuuint64_t)batch};
+    const cuuint64_t strides[3] = {256, (cuuint64_t)q_heads * 256, (cuuint64_t)q_tokens * q_heads * 256};
+    const cuuint32_t box[4] = {64, (cuuint32_t)group, (cuuint32_t)q_tokens, 1};
+    const cuuint32_t elem[4] = {1, 1, 1, 1};
+    return encode(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 4, const_cast<void *>(q), dims, strides, box, elem,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 template <bool kPaged>
-int launch_grouped_umma(const GroupedParams &p, const CUtensorMap &map_k, const CUtensorMap &map_v, unsigned grid,
-                        cudaStream_t stream)
+int launch_grouped_umma(const GroupedParams &p, unsigned *ticket, const CUtensorMap &map_q, const CUtensorMap &map_k,
+                        const CUtensorMap &map_v, cudaStream_t stream)
 {
     static bool done[kMaxDevices] = {};
     int dev = 0;
@@ -107,8 +122,15 @@ int launch_grouped_umma(const GroupedParams &p, const CUtensorMap &map_k, const 
         }
         done[dev] = true;
     }
+    // One block per SM draws chunks from the ticket counter, which starts at zero.
+    if (cudaMemsetAsync(ticket, 0, sizeof(unsigned), stream) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return INSTINFER_ERR_CUDA;
+    }
+    const int64_t chunks = (int64_t)p.a.pairs * p.a.n_splits;
+    const unsigned grid = (unsigned)(chunks < sm_count() ? chunks : sm_count());
     cudaError_t err = launch_overlapped(grouped_attn_umma_kernel<kPaged>, grid, kUmmaThreads, kUmmaSmemBytes, stream,
-                                        p, map_k, map_v);
+                                        p, ticket, map_q, map_k, map_v);
     if (err != cudaSuccess || cudaGetLastError() != cudaSuccess) return INSTINFER_ERR_CUDA;
     if (p.a.n_splits > 1) {
         err = launch_overlapped(grouped_merge_kernel<128>, (unsigned)(p.a.pairs * p.rows), 128, 0, stream, p);
@@ -200,11 +222,15 @@ int instinfer_decode_attention_grouped(void *out, float *lse, const void *q, con
         // The cache as the copy engine sees it; a cache of 2^31 rows or more, or a driver
         // without the encoder, takes the warp-level form below.
         const int64_t rows = p.a.kv_bytes / (2 * 128);
-        CUtensorMap map_k, map_v;
-        if (make_cache_map(&map_k, k_cache, rows, paged ? block_tokens : kUmmaTile) &&
+        CUtensorMap map_q, map_k, map_v;
+        // the ticket counter sits in the last 256 bytes of the workspace, behind the partials
+        unsigned *ticket = reinterpret_cast<unsigned *>(
+            static_cast<unsigned char *>(workspace) + grouped_workspace_for(pairs, p.rows, head_dim, plan) - 256);
+        if (make_query_map(&map_q, q, batch, q_tokens, q_heads, p.group) &&
+            make_cache_map(&map_k, k_cache, rows, paged ? block_tokens : kUmmaTile) &&
             make_cache_map(&map_v, v_cache, rows, paged ? block_tokens : kUmmaTile))
-            return paged ? launch_grouped_umma<true>(p, map_k, map_v, grid, stream)
-                         : launch_grouped_umma<false>(p, map_k, map_v, grid, stream);
+            return paged ? launch_grouped_umma<true>(p, ticket, map_q, map_k, map_v, stream)
+                         : launch_grouped_umma<false>(p, ticket, map_q, map_k, map_v, stream);
     }
     switch (head_dim) {
     case 64: return paged ? launch_grouped<64, true>(p, grid, stream) : launch_grouped<64, false>(p, grid, stream);

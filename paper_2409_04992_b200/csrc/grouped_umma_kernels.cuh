@@ -11,12 +11,15 @@
 // where the 32 columns of P^T are the fp16 high and low parts of the 16 rows' softmax weights
 // (so that the result keeps fp32-level accuracy), added up in the epilogue.
 //
-// A block owns one chunk of token positions of one (sequence, KV head) and is specialised by
-// warp:
+// The kernel is persistent: one block per SM draws chunks (token ranges of one (sequence, KV
+// head), the same list one block per chunk would run) from a ticket counter, and its copy
+// pipeline runs on across chunk boundaries.  A block is specialised by warp:
 //   * warp 4 (producer) moves 128-token tiles of K and of V with tensor-map copies
 //     (cp.async.bulk.tensor, 128-byte swizzle, this GPU's memory, no multicast) into a ring of
 //     32 KiB slots; a paged tile is 128 / T copies of one (block, head) run each, the block
-//     ids read one tile ahead; a block with a bad id is not fetched but zero-filled;
+//     ids read one tile ahead; a block with a bad id is not fetched but zero-filled.  It also
+//     draws the tickets (one chunk ahead), announces each chunk to the other warps through a
+//     small queue in shared memory and fetches the chunk's query rows;
 //   * one lane of warp 5 issues the MMAs: K tile (K-major, as it lies in the cache) against the
 //     query rows held in shared memory -> logits in tensor memory (two buffers, so the next
 //     tile's logits are computed while this tile's are being exponentiated); V tile (the same
@@ -43,28 +46,65 @@ namespace instinfer {
 constexpr int kUmmaTile = 128;                         // tokens per tile
 constexpr int kUmmaPanelBytes = kUmmaTile * 128;       // 64 dims of 128 tokens (rows of 128 bytes)
 constexpr int kUmmaItemBytes = 2 * kUmmaPanelBytes;    // a K tile, or a V tile: 32 KiB
-constexpr int kUmmaSlots = 3;
-constexpr int kUmmaQBytes = kGroupRows * 256;          // 16 query rows, core-matrix order
+constexpr int kUmmaKSlots = 3;                         // ring depth of K tiles
+constexpr int kUmmaVSlots = 3;                         // ring depth of V tiles
+constexpr int kUmmaQBytes = kGroupRows * 256;          // 16 query rows as two 64-dim panels
+constexpr int kUmmaQBuffers = 2;                       // the next chunk's query rows arrive early
 constexpr int kUmmaPBytes = 32 * kUmmaTile * 2;        // 32 weight columns of 128 tokens
-constexpr int kUmmaMiscBytes = 1024;                   // barriers, tensor-memory address, reductions
-constexpr int kUmmaCarveBytes = kUmmaSlots * kUmmaItemBytes + kUmmaQBytes + kUmmaPBytes + kUmmaMiscBytes;
+constexpr int kUmmaMiscBytes = 2048;                   // barriers, work queue, tensor-memory address, reductions
+constexpr int kUmmaCarveBytes = (kUmmaKSlots + kUmmaVSlots) * kUmmaItemBytes + kUmmaQBuffers * kUmmaQBytes + kUmmaPBytes + kUmmaMiscBytes;
 constexpr int kUmmaSmemBytes = kUmmaCarveBytes + 1024; // room to align the ring to 1024 bytes
-constexpr int kUmmaThreads = 192;                      // 4 softmax warps, producer warp, MMA warp
-constexpr int kUmmaCtasPerSm = 2;
-constexpr int kUmmaTmemCols = 64;                      // 2 x 16 logits, 32 output accumulator
+constexpr int kUmmaThreads = 256;                      // 4 softmax warps, K and V producers, logit and output MMA issuers
+constexpr int kUmmaWarpK = 4, kUmmaWarpV = 5, kUmmaWarpLogits = 6, kUmmaWarpOutput = 7;
+constexpr int kUmmaTmemCols = 128;                     // 2 x 16 logits, 2 x 32 output accumulator (96 used)
+constexpr int kUmmaQueue = 4;                          // chunks the producer may be ahead of the consumers
 
 // offsets inside the misc region
-constexpr int kUmmaBarFull = 0;        // [kUmmaSlots] tile landed
-constexpr int kUmmaBarEmpty = 24;      // [kUmmaSlots] the MMAs that read the slot are complete
-constexpr int kUmmaBarSFull = 48;      // [2] logits of a tile are in tensor memory
-constexpr int kUmmaBarSFree = 64;      // [2] the softmax warps have read them
-constexpr int kUmmaBarPFull = 80;      // weights of a tile are in shared memory
-constexpr int kUmmaBarPvDone = 88;     // the second MMA of a tile is complete
-constexpr int kUmmaTmemPtr = 96;
-constexpr int kUmmaAbort = 100;        // set by a softmax thread whose wait ran out
-constexpr int kUmmaRed = 128;          // [4][16] floats: per-warp row maxima, later row sums
+constexpr int kUmmaBarKFull = 0;       // [kUmmaKSlots] K tile landed
+constexpr int kUmmaBarKEmpty = 24;     // [kUmmaKSlots] the logit MMAs that read the slot are complete
+constexpr int kUmmaBarVFull = 48;      // [kUmmaVSlots] V tile landed
+constexpr int kUmmaBarVEmpty = 72;     // [kUmmaVSlots] the output MMAs that read the slot are complete
+constexpr int kUmmaBarSFull = 96;      // [2] logits of a tile are in tensor memory
+constexpr int kUmmaBarSFree = 112;     // [2] the softmax warps have read them
+constexpr int kUmmaBarPFull = 128;     // weights of a tile are in shared memory
+constexpr int kUmmaBarPvDone = 136;    // the second MMA of a tile is complete
+constexpr int kUmmaBarQFull = 144;     // [2] query rows of a chunk landed
+constexpr int kUmmaBarQEmpty = 160;    // [2] the chunk's last logit MMA is complete
+constexpr int kUmmaBarWorkFull = 176;  // [kUmmaQueue] a chunk is announced
+constexpr int kUmmaBarWorkEmpty = 208; // [kUmmaQueue] all seven consumers have read the announcement
+constexpr int kUmmaTmemPtr = 240;
+constexpr int kUmmaAbort = 244;        // set by a softmax thread whose wait ran out
+constexpr int kUmmaWork = 256;         // [kUmmaQueue] int2 {chunk number or -1, sequence length}
+constexpr int kUmmaBarAccFree = 288;   // [2] the epilogue has read the accumulator of a chunk of this parity
+constexpr int kUmmaRed = 384;          // [4][16] floats: per-warp row maxima of a tile
+constexpr int kUmmaSavedM = 640;       // [2][16] floats: a finished chunk's references, by chunk parity
+constexpr int kUmmaSavedL = 768;       // [2][4][16] floats: its per-warp row sums
+static_assert(kUmmaSavedL + 512 <= kUmmaMiscBytes, "misc region too small");
+static_assert(kUmmaSmemBytes <= 227 * 1024, "one block per SM must fit");
 
 // ---- tcgen05 / TMA wrappers ----------------------------------------------------------------
+// The roles of this kernel hand tiles to one another in a chain (copy -> MMA -> softmax -> MMA),
+// one or two warps per role, so the time a waiter takes to notice a completed phase adds to
+// every tile: these waits poll (no suspend-time hint), still bounded by the clock.
+__device__ __forceinline__ bool mbarrier_test(unsigned bar, unsigned parity)
+{
+    unsigned done;
+    asm volatile("{\n\t.reg .pred p;\n\t"
+                 "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+                 "selp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+    return done != 0;
+}
+__device__ __forceinline__ bool mbarrier_poll_bounded(unsigned bar, unsigned parity)
+{
+    for (int i = 0; i < 64; ++i)
+        if (mbarrier_test(bar, parity)) return true;
+    const long long start = clock64();
+    for (;;) {
+        if (mbarrier_test(bar, parity)) return true;
+        if (clock64() - start > kWaitCycles) return false;
+    }
+}
 __device__ __forceinline__ void mbarrier_arrive(unsigned bar)
 {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" :: "r"(bar) : "memory");
@@ -143,86 +183,135 @@ __device__ __forceinline__ bool softmax_any(bool mine)
 }
 __device__ __forceinline__ void softmax_sync() { asm volatile("bar.sync 2, 128;" ::: "memory"); }
 
+// Reduces 16 per-lane values over the warp (maximum or sum) in 16 shuffles: each step halves the
+// number of values a lane carries and exchanges the other half with the lane `offset` away.
+// Lane L ends up with the result for row warp_reduce16_row(L) (lanes L and L ^ 1 hold the same).
+template <bool kMax>
+__device__ __forceinline__ float warp_reduce16(const float (&v)[16], int lane)
+{
+    auto both = [](float x, float y) { return kMax ? fmaxf(x, y) : x + y; };
+    float a8[8], a4[4], a2[2];
+    const bool up16 = (lane & 16) != 0, up8 = (lane & 8) != 0, up4 = (lane & 4) != 0, up2 = (lane & 2) != 0;
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+        a8[i] = both(up16 ? v[i + 8] : v[i], __shfl_xor_sync(0xffffffffu, up16 ? v[i] : v[i + 8], 16));
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+        a4[i] = both(up8 ? a8[i + 4] : a8[i], __shfl_xor_sync(0xffffffffu, up8 ? a8[i] : a8[i + 4], 8));
+#pragma unroll
+    for (int i = 0; i < 2; ++i)
+        a2[i] = both(up4 ? a4[i + 2] : a4[i], __shfl_xor_sync(0xffffffffu, up4 ? a4[i] : a4[i + 2], 4));
+    const float a1 = both(up2 ? a2[1] : a2[0], __shfl_xor_sync(0xffffffffu, up2 ? a2[0] : a2[1], 2));
+    return both(a1, __shfl_xor_sync(0xffffffffu, a1, 1));
+}
+__device__ __forceinline__ int warp_reduce16_row(int lane) { return ((lane >> 4) & 1) * 8 + ((lane >> 3) & 1) * 4 + ((lane >> 2) & 1) * 2 + ((lane >> 1) & 1); }
+
+__device__ __forceinline__ void tma_load_4d(unsigned dst, const CUtensorMap *map, int x, int y, int z, int w,
+                                            unsigned bar)
+{
+    asm volatile("cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes "
+                 "[%0], [%1, {%2, %3, %4, %5}], [%6];"
+                 :: "r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(z), "r"(w), "r"(bar) : "memory");
+}
+
+// A chunk of the grid's work list: number w counts (order, pair) with the order (long chunks
+// first) slowest, exactly the order in which one block per chunk would be scheduled.
+struct UmmaChunk {
+    int pair, split, b, hk, begin, end, n_tiles;
+};
+__device__ __forceinline__ UmmaChunk umma_chunk(const AttnParams &a, int w, int len)
+{
+    UmmaChunk c;
+    const int order = w / a.pairs;
+    c.pair = w - order * a.pairs;
+    c.split = scheduled_chunk(a, order);
+    c.b = c.pair / a.heads;
+    c.hk = c.pair - c.b * a.heads;
+    int size;
+    chunk_range(a, c.split, c.begin, size);
+    c.end = min(c.begin + size, len);
+    c.n_tiles = c.end > c.begin ? (c.end - c.begin + kUmmaTile - 1) / kUmmaTile : 0;
+    return c;
+}
+
+// Persistent: one block per SM; blocks draw chunks from a ticket counter (`ticket`, zeroed by
+// the host before the launch) until the list is exhausted, and the producers stream tiles
+// across chunk boundaries, so the copy pipeline never drains between chunks.
 template <bool kPaged>
-__global__ void __launch_bounds__(kUmmaThreads, kUmmaCtasPerSm)
-grouped_attn_umma_kernel(const GroupedParams p, const __grid_constant__ CUtensorMap map_k,
-                         const __grid_constant__ CUtensorMap map_v)
+__global__ void __launch_bounds__(kUmmaThreads, 1)
+grouped_attn_umma_kernel(const GroupedParams p, unsigned *ticket, const __grid_constant__ CUtensorMap map_q,
+                         const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v)
 {
     constexpr int D = 128;
     extern __shared__ unsigned char smem_raw[];
     const AttnParams &a = p.a;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int order = blockIdx.x / a.pairs;
-    const int pair = blockIdx.x - order * a.pairs;
-    const int split = scheduled_chunk(a, order);
-    const int b = pair / a.heads, hk = pair - b * a.heads;
     const bool final_writer = a.n_splits == 1;
+    const int total = a.pairs * a.n_splits;
     allow_next_kernel();
     wait_for_previous_kernels();
 
-    const int len = checked_seq_len(a, b, threadIdx.x == 0 && hk == 0 && final_writer);
-    int begin, chunk_size;
-    chunk_range(a, split, begin, chunk_size);
-    if (begin >= len) {                        // the whole block leaves before anything is set up
-        if (final_writer) {                    // inactive slot: zero output, lse = -inf
-            for (int i = threadIdx.x; i < p.rows * D; i += kUmmaThreads) {
-                const int r = i / D, d = i - r * D;
-                const int64_t row = grouped_row_index(p, b, hk, r);
-                a.out[row * D + d] = __float2half_rn(0.f);
-                if (a.lse && d == 0) a.lse[row] = -INFINITY;
-            }
-        }
-        return;
-    }
-    const int end = min(begin + chunk_size, len);
-    const int n_tiles = (end - begin + kUmmaTile - 1) / kUmmaTile;
-
-    // Shared memory: ring (1024-byte aligned: the 128-byte swizzle is a function of the address),
-    // query rows, weights, misc.
+    // Shared memory: K ring, V ring (1024-byte aligned: the 128-byte swizzle is a function of the
+    // address), query rows, weights, misc.
     const unsigned raw = static_cast<unsigned>(__cvta_generic_to_shared(smem_raw));
     const unsigned ring = (raw + 1023u) & ~1023u;
     unsigned char *smem = smem_raw + (ring - raw);
-    const unsigned q_smem = ring + kUmmaSlots * kUmmaItemBytes;
-    const unsigned p_smem = q_smem + kUmmaQBytes;
-    const unsigned misc = p_smem + kUmmaPBytes;
-    unsigned char *misc_ptr = smem + kUmmaSlots * kUmmaItemBytes + kUmmaQBytes + kUmmaPBytes;
+    constexpr int kVOffset = kUmmaKSlots * kUmmaItemBytes;
+    constexpr int kQOffset = kVOffset + kUmmaVSlots * kUmmaItemBytes;
+    constexpr int kPOffset = kQOffset + kUmmaQBuffers * kUmmaQBytes;
+    constexpr int kMiscOffset = kPOffset + kUmmaPBytes;
+    const unsigned q_smem = ring + kQOffset;
+    const unsigned p_smem = ring + kPOffset;
+    const unsigned misc = ring + kMiscOffset;
+    unsigned char *misc_ptr = smem + kMiscOffset;
     volatile unsigned *abort_word = reinterpret_cast<volatile unsigned *>(misc_ptr + kUmmaAbort);
+    volatile int2 *work = reinterpret_cast<volatile int2 *>(misc_ptr + kUmmaWork);
     float *red = reinterpret_cast<float *>(misc_ptr + kUmmaRed);
 
     // ---- set-up ----
-    if (warp == 5) {                           // tensor memory: one warp allocates and later frees
+    if (warp == kUmmaWarpLogits) {             // tensor memory: one warp allocates and later frees
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
                      :: "r"(misc + kUmmaTmemPtr), "n"(kUmmaTmemCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-    } else if (warp == 4) {
+    } else if (warp == kUmmaWarpK) {
         if (lane == 0) {
 #pragma unroll
-            for (int s = 0; s < kUmmaSlots; ++s) {
-                mbarrier_init(misc + kUmmaBarFull + s * 8, 1);
-                mbarrier_init(misc + kUmmaBarEmpty + s * 8, 1);
+            for (int s = 0; s < kUmmaKSlots; ++s) {
+                mbarrier_init(misc + kUmmaBarKFull + s * 8, 1);
+                mbarrier_init(misc + kUmmaBarKEmpty + s * 8, 1);
+            }
+#pragma unroll
+            for (int s = 0; s < kUmmaVSlots; ++s) {
+                mbarrier_init(misc + kUmmaBarVFull + s * 8, 1);
+                mbarrier_init(misc + kUmmaBarVEmpty + s * 8, 1);
             }
 #pragma unroll
             for (int s = 0; s < 2; ++s) {
                 mbarrier_init(misc + kUmmaBarSFull + s * 8, 1);
                 mbarrier_init(misc + kUmmaBarSFree + s * 8, 4);
+                mbarrier_init(misc + kUmmaBarQFull + s * 8, 1);
+                mbarrier_init(misc + kUmmaBarQEmpty + s * 8, 1);
+                mbarrier_init(misc + kUmmaBarAccFree + s * 8, 4);
+            }
+#pragma unroll
+            for (int s = 0; s < kUmmaQueue; ++s) {
+                mbarrier_init(misc + kUmmaBarWorkFull + s * 8, 1);
+                mbarrier_init(misc + kUmmaBarWorkEmpty + s * 8, 7);       // V producer, 2 MMA lanes, 4 softmax warps
             }
             mbarrier_init(misc + kUmmaBarPFull, 4);
             mbarrier_init(misc + kUmmaBarPvDone, 1);
             mbarrier_init_fence();
             *abort_word = 0u;
+            asm volatile("prefetch.tensormap [%0];" :: "l"(reinterpret_cast<uint64_t>(&map_q)) : "memory");
             asm volatile("prefetch.tensormap [%0];" :: "l"(reinterpret_cast<uint64_t>(&map_k)) : "memory");
             asm volatile("prefetch.tensormap [%0];" :: "l"(reinterpret_cast<uint64_t>(&map_v)) : "memory");
         }
-    } else {
-        // Query rows as operand B of the first MMA (N = 16 rows, K = D, K-major, no swizzle):
-        // 8 x 16-byte core matrices, 128 bytes each; along K at 128 bytes, the second group of
-        // 8 rows at 2048 bytes.  Rows beyond p.rows are zero.
-        for (int i = threadIdx.x; i < kGroupRows * 16; i += 128) {
-            const int r = i >> 4, seg = i & 15;
-            uint4 v = make_uint4(0u, 0u, 0u, 0u);
-            if (r < p.rows) v = reinterpret_cast<const uint4 *>(a.q + grouped_row_index(p, b, hk, r) * D)[seg];
-            *reinterpret_cast<uint4 *>(smem + kUmmaSlots * kUmmaItemBytes + (r >> 3) * 2048 + seg * 128 + (r & 7) * 16) = v;
-        }
+    } else if (warp < 4) {
+        // The query buffers start as zeros: a chunk's copy overwrites rows < p.rows only, so the
+        // padding rows of the 16-row operand stay zero for the whole launch.
+        const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
+        for (int i = threadIdx.x; i < kUmmaQBuffers * kUmmaQBytes / 16; i += 128)
+            *reinterpret_cast<uint4 *>(smem + kQOffset + i * 16) = zero;
         fence_async_proxy();
     }
     tc_fence_before();
@@ -230,25 +319,26 @@ grouped_attn_umma_kernel(const GroupedParams p, const __grid_constant__ CUtensor
     tc_fence_after();
     const unsigned tmem = *reinterpret_cast<volatile unsigned *>(misc_ptr + kUmmaTmemPtr);
 
-    if (warp == 4) {
-        // ================================ producer ================================
-        const int T = kPaged ? a.block_tokens : kUmmaTile;
-        const int32_t *table_row = kPaged ? a.block_table + (int64_t)b * a.max_blocks_per_seq : nullptr;
+    // What both producers do for one chunk: the chunk's tiles of one cache (K or V) into that
+    // cache's ring, tile `count` of this block going to slot count % slots; returns false if a
+    // wait ran out.
+    const int T = kPaged ? a.block_tokens : kUmmaTile;
+    auto stream_chunk = [&](const UmmaChunk &c, const CUtensorMap *map, int ring_offset, int slots, int bar_full,
+                            int bar_empty, int &count) -> bool {
         const int64_t total_rows = a.kv_bytes / (2 * D);
-        auto fetch_ids = [&](int j) -> int {           // lane i: physical block of the tile's i-th block
+        const int32_t *table_row = kPaged ? a.block_table + (int64_t)c.b * a.max_blocks_per_seq : nullptr;
+        auto fetch_ids = [&](int j) -> int {            // lane i: physical block of the tile's i-th block
             if (!kPaged) return 0;
-            const int tile_start = begin + j * kUmmaTile;
-            const int nb = (min(end - tile_start, kUmmaTile) + T - 1) / T;
+            const int tile_start = c.begin + j * kUmmaTile;
+            const int nb = (min(c.end - tile_start, kUmmaTile) + T - 1) / T;
             const int idx = tile_start / T + lane;
-            if (j >= n_tiles || lane >= nb || !bounds_ok(idx < a.max_blocks_per_seq, a.status)) return -1;
+            if (j >= c.n_tiles || lane >= nb || !bounds_ok(idx < a.max_blocks_per_seq, a.status)) return -1;
             return __ldg(table_row + idx);
         };
         int ids_next = fetch_ids(0);
-        int issued = 0;
-        bool fine = true;
-        for (int j = 0; j < n_tiles && fine; ++j) {
-            const int tile_start = begin + j * kUmmaTile;
-            const int nb = kPaged ? (min(end - tile_start, kUmmaTile) + T - 1) / T : 1;
+        for (int j = 0; j < c.n_tiles; ++j, ++count) {
+            const int tile_start = c.begin + j * kUmmaTile;
+            const int nb = kPaged ? (min(c.end - tile_start, kUmmaTile) + T - 1) / T : 1;
             const int phys = ids_next;
             ids_next = fetch_ids(j + 1);
             bool good = lane < nb;
@@ -256,94 +346,239 @@ grouped_attn_umma_kernel(const GroupedParams p, const __grid_constant__ CUtensor
             if (kPaged) {
                 const bool in_range = phys >= 0 && (int64_t)phys < a.num_phys_blocks;
                 if (good && !in_range && a.status) atomicOr(a.status, kFlagBlockRange);
-                row0 = in_range ? (phys * a.heads + hk) * T : 0;      // < 2^31 rows: checked by the host
+                row0 = in_range ? (phys * a.heads + c.hk) * T : 0;           // < 2^31 rows: checked by the host
                 good = good && in_range && bounds_ok((int64_t)row0 + T <= total_rows, a.status);
             } else {
-                row0 = pair * a.s_max + tile_start;            // rows past the tensor's end read as zeros
+                row0 = c.pair * a.s_max + tile_start;          // rows past the tensor's end read as zeros
             }
-            for (int which = 0; which < 2 && fine; ++which) {
-                const int item = 2 * j + which;
-                const int slot = item % kUmmaSlots;
-                if (item >= kUmmaSlots)
-                    fine = __all_sync(0xffffffffu, mbarrier_wait_bounded(misc + kUmmaBarEmpty + slot * 8,
-                                                                         (item / kUmmaSlots - 1) & 1));
-                if (!fine) break;
-                const unsigned dst = ring + slot * kUmmaItemBytes + (kPaged ? lane * T * 128 : 0);
-                const unsigned bar = misc + kUmmaBarFull + slot * 8;
-                if (kPaged && lane < nb && !good) {            // a block that cannot be read counts as zeros
-                    const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
-                    unsigned char *z = smem + slot * kUmmaItemBytes + lane * T * 128;
-                    for (int i = 0; i < T * 8; ++i) {
-                        *reinterpret_cast<uint4 *>(z + i * 16) = zero;
-                        *reinterpret_cast<uint4 *>(z + kUmmaPanelBytes + i * 16) = zero;
+            const int slot = count % slots;
+            if (count >= slots &&
+                !__all_sync(0xffffffffu, mbarrier_poll_bounded(misc + bar_empty + slot * 8, (count / slots - 1) & 1)))
+                return false;
+            const int slot_offset = ring_offset + slot * kUmmaItemBytes + (kPaged ? lane * T * 128 : 0);
+            const unsigned bar = misc + bar_full + slot * 8;
+            if (kPaged && lane < nb && !good) {                // a block that cannot be read counts as zeros
+                const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
+                for (int i = 0; i < T * 8; ++i) {
+                    *reinterpret_cast<uint4 *>(smem + slot_offset + i * 16) = zero;
+                    *reinterpret_cast<uint4 *>(smem + slot_offset + kUmmaPanelBytes + i * 16) = zero;
+                }
+                fence_async_proxy();
+            }
+            const unsigned fetched = __popc(__ballot_sync(0xffffffffu, good));
+            if (lane == 0) mbarrier_expect_bytes(bar, fetched * (unsigned)T * 256u);
+            __syncwarp();
+            if (good) {
+                tma_load_2d(ring + slot_offset, map, 0, row0, bar);
+                tma_load_2d(ring + slot_offset + kUmmaPanelBytes, map, 64, row0, bar);
+            }
+        }
+        return true;
+    };
+    // copies in flight must land (or be given up, bounded) before shared memory is handed on
+    auto drain = [&](int slots, int bar_full, int count) {
+        for (int i = max(count - slots, 0); i < count; ++i)
+            (void)mbarrier_poll_bounded(misc + bar_full + (i % slots) * 8, (i / slots) & 1);
+    };
+
+    if (warp == kUmmaWarpK) {
+        // ================== K producer: also draws the tickets and announces the chunks ==================
+        // Tickets are drawn two chunks ahead and lengths read one chunk ahead: the atomic and the
+        // load are issued at the start of a chunk and their results first used at its end, so
+        // their round trips through a busy memory system overlap with the chunk's copies.
+        auto issue_draw = [&]() -> unsigned {           // lane 0's return value is the ticket
+            unsigned w = 0;
+            if (lane == 0) w = atomicAdd(ticket, 1u);
+            return w;
+        };
+        auto ticket_of = [&](unsigned raw_ticket) -> int {     // chunk number (total: none left)
+            raw_ticket = __shfl_sync(0xffffffffu, raw_ticket, 0);
+            return raw_ticket < (unsigned)total ? (int)raw_ticket : total;
+        };
+        auto issue_length = [&](int w) -> int {         // raw length of the chunk's sequence
+            int len = 0;
+            if (w < total) {
+                const int b = (w % a.pairs) / a.heads;
+                asm volatile("ld.global.nc.b32 %0, [%1];" : "=r"(len) : "l"(a.seq_lens + b) : "memory");
+            }
+            return len;
+        };
+        auto checked_length = [&](int w, int len) -> int {    // out-of-range lengths make the slot inactive
+            if (w >= total) return 0;
+            if (len < 0 || len > a.max_seq_len) {
+                const int order = w / a.pairs, pair = w - order * a.pairs;
+                if (lane == 0 && order == 0 && pair % a.heads == 0 && a.status) atomicOr(a.status, kFlagSeqLenRange);
+                return 0;
+            }
+            return len;
+        };
+        int w_now = ticket_of(issue_draw());
+        int w_next = ticket_of(issue_draw());
+        int len_now = checked_length(w_now, issue_length(w_now));
+        int count = 0;                                  // K tiles issued so far (ring position)
+        int k = 0;                                      // chunks announced so far
+        bool fine = true;
+        bool first = true;
+        unsigned raw_after = 0;
+        int raw_len_next = 0;
+        while (fine) {
+            if (!first) {                               // what was requested a chunk ago has arrived by now
+                w_now = w_next;
+                len_now = checked_length(w_now, raw_len_next);
+                w_next = ticket_of(raw_after);
+            }
+            first = false;
+            const int w = w_now, len = len_now;
+            if (w >= total) break;
+            raw_after = issue_draw();
+            raw_len_next = issue_length(w_next);
+            const UmmaChunk c = umma_chunk(a, w, len);
+            if (c.n_tiles == 0) {
+                if (final_writer) {                     // inactive sequence: zero output, lse = -inf
+                    for (int i = lane; i < p.rows * D; i += 32) {
+                        const int r = i / D, d = i - r * D;
+                        const int64_t row = grouped_row_index(p, c.b, c.hk, r);
+                        a.out[row * D + d] = __float2half_rn(0.f);
+                        if (a.lse && d == 0) a.lse[row] = -INFINITY;
                     }
-                    fence_async_proxy();
                 }
-                const unsigned fetched = __popc(__ballot_sync(0xffffffffu, good));
-                __syncwarp();
-                if (lane == 0) mbarrier_expect_bytes(bar, fetched * (unsigned)T * 256u);
-                __syncwarp();
-                if (good) {
-                    const CUtensorMap *map = which == 0 ? &map_k : &map_v;
-                    tma_load_2d(dst, map, 0, row0, bar);
-                    tma_load_2d(dst + kUmmaPanelBytes, map, 64, row0, bar);
-                }
-                ++issued;
+                continue;
+            }
+            // announce the chunk to the other warps
+            const int wq = k % kUmmaQueue;
+            if (k >= kUmmaQueue)
+                fine = __all_sync(0xffffffffu, mbarrier_poll_bounded(misc + kUmmaBarWorkEmpty + wq * 8,
+                                                                     (k / kUmmaQueue - 1) & 1));
+            if (!fine) break;
+            if (lane == 0) {
+                work[wq].x = w;
+                work[wq].y = len;
+                mbarrier_arrive(misc + kUmmaBarWorkFull + wq * 8);
+            }
+            // its query rows: rows t * group + g of (sequence, KV head), 64 dims per panel
+            const int qb = k & 1;
+            if (k >= 2)
+                fine = __all_sync(0xffffffffu, mbarrier_poll_bounded(misc + kUmmaBarQEmpty + qb * 8, (k / 2 - 1) & 1));
+            if (!fine) break;
+            if (lane == 0) {
+                const unsigned bar = misc + kUmmaBarQFull + qb * 8;
+                mbarrier_expect_bytes(bar, (unsigned)p.rows * 256u);
+                tma_load_4d(q_smem + qb * kUmmaQBytes, &map_q, 0, c.hk * p.group, 0, c.b, bar);
+                tma_load_4d(q_smem + qb * kUmmaQBytes + kUmmaQBytes / 2, &map_q, 64, c.hk * p.group, 0, c.b, bar);
+            }
+            ++k;
+            fine = stream_chunk(c, &map_k, 0, kUmmaKSlots, kUmmaBarKFull, kUmmaBarKEmpty, count);
+        }
+        if (fine) {                                     // no chunk is left: tell the others
+            const int wq = k % kUmmaQueue;
+            if (k >= kUmmaQueue)
+                fine = __all_sync(0xffffffffu, mbarrier_poll_bounded(misc + kUmmaBarWorkEmpty + wq * 8,
+                                                                     (k / kUmmaQueue - 1) & 1));
+            if (fine && lane == 0) {
+                work[wq].x = -1;
+                work[wq].y = 0;
+                mbarrier_arrive(misc + kUmmaBarWorkFull + wq * 8);
             }
         }
         if (!fine) {
             if (lane == 0 && a.status) atomicOr(a.status, kFlagCopyTimeout);
-            // copies in flight must land (or be given up, bounded) before shared memory is handed on
-            for (int item = max(issued - kUmmaSlots, 0); item < issued; ++item)
-                (void)mbarrier_wait_bounded(misc + kUmmaBarFull + (item % kUmmaSlots) * 8, (item / kUmmaSlots) & 1);
+            drain(kUmmaKSlots, kUmmaBarKFull, count);
         }
-    } else if (warp == 5) {
-        // ================================ MMA issue ================================
+    } else if (warp == kUmmaWarpV) {
+        // ================================ V producer ================================
+        int count = 0;
+        bool fine = true;
+        for (int k = 0; fine; ++k) {
+            const int wq = k % kUmmaQueue;
+            fine = __all_sync(0xffffffffu, mbarrier_poll_bounded(misc + kUmmaBarWorkFull + wq * 8, (k / kUmmaQueue) & 1));
+            if (!fine) break;
+            const int w = work[wq].x, len = work[wq].y;
+            __syncwarp();
+            if (lane == 0) mbarrier_arrive(misc + kUmmaBarWorkEmpty + wq * 8);
+            if (w < 0) break;
+            fine = stream_chunk(umma_chunk(a, w, len), &map_v, kVOffset, kUmmaVSlots, kUmmaBarVFull, kUmmaBarVEmpty, count);
+        }
+        if (!fine) {
+            if (lane == 0 && a.status) atomicOr(a.status, kFlagCopyTimeout);
+            drain(kUmmaVSlots, kUmmaBarVFull, count);
+        }
+    } else if (warp == kUmmaWarpLogits) {
+        // ================================ logit MMAs ================================
+        // One lane issues S^T = K_tile Q^T for every tile of every chunk of this block, as far
+        // ahead of the softmax warps as the two logit buffers allow.
         if (lane == 0) {
-            constexpr unsigned idesc_logits = umma_idesc(128, 16, 0, 0);   // K tile K-major, Q K-major
-            constexpr unsigned idesc_output = umma_idesc(128, 32, 1, 1);   // V tile MN-major, weights MN-major
-            auto logits = [&](int j) -> bool {
-                const int item = 2 * j, slot = item % kUmmaSlots;
-                if (!mbarrier_wait_bounded(misc + kUmmaBarFull + slot * 8, (item / kUmmaSlots) & 1)) return false;
-                if (j >= 2 && !mbarrier_wait_bounded(misc + kUmmaBarSFree + (j & 1) * 8, ((j >> 1) - 1) & 1)) return false;
-                tc_fence_after();
-                const unsigned k_tile = ring + slot * kUmmaItemBytes;
+            constexpr unsigned idesc = umma_idesc(128, 16, 0, 0);          // K tile K-major, Q K-major
+            bool fine = true;
+            int g = 0;                                                      // tiles of all chunks so far
+            for (int k = 0; fine; ++k) {
+                const int wq = k % kUmmaQueue;
+                fine = mbarrier_poll_bounded(misc + kUmmaBarWorkFull + wq * 8, (k / kUmmaQueue) & 1);
+                if (!fine) break;
+                const int w = work[wq].x, len = work[wq].y;
+                mbarrier_arrive(misc + kUmmaBarWorkEmpty + wq * 8);
+                if (w < 0) break;
+                const int n_tiles = umma_chunk(a, w, len).n_tiles;
+                fine = mbarrier_poll_bounded(misc + kUmmaBarQFull + (k & 1) * 8, (k / 2) & 1);
+                // K tile and query rows alike: rows of 128 bytes per 64-dim panel, 8-row groups 1024
+                // bytes apart, 128-byte swizzle; a k-step of 16 dims is 32 bytes along the row
+                const uint64_t q_desc = umma_desc(q_smem + (k & 1) * kUmmaQBytes, 16, 1024, 2);
+                for (int j = 0; j < n_tiles && fine; ++j, ++g) {
+                    const int slot = g % kUmmaKSlots;
+                    fine = mbarrier_poll_bounded(misc + kUmmaBarKFull + slot * 8, (g / kUmmaKSlots) & 1) &&
+                           (g < 2 || mbarrier_poll_bounded(misc + kUmmaBarSFree + (g & 1) * 8, ((g >> 1) - 1) & 1));
+                    if (!fine) break;
+                    tc_fence_after();
+                    const uint64_t k_desc = umma_desc(ring + slot * kUmmaItemBytes, 16, 1024, 2);
 #pragma unroll
-                for (int ks = 0; ks < 8; ++ks) {
-                    // K tile: rows of 128 bytes per 64-dim panel, 8-row groups 1024 bytes apart,
-                    // 128-byte swizzle; a k-step of 16 dims is 32 bytes further along the row
-                    const uint64_t ad = umma_desc(k_tile + (ks >> 2) * kUmmaPanelBytes + (ks & 3) * 32, 16, 1024, 2);
-                    const uint64_t bd = umma_desc(q_smem + ks * 256, 128, 2048, 0);
-                    tc_mma_f16(tmem + (j & 1) * 16, ad, bd, idesc_logits, ks > 0);
+                    for (int ks = 0; ks < 8; ++ks)
+                        tc_mma_f16(tmem + (g & 1) * 16, k_desc + (uint64_t)(((ks >> 2) * kUmmaPanelBytes + (ks & 3) * 32) >> 4),
+                                   q_desc + (uint64_t)(((ks >> 2) * (kUmmaQBytes / 2) + (ks & 3) * 32) >> 4), idesc, ks > 0);
+                    tc_commit(misc + kUmmaBarSFull + (g & 1) * 8);
+                    tc_commit(misc + kUmmaBarKEmpty + slot * 8);
+                    // after the chunk's last logit MMA its query rows may be replaced
+                    if (j + 1 == n_tiles) tc_commit(misc + kUmmaBarQEmpty + (k & 1) * 8);
                 }
-                tc_commit(misc + kUmmaBarSFull + (j & 1) * 8);
-                tc_commit(misc + kUmmaBarEmpty + slot * 8);
-                return true;
-            };
-            auto output = [&](int j) -> bool {
-                const int item = 2 * j + 1, slot = item % kUmmaSlots;
-                if (!mbarrier_wait_bounded(misc + kUmmaBarFull + slot * 8, (item / kUmmaSlots) & 1)) return false;
-                if (!mbarrier_wait_bounded(misc + kUmmaBarPFull, j & 1)) return false;
-                tc_fence_after();
-                const unsigned v_tile = ring + slot * kUmmaItemBytes;
+            }
+            if (!fine && a.status) atomicOr(a.status, kFlagCopyTimeout);
+        }
+        __syncwarp();
+    } else if (warp == kUmmaWarpOutput) {
+        // ================================ output MMAs ================================
+        // One lane issues O^T += V_tile^T P^T for every tile, into the accumulator of the chunk's parity.
+        if (lane == 0) {
+            constexpr unsigned idesc = umma_idesc(128, 32, 1, 1);          // V tile MN-major, weights MN-major
+            // Weights: 8-column blocks of [128 tokens][16 bytes], 2048 bytes apart; 8-token groups
+            // 128 bytes apart; a k-step is 16 tokens = 256 bytes.
+            const uint64_t p_desc = umma_desc(p_smem, 128, 2048, 0);
+            bool fine = true;
+            int g = 0;
+            for (int k = 0; fine; ++k) {
+                const int wq = k % kUmmaQueue;
+                fine = mbarrier_poll_bounded(misc + kUmmaBarWorkFull + wq * 8, (k / kUmmaQueue) & 1);
+                if (!fine) break;
+                const int w = work[wq].x, len = work[wq].y;
+                mbarrier_arrive(misc + kUmmaBarWorkEmpty + wq * 8);
+                if (w < 0) break;
+                const int n_tiles = umma_chunk(a, w, len).n_tiles;
+                // the accumulator of this parity was last used two chunks ago: its epilogue must have read it
+                if (k >= 2) fine = mbarrier_poll_bounded(misc + kUmmaBarAccFree + (k & 1) * 8, (k / 2 - 1) & 1);
+                const unsigned acc = tmem + 32 + (k & 1) * 32;
+                for (int j = 0; j < n_tiles && fine; ++j, ++g) {
+                    const int slot = g % kUmmaVSlots;
+                    fine = mbarrier_poll_bounded(misc + kUmmaBarVFull + slot * 8, (g / kUmmaVSlots) & 1) &&
+                           mbarrier_poll_bounded(misc + kUmmaBarPFull, g & 1);
+                    if (!fine) break;
+                    tc_fence_after();
+                    // V tile read MN-major (M = dims): the two 64-dim panels are kUmmaPanelBytes apart
+                    // (leading offset), 8-token groups 1024 bytes apart; a k-step is 16 tokens = 2048 bytes
+                    const uint64_t v_desc = umma_desc(ring + kVOffset + slot * kUmmaItemBytes, kUmmaPanelBytes, 1024, 2);
 #pragma unroll
-                for (int ks = 0; ks < 8; ++ks) {
-                    // V tile read MN-major (M = dims): the two 64-dim panels are kUmmaPanelBytes
-                    // apart (leading offset), 8-token groups 1024 bytes apart; a k-step is 16 tokens.
-                    // Weights: 8-column blocks of [128 tokens][16 bytes], 2048 bytes apart; 8-token
-                    // groups 128 bytes apart.
-                    const uint64_t ad = umma_desc(v_tile + ks * 2048, kUmmaPanelBytes, 1024, 2);
-                    const uint64_t bd = umma_desc(p_smem + ks * 256, 128, 2048, 0);
-                    tc_mma_f16(tmem + 32, ad, bd, idesc_output, j > 0 || ks > 0);
+                    for (int ks = 0; ks < 8; ++ks)
+                        tc_mma_f16(acc, v_desc + (uint64_t)((ks * 2048) >> 4), p_desc + (uint64_t)((ks * 256) >> 4), idesc,
+                                   j > 0 || ks > 0);
+                    tc_commit(misc + kUmmaBarVEmpty + slot * 8);
+                    tc_commit(misc + kUmmaBarPvDone);
                 }
-                tc_commit(misc + kUmmaBarEmpty + slot * 8);
-                tc_commit(misc + kUmmaBarPvDone);
-                return true;
-            };
-            bool fine = logits(0);
-            for (int j = 0; j < n_tiles && fine; ++j) {
-                if (j + 1 < n_tiles) fine = logits(j + 1);
-                if (fine) fine = output(j);
             }
             if (!fine && a.status) atomicOr(a.status, kFlagCopyTimeout);
         }
@@ -352,189 +587,218 @@ grouped_attn_umma_kernel(const GroupedParams p, const __grid_constant__ CUtensor
         // ================================ softmax and epilogue ================================
         const int t = threadIdx.x;                                 // token of the tile = lane of tensor memory
         const unsigned lane_base = tmem + ((unsigned)(warp * 32) << 16);
-        float m[16], l[16];
-#pragma unroll
-        for (int r = 0; r < 16; ++r) {
-            m[r] = kMinusHuge;
-            l[r] = 0.f;
-        }
-        const int unmasked_end = min(end, len - (p.q_tokens - 1));  // tiles ending here or before need no mask
-        bool aborted = false;
-        for (int j = 0; j < n_tiles; ++j) {
-            const int sb = j & 1;
-            // (warp-uniform: the tensor-memory loads below are warp-wide instructions)
-            bool fine = __all_sync(0xffffffffu, mbarrier_wait_bounded(misc + kUmmaBarSFull + sb * 8, (j >> 1) & 1));
-            float s[16];
-            if (fine) {
-                tc_fence_after();
-                tc_load16(s, lane_base + sb * 16);
-                tc_fence_before();
-            } else {
-#pragma unroll
-                for (int r = 0; r < 16; ++r) s[r] = 0.f;
-            }
-            __syncwarp();
-            if (lane == 0) mbarrier_arrive(misc + kUmmaBarSFree + sb * 8);
-            const int tile_start = begin + j * kUmmaTile;
-            const int tok = tile_start + t;
-#pragma unroll
-            for (int r = 0; r < 16; ++r) s[r] *= a.scale_log2e;
-            if (tile_start + kUmmaTile > unmasked_end) {           // uniform: last tiles of the sequence / chunk
-#pragma unroll
-                for (int r = 0; r < 16; ++r) {
-                    const int vis = r < p.rows ? len - (p.q_tokens - 1 - r / p.group) : 0;
-                    if (tok >= min(vis, end)) s[r] = -INFINITY;
-                }
-                if (tok >= end) {
-                    // The value row of a position outside the chunk gets weight zero, but its bytes
-                    // may be anything (the tail of a block, a slot not fetched): 0 x NaN must not
-                    // reach the accumulator, so the row is cleared once the tile has landed.
-                    const int item = 2 * j + 1, slot = item % kUmmaSlots;
-                    fine = mbarrier_wait_bounded(misc + kUmmaBarFull + slot * 8, (item / kUmmaSlots) & 1) && fine;
-                    const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
-                    unsigned char *vrow = smem + slot * kUmmaItemBytes + t * 128;
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        *reinterpret_cast<uint4 *>(vrow + i * 16) = zero;
-                        *reinterpret_cast<uint4 *>(vrow + kUmmaPanelBytes + i * 16) = zero;
-                    }
-                }
-            }
-            bool moved = false;
-#pragma unroll
-            for (int r = 0; r < 16; ++r) moved = moved || s[r] > m[r] + kGroupLag;
-            if (!fine) *abort_word = 1u;
-            bool waited = false;
-            if (softmax_any(moved || !fine)) {
-                if (*abort_word != 0u) {                            // the same for all 128 threads
-                    aborted = true;
-                    break;
-                }
-                // Some row's reference moves: row maxima over the tile, new references, and the
-                // accumulator (and the sums) rescaled to them.
-#pragma unroll
-                for (int r = 0; r < 16; ++r) {
-                    float top = s[r];
-                    top = fmaxf(top, __shfl_xor_sync(0xffffffffu, top, 1));
-                    top = fmaxf(top, __shfl_xor_sync(0xffffffffu, top, 2));
-                    top = fmaxf(top, __shfl_xor_sync(0xffffffffu, top, 4));
-                    top = fmaxf(top, __shfl_xor_sync(0xffffffffu, top, 8));
-                    top = fmaxf(top, __shfl_xor_sync(0xffffffffu, top, 16));
-                    if (lane == 0) red[warp * 16 + r] = top;
-                }
-                softmax_sync();
-                float alpha[16];
-                bool any_change = false;
-#pragma unroll
-                for (int r = 0; r < 16; ++r) {
-                    const float top = fmaxf(fmaxf(red[r], red[16 + r]), fmaxf(red[32 + r], red[48 + r]));
-                    alpha[r] = 1.f;
-                    if (top > m[r] + kGroupLag) {
-                        alpha[r] = fast_exp2(m[r] - top);
-                        m[r] = top;
-                        any_change = true;
-                    }
-                    l[r] *= alpha[r];
-                }
-                if (j > 0 && any_change) {
-                    // the accumulator holds tiles 0 .. j-1 once the previous tile's MMA is complete
-                    fine = __all_sync(0xffffffffu, mbarrier_wait_bounded(misc + kUmmaBarPvDone, (j - 1) & 1));
-                    waited = true;
-                    if (fine) {
-                        tc_fence_after();
-                        float o[16];
-#pragma unroll
-                        for (int half = 0; half < 2; ++half) {      // columns 0-15: high parts, 16-31: low parts
-                            tc_load16(o, lane_base + 32 + half * 16);
-#pragma unroll
-                            for (int r = 0; r < 16; ++r) o[r] *= alpha[r];
-                            tc_store16(lane_base + 32 + half * 16, o);
-                        }
-                    } else {
-                        *abort_word = 1u;                           // seen by all at the next tile's vote
-                    }
-                }
-            }
-            // Weights against the references (scaled by kGroupWeightScale inside the exponent),
-            // their sums, and the fp16 high and low parts: thread t holds row t of operand B
-            // (MN-major: 8 columns = 16 bytes per token and column block).
-            unsigned hi[8], lo[8];
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                const float w0 = fast_exp2(s[2 * i] - (m[2 * i] - kGroupWeightLog2));
-                const float w1 = fast_exp2(s[2 * i + 1] - (m[2 * i + 1] - kGroupWeightLog2));
-                l[2 * i] += w0;
-                l[2 * i + 1] += w1;
-                hi[i] = pack_half2(w0, w1);
-                const float2 back = __half22float2(*reinterpret_cast<const __half2 *>(&hi[i]));
-                lo[i] = pack_half2(w0 - back.x, w1 - back.y);
-            }
-            if (j > 0 && !waited && fine) {                         // the previous MMA has read the weights
-                fine = mbarrier_wait_bounded(misc + kUmmaBarPvDone, (j - 1) & 1);
-                if (!fine) *abort_word = 1u;
-            }
-            unsigned char *prow = smem + kUmmaSlots * kUmmaItemBytes + kUmmaQBytes + t * 16;
-            *reinterpret_cast<uint4 *>(prow) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-            *reinterpret_cast<uint4 *>(prow + 2048) = make_uint4(hi[4], hi[5], hi[6], hi[7]);
-            *reinterpret_cast<uint4 *>(prow + 4096) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
-            *reinterpret_cast<uint4 *>(prow + 6144) = make_uint4(lo[4], lo[5], lo[6], lo[7]);
-            fence_async_proxy();
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbarrier_arrive(misc + kUmmaBarPFull);
-        }
-        if (!aborted) aborted = softmax_any(*abort_word != 0u) || false;
-        if (aborted) {
-            if (t == 0 && a.status) atomicOr(a.status, kFlagCopyTimeout);
-        } else if (!mbarrier_wait_bounded(misc + kUmmaBarPvDone, (n_tiles - 1) & 1)) {
-            if (a.status) atomicOr(a.status, kFlagCopyTimeout);
-            aborted = true;
-        }
-        // Row sums over the block (every thread joins the barrier, also after a give-up).
-#pragma unroll
-        for (int r = 0; r < 16; ++r) {
-            float sum = l[r];
-            sum += __shfl_xor_sync(0xffffffffu, sum, 1);
-            sum += __shfl_xor_sync(0xffffffffu, sum, 2);
-            sum += __shfl_xor_sync(0xffffffffu, sum, 4);
-            sum += __shfl_xor_sync(0xffffffffu, sum, 8);
-            sum += __shfl_xor_sync(0xffffffffu, sum, 16);
-            if (lane == 0) red[warp * 16 + r] = sum;
-        }
-        softmax_sync();
-        if (!softmax_any(aborted)) {
-            // Epilogue: thread t owns output dim t; columns r and 16 + r are the high and low
-            // parts of row r.  Sums and accumulator both carry kGroupWeightScale.
+        float *saved_m = reinterpret_cast<float *>(misc_ptr + kUmmaSavedM);     // [2][16]
+        float *saved_l = reinterpret_cast<float *>(misc_ptr + kUmmaSavedL);     // [2][4][16]
+        // The epilogue of a chunk (accumulator -> partial result) runs after the first tile of the
+        // next chunk has been handed to the MMA, so that the tensor pipe and the copies go on
+        // meanwhile; the accumulators alternate between two regions of tensor memory.
+        auto epilogue = [&](const UmmaChunk &c, int parity) {
+            // Thread t owns output dim t; columns r and 16 + r are the high and low parts of row
+            // r.  Sums and accumulator both carry kGroupWeightScale.
             tc_fence_after();
             float o_hi[16], o_lo[16];
-            tc_load16(o_hi, lane_base + 32);
-            tc_load16(o_lo, lane_base + 48);
+            tc_load16(o_hi, lane_base + 32 + parity * 32);
+            tc_load16(o_lo, lane_base + 48 + parity * 32);
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbarrier_arrive(misc + kUmmaBarAccFree + parity * 8);
+            const float *sl = saved_l + parity * 64, *sm = saved_m + parity * 16;
 #pragma unroll
             for (int r = 0; r < 16; ++r) {
                 if (r < p.rows) {
-                    const float total = (red[r] + red[16 + r]) + (red[32 + r] + red[48 + r]);
+                    const float total_w = (sl[r] + sl[16 + r]) + (sl[32 + r] + sl[48 + r]);
                     // A row that sees no position of this chunk (causal limit before the chunk) has total 0.
-                    const bool empty = !(total > 0.f);
-                    const float value = empty ? 0.f : (o_hi[r] + o_lo[r]) / total;
-                    const float lse2 = empty ? kMinusHuge : m[r] + log2f(total) - kGroupWeightLog2;
+                    const bool empty = !(total_w > 0.f);
+                    const float value = empty ? 0.f : (o_hi[r] + o_lo[r]) / total_w;
+                    const float lse2 = empty ? kMinusHuge : sm[r] + log2f(total_w) - kGroupWeightLog2;
                     if (final_writer) {
-                        const int64_t row = grouped_row_index(p, b, hk, r);
+                        const int64_t row = grouped_row_index(p, c.b, c.hk, r);
                         a.out[row * D + t] = __float2half_rn(value);
                         if (a.lse && t == 0) a.lse[row] = empty ? -INFINITY : lse2 * kLn2;
                     } else {
-                        const int64_t slot = ((int64_t)pair * a.n_splits + split) * p.rows + r;
+                        const int64_t slot = ((int64_t)c.pair * a.n_splits + c.split) * p.rows + r;
                         a.part_o[slot * D + t] = value;
                         if (t == 0) a.part_lse[slot] = lse2;
                     }
                 }
             }
+        };
+        bool aborted = false, pending = false;
+        UmmaChunk before = {};                                      // the chunk whose epilogue is pending
+        int g = 0;                                                  // tiles of all chunks so far
+        int k = 0;
+        for (; !aborted; ++k) {
+            const int wq = k % kUmmaQueue;
+            bool fine = mbarrier_poll_bounded(misc + kUmmaBarWorkFull + wq * 8, (k / kUmmaQueue) & 1);
+            if (softmax_any(!fine)) {                               // one decision for the four warps
+                aborted = true;
+                break;
+            }
+            const int w = work[wq].x, len = work[wq].y;
+            __syncwarp();
+            if (lane == 0) mbarrier_arrive(misc + kUmmaBarWorkEmpty + wq * 8);
+            if (w < 0) break;
+            const UmmaChunk c = umma_chunk(a, w, len);
+            const int n_tiles = c.n_tiles;
+            const unsigned acc = lane_base + 32 + (k & 1) * 32;     // this chunk's accumulator
+            float m[16], l[16];
+#pragma unroll
+            for (int r = 0; r < 16; ++r) {
+                m[r] = kMinusHuge;
+                l[r] = 0.f;
+            }
+            const int unmasked_end = min(c.end, len - (p.q_tokens - 1));   // tiles ending here or before need no mask
+            for (int j = 0; j < n_tiles; ++j, ++g) {
+                const int sb = g & 1;
+                // (warp-uniform: the tensor-memory loads below are warp-wide instructions)
+                if (fine) fine = __all_sync(0xffffffffu, mbarrier_poll_bounded(misc + kUmmaBarSFull + sb * 8, (g >> 1) & 1));
+                float s[16];
+                if (fine) {
+                    tc_fence_after();
+                    tc_load16(s, lane_base + sb * 16);
+                    tc_fence_before();
+                } else {
+#pragma unroll
+                    for (int r = 0; r < 16; ++r) s[r] = 0.f;
+                }
+                __syncwarp();
+                if (lane == 0) mbarrier_arrive(misc + kUmmaBarSFree + sb * 8);
+                const int tile_start = c.begin + j * kUmmaTile;
+                const int tok = tile_start + t;
+#pragma unroll
+                for (int r = 0; r < 16; ++r) s[r] *= a.scale_log2e;
+                if (tile_start + kUmmaTile > unmasked_end) {       // uniform: last tiles of the sequence / chunk
+#pragma unroll
+                    for (int r = 0; r < 16; ++r) {
+                        const int vis = r < p.rows ? len - (p.q_tokens - 1 - r / p.group) : 0;
+                        if (tok >= min(vis, c.end)) s[r] = -INFINITY;
+                    }
+                    if (tok >= c.end && fine) {
+                        // The value row of a position outside the chunk gets weight zero, but its bytes
+                        // may be anything (the tail of a block, a slot not fetched): 0 x NaN must not
+                        // reach the accumulator, so the row is cleared once the tile has landed.
+                        const int slot = g % kUmmaVSlots;
+                        fine = mbarrier_poll_bounded(misc + kUmmaBarVFull + slot * 8, (g / kUmmaVSlots) & 1);
+                        const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
+                        unsigned char *vrow = smem + kVOffset + slot * kUmmaItemBytes + t * 128;
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) {
+                            *reinterpret_cast<uint4 *>(vrow + i * 16) = zero;
+                            *reinterpret_cast<uint4 *>(vrow + kUmmaPanelBytes + i * 16) = zero;
+                        }
+                    }
+                }
+                bool moved = false;
+#pragma unroll
+                for (int r = 0; r < 16; ++r) moved = moved || s[r] > m[r] + kGroupLag;
+                if (!fine) *abort_word = 1u;
+                bool waited = false;
+                if (softmax_any(moved || !fine)) {
+                    if (*abort_word != 0u) {                        // the same for all 128 threads
+                        aborted = true;
+                        break;
+                    }
+                    // Some row's reference moves: row maxima over the tile, new references, and the
+                    // accumulator (and the sums) rescaled to them.
+                    float tops[16];
+#pragma unroll
+                    for (int r = 0; r < 16; ++r) tops[r] = s[r];
+                    const float top_mine = warp_reduce16<true>(tops, lane);
+                    if ((lane & 1) == 0) red[warp * 16 + warp_reduce16_row(lane)] = top_mine;
+                    softmax_sync();
+                    float alpha[16];
+                    bool any_change = false;
+#pragma unroll
+                    for (int r = 0; r < 16; ++r) {
+                        const float top = fmaxf(fmaxf(red[r], red[16 + r]), fmaxf(red[32 + r], red[48 + r]));
+                        alpha[r] = 1.f;
+                        if (top > m[r] + kGroupLag) {
+                            alpha[r] = fast_exp2(m[r] - top);
+                            m[r] = top;
+                            any_change = true;
+                        }
+                        l[r] *= alpha[r];
+                    }
+                    if (j > 0 && any_change) {
+                        // the accumulator holds tiles 0 .. j-1 once the previous tile's MMA is complete
+                        fine = __all_sync(0xffffffffu, mbarrier_poll_bounded(misc + kUmmaBarPvDone, (g - 1) & 1));
+                        waited = true;
+                        if (fine) {
+                            tc_fence_after();
+                            float o[16];
+#pragma unroll
+                            for (int half = 0; half < 2; ++half) {  // columns 0-15: high parts, 16-31: low parts
+                                tc_load16(o, acc + half * 16);
+#pragma unroll
+                                for (int r = 0; r < 16; ++r) o[r] *= alpha[r];
+                                tc_store16(acc + half * 16, o);
+                            }
+                        } else {
+                            *abort_word = 1u;                       // seen by all at the next vote
+                        }
+                    }
+                }
+                // Weights against the references (scaled by kGroupWeightScale inside the exponent),
+                // their sums, and the fp16 high and low parts: thread t holds row t of operand B
+                // (MN-major: 8 columns = 16 bytes per token and column block).
+                unsigned hi[8], lo[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const float w0 = fast_exp2(s[2 * i] - (m[2 * i] - kGroupWeightLog2));
+                    const float w1 = fast_exp2(s[2 * i + 1] - (m[2 * i + 1] - kGroupWeightLog2));
+                    l[2 * i] += w0;
+                    l[2 * i + 1] += w1;
+                    hi[i] = pack_half2(w0, w1);
+                    const float2 back = __half22float2(*reinterpret_cast<const __half2 *>(&hi[i]));
+                    lo[i] = pack_half2(w0 - back.x, w1 - back.y);
+                }
+                if (g > 0 && !waited && fine) {                     // the previous MMA has read the weights
+                    fine = mbarrier_poll_bounded(misc + kUmmaBarPvDone, (g - 1) & 1);
+                    if (!fine) *abort_word = 1u;
+                }
+                unsigned char *prow = smem + kPOffset + t * 16;
+                *reinterpret_cast<uint4 *>(prow) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+                *reinterpret_cast<uint4 *>(prow + 2048) = make_uint4(hi[4], hi[5], hi[6], hi[7]);
+                *reinterpret_cast<uint4 *>(prow + 4096) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+                *reinterpret_cast<uint4 *>(prow + 6144) = make_uint4(lo[4], lo[5], lo[6], lo[7]);
+                fence_async_proxy();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbarrier_arrive(misc + kUmmaBarPFull);
+                if (j == 0 && pending) {
+                    // The previous chunk's last MMA is complete (this thread waited for it before
+                    // writing this tile's weights) and its sums were stored before this tile's vote.
+                    if (__all_sync(0xffffffffu, fine)) epilogue(before, (k - 1) & 1);
+                    pending = false;
+                }
+            }
+            if (aborted) break;
+            // the chunk's references and row sums, for its epilogue
+            const float sum_mine = warp_reduce16<false>(l, lane);
+            if ((lane & 1) == 0) saved_l[(k & 1) * 64 + warp * 16 + warp_reduce16_row(lane)] = sum_mine;
+            if (t < 16) {
+                float mine = m[0];
+#pragma unroll
+                for (int r = 1; r < 16; ++r) mine = t == r ? m[r] : mine;
+                saved_m[(k & 1) * 16 + t] = mine;
+            }
+            before = c;
+            pending = true;
+            if (!fine) *abort_word = 1u;
         }
+        if (!aborted && pending) {
+            // the last chunk: its last MMA has not been waited for yet
+            const bool fine = __all_sync(0xffffffffu, mbarrier_poll_bounded(misc + kUmmaBarPvDone, (g - 1) & 1));
+            if (!softmax_any(!fine || *abort_word != 0u)) epilogue(before, (k - 1) & 1);
+            else aborted = true;
+        }
+        if (aborted && t == 0 && a.status) atomicOr(a.status, kFlagCopyTimeout);
     }
 
     // ---- teardown: everyone is done with tensor memory before it is released ----
     tc_fence_before();
     __syncthreads();
-    if (warp == 5) {
+    if (warp == kUmmaWarpLogits) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(tmem), "n"(kUmmaTmemCols) : "memory");
     }
