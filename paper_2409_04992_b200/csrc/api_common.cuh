@@ -128,9 +128,10 @@ struct PlanRules {
     int tail_chunk_tokens;       // 0: no short chunks at the end of long sequences
     int block_overhead_tokens;   // > 0: choose the chunk count by modelled time (see make_plan)
     bool allow_cluster;          // the kernel has the cluster form for small problems
+    int chunk_granule;           // chunk lengths are multiples of this (0: kChunkGranule)
 };
-constexpr PlanRules kOneRowRules = {kCtasPerSm, kTargetWaves, kChunkCeiling, kTailChunk, 0, true};
-constexpr PlanRules kNoClusterRules = {kCtasPerSm, kTargetWaves, kChunkCeiling, kTailChunk, 0, false};
+constexpr PlanRules kOneRowRules = {kCtasPerSm, kTargetWaves, kChunkCeiling, kTailChunk, 0, true, 0};
+constexpr PlanRules kNoClusterRules = {kCtasPerSm, kTargetWaves, kChunkCeiling, kTailChunk, 0, false, 0};
 constexpr int kClusterMaxChunks = 8;     // portable cluster size
 constexpr int kClusterMaxChunkTokens = 512;
 
@@ -145,6 +146,7 @@ inline SplitPlan make_plan(int64_t pairs, int32_t max_seq_len, const PlanRules &
         return plan;
     }
     const int64_t slots = (int64_t)sm_count() * rules.ctas_per_sm;
+    const int64_t granule = rules.chunk_granule > 0 ? rules.chunk_granule : kChunkGranule;
     if (rules.allow_cluster) {
         // Small problems are bound by launch and memory latency, not by bandwidth: at most 8
         // chunks per sequence, all resident at once, merged inside the kernel by a cluster.
@@ -172,7 +174,7 @@ inline SplitPlan make_plan(int64_t pairs, int32_t max_seq_len, const PlanRules &
         int64_t best = -1;
         const int64_t last = most < fewest + 96 ? most : fewest + 96;
         for (int64_t c = fewest; c <= last; ++c) {
-            const int64_t len = ceil_div(ceil_div(max_seq_len, c), kChunkGranule) * kChunkGranule;
+            const int64_t len = ceil_div(ceil_div(max_seq_len, c), granule) * granule;
             const int64_t cost = ceil_div(pairs * ceil_div(max_seq_len, len), slots) *
                                  (len + rules.block_overhead_tokens);
             if (best < 0 || cost < best) {
@@ -181,7 +183,7 @@ inline SplitPlan make_plan(int64_t pairs, int32_t max_seq_len, const PlanRules &
             }
         }
     }
-    int64_t chunk = ceil_div(ceil_div(max_seq_len, n), kChunkGranule) * kChunkGranule;
+    int64_t chunk = ceil_div(ceil_div(max_seq_len, n), granule) * granule;
     // Short region: about kTailWaves waves of tail_chunk-token blocks at the start of every
     // sequence, at most a quarter of the longest; none when the chunks are that short anyway.
     const int64_t tail_chunk = rules.tail_chunk_tokens > 0 ? rules.tail_chunk_tokens : kTailChunk;
@@ -189,7 +191,7 @@ inline SplitPlan make_plan(int64_t pairs, int32_t max_seq_len, const PlanRules &
     if (short_tokens > max_seq_len / 4) short_tokens = max_seq_len / 4 / tail_chunk * tail_chunk;
     if (chunk <= 2 * tail_chunk || short_tokens < tail_chunk || rules.tail_chunk_tokens <= 0) short_tokens = 0;
     if (short_tokens > 0)
-        chunk = ceil_div(ceil_div(max_seq_len - short_tokens, n), kChunkGranule) * kChunkGranule;
+        chunk = ceil_div(ceil_div(max_seq_len - short_tokens, n), granule) * granule;
     const int64_t n_short = short_tokens > 0 ? short_tokens / tail_chunk : 0;
     plan.chunk_tokens = (int32_t)chunk;
     plan.n_big = (int32_t)ceil_div(max_seq_len - short_tokens, chunk);

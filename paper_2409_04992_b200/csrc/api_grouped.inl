@@ -16,8 +16,13 @@ PlanRules grouped_rules(int32_t head_dim)
 {
     const int ctas = head_dim == 64 ? GroupedGeometry<64>::kCtasPerSm
                    : head_dim == 128 ? GroupedGeometry<128>::kCtasPerSm : GroupedGeometry<256>::kCtasPerSm;
-    return PlanRules{ctas, 2, 4096, 1024, 320, false};
+    return PlanRules{ctas, 2, 4096, 1024, 320, false, 0};
 }
+
+// The tcgen05 form is persistent (one block per SM draws chunks from a counter), so waves do not
+// matter; chunks are whole 128-token tiles, long enough (up to 4096 tokens) that the per-chunk
+// epilogue is small, with 1024-token chunks drawn last to even out the end of the launch.
+PlanRules umma_rules() { return PlanRules{1, 8, 4096, 1024, 0, false, 128}; }
 
 size_t grouped_workspace_for(int64_t pairs, int32_t rows, int32_t head_dim, const SplitPlan &plan)
 {
@@ -183,11 +188,19 @@ int instinfer_decode_attention_grouped(void *out, float *lse, const void *q, con
         return INSTINFER_ERR_INVALID_ARG;
 
     const int64_t pairs = (int64_t)batch * kv_heads;
-    const SplitPlan plan = make_plan(pairs, max_seq_len, grouped_rules(head_dim));
     GroupedParams p = {};
     p.group = q_heads / kv_heads;
     p.q_tokens = q_tokens;
     p.rows = p.group * q_tokens;
+    const int64_t kv_bytes = (paged ? num_phys_blocks * kv_heads * block_tokens : (int64_t)batch * kv_heads * s_max) * head_dim * 2;
+    // The tcgen05 form needs the caches and the query as the copy engine sees them; a cache of
+    // 2^31 rows or more, or a driver without the encoder, takes the warp-level form.
+    CUtensorMap map_q, map_k, map_v;
+    const bool umma = g_grouped_path != 1 && umma_shape(head_dim, paged, block_tokens) &&
+                      make_query_map(&map_q, q, batch, q_tokens, q_heads, p.group) &&
+                      make_cache_map(&map_k, k_cache, kv_bytes / 256, paged ? block_tokens : kUmmaTile) &&
+                      make_cache_map(&map_v, v_cache, kv_bytes / 256, paged ? block_tokens : kUmmaTile);
+    const SplitPlan plan = make_plan(pairs, max_seq_len, umma ? umma_rules() : grouped_rules(head_dim));
     if (workspace == nullptr || !aligned16(workspace) ||
         workspace_bytes < grouped_workspace_for(pairs, p.rows, head_dim, plan))
         return INSTINFER_ERR_WORKSPACE;
@@ -211,26 +224,19 @@ int instinfer_decode_attention_grouped(void *out, float *lse, const void *q, con
     p.a.tail_chunk = plan.tail_chunk;
     p.a.n_splits = plan.n_splits;
     p.a.max_seq_len = max_seq_len;
-    p.a.kv_bytes = (paged ? num_phys_blocks * kv_heads * block_tokens : (int64_t)batch * kv_heads * s_max) * head_dim * 2;
+    p.a.kv_bytes = kv_bytes;
     p.a.scale_log2e = scale * 1.44269504088896340736f;
     p.a.part_o = static_cast<float *>(workspace);
     p.a.part_lse = p.a.part_o + (size_t)pairs * plan.n_splits * p.rows * head_dim;
 
     const unsigned grid = (unsigned)(pairs * plan.n_splits);
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    if (g_grouped_path == 2 && umma_shape(head_dim, paged, block_tokens)) {     // automatic: warp-level, for now
-        // The cache as the copy engine sees it; a cache of 2^31 rows or more, or a driver
-        // without the encoder, takes the warp-level form below.
-        const int64_t rows = p.a.kv_bytes / (2 * 128);
-        CUtensorMap map_q, map_k, map_v;
+    if (umma) {
         // the ticket counter sits in the last 256 bytes of the workspace, behind the partials
         unsigned *ticket = reinterpret_cast<unsigned *>(
             static_cast<unsigned char *>(workspace) + grouped_workspace_for(pairs, p.rows, head_dim, plan) - 256);
-        if (make_query_map(&map_q, q, batch, q_tokens, q_heads, p.group) &&
-            make_cache_map(&map_k, k_cache, rows, paged ? block_tokens : kUmmaTile) &&
-            make_cache_map(&map_v, v_cache, rows, paged ? block_tokens : kUmmaTile))
-            return paged ? launch_grouped_umma<true>(p, ticket, map_q, map_k, map_v, stream)
-                         : launch_grouped_umma<false>(p, ticket, map_q, map_k, map_v, stream);
+        return paged ? launch_grouped_umma<true>(p, ticket, map_q, map_k, map_v, stream)
+                     : launch_grouped_umma<false>(p, ticket, map_q, map_k, map_v, stream);
     }
     switch (head_dim) {
     case 64: return paged ? launch_grouped<64, true>(p, grid, stream) : launch_grouped<64, false>(p, grid, stream);
@@ -245,8 +251,14 @@ size_t instinfer_grouped_workspace_bytes(int32_t batch, int32_t q_tokens, int32_
     if (grouped_shape(batch, q_tokens, q_heads, kv_heads, head_dim, max_seq_len) != INSTINFER_OK) return 0;
     const int64_t pairs = (int64_t)batch * kv_heads;
     if (pairs == 0) return 256;
-    return grouped_workspace_for(pairs, q_heads / kv_heads * q_tokens, head_dim,
-                                 make_plan(pairs, max_seq_len, grouped_rules(head_dim)));
+    // enough for either implementation: which one runs also depends on the cache layout
+    const int32_t rows = q_heads / kv_heads * q_tokens;
+    size_t bytes = grouped_workspace_for(pairs, rows, head_dim, make_plan(pairs, max_seq_len, grouped_rules(head_dim)));
+    if (head_dim == 128) {
+        const size_t other = grouped_workspace_for(pairs, rows, head_dim, make_plan(pairs, max_seq_len, umma_rules()));
+        if (other > bytes) bytes = other;
+    }
+    return bytes;
 }
 
 int instinfer_set_grouped_path(int32_t path)

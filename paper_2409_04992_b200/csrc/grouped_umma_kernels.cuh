@@ -13,26 +13,34 @@
 //
 // The kernel is persistent: one block per SM draws chunks (token ranges of one (sequence, KV
 // head), the same list one block per chunk would run) from a ticket counter, and its copy
-// pipeline runs on across chunk boundaries.  A block is specialised by warp:
-//   * warp 4 (producer) moves 128-token tiles of K and of V with tensor-map copies
-//     (cp.async.bulk.tensor, 128-byte swizzle, this GPU's memory, no multicast) into a ring of
-//     32 KiB slots; a paged tile is 128 / T copies of one (block, head) run each, the block
-//     ids read one tile ahead; a block with a bad id is not fetched but zero-filled.  It also
-//     draws the tickets (one chunk ahead), announces each chunk to the other warps through a
-//     small queue in shared memory and fetches the chunk's query rows;
-//   * one lane of warp 5 issues the MMAs: K tile (K-major, as it lies in the cache) against the
-//     query rows held in shared memory -> logits in tensor memory (two buffers, so the next
-//     tile's logits are computed while this tile's are being exponentiated); V tile (the same
-//     bytes read MN-major: no transpose anywhere) against the weights in shared memory ->
-//     the output accumulator in tensor memory;
+// pipeline runs on across chunk boundaries.  A block has eight warps, each with one job, that
+// hand tiles to one another through mbarriers:
+//   * warp 4 (K producer) moves 128-token tiles of K with tensor-map copies (cp.async.bulk.tensor,
+//     128-byte swizzle, this GPU's memory, no multicast) into a ring of three 32 KiB slots; a
+//     paged tile is 128 / T copies of one (block, head) run each, the block ids read one tile
+//     ahead; a block with a bad id is not fetched but zero-filled.  It also draws the tickets
+//     (two chunks ahead, so the atomic's round trip is hidden), announces each chunk to the
+//     other warps through a small queue in shared memory and fetches the chunk's query rows;
+//   * warp 5 (V producer) does the same for the V tiles into a ring of its own;
+//   * warp 6 issues the logit MMAs: K tile (K-major, as it lies in the cache) against the query
+//     rows -> logits in tensor memory (two buffers, so it runs up to two tiles ahead of the
+//     softmax); warp 7 issues the output MMAs: V tile (the same bytes read MN-major: no
+//     transpose anywhere) against the weights in shared memory -> the accumulator in tensor
+//     memory (one per chunk parity).  One thread issuing both took 2250 cycles per tile, more
+//     than the tile's copy time: two issuers halve that.  Both warps run converged and
+//     predicate only the issue, so descriptors stay warp-uniform values;
 //   * warps 0-3 (softmax): thread t owns token t of the tile, i.e. lane t of tensor memory: it
 //     reads its 16 logits, masks, exponentiates against per-row references that all threads
 //     hold alike and that follow the maximum lazily (a reference moves only when a logit
 //     exceeds it by more than kGroupLag; then the accumulator in tensor memory is rescaled,
-//     which is rare), and writes its 32 fp16 weights where the second MMA expects them;
-//   * the epilogue reads the accumulator (thread = output dim), adds the high and low halves,
-//     divides by the row sums and writes the chunk's partial (or the result itself when the
-//     sequence is one chunk).
+//     which is rare), and writes its 32 fp16 weights where the output MMA expects them;
+//   * a chunk's epilogue (thread = output dim: accumulator columns r and 16 + r added, divided
+//     by the row sum, written as the chunk's partial, or as the result when the sequence is
+//     one chunk) runs after the first tile of the next chunk has been handed on, so that
+//     nothing waits for it.
+// Waits of the warps that run ahead (producers, logit issuer) let the hardware park the warp;
+// the waits on the chain softmax -> output MMA -> softmax poll, because there the time to
+// notice a completed phase adds to every tile.
 // Every wait is on an mbarrier and bounded by the clock; a wait that runs out sets
 // kFlagCopyTimeout, the block stops waiting, releases its tensor memory and ends.
 #pragma once
@@ -172,6 +180,14 @@ __host__ __device__ constexpr unsigned umma_idesc(int m, int n, int a_mn_major, 
 {
     return 1u << 4 | (unsigned)a_mn_major << 15 | (unsigned)b_mn_major << 16 | (unsigned)(n >> 3) << 17 |
            (unsigned)(m >> 4) << 24;
+}
+// One lane of a converged warp (the MMA warps run converged so that descriptors and addresses
+// stay warp-uniform values; only the issue itself is predicated).
+__device__ __forceinline__ bool elect_one()
+{
+    unsigned chosen;
+    asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(chosen));
+    return chosen != 0;
 }
 // Barrier over the 128 softmax threads that also ORs a predicate.
 __device__ __forceinline__ bool softmax_any(bool mine)
@@ -353,7 +369,7 @@ grouped_attn_umma_kernel(const GroupedParams p, unsigned *ticket, const __grid_c
             }
             const int slot = count % slots;
             if (count >= slots &&
-                !__all_sync(0xffffffffu, mbarrier_poll_bounded(misc + bar_empty + slot * 8, (count / slots - 1) & 1)))
+                !__all_sync(0xffffffffu, mbarrier_wait_bounded(misc + bar_empty + slot * 8, (count / slots - 1) & 1)))
                 return false;
             const int slot_offset = ring_offset + slot * kUmmaItemBytes + (kPaged ? lane * T * 128 : 0);
             const unsigned bar = misc + bar_full + slot * 8;
@@ -506,46 +522,51 @@ grouped_attn_umma_kernel(const GroupedParams p, unsigned *ticket, const __grid_c
         // ================================ logit MMAs ================================
         // One lane issues S^T = K_tile Q^T for every tile of every chunk of this block, as far
         // ahead of the softmax warps as the two logit buffers allow.
-        if (lane == 0) {
+        {
             constexpr unsigned idesc = umma_idesc(128, 16, 0, 0);          // K tile K-major, Q K-major
             bool fine = true;
             int g = 0;                                                      // tiles of all chunks so far
             for (int k = 0; fine; ++k) {
                 const int wq = k % kUmmaQueue;
-                fine = mbarrier_poll_bounded(misc + kUmmaBarWorkFull + wq * 8, (k / kUmmaQueue) & 1);
+                fine = __all_sync(0xffffffffu, mbarrier_wait_bounded(misc + kUmmaBarWorkFull + wq * 8, (k / kUmmaQueue) & 1));
                 if (!fine) break;
-                const int w = work[wq].x, len = work[wq].y;
-                mbarrier_arrive(misc + kUmmaBarWorkEmpty + wq * 8);
+                const int w = __shfl_sync(0xffffffffu, work[wq].x, 0), len = __shfl_sync(0xffffffffu, work[wq].y, 0);
+                __syncwarp();
+                if (elect_one()) mbarrier_arrive(misc + kUmmaBarWorkEmpty + wq * 8);
                 if (w < 0) break;
                 const int n_tiles = umma_chunk(a, w, len).n_tiles;
-                fine = mbarrier_poll_bounded(misc + kUmmaBarQFull + (k & 1) * 8, (k / 2) & 1);
+                fine = __all_sync(0xffffffffu, mbarrier_wait_bounded(misc + kUmmaBarQFull + (k & 1) * 8, (k / 2) & 1));
                 // K tile and query rows alike: rows of 128 bytes per 64-dim panel, 8-row groups 1024
                 // bytes apart, 128-byte swizzle; a k-step of 16 dims is 32 bytes along the row
                 const uint64_t q_desc = umma_desc(q_smem + (k & 1) * kUmmaQBytes, 16, 1024, 2);
                 for (int j = 0; j < n_tiles && fine; ++j, ++g) {
                     const int slot = g % kUmmaKSlots;
-                    fine = mbarrier_poll_bounded(misc + kUmmaBarKFull + slot * 8, (g / kUmmaKSlots) & 1) &&
-                           (g < 2 || mbarrier_poll_bounded(misc + kUmmaBarSFree + (g & 1) * 8, ((g >> 1) - 1) & 1));
+                    fine = __all_sync(0xffffffffu,
+                                      mbarrier_wait_bounded(misc + kUmmaBarKFull + slot * 8, (g / kUmmaKSlots) & 1) &&
+                                      (g < 2 || mbarrier_wait_bounded(misc + kUmmaBarSFree + (g & 1) * 8, ((g >> 1) - 1) & 1)));
                     if (!fine) break;
                     tc_fence_after();
                     const uint64_t k_desc = umma_desc(ring + slot * kUmmaItemBytes, 16, 1024, 2);
+                    if (elect_one()) {
 #pragma unroll
-                    for (int ks = 0; ks < 8; ++ks)
-                        tc_mma_f16(tmem + (g & 1) * 16, k_desc + (uint64_t)(((ks >> 2) * kUmmaPanelBytes + (ks & 3) * 32) >> 4),
-                                   q_desc + (uint64_t)(((ks >> 2) * (kUmmaQBytes / 2) + (ks & 3) * 32) >> 4), idesc, ks > 0);
-                    tc_commit(misc + kUmmaBarSFull + (g & 1) * 8);
-                    tc_commit(misc + kUmmaBarKEmpty + slot * 8);
-                    // after the chunk's last logit MMA its query rows may be replaced
-                    if (j + 1 == n_tiles) tc_commit(misc + kUmmaBarQEmpty + (k & 1) * 8);
+                        for (int ks = 0; ks < 8; ++ks)
+                            tc_mma_f16(tmem + (g & 1) * 16, k_desc + (uint64_t)(((ks >> 2) * kUmmaPanelBytes + (ks & 3) * 32) >> 4),
+                                       q_desc + (uint64_t)(((ks >> 2) * (kUmmaQBytes / 2) + (ks & 3) * 32) >> 4), idesc, ks > 0);
+                        tc_commit(misc + kUmmaBarSFull + (g & 1) * 8);
+                        tc_commit(misc + kUmmaBarKEmpty + slot * 8);
+                        // after the chunk's last logit MMA its query rows may be replaced
+                        if (j + 1 == n_tiles) tc_commit(misc + kUmmaBarQEmpty + (k & 1) * 8);
+                    }
+                    __syncwarp();
                 }
             }
-            if (!fine && a.status) atomicOr(a.status, kFlagCopyTimeout);
+            if (!fine && lane == 0 && a.status) atomicOr(a.status, kFlagCopyTimeout);
         }
         __syncwarp();
     } else if (warp == kUmmaWarpOutput) {
         // ================================ output MMAs ================================
         // One lane issues O^T += V_tile^T P^T for every tile, into the accumulator of the chunk's parity.
-        if (lane == 0) {
+        {
             constexpr unsigned idesc = umma_idesc(128, 32, 1, 1);          // V tile MN-major, weights MN-major
             // Weights: 8-column blocks of [128 tokens][16 bytes], 2048 bytes apart; 8-token groups
             // 128 bytes apart; a k-step is 16 tokens = 256 bytes.
@@ -554,33 +575,39 @@ grouped_attn_umma_kernel(const GroupedParams p, unsigned *ticket, const __grid_c
             int g = 0;
             for (int k = 0; fine; ++k) {
                 const int wq = k % kUmmaQueue;
-                fine = mbarrier_poll_bounded(misc + kUmmaBarWorkFull + wq * 8, (k / kUmmaQueue) & 1);
+                fine = __all_sync(0xffffffffu, mbarrier_poll_bounded(misc + kUmmaBarWorkFull + wq * 8, (k / kUmmaQueue) & 1));
                 if (!fine) break;
-                const int w = work[wq].x, len = work[wq].y;
-                mbarrier_arrive(misc + kUmmaBarWorkEmpty + wq * 8);
+                const int w = __shfl_sync(0xffffffffu, work[wq].x, 0), len = __shfl_sync(0xffffffffu, work[wq].y, 0);
+                __syncwarp();
+                if (elect_one()) mbarrier_arrive(misc + kUmmaBarWorkEmpty + wq * 8);
                 if (w < 0) break;
                 const int n_tiles = umma_chunk(a, w, len).n_tiles;
                 // the accumulator of this parity was last used two chunks ago: its epilogue must have read it
-                if (k >= 2) fine = mbarrier_poll_bounded(misc + kUmmaBarAccFree + (k & 1) * 8, (k / 2 - 1) & 1);
+                if (k >= 2)
+                    fine = __all_sync(0xffffffffu, mbarrier_poll_bounded(misc + kUmmaBarAccFree + (k & 1) * 8, (k / 2 - 1) & 1));
                 const unsigned acc = tmem + 32 + (k & 1) * 32;
                 for (int j = 0; j < n_tiles && fine; ++j, ++g) {
                     const int slot = g % kUmmaVSlots;
-                    fine = mbarrier_poll_bounded(misc + kUmmaBarVFull + slot * 8, (g / kUmmaVSlots) & 1) &&
-                           mbarrier_poll_bounded(misc + kUmmaBarPFull, g & 1);
+                    fine = __all_sync(0xffffffffu,
+                                      mbarrier_poll_bounded(misc + kUmmaBarVFull + slot * 8, (g / kUmmaVSlots) & 1) &&
+                                      mbarrier_poll_bounded(misc + kUmmaBarPFull, g & 1));
                     if (!fine) break;
                     tc_fence_after();
                     // V tile read MN-major (M = dims): the two 64-dim panels are kUmmaPanelBytes apart
                     // (leading offset), 8-token groups 1024 bytes apart; a k-step is 16 tokens = 2048 bytes
                     const uint64_t v_desc = umma_desc(ring + kVOffset + slot * kUmmaItemBytes, kUmmaPanelBytes, 1024, 2);
+                    if (elect_one()) {
 #pragma unroll
-                    for (int ks = 0; ks < 8; ++ks)
-                        tc_mma_f16(acc, v_desc + (uint64_t)((ks * 2048) >> 4), p_desc + (uint64_t)((ks * 256) >> 4), idesc,
-                                   j > 0 || ks > 0);
-                    tc_commit(misc + kUmmaBarVEmpty + slot * 8);
-                    tc_commit(misc + kUmmaBarPvDone);
+                        for (int ks = 0; ks < 8; ++ks)
+                            tc_mma_f16(acc, v_desc + (uint64_t)((ks * 2048) >> 4), p_desc + (uint64_t)((ks * 256) >> 4), idesc,
+                                       j > 0 || ks > 0);
+                        tc_commit(misc + kUmmaBarVEmpty + slot * 8);
+                        tc_commit(misc + kUmmaBarPvDone);
+                    }
+                    __syncwarp();
                 }
             }
-            if (!fine && a.status) atomicOr(a.status, kFlagCopyTimeout);
+            if (!fine && lane == 0 && a.status) atomicOr(a.status, kFlagCopyTimeout);
         }
         __syncwarp();
     } else {
