@@ -33,7 +33,8 @@ SparfLayout sparf_layout(int64_t pairs, int32_t max_seq_len, int32_t max_k)
     w.row_ids = w.stage_pos + round256((size_t)pairs * w.score_stride * sizeof(int32_t));
     w.stats = w.row_ids + round256((size_t)pairs * max_k * sizeof(int32_t));
     w.rows_state = w.stats + round256((size_t)pairs * sizeof(float2));
-    w.row_cand = w.rows_state + round256((size_t)pairs * sizeof(SelectRow));
+    // (+ one counter behind the rows: how many rows the chain left unsolved)
+    w.row_cand = w.rows_state + round256(((size_t)pairs + 1) * sizeof(SelectRow));
     w.zeroed_bytes = w.row_cand - w.rows_state;
     w.seg_count = w.row_cand + round256((size_t)pairs * w.cand_capacity * sizeof(uint2));
     w.seg_final = w.seg_count + round256((size_t)pairs * w.segments * sizeof(int32_t));
@@ -232,6 +233,7 @@ int instinfer_sparf_decode_attention(void *out, float *alpha, int32_t *selected,
     sp.scale_log2e = scale * 1.44269504088896340736f;
 
     sp.rows_state = reinterpret_cast<SelectRow *>(ws + w.rows_state);
+    sp.unsolved = reinterpret_cast<int *>(sp.rows_state + pairs);
     sp.row_cand = reinterpret_cast<uint2 *>(ws + w.row_cand);
     sp.seg_count = reinterpret_cast<int32_t *>(ws + w.seg_count);
     sp.seg_final = reinterpret_cast<int32_t *>(ws + w.seg_final);

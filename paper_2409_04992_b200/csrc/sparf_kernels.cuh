@@ -62,6 +62,7 @@ struct SparfParams {
     int32_t *row_ids;          // [pairs, max_k]
     float2 *stats;             // [pairs] (alpha, number of selected rows)
     struct SelectRow *rows_state;   // [pairs], zeroed before each call
+    int *unsolved;             // rows the staged chain could not settle (zeroed with rows_state)
     uint2 *row_cand;           // [pairs, cand_capacity] (ordered key, token index)
     int32_t *seg_count;        // [pairs, segments] staged tokens per segment
     int32_t *seg_final;        // [pairs, segments] selected tokens per segment
@@ -311,6 +312,7 @@ sparf_scores_kernel(const SparfParams p)
     wait_for_previous_kernels();
     __shared__ ScoreShared ss;
     const int d = threadIdx.x;
+    if (*p.unsolved == 0) return;                            // the usual case: the chain settled every row
     const int64_t items = (int64_t)p.batch * p.heads * p.score_blocks;
     for (int64_t item = blockIdx.x; item < items; item += gridDim.x) {
         const int pair = (int)(item / p.score_blocks);
@@ -707,6 +709,7 @@ sparf_select_kernel(const SparfParams p)
     allow_next_kernel();
     wait_for_previous_kernels();
     __shared__ SelectShared sh;
+    if (*p.unsolved == 0) return;                            // the usual case: the chain settled every row
     const int pairs = p.batch * p.heads;
     for (int pair = blockIdx.x; pair < pairs; pair += gridDim.x) {
         if (p.rows_state[pair].solved) continue;             // done by the staged chain

@@ -313,7 +313,10 @@ sparf_resolve_kernel(const SparfParams p)
     const int n = row->n_cand, need = k - sure;
     // The bracket must hold the threshold: the sure tokens do not exceed k, and together with
     // the candidates they reach it.
-    if (row->overflow || n > p.cand_capacity || need < 0 || need > n) return;       // unsolved
+    if (row->overflow || n > p.cand_capacity || need < 0 || need > n) {               // unsolved
+        if (tid == 0) atomicAdd(p.unsolved, 1);
+        return;
+    }
     if (need == 0) {                     // exactly the sure tokens: every logit above the upper bound, no candidate
         if (tid == 0) {
             row->tau = ordered_key(row->hi);
