@@ -437,6 +437,14 @@ int instinfer_set_sparse_path(int32_t path);
  */
 int instinfer_set_grouped_path(int32_t path);
 
+/*
+ * Which of the two implementations instinfer_decode_attention_grouped takes for a head size
+ * and a cache layout (block_tokens = 0: contiguous), under the current setting of
+ * instinfer_set_grouped_path: 1 warp-level, 2 tcgen05, 0 for a shape the entry point refuses.
+ * (A cache of 2^31 rows or more still takes the warp-level form at call time.)  Host only.
+ */
+int32_t instinfer_grouped_path_for(int32_t head_dim, int32_t block_tokens);
+
 
 /*
  * Measurement aid (no counterpart in the paper).  Given two cudaEvent_t (as void*, owned by

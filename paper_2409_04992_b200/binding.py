@@ -87,6 +87,8 @@ def load() -> ctypes.CDLL:
         lib.instinfer_set_sparse_path.argtypes = [i32]
         lib.instinfer_set_grouped_path.restype = ctypes.c_int
         lib.instinfer_set_grouped_path.argtypes = [i32]
+        lib.instinfer_grouped_path_for.restype = i32
+        lib.instinfer_grouped_path_for.argtypes = [i32, i32]
         lib.instinfer_sparf_workspace_bytes.restype = sz
         lib.instinfer_sparf_workspace_bytes.argtypes = [i32, i32, i32, i32, i32]
         lib.instinfer_workspace_bytes.restype = sz
@@ -344,6 +346,11 @@ def sparf_append_bulk(k_pool: torch.Tensor, v_pool: torch.Tensor, kt_pool: torch
         _ptr(seq_lens), _ptr(new_lens), _ptr(block_table), block_table.shape[1], k_pool.shape[2],
         k_pool.shape[0], _ptr(kt_block_table), kt_block_table.shape[1], kt_pool.shape[3],
         kt_pool.shape[0], batch, max_new, heads, head_dim, _ptr(status_flags), _stream(stream)))
+
+
+def grouped_path_for(head_dim: int, block_tokens: int) -> int:
+    """instinfer_grouped_path_for: 1 warp-level MMAs, 2 tcgen05, 0 unsupported (block_tokens 0: contiguous)."""
+    return int(load().instinfer_grouped_path_for(int(head_dim), int(block_tokens)))
 
 
 def set_grouped_path(path: int) -> None:

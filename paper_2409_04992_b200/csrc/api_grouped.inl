@@ -261,6 +261,14 @@ size_t instinfer_grouped_workspace_bytes(int32_t batch, int32_t q_tokens, int32_
     return bytes;
 }
 
+int32_t instinfer_grouped_path_for(int32_t head_dim, int32_t block_tokens)
+{
+    if (head_dim != 64 && head_dim != 128 && head_dim != 256) return 0;
+    if (block_tokens < 0 || (block_tokens > 0 && block_tokens % kGroupTile != 0)) return 0;
+    const bool paged = block_tokens > 0;
+    return g_grouped_path != 1 && umma_shape(head_dim, paged, block_tokens) && tensor_map_encoder() != nullptr ? 2 : 1;
+}
+
 int instinfer_set_grouped_path(int32_t path)
 {
     if (path < 0 || path > 2) return INSTINFER_ERR_INVALID_ARG;

@@ -136,6 +136,7 @@ int main(void)
     expect("sparse path range", instinfer_set_sparse_path(3), INSTINFER_ERR_INVALID_ARG);
     expect("grouped path range", instinfer_set_grouped_path(3), INSTINFER_ERR_INVALID_ARG);
     expect("grouped path automatic", instinfer_set_grouped_path(0), INSTINFER_OK);
+    expect("grouped path of a refused head size", instinfer_grouped_path_for(96, 16), 0);
     expect("timing events one null", instinfer_set_timing_events(fake, NULL), INSTINFER_ERR_INVALID_ARG);
     expect("timing events off", instinfer_set_timing_events(NULL, NULL), INSTINFER_OK);
     if (strcmp(instinfer_status_string(INSTINFER_OK), "ok") != 0) {

@@ -109,6 +109,27 @@ def test_other_head_sizes(dim, layout, tokens, q_tokens, q_heads, kv_heads):
               f"D={dim} {layout} Tq={q_tokens} Hq={q_heads} Hkv={kv_heads} chunk={chunk}")
 
 
+def test_the_tcgen05_form_is_the_one_that_runs(grouped_path):
+    """On a GPU machine the driver has the tensor-map encoder, so head size 128 with a contiguous
+    cache or 16/32/64-token blocks takes the tcgen05 kernel unless the warp-level one is forced."""
+    want = 2 if grouped_path == 2 else 1
+    for tokens in (0, 16, 32, 64):
+        assert binding.grouped_path_for(128, tokens) == want
+    binding.set_grouped_path(0)
+    assert binding.grouped_path_for(128, 16) == 2                                 # the default
+    assert binding.grouped_path_for(128, 48) == 1 and binding.grouped_path_for(128, 128) == 1
+    assert binding.grouped_path_for(64, 16) == 1 and binding.grouped_path_for(256, 0) == 1
+    assert binding.grouped_path_for(96, 16) == 0 and binding.grouped_path_for(128, 8) == 0
+
+
+def test_tiny_contiguous_cache_smaller_than_one_tile():
+    # fewer rows in the whole cache than one 128-token copy box
+    g = make("contiguous", 0, 1, 2, 4, lens=[20])
+    check(g, 0, "one sequence of 20 tokens, contiguous")
+    g = make("contiguous", 0, 2, 1, 2, lens=[1, 3])
+    check(g, 0, "two sequences of 1 and 3 tokens, contiguous")
+
+
 def test_peaked_logits():
     for chunk in (0, 64):
         g = make("paged", 32, 2, 2, 8, lens=[700, 1500, 40])
