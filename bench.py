@@ -690,6 +690,9 @@ def measure_grouped(device, steps: int = 20) -> dict:
         results[name] = {"value": kv_bytes / seconds / 1e9, "unit": UNIT, "ms_per_step": seconds * 1e3,
                          "kv_bytes_per_step": kv_bytes, "query_rows_per_kv_head": q_heads // kv_heads * q_tokens,
                          "roofline": sub_roofline(kv_bytes, seconds),
+                         "kernel": {1: "grouped_attn_split_kernel (warp-level mma.sync)",
+                                    2: "grouped_attn_umma_kernel (tcgen05, tensor memory, tensor-map copies)"}.get(
+                                        binding.grouped_path_for(dim, tokens), "?"),
                          "status_flags": int(flags.item())}
         del g, c, out, ws
         torch.cuda.empty_cache()
