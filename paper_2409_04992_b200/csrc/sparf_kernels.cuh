@@ -355,14 +355,16 @@ __device__ __forceinline__ T block_sum(T v, T *scratch)      // scratch: 32 entr
 constexpr int kLinearBins = 2048;        // select: linear bins between the smallest and largest logit
 constexpr int kCandidates = 8192;        // select: keys of the threshold bin resolved in shared memory
 
-struct SelectShared {
+struct SelectCore {
     unsigned hist[kLinearBins + 1];      // bin kLinearBins: the forced local window
-    unsigned cand[kCandidates];
     float red_f[32];
     unsigned red_u[2][32];
     int scan_gt[32], scan_eq[32];
     unsigned tau;
     int take_equal, bin, above, n_cand;
+};
+struct SelectShared : SelectCore {
+    unsigned cand[kCandidates];
 };
 
 // Streams a score row as float4 with 4 loads in flight per thread; fn(first_index, values[4]).
@@ -419,7 +421,7 @@ __device__ __forceinline__ void locate_bucket(const unsigned *hist, int remainin
 // a set of (nearly) equal keys costs nothing.  Returns through sh.tau / sh.take_equal the
 // threshold key and how many keys equal to it are among the `need` largest.
 template <int NT, typename Member, typename KeyAt>
-__device__ __forceinline__ void exact_threshold(SelectShared &sh, int n, int need, Member member, KeyAt key_at)
+__device__ __forceinline__ void exact_threshold(SelectCore &sh, int n, int need, Member member, KeyAt key_at)
 {
     const int tid = threadIdx.x;
     unsigned any = 0u, all = 0xffffffffu;

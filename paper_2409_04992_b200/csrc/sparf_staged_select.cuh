@@ -289,16 +289,18 @@ sparf_stage_kernel(const SparfParams p)
     if (far_above) row->overflow = 1;
 }
 
-// grid pairs, kResolveThreads threads (512, or 256 when the candidate lists are short), dynamic shared memory cand_capacity * 4 bytes (positions;
-// the keys sit in the select scratch).  cand_capacity <= kCandidates.
+// grid pairs, kResolveThreads threads (512, or 256 when the candidate lists are short), dynamic
+// shared memory cand_capacity * 4 bytes (the candidates' keys; their positions are read from
+// the list in global memory, which keeps the block small enough for many to share an SM).
+// cand_capacity <= kCandidates.
 template <int kResolveThreads>
 __global__ void __launch_bounds__(kResolveThreads)
 sparf_resolve_kernel(const SparfParams p)
 {
     allow_next_kernel();
     wait_for_previous_kernels();
-    extern __shared__ __align__(16) int where[];
-    __shared__ SelectShared sh;
+    extern __shared__ __align__(16) unsigned keys[];
+    __shared__ SelectCore sh;
     const int pair = blockIdx.x, tid = threadIdx.x;
     const int b = pair / p.heads;
     SelectRow *row = p.rows_state + pair;
@@ -325,13 +327,8 @@ sparf_resolve_kernel(const SparfParams p)
         }
         return;
     }
-    unsigned *keys = sh.cand;
     const uint2 *cand = p.row_cand + (int64_t)pair * p.cand_capacity;
-    for (int t = tid; t < n; t += kResolveThreads) {
-        const uint2 c = cand[t];
-        keys[t] = c.x;
-        where[t] = (int)c.y;
-    }
+    for (int t = tid; t < n; t += kResolveThreads) keys[t] = cand[t].x;
     __syncthreads();
     // the need-th largest key, and how many of the keys equal to it are taken
     exact_threshold<kResolveThreads>(sh, n, need, [](int) { return true; }, [&](int i) { return keys[i]; });
@@ -346,11 +343,14 @@ sparf_resolve_kernel(const SparfParams p)
     int cut = 0x7fffffff;                                    // every token that ties with tau is taken ...
     if (take < ties) {                                       // ... unless the cut falls among them (uniform)
         exact_threshold<kResolveThreads>(sh, n, take, [&](int i) { return keys[i] == tau; },
-                                         [&](int i) { return ~(unsigned)where[i]; });
+                                         [&](int i) { return ~cand[i].y; });
         cut = (int)~sh.tau;
     }
     for (int t = tid; t < n; t += kResolveThreads) {
-        if (keys[t] > tau || (keys[t] == tau && where[t] <= cut)) atomicAdd(&seg_final[where[t] / kSegmentTokens], 1);
+        if (keys[t] >= tau) {
+            const int where = (int)cand[t].y;
+            if (keys[t] > tau || where <= cut) atomicAdd(&seg_final[where / kSegmentTokens], 1);
+        }
     }
     if (tid == 0) {
         row->tau = tau;
