@@ -252,6 +252,7 @@ class Layer:
         self.chunk_tokens = binding.plan_chunk_tokens(B, H, self.max_len)
         self.n_splits = binding.plan_num_splits(B, H, self.max_len)
         self.clustered = binding.plan_merges_in_cluster(B, H, self.max_len)
+        self.events = None
 
     @property
     def launches(self) -> int:
@@ -280,6 +281,20 @@ class Layer:
         binding.decode_step_host(self.host_out, self.host_qkv, self.qkv, self.out, self.lse, c.k_cache,
                                  c.v_cache, c.seq_lens, c.block_table, self.max_len, c.scale,
                                  self.workspace, flags)
+
+    def run_from_host_overlapped(self, flags, compute, upload, download):
+        """The same, with the upload and the download on streams of their own, so that a step of
+        many layers overlaps layer L+1's upload and layer L-1's download with layer L's kernels."""
+        from paper_2409_04992_b200 import binding
+        c = self.case
+        if self.events is None:                   # torch creates a CUDA event at its first record
+            self.events = (torch.cuda.Event(), torch.cuda.Event())
+            for e in self.events:
+                e.record(compute)
+        binding.decode_step_host_overlapped(self.host_out, self.host_qkv, self.qkv, self.out, self.lse,
+                                            c.k_cache, c.v_cache, c.seq_lens, c.block_table, self.max_len,
+                                            c.scale, self.workspace, flags, compute, upload, download,
+                                            self.events[0], self.events[1])
 
     @property
     def h2d_bytes(self) -> int:
@@ -313,7 +328,32 @@ def build_layers(w: wl.Workload, device, rank: int):
     return [layers[i % distinct] for i in range(w.layers)], distinct
 
 
+_copy_streams = {}
+
+
 def run_step(layers, flags, from_host=False):
+    """One step.  From host buffers, with every layer owning its staging buffers, the copies run
+    on two streams of their own (forked from the current stream and joined at the end of the
+    step, so the step is still one unit of work on the current stream)."""
+    if from_host and len({id(layer) for layer in layers}) == len(layers) and len(layers) > 1:
+        compute = torch.cuda.current_stream()
+        dev = compute.device
+        if dev not in _copy_streams:
+            _copy_streams[dev] = (torch.cuda.Stream(dev), torch.cuda.Stream(dev))
+        upload, download = _copy_streams[dev]
+        if any(layer.events is None for layer in layers):        # creates the events, outside any capture
+            for layer in layers:
+                if layer.events is None:
+                    layer.events = (torch.cuda.Event(), torch.cuda.Event())
+                    for e in layer.events:
+                        e.record(compute)
+        upload.wait_stream(compute)
+        download.wait_stream(compute)
+        for layer in layers:
+            layer.run_from_host_overlapped(flags, compute, upload, download)
+        compute.wait_stream(upload)
+        compute.wait_stream(download)
+        return
     for layer in layers:
         if from_host:
             layer.run_from_host(flags)

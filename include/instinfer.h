@@ -275,6 +275,32 @@ int instinfer_decode_step_host(void *out_host, const void *qkv_host, void *qkv_d
                                int32_t *status_flags, void *cuda_stream);
 
 /*
+ * The same step with the two copies taken off the compute stream, so that a caller that runs
+ * one step per layer overlaps layer L+1's upload and layer L-1's download with layer L's
+ * kernels (the paper pipelines the transfers to and from the drive in the same way,
+ * Sec. IV-D).  Streams and events are the caller's (cudaStream_t / cudaEvent_t as void*):
+ *   upload_stream:    copy qkv_host -> qkv_dev, then record uploaded_event
+ *   compute_stream:   wait for uploaded_event, instinfer_kv_append, attention, record attended_event
+ *   download_stream:  wait for attended_event, copy out_dev -> out_host
+ * A copy stream may be the compute stream itself (then its event is not used and may be
+ * NULL); otherwise its event must not be NULL.  Nothing else orders the three streams: the
+ * caller keeps qkv_dev, out_dev, the workspace and the events of a call untouched until that
+ * call's part of each stream has run (one set per call in flight), and if the streams are
+ * being captured into a graph it forks the copy streams from the capturing stream before the
+ * first call and joins them after the last.  out_host holds the result once download_stream
+ * has reached that point.  Arguments and errors otherwise as instinfer_decode_step_host.
+ */
+int instinfer_decode_step_host_overlapped(void *out_host, const void *qkv_host, void *qkv_dev, void *out_dev,
+                                          float *lse, void *k_cache, void *v_cache, const int32_t *seq_lens,
+                                          const int32_t *block_table, int32_t max_blocks_per_seq,
+                                          int32_t block_tokens, int64_t num_phys_blocks,
+                                          int32_t batch, int32_t heads, int32_t head_dim, int32_t s_max,
+                                          int32_t max_seq_len, float scale,
+                                          void *workspace, size_t workspace_bytes, int32_t *status_flags,
+                                          void *compute_stream, void *upload_stream, void *download_stream,
+                                          void *uploaded_event, void *attended_event);
+
+/*
  * ---- Sparse decode attention (the paper's Algorithm 1, SparF; SparQ's arithmetic) ----
  * Paged layout only.  Besides the K and V pools the cache keeps
  *   kt_pool  fp16 [num_kt_blocks, heads, head_dim, kt_block_tokens]: K a second time,

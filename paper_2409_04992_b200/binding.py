@@ -72,6 +72,10 @@ def load() -> ctypes.CDLL:
         lib.instinfer_decode_step_host.argtypes = [ptr, ptr, ptr, ptr, ptr, ptr, ptr, ptr, ptr,
                                                    i32, i32, i64, i32, i32, i32, i32, i32, f32,
                                                    ptr, sz, ptr, ptr]
+        lib.instinfer_decode_step_host_overlapped.restype = ctypes.c_int
+        lib.instinfer_decode_step_host_overlapped.argtypes = [ptr, ptr, ptr, ptr, ptr, ptr, ptr, ptr, ptr,
+                                                              i32, i32, i64, i32, i32, i32, i32, i32, f32,
+                                                              ptr, sz, ptr, ptr, ptr, ptr, ptr, ptr]
         lib.instinfer_sparf_append.restype = ctypes.c_int
         lib.instinfer_sparf_append.argtypes = [ptr, ptr, ptr, ptr, ptr, ptr, ptr, ptr, i32, i32, i64,
                                                ptr, i32, i32, i64, i32, i32, i32, ptr, ptr]
@@ -317,6 +321,32 @@ def decode_step_host(out_host: torch.Tensor, qkv_host: torch.Tensor, qkv_dev: to
         _ptr(v_cache), _ptr(seq_lens), _ptr(block_table), max_blocks, block_tokens, phys, batch,
         heads, head_dim, s_max, int(max_seq_len), float(scale), _ptr(workspace),
         workspace.numel() * workspace.element_size(), _ptr(status_flags), _stream(stream)))
+
+
+def decode_step_host_overlapped(out_host: torch.Tensor, qkv_host: torch.Tensor, qkv_dev: torch.Tensor,
+                                out_dev: torch.Tensor, lse: Optional[torch.Tensor], k_cache: torch.Tensor,
+                                v_cache: torch.Tensor, seq_lens: torch.Tensor,
+                                block_table: Optional[torch.Tensor], max_seq_len: int, scale: float,
+                                workspace: torch.Tensor, status_flags: Optional[torch.Tensor],
+                                compute: torch.cuda.Stream, upload: torch.cuda.Stream,
+                                download: torch.cuda.Stream, uploaded: torch.cuda.Event,
+                                attended: torch.cuda.Event) -> None:
+    """instinfer_decode_step_host_overlapped: as decode_step_host, with the upload on `upload`
+    and the download on `download`; `uploaded` and `attended` are events that have been
+    recorded at least once (torch creates the CUDA event at its first record)."""
+    _, batch, heads, head_dim = qkv_host.shape
+    if block_table is None:
+        max_blocks, block_tokens, phys, s_max = 0, 0, 0, k_cache.shape[2]
+    else:
+        max_blocks, block_tokens, phys, s_max = (block_table.shape[1], k_cache.shape[2],
+                                                 k_cache.shape[0], 0)
+    _check(load().instinfer_decode_step_host_overlapped(
+        _ptr(out_host), _ptr(qkv_host), _ptr(qkv_dev), _ptr(out_dev), _ptr(lse), _ptr(k_cache),
+        _ptr(v_cache), _ptr(seq_lens), _ptr(block_table), max_blocks, block_tokens, phys, batch,
+        heads, head_dim, s_max, int(max_seq_len), float(scale), _ptr(workspace),
+        workspace.numel() * workspace.element_size(), _ptr(status_flags), compute.cuda_stream or None,
+        upload.cuda_stream or None, download.cuda_stream or None, uploaded.cuda_event or None,
+        attended.cuda_event or None))
 
 
 def sparf_append(k_pool: torch.Tensor, v_pool: torch.Tensor, kt_pool: torch.Tensor,

@@ -377,13 +377,15 @@ size_t instinfer_allgather_workspace_bytes(int32_t batch, int32_t heads, int32_t
     if (pairs == 0) return 256;
     return workspace_for(pairs, make_plan(pairs, max_seq_len)) + staging_for(pairs);
 }
-int instinfer_decode_step_host(void *out_host, const void *qkv_host, void *qkv_dev, void *out_dev,
-                               float *lse, void *k_cache, void *v_cache, const int32_t *seq_lens,
-                               const int32_t *block_table, int32_t max_blocks_per_seq,
-                               int32_t block_tokens, int64_t num_phys_blocks, int32_t batch,
-                               int32_t heads, int32_t head_dim, int32_t s_max, int32_t max_seq_len,
-                               float scale, void *workspace, size_t workspace_bytes,
-                               int32_t *status_flags, void *cuda_stream)
+// The host-vector step.  With `up` and `down` equal to the compute stream and no events this
+// is one stream in order; otherwise the upload runs on `up`, the kernels on `compute` after
+// `uploaded`, the download on `down` after `attended`.
+static int host_step(void *out_host, const void *qkv_host, void *qkv_dev, void *out_dev, float *lse,
+                     void *k_cache, void *v_cache, const int32_t *seq_lens, const int32_t *block_table,
+                     int32_t max_blocks_per_seq, int32_t block_tokens, int64_t num_phys_blocks, int32_t batch,
+                     int32_t heads, int32_t head_dim, int32_t s_max, int32_t max_seq_len, float scale,
+                     void *workspace, size_t workspace_bytes, int32_t *status_flags, cudaStream_t compute,
+                     cudaStream_t up, cudaStream_t down, cudaEvent_t uploaded, cudaEvent_t attended)
 {
     // Everything the host can check is checked here, for all the calls this one is made of,
     // so that a refused call has put nothing on the stream (not even the upload).
@@ -398,6 +400,8 @@ int instinfer_decode_step_host(void *out_host, const void *qkv_host, void *qkv_d
         return INSTINFER_ERR_INVALID_ARG;
     }
     if (head_dim != kHeadDim || (paged && block_tokens % 8 != 0)) return INSTINFER_ERR_UNSUPPORTED;
+    if ((up != compute && uploaded == nullptr) || (down != compute && attended == nullptr))
+        return INSTINFER_ERR_INVALID_ARG;
     if (batch == 0) return INSTINFER_OK;
     if (out_host == nullptr || qkv_host == nullptr || !usable(qkv_dev) || !usable(out_dev) ||
         !usable(k_cache) || !usable(v_cache) || seq_lens == nullptr)
@@ -408,33 +412,70 @@ int instinfer_decode_step_host(void *out_host, const void *qkv_host, void *qkv_d
             workspace_bytes < workspace_for(pairs, make_plan(pairs, max_seq_len)))
             return INSTINFER_ERR_WORKSPACE;
     }
-    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     const size_t one = (size_t)batch * heads * head_dim * sizeof(__half);
-    if (cudaMemcpyAsync(qkv_dev, qkv_host, 3 * one, cudaMemcpyHostToDevice, stream) != cudaSuccess) {
+    bool fine = cudaMemcpyAsync(qkv_dev, qkv_host, 3 * one, cudaMemcpyHostToDevice, up) == cudaSuccess;
+    if (fine && up != compute)
+        fine = cudaEventRecord(uploaded, up) == cudaSuccess && cudaStreamWaitEvent(compute, uploaded, 0) == cudaSuccess;
+    if (!fine) {
         (void)cudaGetLastError();
         return INSTINFER_ERR_CUDA;
     }
     const unsigned char *staged = static_cast<const unsigned char *>(qkv_dev);
     int rc = instinfer_kv_append(k_cache, v_cache, staged + one, staged + 2 * one, seq_lens, block_table,
                                  max_blocks_per_seq, block_tokens, num_phys_blocks, batch, heads,
-                                 head_dim, s_max, status_flags, cuda_stream);
+                                 head_dim, s_max, status_flags, compute);
     if (rc != INSTINFER_OK) return rc;
     if (block_table == nullptr)
         rc = instinfer_decode_attention(out_dev, lse, staged, k_cache, v_cache, seq_lens, batch, heads,
                                         head_dim, s_max, max_seq_len, scale, workspace,
-                                        workspace_bytes, status_flags, cuda_stream);
+                                        workspace_bytes, status_flags, compute);
     else
         rc = instinfer_decode_attention_paged(out_dev, lse, staged, k_cache, v_cache, block_table,
                                               seq_lens, batch, heads, head_dim, block_tokens,
                                               max_blocks_per_seq, num_phys_blocks, max_seq_len,
                                               scale, workspace, workspace_bytes, status_flags,
-                                              cuda_stream);
+                                              compute);
     if (rc != INSTINFER_OK) return rc;
-    if (cudaMemcpyAsync(out_host, out_dev, one, cudaMemcpyDeviceToHost, stream) != cudaSuccess) {
+    if (down != compute)
+        fine = cudaEventRecord(attended, compute) == cudaSuccess && cudaStreamWaitEvent(down, attended, 0) == cudaSuccess;
+    fine = fine && cudaMemcpyAsync(out_host, out_dev, one, cudaMemcpyDeviceToHost, down) == cudaSuccess;
+    if (!fine) {
         (void)cudaGetLastError();
         return INSTINFER_ERR_CUDA;
     }
     return INSTINFER_OK;
+}
+
+int instinfer_decode_step_host(void *out_host, const void *qkv_host, void *qkv_dev, void *out_dev,
+                               float *lse, void *k_cache, void *v_cache, const int32_t *seq_lens,
+                               const int32_t *block_table, int32_t max_blocks_per_seq,
+                               int32_t block_tokens, int64_t num_phys_blocks, int32_t batch,
+                               int32_t heads, int32_t head_dim, int32_t s_max, int32_t max_seq_len,
+                               float scale, void *workspace, size_t workspace_bytes,
+                               int32_t *status_flags, void *cuda_stream)
+{
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    return host_step(out_host, qkv_host, qkv_dev, out_dev, lse, k_cache, v_cache, seq_lens, block_table,
+                     max_blocks_per_seq, block_tokens, num_phys_blocks, batch, heads, head_dim, s_max,
+                     max_seq_len, scale, workspace, workspace_bytes, status_flags, stream, stream, stream,
+                     nullptr, nullptr);
+}
+
+int instinfer_decode_step_host_overlapped(void *out_host, const void *qkv_host, void *qkv_dev, void *out_dev,
+                                          float *lse, void *k_cache, void *v_cache, const int32_t *seq_lens,
+                                          const int32_t *block_table, int32_t max_blocks_per_seq,
+                                          int32_t block_tokens, int64_t num_phys_blocks, int32_t batch,
+                                          int32_t heads, int32_t head_dim, int32_t s_max, int32_t max_seq_len,
+                                          float scale, void *workspace, size_t workspace_bytes,
+                                          int32_t *status_flags, void *compute_stream, void *upload_stream,
+                                          void *download_stream, void *uploaded_event, void *attended_event)
+{
+    return host_step(out_host, qkv_host, qkv_dev, out_dev, lse, k_cache, v_cache, seq_lens, block_table,
+                     max_blocks_per_seq, block_tokens, num_phys_blocks, batch, heads, head_dim, s_max,
+                     max_seq_len, scale, workspace, workspace_bytes, status_flags,
+                     static_cast<cudaStream_t>(compute_stream), static_cast<cudaStream_t>(upload_stream),
+                     static_cast<cudaStream_t>(download_stream), static_cast<cudaEvent_t>(uploaded_event),
+                     static_cast<cudaEvent_t>(attended_event));
 }
 size_t instinfer_workspace_bytes(int32_t batch, int32_t heads, int32_t head_dim, int32_t max_seq_len)
 {

@@ -113,6 +113,8 @@ int main(void)
            INSTINFER_ERR_UNSUPPORTED);
     expect("host step workspace", instinfer_decode_step_host(fake, fake, fake, fake, NULL, fake, fake, lens, NULL, 0, 0, 0, 2, 4, 128, 256, 256, 0.1f, fake, 16, NULL, NULL),
            INSTINFER_ERR_WORKSPACE);
+    expect("overlapped host step without its upload event", instinfer_decode_step_host_overlapped(fake, fake, fake, fake, NULL, fake, fake, lens, NULL, 0, 0, 0, 2, 4, 128, 256, 256, 0.1f, fake, big, NULL, NULL, fake, NULL, NULL, NULL),
+           INSTINFER_ERR_INVALID_ARG);
 
     /* sparse path */
     expect("sparse append kt table", instinfer_sparf_append(fake, fake, fake, (float *)fake, fake, fake, lens, table, 16, 16, 40, NULL, 2, 128, 9, 2, 4, 128, NULL, NULL),
