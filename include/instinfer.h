@@ -275,10 +275,10 @@ int instinfer_decode_step_host(void *out_host, const void *qkv_host, void *qkv_d
                                int32_t *status_flags, void *cuda_stream);
 
 /*
- * The same step with the two copies taken off the compute stream, so that a caller that runs
- * one step per layer overlaps layer L+1's upload and layer L-1's download with layer L's
- * kernels (the paper pipelines the transfers to and from the drive in the same way,
- * Sec. IV-D).  Streams and events are the caller's (cudaStream_t / cudaEvent_t as void*):
+ * The same step with the two copies taken off the compute stream, so that a caller with
+ * several independent steps in flight (the paper's mini-batches, Sec. IV-D: one mini-batch's
+ * vectors travel while another's attention runs) overlaps the next step's upload and the
+ * previous step's download with this step's kernels.  Streams and events are the caller's (cudaStream_t / cudaEvent_t as void*):
  *   upload_stream:    copy qkv_host -> qkv_dev, then record uploaded_event
  *   compute_stream:   wait for uploaded_event, instinfer_kv_append, attention, record attended_event
  *   download_stream:  wait for attended_event, copy out_dev -> out_host
