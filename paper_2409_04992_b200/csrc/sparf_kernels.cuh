@@ -21,6 +21,7 @@
 //                         out = alpha * attended + (1 - alpha) * v_sum / S.
 #pragma once
 
+#include <cstddef>
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -206,7 +207,7 @@ __device__ __forceinline__ unsigned ordered_key(float x)
 
 // Step 1 and the temperature of steps 2-4, shared by the kernels that compute approximate
 // logits.  Threads d < 128 each own one head dim; every thread of the block must call it.
-struct ScoreShared {
+struct __align__(16) ScoreShared {       // 16 bytes: the keys of step 1 are read four at a time
     float abs_q[kHeadDim];
     unsigned short q_bits[kHeadDim];   // q of the selected dims as fp16 bit patterns, in rank order
     int dim[kHeadDim];          // the selected dims, in rank order
@@ -214,26 +215,39 @@ struct ScoreShared {
     float approx_scale;
 };
 
+static_assert(offsetof(ScoreShared, dim) % 16 == 0, "the keys of step 1 are read as uint4");
+
 __device__ __forceinline__ void score_setup(const SparfParams &p, int pair, ScoreShared &ss)
 {
     const int d = threadIdx.x;
     // Step 1: rank of |q_d| (exact comparisons of fp16 magnitudes, ties to the lower index).
-    float qd = 0.f;
+    // The 15 magnitude bits of an fp16 number order like the magnitude itself, so one integer
+    // key per dim -- magnitude bits, then 127 - d -- makes every comparison a single one:
+    // rank = number of larger keys.  (ss.dim doubles as the key array until the ranks are known.)
+    unsigned short bits = 0;
+    unsigned *keys = reinterpret_cast<unsigned *>(ss.dim);
     if (d < kHeadDim) {
-        qd = __half2float(p.q[(int64_t)pair * kHeadDim + d]);
-        ss.abs_q[d] = fabsf(qd);
+        bits = __half_as_ushort(p.q[(int64_t)pair * kHeadDim + d]);
+        ss.abs_q[d] = fabsf(__half2float(__ushort_as_half(bits)));
+        keys[d] = (unsigned)(bits & 0x7fffu) << 8 | (unsigned)(kHeadDim - 1 - d);
     }
     __syncthreads();
+    int rank = 0;
     if (d < kHeadDim) {
-        int rank = 0;
-        for (int e = 0; e < kHeadDim; ++e) {
-            const float other = ss.abs_q[e];
-            rank += (other > ss.abs_q[d]) || (other == ss.abs_q[d] && e < d);
+        const unsigned mine = keys[d];
+        const uint4 *four = reinterpret_cast<const uint4 *>(keys);
+#pragma unroll 8
+        for (int e = 0; e < kHeadDim / 4; ++e) {
+            const uint4 other = four[e];
+            rank += (int)(other.x > mine) + (int)(other.y > mine) + (int)(other.z > mine) + (int)(other.w > mine);
         }
+    }
+    __syncthreads();                                         // every key has been read: ss.dim is free
+    if (d < kHeadDim) {
         const bool kept = rank < p.r;
         if (kept) {
             ss.dim[rank] = d;
-            ss.q_bits[rank] = __half_as_ushort(p.q[(int64_t)pair * kHeadDim + d]);
+            ss.q_bits[rank] = bits;
         }
         ss.kept[d] = kept;
     }
