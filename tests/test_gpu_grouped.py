@@ -137,6 +137,59 @@ def test_peaked_logits():
         check(g, chunk, f"peaked chunk={chunk}")
 
 
+@pytest.mark.parametrize("layout,tokens", [("contiguous", 0), ("paged", 16), ("paged", 64)])
+def test_reference_moves_in_the_middle_of_a_chunk(layout, tokens):
+    """Keys aligned with the query at a few late positions, each with a logit far above all
+    earlier ones: the softmax reference moves (and the accumulator is rescaled) several times
+    inside one chunk, not only at its first tile."""
+    lens = [1700, 900]
+    g = make(layout, tokens, 1, 1, 4, lens=lens)
+    c = g.base
+    T = tokens
+    for b, n in enumerate(lens):
+        for pos, gain in ((n // 3, 2.0), (n // 2 + 5, 4.0), (n - 140, 7.0)):
+            row = (g.q[b, 0, 0].float() * gain).half()          # logit = gain * |q|^2 * scale: tens of units apart
+            if c.block_table is None:
+                c.k_cache[b, 0, pos] = row
+            else:
+                c.k_cache[int(c.block_table[b, pos // T]), 0, pos % T] = row
+    for chunk in (0, 2048, 256):
+        check(g, chunk, f"moving reference, {layout} T={tokens} chunk={chunk}")
+
+
+def test_a_block_that_cannot_be_read_counts_as_zeros():
+    """A block id outside the pool is flagged, and the result is the oracle's on the same cache
+    with that block's keys and values zeroed (every form of the kernel)."""
+    lens = [200, 330]
+    g = make("paged", 16, 2, 2, 4, lens=lens)
+    dev = to_device(g)
+    c = dev.base
+    # append first with the good table, then break one entry for the attention call only
+    out_ok, _, _ = gpu_step(dev)
+    table = c.block_table.clone()
+    victim_block = 3
+    phys = int(table[1, victim_block])
+    table[1, victim_block] = c.k_cache.shape[0] + 7
+    B, Tq, Hq, D = g.q.shape
+    out = torch.zeros_like(dev.q)
+    lse = torch.zeros((B, Tq, Hq), dtype=torch.float32, device="cuda")
+    flags = torch.zeros(1, dtype=torch.int32, device="cuda")
+    ws = torch.empty(binding.grouped_workspace_bytes(B, Tq, Hq, 2, D, max(lens)), dtype=torch.uint8, device="cuda")
+    binding.decode_attention_grouped(out, lse, dev.q, c.k_cache, c.v_cache, table, c.seq_lens, max(lens),
+                                     c.scale, ws, flags)
+    torch.cuda.synchronize()
+    assert int(flags.item()) == binding.FLAG_BLOCK_RANGE
+    k = c.k_cache.cpu().numpy().copy()
+    v = c.v_cache.cpu().numpy().copy()
+    k[phys] = 0
+    v[phys] = 0
+    want, want_lse = capi.decode_attention_grouped(g.q.numpy(), k, v, np.array(lens, dtype=np.int32), g.base.scale,
+                                                   block_table=g.base.block_table.numpy())
+    gu.assert_close(out.cpu().reshape(B, Tq * Hq, D), want.reshape(B, Tq * Hq, D),
+                    lse.cpu().reshape(B, Tq * Hq), want_lse.reshape(B, Tq * Hq), "zeroed block")
+    assert torch.equal(out[0], out_ok.cuda()[0])            # the other sequence is untouched
+
+
 def test_one_row_case_agrees_with_the_one_row_entry_point():
     g = make("paged", 16, 3, 1, 3)
     dev = to_device(g)
