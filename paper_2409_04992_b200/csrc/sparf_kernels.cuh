@@ -274,7 +274,8 @@ __device__ __forceinline__ void score_group(const SparfParams &p, const ScoreSha
                                             const int32_t *table_row, int h, int i, float (&dot)[8])
 {
     const int T = p.kt_block_tokens;
-    const int blk = i / T, slot = i - blk * T;
+    const int t_shift = (T & (T - 1)) == 0 ? __ffs(T) - 1 : -1;      // blocks of 2^n tokens: no division
+    const int blk = t_shift >= 0 ? i >> t_shift : i / T, slot = i - blk * T;
     const int phys = bounds_ok(blk < p.kt_max_blocks_per_seq, p.status) ? table_row[blk] : -1;
 #pragma unroll
     for (int e = 0; e < 8; ++e) dot[e] = 0.f;
@@ -644,6 +645,7 @@ __device__ __forceinline__ void select_row(const SparfParams &p, SelectShared &s
 
     // Ordered compaction: position = #greater before + min(#equal before, take_equal).
     const int T = p.block_tokens;
+    const int t_shift = (T & (T - 1)) == 0 ? __ffs(T) - 1 : -1;      // blocks of 2^n tokens: no division per token
     const int32_t *table_row = p.block_table + (int64_t)b * p.max_blocks_per_seq;
     int base_gt = 0, base_eq = 0;
     float mass = 0.f;
@@ -692,7 +694,7 @@ __device__ __forceinline__ void select_row(const SparfParams &p, SelectShared &s
             if (gt[e] || (eq[e] && eq_before < take_equal)) {
                 const int i = 4 * g + e;
                 const int pos = gt_before + min(eq_before, take_equal);
-                const int blk = i / T, slot = i - blk * T;
+                const int blk = t_shift >= 0 ? i >> t_shift : i / T, slot = i - blk * T;
                 const int phys = bounds_ok(blk < p.max_blocks_per_seq && pos < p.max_k, p.status) ? table_row[blk] : -1;
                 const bool ok = phys >= 0 && (int64_t)phys < p.num_phys_blocks;
                 if (!ok && p.status) atomicOr(p.status, kFlagBlockRange);

@@ -399,6 +399,7 @@ sparf_emit_kernel(const SparfParams p)
     const int own_excl = own_incl - own;                     // lane j: selected in the block's segments before j
 
     const int T = p.block_tokens;
+    const int t_shift = (T & (T - 1)) == 0 ? __ffs(T) - 1 : -1;      // blocks of 2^n tokens: no division per token
     const int32_t *table_row = p.block_table + (int64_t)b * p.max_blocks_per_seq;
     const float *stage_x = p.scores + (int64_t)pair * p.score_stride;
     const int32_t *stage_pos = p.stage_pos + (int64_t)pair * p.score_stride;
@@ -448,7 +449,7 @@ sparf_emit_kernel(const SparfParams p)
         for (int e = 0; e < 4; ++e) {
             if (take >> e & 1u) {
                 const int i = pos[e];
-                const int blk = i / T, slot = i - blk * T;
+                const int blk = t_shift >= 0 ? i >> t_shift : i / T, slot = i - blk * T;
                 const int phys = bounds_ok(blk < p.max_blocks_per_seq && dst < p.max_k, p.status) ? table_row[blk] : -1;
                 const bool ok = phys >= 0 && (int64_t)phys < p.num_phys_blocks;
                 if (!ok && p.status) atomicOr(p.status, kFlagBlockRange);
