@@ -131,6 +131,17 @@ def test_transposed_copy_with_its_own_block_size(tokens, kt_tokens):
     run_and_check(cpu, state, 16, 4, f"T={tokens} Tk={kt_tokens}")
 
 
+@pytest.mark.parametrize("tokens,kt_tokens", [(16, 1024), (64, 2048)])
+def test_transposed_copy_in_blocks_of_1024_tokens_and_more(tokens, kt_tokens):
+    """Large blocks of the transposed copy (the paper gives its embedding-indexed mapping groups
+    of up to 1K tokens): rows that end inside a block, on a 1024-token edge, rows of a few
+    tokens, and rows of more than one 8192-token score block."""
+    cpu, state = make([1, 9, 1023, 1024, 1025, 3000, 0, 9000, 2048 + 255], tokens, kt_tokens=kt_tokens)
+    assert state.kt_block_tokens == kt_tokens
+    run_and_check(cpu, state, 16, 4, f"T={tokens} Tk={kt_tokens}")
+    run_and_check(cpu, state, 5, 0, f"T={tokens} Tk={kt_tokens} r=5")
+
+
 def test_long_peaked_sequences_and_forty_heads():
     cpu, state = make([5000, 3000], tokens=32, heads=40, index=3, peaked=0.02)
     out, alpha, sel, own = run_and_check(cpu, state, 16, 16, "long peaked")

@@ -57,9 +57,9 @@ def check_pair(pb, k_tokens, scale, sel_row, out_row, alpha_value, what):
     return in_band
 
 
-def run_workload(index, pairs, path):
+def run_workload(index, pairs, path, kt_tokens=256):
     case = wl.generate(wl.STANDARD[index], device="cuda", poison=False)
-    state = wl.make_sparf_state(case, 0.125, 256)
+    state = wl.make_sparf_state(case, 0.125, kt_tokens)
     B, H, D = case.q.shape
     max_len, max_k = case.max_seq_len, max(state.k_tokens_host)
     out = torch.empty((B, H, D), dtype=torch.float16, device="cuda")
@@ -104,6 +104,11 @@ def test_long_context_workload_sampled_pairs():
     if free < 45 * 2 ** 30:
         pytest.skip("needs 45 GiB of free device memory")
     run_workload(3, spread_pairs(8, 40, 32, 3), 0)
+
+
+def test_long_context_workload_with_1024_token_transposed_blocks():
+    """The same workload with the transposed copy in 1024-token blocks."""
+    run_workload(3, spread_pairs(8, 40, 16, 5), 0, kt_tokens=1024)
 
 
 @pytest.mark.parametrize("path", [1, 2], ids=["chunk-parallel", "block-per-row"])
