@@ -197,6 +197,7 @@ sparf_sample_kernel(const SparfParams p)
 struct StageShared {
     ScoreShared score;
     float red[32];
+    uint2 staged[kSparfThreads / 32][kSegmentTokens];       // per warp: a segment's staged tokens (logit bits, position)
 };
 
 // grid pairs * score_blocks, kSparfThreads threads: kScoreBlockTokens tokens of one row.  Each
@@ -228,6 +229,7 @@ sparf_stage_kernel(const SparfParams p)
     float *stage_x = p.scores + (int64_t)pair * p.score_stride;
     int32_t *stage_pos = p.stage_pos + (int64_t)pair * p.score_stride;
     uint2 *cand = p.row_cand + (int64_t)pair * p.cand_capacity;
+    const unsigned buf = static_cast<unsigned>(__cvta_generic_to_shared(sh.staged[warp]));
     float z = 0.f;
     bool far_above = false;
     for (int seg_begin = begin + warp * kSegmentTokens; seg_begin < end; seg_begin += kWarpsPerBlock * kSegmentTokens) {
@@ -269,20 +271,37 @@ sparf_stage_kernel(const SparfParams p)
             if ((total >> 10 & 1023) != 0) cand_base = atomicAdd(&row->n_cand, total >> 10 & 1023);
         }
         cand_base = __shfl_sync(0xffffffffu, cand_base, 0);
-        int at = (incl - mine) & 1023, cand_at = cand_base + ((incl - mine) >> 10 & 1023);
+        // The staged tokens go, in position order, through the warp's piece of shared memory (one
+        // predicated 8-byte store per token, no branch), and from there to global memory as whole
+        // runs written by consecutive lanes; which of them are candidates (not surely selected,
+        // not in the window) is decided again on the way out, their slots come from a vote.
+        unsigned at = buf + ((incl - mine) & 1023) * 8;
 #pragma unroll
         for (int e = 0; e < 8; ++e) {
-            if (staged >> e & 1u) {
-                if (!bounds_ok(seg_begin + at < p.score_stride, p.status)) continue;
-                stage_x[seg_begin + at] = dot[e];
-                stage_pos[seg_begin + at] = i + e;
-                ++at;
-                if (cands >> e & 1u) {           // between the bounds: a candidate for the exact threshold
-                    if (cand_at < p.cand_capacity) cand[cand_at] = make_uint2(ordered_key(dot[e]), (unsigned)(i + e));
-                    ++cand_at;
-                }
-            }
+            asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %0, 0;\n\t@p st.shared.v2.b32 [%1], {%2, %3};\n\t}"
+                         :: "r"(staged >> e & 1u), "r"(at), "r"(__float_as_uint(dot[e])), "r"(i + e) : "memory");
+            at += (staged >> e & 1u) * 8;
         }
+        __syncwarp();
+        const int n = total & 1023;
+        for (int t0 = 0; t0 < n; t0 += 32) {
+            const int t = t0 + lane;
+            const bool have = t < n && bounds_ok(seg_begin + t < p.score_stride, p.status);
+            uint2 v = make_uint2(0u, 0u);
+            if (have) {
+                asm volatile("ld.shared.v2.b32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(buf + t * 8));
+                stage_x[seg_begin + t] = __uint_as_float(v.x);
+                stage_pos[seg_begin + t] = (int)v.y;
+            }
+            const bool between = have && !(__uint_as_float(v.x) > hi) && (int)v.y < window_from;
+            const unsigned votes = __ballot_sync(0xffffffffu, between);
+            if (between) {
+                const int slot = cand_base + __popc(votes & ((1u << lane) - 1u));
+                if (slot < p.cand_capacity) cand[slot] = make_uint2(ordered_key(__uint_as_float(v.x)), v.y);
+            }
+            cand_base += __popc(votes);
+        }
+        __syncwarp();                        // the piece of shared memory is reused by the next segment
     }
     z = block_sum(z, sh.red);
     if (tid == 0) p.blk_z[(int64_t)pair * p.score_blocks + block_in_row] = z;
