@@ -16,7 +16,7 @@
 // pipeline runs on across chunk boundaries.  A block has eight warps, each with one job, that
 // hand tiles to one another through mbarriers:
 //   * warp 4 (K producer) moves 128-token tiles of K with tensor-map copies (cp.async.bulk.tensor,
-//     128-byte swizzle, this GPU's memory, no multicast) into a ring of three 32 KiB slots; a
+//     128-byte swizzle, this GPU's memory, every block fetching its own tiles) into a ring of three 32 KiB slots; a
 //     paged tile is 128 / T copies of one (block, head) run each, the block ids read one tile
 //     ahead; a block with a bad id is not fetched but zero-filled.  It also draws the tickets
 //     (two chunks ahead, so the atomic's round trip is hidden), announces each chunk to the
