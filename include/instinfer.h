@@ -453,7 +453,7 @@ int instinfer_set_sparse_path(int32_t path);
 /*
  * instinfer_decode_attention_grouped has two implementations of the same arithmetic: warp-level
  * tensor-core MMAs (every head size and block size the entry point takes) and, for head size
- * 128 with a contiguous cache or 16, 32 or 64 tokens per block, asynchronous tcgen05 MMAs that
+ * 128 with a contiguous cache or blocks of 16, 32, 64 or a multiple of 128 tokens, asynchronous tcgen05 MMAs that
  * take 128-token tiles as the long side, with accumulators in tensor memory and tiles moved by
  * tensor-map copies.  The library picks the second where the shape allows;
  * instinfer_set_grouped_path forces the choice for later calls of this process: 0 automatic,

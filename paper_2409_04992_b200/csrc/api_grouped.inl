@@ -55,7 +55,7 @@ int launch_grouped(const GroupedParams &p, unsigned grid, cudaStream_t stream)
     return INSTINFER_OK;
 }
 
-// ---- the tcgen05 form (head size 128; contiguous, or paged with 16, 32 or 64 tokens per block) ----
+// ---- the tcgen05 form (head size 128; contiguous, or paged in blocks of 16, 32, 64 or a multiple of 128 tokens) ----
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
@@ -94,7 +94,10 @@ bool make_cache_map(CUtensorMap *map, const void *cache, int64_t rows, int32_t b
 
 bool umma_shape(int32_t head_dim, bool paged, int32_t block_tokens)
 {
-    return head_dim == 128 && (!paged || block_tokens == 16 || block_tokens == 32 || block_tokens == 64);
+    // blocks of 16, 32 or 64 tokens, or of a multiple of 128 (then a forced chunk length must be one too,
+    // so that no 128-token tile straddles two blocks)
+    return head_dim == 128 && (!paged || block_tokens == 16 || block_tokens == 32 || block_tokens == 64 ||
+                               (block_tokens % kUmmaTile == 0 && g_forced_chunk % kUmmaTile == 0));
 }
 
 // The query tensor [B, Tq, Hq, 128] as the copy engine sees it: a box is 64 dims of the `group`
@@ -198,8 +201,8 @@ int instinfer_decode_attention_grouped(void *out, float *lse, const void *q, con
     CUtensorMap map_q, map_k, map_v;
     const bool umma = g_grouped_path != 1 && umma_shape(head_dim, paged, block_tokens) &&
                       make_query_map(&map_q, q, batch, q_tokens, q_heads, p.group) &&
-                      make_cache_map(&map_k, k_cache, kv_bytes / 256, paged ? block_tokens : kUmmaTile) &&
-                      make_cache_map(&map_v, v_cache, kv_bytes / 256, paged ? block_tokens : kUmmaTile);
+                      make_cache_map(&map_k, k_cache, kv_bytes / 256, paged && block_tokens < kUmmaTile ? block_tokens : kUmmaTile) &&
+                      make_cache_map(&map_v, v_cache, kv_bytes / 256, paged && block_tokens < kUmmaTile ? block_tokens : kUmmaTile);
     const SplitPlan plan = make_plan(pairs, max_seq_len, umma ? umma_rules() : grouped_rules(head_dim));
     if (workspace == nullptr || !aligned16(workspace) ||
         workspace_bytes < grouped_workspace_for(pairs, p.rows, head_dim, plan))

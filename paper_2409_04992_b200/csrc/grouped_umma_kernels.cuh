@@ -17,7 +17,8 @@
 // hand tiles to one another through mbarriers:
 //   * warp 4 (K producer) moves 128-token tiles of K with tensor-map copies (cp.async.bulk.tensor,
 //     128-byte swizzle, this GPU's memory, every block fetching its own tiles) into a ring of three 32 KiB slots; a
-//     paged tile is 128 / T copies of one (block, head) run each, the block ids read one tile
+//     paged tile is 128 / T copies of one (block, head) run each (one copy of 128 rows where a
+//     block holds a multiple of 128 tokens), the block ids read one tile
 //     ahead; a block with a bad id is not fetched but zero-filled.  It also draws the tickets
 //     (two chunks ahead, so the atomic's round trip is hidden), announces each chunk to the
 //     other warps through a small queue in shared memory and fetches the chunk's query rows;
@@ -338,7 +339,10 @@ grouped_attn_umma_kernel(const GroupedParams p, unsigned *ticket, const __grid_c
     // What both producers do for one chunk: the chunk's tiles of one cache (K or V) into that
     // cache's ring, tile `count` of this block going to slot count % slots; returns false if a
     // wait ran out.
-    const int T = kPaged ? a.block_tokens : kUmmaTile;
+    // A copy moves `T` rows: a whole block of 16, 32 or 64 tokens, or 128 rows of a larger block
+    // (a multiple of 128 tokens: tiles start on multiples of 128 then and never straddle a block),
+    // or of a contiguous cache.
+    const int T = kPaged ? min(a.block_tokens, kUmmaTile) : kUmmaTile;
     auto stream_chunk = [&](const UmmaChunk &c, const CUtensorMap *map, int ring_offset, int slots, int bar_full,
                             int bar_empty, int &count) -> bool {
         const int64_t total_rows = a.kv_bytes / (2 * D);
@@ -347,7 +351,7 @@ grouped_attn_umma_kernel(const GroupedParams p, unsigned *ticket, const __grid_c
             if (!kPaged) return 0;
             const int tile_start = c.begin + j * kUmmaTile;
             const int nb = (min(c.end - tile_start, kUmmaTile) + T - 1) / T;
-            const int idx = tile_start / T + lane;
+            const int idx = (tile_start + lane * T) / a.block_tokens;
             if (j >= c.n_tiles || lane >= nb || !bounds_ok(idx < a.max_blocks_per_seq, a.status)) return -1;
             return __ldg(table_row + idx);
         };
@@ -362,7 +366,8 @@ grouped_attn_umma_kernel(const GroupedParams p, unsigned *ticket, const __grid_c
             if (kPaged) {
                 const bool in_range = phys >= 0 && (int64_t)phys < a.num_phys_blocks;
                 if (good && !in_range && a.status) atomicOr(a.status, kFlagBlockRange);
-                row0 = in_range ? (phys * a.heads + c.hk) * T : 0;           // < 2^31 rows: checked by the host
+                // (< 2^31 rows: checked by the host)
+                row0 = in_range ? (phys * a.heads + c.hk) * a.block_tokens + (tile_start + lane * T) % a.block_tokens : 0;
                 good = good && in_range && bounds_ok((int64_t)row0 + T <= total_rows, a.status);
             } else {
                 row0 = c.pair * a.s_max + tile_start;          // rows past the tensor's end read as zeros

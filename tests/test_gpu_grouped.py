@@ -113,13 +113,25 @@ def test_the_tcgen05_form_is_the_one_that_runs(grouped_path):
     """On a GPU machine the driver has the tensor-map encoder, so head size 128 with a contiguous
     cache or 16/32/64-token blocks takes the tcgen05 kernel unless the warp-level one is forced."""
     want = 2 if grouped_path == 2 else 1
-    for tokens in (0, 16, 32, 64):
+    for tokens in (0, 16, 32, 64, 128, 256):
         assert binding.grouped_path_for(128, tokens) == want
     binding.set_grouped_path(0)
     assert binding.grouped_path_for(128, 16) == 2                                 # the default
-    assert binding.grouped_path_for(128, 48) == 1 and binding.grouped_path_for(128, 128) == 1
+    assert binding.grouped_path_for(128, 48) == 1 and binding.grouped_path_for(128, 192) == 1
+    binding.set_chunk_tokens(192)                                                # tiles would straddle 128-token blocks
+    try:
+        assert binding.grouped_path_for(128, 128) == 1 and binding.grouped_path_for(128, 64) == 2
+    finally:
+        binding.set_chunk_tokens(0)
     assert binding.grouped_path_for(64, 16) == 1 and binding.grouped_path_for(256, 0) == 1
     assert binding.grouped_path_for(96, 16) == 0 and binding.grouped_path_for(128, 8) == 0
+
+
+@pytest.mark.parametrize("tokens", [128, 256])
+@pytest.mark.parametrize("q_tokens,q_heads,kv_heads", [(1, 8, 2), (3, 4, 1)])
+def test_blocks_of_128_tokens_and_more(tokens, q_tokens, q_heads, kv_heads):
+    for chunk in (0, 128, 64):          # chunk 64: tiles would straddle blocks, the warp-level form takes over
+        check(make("paged", tokens, kv_heads, q_tokens, q_heads), chunk, f"T={tokens} chunk={chunk}")
 
 
 def test_tiny_contiguous_cache_smaller_than_one_tile():
