@@ -453,9 +453,9 @@ int instinfer_set_sparse_path(int32_t path);
 /*
  * instinfer_decode_attention_grouped has two implementations of the same arithmetic: warp-level
  * tensor-core MMAs (every head size and block size the entry point takes) and, for head size
- * 128 with a contiguous cache or blocks of 16, 32, 64 or a multiple of 128 tokens, asynchronous tcgen05 MMAs that
- * take 128-token tiles as the long side, with accumulators in tensor memory and tiles moved by
- * tensor-map copies.  The library picks the second where the shape allows;
+ * 128 or 256 with a contiguous cache or blocks of 16, 32, 64 or a multiple of 128 tokens,
+ * asynchronous tcgen05 MMAs that take 128-token tiles as the long side, with accumulators in
+ * tensor memory and tiles moved by tensor-map copies.  The library picks the second where the shape allows;
  * instinfer_set_grouped_path forces the choice for later calls of this process: 0 automatic,
  * 1 warp-level, 2 tcgen05 where the shape allows (a tuning and test aid; returns INSTINFER_OK
  * or INSTINFER_ERR_INVALID_ARG; not thread-safe against concurrent calls).  Both meet the

@@ -55,7 +55,7 @@ int launch_grouped(const GroupedParams &p, unsigned grid, cudaStream_t stream)
     return INSTINFER_OK;
 }
 
-// ---- the tcgen05 form (head size 128; contiguous, or paged in blocks of 16, 32, 64 or a multiple of 128 tokens) ----
+// ---- the tcgen05 form (head sizes 128 and 256; contiguous, or paged in blocks of 16, 32, 64 or a multiple of 128 tokens) ----
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
@@ -77,14 +77,14 @@ EncodeTiledFn tensor_map_encoder()
     return fn;
 }
 
-// A K or V cache as a 2-D fp16 tensor [rows][128] (a row is one token of one head, 256 bytes);
+// A K or V cache as a 2-D fp16 tensor [rows][head_dim] (a row is one token of one head);
 // a box is 64 dims (128 bytes, the swizzle span) by `box_rows` tokens.
-bool make_cache_map(CUtensorMap *map, const void *cache, int64_t rows, int32_t box_rows)
+bool make_cache_map(CUtensorMap *map, const void *cache, int64_t rows, int32_t head_dim, int32_t box_rows)
 {
     EncodeTiledFn encode = tensor_map_encoder();
     if (encode == nullptr || rows <= 0 || rows >= ((int64_t)1 << 31)) return false;
-    const cuuint64_t dims[2] = {128, (cuuint64_t)rows};
-    const cuuint64_t strides[1] = {256};
+    const cuuint64_t dims[2] = {(cuuint64_t)head_dim, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)head_dim * 2};
     const cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
     const cuuint32_t elem[2] = {1, 1};
     return encode(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void *>(cache), dims, strides, box, elem,
@@ -96,18 +96,21 @@ bool umma_shape(int32_t head_dim, bool paged, int32_t block_tokens)
 {
     // blocks of 16, 32 or 64 tokens, or of a multiple of 128 (then a forced chunk length must be one too,
     // so that no 128-token tile straddles two blocks)
-    return head_dim == 128 && (!paged || block_tokens == 16 || block_tokens == 32 || block_tokens == 64 ||
-                               (block_tokens % kUmmaTile == 0 && g_forced_chunk % kUmmaTile == 0));
+    return (head_dim == 128 || head_dim == 256) &&
+           (!paged || block_tokens == 16 || block_tokens == 32 || block_tokens == 64 ||
+            (block_tokens % kUmmaTile == 0 && g_forced_chunk % kUmmaTile == 0));
 }
 
-// The query tensor [B, Tq, Hq, 128] as the copy engine sees it: a box is 64 dims of the `group`
+// The query tensor [B, Tq, Hq, head_dim] as the copy engine sees it: a box is 64 dims of the `group`
 // heads of one KV head for all Tq new tokens, i.e. the chunk's rows t * group + g in order.
-bool make_query_map(CUtensorMap *map, const void *q, int32_t batch, int32_t q_tokens, int32_t q_heads, int32_t group)
+bool make_query_map(CUtensorMap *map, const void *q, int32_t batch, int32_t q_tokens, int32_t q_heads, int32_t group,
+                    int32_t head_dim)
 {
     EncodeTiledFn encode = tensor_map_encoder();
     if (encode == nullptr) return false;
-    const cuuint64_t dims[4] = {128, (cuuint64_t)q_heads, (cuuint64_t)q_tokens, (cuuint64_t)batch};
-    const cuuint64_t strides[3] = {256, (cuuint64_t)q_heads * 256, (cuuint64_t)q_tokens * q_heads * 256};
+    const cuuint64_t row = (cuuint64_t)head_dim * 2;
+    const cuuint64_t dims[4] = {(cuuint64_t)head_dim, (cuuint64_t)q_heads, (cuuint64_t)q_tokens, (cuuint64_t)batch};
+    const cuuint64_t strides[3] = {row, (cuuint64_t)q_heads * row, (cuuint64_t)q_tokens * q_heads * row};
     const cuuint32_t box[4] = {64, (cuuint32_t)group, (cuuint32_t)q_tokens, 1};
     const cuuint32_t elem[4] = {1, 1, 1, 1};
     return encode(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 4, const_cast<void *>(q), dims, strides, box, elem,
@@ -115,7 +118,7 @@ bool make_query_map(CUtensorMap *map, const void *q, int32_t batch, int32_t q_to
                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <bool kPaged>
+template <int D, bool kPaged>
 int launch_grouped_umma(const GroupedParams &p, unsigned *ticket, const CUtensorMap &map_q, const CUtensorMap &map_k,
                         const CUtensorMap &map_v, cudaStream_t stream)
 {
@@ -123,8 +126,8 @@ int launch_grouped_umma(const GroupedParams &p, unsigned *ticket, const CUtensor
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return INSTINFER_ERR_CUDA;
     if (!done[dev]) {
-        if (cudaFuncSetAttribute(grouped_attn_umma_kernel<kPaged>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 kUmmaSmemBytes) != cudaSuccess) {
+        if (cudaFuncSetAttribute(grouped_attn_umma_kernel<D, kPaged>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 UmmaGeometry<D>::kSmemBytes) != cudaSuccess) {
             (void)cudaGetLastError();
             return INSTINFER_ERR_CUDA;
         }
@@ -137,11 +140,11 @@ int launch_grouped_umma(const GroupedParams &p, unsigned *ticket, const CUtensor
     }
     const int64_t chunks = (int64_t)p.a.pairs * p.a.n_splits;
     const unsigned grid = (unsigned)(chunks < sm_count() ? chunks : sm_count());
-    cudaError_t err = launch_overlapped(grouped_attn_umma_kernel<kPaged>, grid, kUmmaThreads, kUmmaSmemBytes, stream,
-                                        p, ticket, map_q, map_k, map_v);
+    cudaError_t err = launch_overlapped(grouped_attn_umma_kernel<D, kPaged>, grid, kUmmaThreads,
+                                        UmmaGeometry<D>::kSmemBytes, stream, p, ticket, map_q, map_k, map_v);
     if (err != cudaSuccess || cudaGetLastError() != cudaSuccess) return INSTINFER_ERR_CUDA;
     if (p.a.n_splits > 1) {
-        err = launch_overlapped(grouped_merge_kernel<128>, (unsigned)(p.a.pairs * p.rows), 128, 0, stream, p);
+        err = launch_overlapped(grouped_merge_kernel<D>, (unsigned)(p.a.pairs * p.rows), D, 0, stream, p);
         if (err != cudaSuccess || cudaGetLastError() != cudaSuccess) return INSTINFER_ERR_CUDA;
     }
     return INSTINFER_OK;
@@ -200,9 +203,11 @@ int instinfer_decode_attention_grouped(void *out, float *lse, const void *q, con
     // 2^31 rows or more, or a driver without the encoder, takes the warp-level form.
     CUtensorMap map_q, map_k, map_v;
     const bool umma = g_grouped_path != 1 && umma_shape(head_dim, paged, block_tokens) &&
-                      make_query_map(&map_q, q, batch, q_tokens, q_heads, p.group) &&
-                      make_cache_map(&map_k, k_cache, kv_bytes / 256, paged && block_tokens < kUmmaTile ? block_tokens : kUmmaTile) &&
-                      make_cache_map(&map_v, v_cache, kv_bytes / 256, paged && block_tokens < kUmmaTile ? block_tokens : kUmmaTile);
+                      make_query_map(&map_q, q, batch, q_tokens, q_heads, p.group, head_dim) &&
+                      make_cache_map(&map_k, k_cache, kv_bytes / (2 * head_dim), head_dim,
+                                     paged && block_tokens < kUmmaTile ? block_tokens : kUmmaTile) &&
+                      make_cache_map(&map_v, v_cache, kv_bytes / (2 * head_dim), head_dim,
+                                     paged && block_tokens < kUmmaTile ? block_tokens : kUmmaTile);
     const SplitPlan plan = make_plan(pairs, max_seq_len, umma ? umma_rules() : grouped_rules(head_dim));
     if (workspace == nullptr || !aligned16(workspace) ||
         workspace_bytes < grouped_workspace_for(pairs, p.rows, head_dim, plan))
@@ -238,8 +243,11 @@ int instinfer_decode_attention_grouped(void *out, float *lse, const void *q, con
         // the ticket counter sits in the last 256 bytes of the workspace, behind the partials
         unsigned *ticket = reinterpret_cast<unsigned *>(
             static_cast<unsigned char *>(workspace) + grouped_workspace_for(pairs, p.rows, head_dim, plan) - 256);
-        return paged ? launch_grouped_umma<true>(p, ticket, map_q, map_k, map_v, stream)
-                     : launch_grouped_umma<false>(p, ticket, map_q, map_k, map_v, stream);
+        if (head_dim == 128)
+            return paged ? launch_grouped_umma<128, true>(p, ticket, map_q, map_k, map_v, stream)
+                         : launch_grouped_umma<128, false>(p, ticket, map_q, map_k, map_v, stream);
+        return paged ? launch_grouped_umma<256, true>(p, ticket, map_q, map_k, map_v, stream)
+                     : launch_grouped_umma<256, false>(p, ticket, map_q, map_k, map_v, stream);
     }
     switch (head_dim) {
     case 64: return paged ? launch_grouped<64, true>(p, grid, stream) : launch_grouped<64, false>(p, grid, stream);
@@ -257,7 +265,7 @@ size_t instinfer_grouped_workspace_bytes(int32_t batch, int32_t q_tokens, int32_
     // enough for either implementation: which one runs also depends on the cache layout
     const int32_t rows = q_heads / kv_heads * q_tokens;
     size_t bytes = grouped_workspace_for(pairs, rows, head_dim, make_plan(pairs, max_seq_len, grouped_rules(head_dim)));
-    if (head_dim == 128) {
+    if (head_dim != 64) {
         const size_t other = grouped_workspace_for(pairs, rows, head_dim, make_plan(pairs, max_seq_len, umma_rules()));
         if (other > bytes) bytes = other;
     }

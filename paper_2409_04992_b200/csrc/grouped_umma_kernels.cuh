@@ -1,5 +1,5 @@
 // Split-KV decode attention for several query rows per KV head on the fifth-generation tensor
-// cores (tcgen05 MMAs with accumulators in tensor memory), head size 128, for sm_100a.
+// cores (tcgen05 MMAs with accumulators in tensor memory), head sizes 128 and 256, for sm_100a.
 //
 // Same operation and same split plan as grouped_attn_split_kernel (grouped heads and several
 // new tokens per step put R <= 16 query rows against one KV head's cache: the paper's "other
@@ -7,16 +7,18 @@
 // contractions are written with the TOKENS as the long side of the MMA, so that nothing is
 // padding:
 //   S^T[128 tokens x 16 rows]  = K_tile[128 x D] Q^T[D x 16]        (M = 128, N = 16, K = D)
-//   O^T[D x 32]               += V_tile^T[D x 128] P^T[128 x 32]    (M = D = 128, N = 32, K = 128)
+//   O^T[D x 32]               += V_tile^T[D x 128] P^T[128 x 32]    (M = 128 dims at a time, N = 32, K = 128)
 // where the 32 columns of P^T are the fp16 high and low parts of the 16 rows' softmax weights
-// (so that the result keeps fp32-level accuracy), added up in the epilogue.
+// (so that the result keeps fp32-level accuracy), added up in the epilogue.  With head size 256
+// the first product takes its K in two halves and the second is two MMAs into two accumulators.
 //
 // The kernel is persistent: one block per SM draws chunks (token ranges of one (sequence, KV
 // head), the same list one block per chunk would run) from a ticket counter, and its copy
 // pipeline runs on across chunk boundaries.  A block has eight warps, each with one job, that
 // hand tiles to one another through mbarriers:
 //   * warp 4 (K producer) moves 128-token tiles of K with tensor-map copies (cp.async.bulk.tensor,
-//     128-byte swizzle, this GPU's memory, every block fetching its own tiles) into a ring of three 32 KiB slots; a
+//     128-byte swizzle, this GPU's memory, every block fetching its own tiles) into a ring of
+//     three 32 KiB slots (128 dims of a tile each: head size 256 takes two per tile); a
 //     paged tile is 128 / T copies of one (block, head) run each (one copy of 128 rows where a
 //     block holds a multiple of 128 tokens), the block ids read one tile
 //     ahead; a block with a bad id is not fetched but zero-filled.  It also draws the tickets
@@ -54,42 +56,56 @@ namespace instinfer {
 
 constexpr int kUmmaTile = 128;                         // tokens per tile
 constexpr int kUmmaPanelBytes = kUmmaTile * 128;       // 64 dims of 128 tokens (rows of 128 bytes)
-constexpr int kUmmaItemBytes = 2 * kUmmaPanelBytes;    // a K tile, or a V tile: 32 KiB
-constexpr int kUmmaKSlots = 3;                         // ring depth of K tiles
-constexpr int kUmmaVSlots = 3;                         // ring depth of V tiles
-constexpr int kUmmaQBytes = kGroupRows * 256;          // 16 query rows as two 64-dim panels
 constexpr int kUmmaQBuffers = 2;                       // the next chunk's query rows arrive early
 constexpr int kUmmaPBytes = 32 * kUmmaTile * 2;        // 32 weight columns of 128 tokens
 constexpr int kUmmaMiscBytes = 2048;                   // barriers, work queue, tensor-memory address, reductions
-constexpr int kUmmaCarveBytes = (kUmmaKSlots + kUmmaVSlots) * kUmmaItemBytes + kUmmaQBuffers * kUmmaQBytes + kUmmaPBytes + kUmmaMiscBytes;
-constexpr int kUmmaSmemBytes = kUmmaCarveBytes + 1024; // room to align the ring to 1024 bytes
 constexpr int kUmmaThreads = 256;                      // 4 softmax warps, K and V producers, logit and output MMA issuers
 constexpr int kUmmaWarpK = 4, kUmmaWarpV = 5, kUmmaWarpLogits = 6, kUmmaWarpOutput = 7;
-constexpr int kUmmaTmemCols = 128;                     // 2 x 16 logits, 2 x 32 output accumulator (96 used)
 constexpr int kUmmaQueue = 4;                          // chunks the producer may be ahead of the consumers
+constexpr int kUmmaSlots = 3;                          // ring depth of each cache, in items (96 KiB)
+constexpr int kUmmaItemPanels = 2;                     // panels per ring item: 128 dims of 128 tokens, 32 KiB
+constexpr int kUmmaItemBytes = kUmmaItemPanels * kUmmaPanelBytes;
+
+// Sizes that follow from the head size D (128 or 256).  A token row is D / 64 panels of 64 dims;
+// the rings hold items of two panels, so a tile of head size 256 is two items per cache and the
+// bytes in flight are the same for both head sizes.  (Head size 64 is not taken: a tile would
+// be half the bytes for the same softmax work per token, and the softmax chain, one thread per
+// token, then bounds the kernel: 4.4 TB/s measured, against 6.8 for the warp-level kernel.)
+template <int D>
+struct UmmaGeometry {
+    static_assert(D == 128 || D == 256, "head sizes of the tcgen05 form");
+    static constexpr int kPanels = D / 64;
+    static constexpr int kItems = kPanels / kUmmaItemPanels;             // ring items per tile and cache
+    static constexpr int kAccs = D / 128;                                // output accumulators of 128 dims
+    static constexpr int kQBytes = kGroupRows * D * 2;                   // 16 query rows, panel by panel
+    static constexpr int kTmemCols = D == 256 ? 256 : 128;               // 2 x 16 logits, 2 x kAccs x 32 output columns
+    static constexpr int kCarveBytes = 2 * kUmmaSlots * kUmmaItemBytes + kUmmaQBuffers * kQBytes + kUmmaPBytes + kUmmaMiscBytes;
+    static constexpr int kSmemBytes = kCarveBytes + 1024;                // room to align the rings to 1024 bytes
+    static_assert(kSmemBytes <= 227 * 1024, "one block per SM must fit");
+};
 
 // offsets inside the misc region
-constexpr int kUmmaBarKFull = 0;       // [kUmmaKSlots] K tile landed
-constexpr int kUmmaBarKEmpty = 24;     // [kUmmaKSlots] the logit MMAs that read the slot are complete
-constexpr int kUmmaBarVFull = 48;      // [kUmmaVSlots] V tile landed
-constexpr int kUmmaBarVEmpty = 72;     // [kUmmaVSlots] the output MMAs that read the slot are complete
-constexpr int kUmmaBarSFull = 96;      // [2] logits of a tile are in tensor memory
-constexpr int kUmmaBarSFree = 112;     // [2] the softmax warps have read them
-constexpr int kUmmaBarPFull = 128;     // weights of a tile are in shared memory
-constexpr int kUmmaBarPvDone = 136;    // the second MMA of a tile is complete
-constexpr int kUmmaBarQFull = 144;     // [2] query rows of a chunk landed
-constexpr int kUmmaBarQEmpty = 160;    // [2] the chunk's last logit MMA is complete
-constexpr int kUmmaBarWorkFull = 176;  // [kUmmaQueue] a chunk is announced
-constexpr int kUmmaBarWorkEmpty = 208; // [kUmmaQueue] all seven consumers have read the announcement
-constexpr int kUmmaTmemPtr = 240;
-constexpr int kUmmaAbort = 244;        // set by a softmax thread whose wait ran out
-constexpr int kUmmaWork = 256;         // [kUmmaQueue] int2 {chunk number or -1, sequence length}
-constexpr int kUmmaBarAccFree = 288;   // [2] the epilogue has read the accumulator of a chunk of this parity
-constexpr int kUmmaRed = 384;          // [4][16] floats: per-warp row maxima of a tile
-constexpr int kUmmaSavedM = 640;       // [2][16] floats: a finished chunk's references, by chunk parity
-constexpr int kUmmaSavedL = 768;       // [2][4][16] floats: its per-warp row sums
+constexpr int kUmmaBarKFull = 0;       // [slots] K item landed
+constexpr int kUmmaBarKEmpty = 48;     // [slots] the logit MMAs that read the slot are complete
+constexpr int kUmmaBarVFull = 96;      // [slots] V item landed
+constexpr int kUmmaBarVEmpty = 144;    // [slots] the output MMAs that read the slot are complete
+constexpr int kUmmaBarSFull = 192;     // [2] logits of a tile are in tensor memory
+constexpr int kUmmaBarSFree = 208;     // [2] the softmax warps have read them
+constexpr int kUmmaBarPFull = 224;     // weights of a tile are in shared memory
+constexpr int kUmmaBarPvDone = 232;    // the output MMAs of a tile are complete
+constexpr int kUmmaBarQFull = 240;     // [2] query rows of a chunk landed
+constexpr int kUmmaBarQEmpty = 256;    // [2] the chunk's last logit MMA is complete
+constexpr int kUmmaBarWorkFull = 272;  // [kUmmaQueue] a chunk is announced
+constexpr int kUmmaBarWorkEmpty = 304; // [kUmmaQueue] all seven consumers have read the announcement
+constexpr int kUmmaBarAccFree = 336;   // [2] the epilogue has read the accumulator of a chunk of this parity
+constexpr int kUmmaTmemPtr = 352;
+constexpr int kUmmaAbort = 356;        // set by a softmax thread whose wait ran out
+constexpr int kUmmaWork = 384;         // [kUmmaQueue] int2 {chunk number or -1, sequence length}
+constexpr int kUmmaRed = 448;          // [4][16] floats: per-warp row maxima of a tile
+constexpr int kUmmaSavedM = 704;       // [2][16] floats: a finished chunk's references, by chunk parity
+constexpr int kUmmaSavedL = 832;       // [2][4][16] floats: its per-warp row sums
+static_assert(kUmmaBarKEmpty - kUmmaBarKFull >= 8 * kUmmaSlots && kUmmaWork + 8 * kUmmaQueue <= kUmmaRed, "barriers overlap");
 static_assert(kUmmaSavedL + 512 <= kUmmaMiscBytes, "misc region too small");
-static_assert(kUmmaSmemBytes <= 227 * 1024, "one block per SM must fit");
 
 // ---- tcgen05 / TMA wrappers ----------------------------------------------------------------
 // The roles of this kernel hand tiles to one another in a chain (copy -> MMA -> softmax -> MMA),
@@ -254,12 +270,15 @@ __device__ __forceinline__ UmmaChunk umma_chunk(const AttnParams &a, int w, int 
 // Persistent: one block per SM; blocks draw chunks from a ticket counter (`ticket`, zeroed by
 // the host before the launch) until the list is exhausted, and the producers stream tiles
 // across chunk boundaries, so the copy pipeline never drains between chunks.
-template <bool kPaged>
+template <int D, bool kPaged>
 __global__ void __launch_bounds__(kUmmaThreads, 1)
 grouped_attn_umma_kernel(const GroupedParams p, unsigned *ticket, const __grid_constant__ CUtensorMap map_q,
                          const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v)
 {
-    constexpr int D = 128;
+    using Geo = UmmaGeometry<D>;
+    constexpr int kSlots = kUmmaSlots, kItems = Geo::kItems, kItemPanels = kUmmaItemPanels, kItemBytes = kUmmaItemBytes;
+    constexpr int kQBytes = Geo::kQBytes, kAccs = Geo::kAccs;
+    constexpr int kQPanelBytes = kGroupRows * 128;              // 16 query rows of 64 dims
     extern __shared__ unsigned char smem_raw[];
     const AttnParams &a = p.a;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -273,9 +292,10 @@ grouped_attn_umma_kernel(const GroupedParams p, unsigned *ticket, const __grid_c
     const unsigned raw = static_cast<unsigned>(__cvta_generic_to_shared(smem_raw));
     const unsigned ring = (raw + 1023u) & ~1023u;
     unsigned char *smem = smem_raw + (ring - raw);
-    constexpr int kVOffset = kUmmaKSlots * kUmmaItemBytes;
-    constexpr int kQOffset = kVOffset + kUmmaVSlots * kUmmaItemBytes;
-    constexpr int kPOffset = kQOffset + kUmmaQBuffers * kUmmaQBytes;
+    constexpr int kKOffset = 0;
+    constexpr int kVOffset = kSlots * kItemBytes;
+    constexpr int kQOffset = kVOffset + kSlots * kItemBytes;
+    constexpr int kPOffset = kQOffset + kUmmaQBuffers * kQBytes;
     constexpr int kMiscOffset = kPOffset + kUmmaPBytes;
     const unsigned q_smem = ring + kQOffset;
     const unsigned p_smem = ring + kPOffset;
@@ -288,17 +308,14 @@ grouped_attn_umma_kernel(const GroupedParams p, unsigned *ticket, const __grid_c
     // ---- set-up ----
     if (warp == kUmmaWarpLogits) {             // tensor memory: one warp allocates and later frees
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                     :: "r"(misc + kUmmaTmemPtr), "n"(kUmmaTmemCols) : "memory");
+                     :: "r"(misc + kUmmaTmemPtr), "n"(Geo::kTmemCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     } else if (warp == kUmmaWarpK) {
         if (lane == 0) {
 #pragma unroll
-            for (int s = 0; s < kUmmaKSlots; ++s) {
+            for (int s = 0; s < kSlots; ++s) {
                 mbarrier_init(misc + kUmmaBarKFull + s * 8, 1);
                 mbarrier_init(misc + kUmmaBarKEmpty + s * 8, 1);
-            }
-#pragma unroll
-            for (int s = 0; s < kUmmaVSlots; ++s) {
                 mbarrier_init(misc + kUmmaBarVFull + s * 8, 1);
                 mbarrier_init(misc + kUmmaBarVEmpty + s * 8, 1);
             }
@@ -327,7 +344,7 @@ grouped_attn_umma_kernel(const GroupedParams p, unsigned *ticket, const __grid_c
         // The query buffers start as zeros: a chunk's copy overwrites rows < p.rows only, so the
         // padding rows of the 16-row operand stay zero for the whole launch.
         const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
-        for (int i = threadIdx.x; i < kUmmaQBuffers * kUmmaQBytes / 16; i += 128)
+        for (int i = threadIdx.x; i < kUmmaQBuffers * kQBytes / 16; i += 128)
             *reinterpret_cast<uint4 *>(smem + kQOffset + i * 16) = zero;
         fence_async_proxy();
     }
@@ -337,13 +354,13 @@ grouped_attn_umma_kernel(const GroupedParams p, unsigned *ticket, const __grid_c
     const unsigned tmem = *reinterpret_cast<volatile unsigned *>(misc_ptr + kUmmaTmemPtr);
 
     // What both producers do for one chunk: the chunk's tiles of one cache (K or V) into that
-    // cache's ring, tile `count` of this block going to slot count % slots; returns false if a
+    // cache's ring, item `count` of this block going to slot count % kSlots; returns false if a
     // wait ran out.
     // A copy moves `T` rows: a whole block of 16, 32 or 64 tokens, or 128 rows of a larger block
     // (a multiple of 128 tokens: tiles start on multiples of 128 then and never straddle a block),
     // or of a contiguous cache.
     const int T = kPaged ? min(a.block_tokens, kUmmaTile) : kUmmaTile;
-    auto stream_chunk = [&](const UmmaChunk &c, const CUtensorMap *map, int ring_offset, int slots, int bar_full,
+    auto stream_chunk = [&](const UmmaChunk &c, const CUtensorMap *map, int ring_offset, int bar_full,
                             int bar_empty, int &count) -> bool {
         const int64_t total_rows = a.kv_bytes / (2 * D);
         const int32_t *table_row = kPaged ? a.block_table + (int64_t)c.b * a.max_blocks_per_seq : nullptr;
@@ -356,7 +373,7 @@ grouped_attn_umma_kernel(const GroupedParams p, unsigned *ticket, const __grid_c
             return __ldg(table_row + idx);
         };
         int ids_next = fetch_ids(0);
-        for (int j = 0; j < c.n_tiles; ++j, ++count) {
+        for (int j = 0; j < c.n_tiles; ++j) {
             const int tile_start = c.begin + j * kUmmaTile;
             const int nb = kPaged ? (min(c.end - tile_start, kUmmaTile) + T - 1) / T : 1;
             const int phys = ids_next;
@@ -372,34 +389,39 @@ grouped_attn_umma_kernel(const GroupedParams p, unsigned *ticket, const __grid_c
             } else {
                 row0 = c.pair * a.s_max + tile_start;          // rows past the tensor's end read as zeros
             }
-            const int slot = count % slots;
-            if (count >= slots &&
-                !__all_sync(0xffffffffu, mbarrier_wait_bounded(misc + bar_empty + slot * 8, (count / slots - 1) & 1)))
-                return false;
-            const int slot_offset = ring_offset + slot * kUmmaItemBytes + (kPaged ? lane * T * 128 : 0);
-            const unsigned bar = misc + bar_full + slot * 8;
-            if (kPaged && lane < nb && !good) {                // a block that cannot be read counts as zeros
-                const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
-                for (int i = 0; i < T * 8; ++i) {
-                    *reinterpret_cast<uint4 *>(smem + slot_offset + i * 16) = zero;
-                    *reinterpret_cast<uint4 *>(smem + slot_offset + kUmmaPanelBytes + i * 16) = zero;
-                }
-                fence_async_proxy();
-            }
             const unsigned fetched = __popc(__ballot_sync(0xffffffffu, good));
-            if (lane == 0) mbarrier_expect_bytes(bar, fetched * (unsigned)T * 256u);
-            __syncwarp();
-            if (good) {
-                tma_load_2d(ring + slot_offset, map, 0, row0, bar);
-                tma_load_2d(ring + slot_offset + kUmmaPanelBytes, map, 64, row0, bar);
+#pragma unroll
+            for (int item = 0; item < kItems; ++item, ++count) {
+                const int slot = count % kSlots;
+                if (count >= kSlots &&
+                    !__all_sync(0xffffffffu, mbarrier_wait_bounded(misc + bar_empty + slot * 8, (count / kSlots - 1) & 1)))
+                    return false;
+                const int slot_offset = ring_offset + slot * kItemBytes + (kPaged ? lane * T * 128 : 0);
+                const unsigned bar = misc + bar_full + slot * 8;
+                if (kPaged && lane < nb && !good) {            // a block that cannot be read counts as zeros
+                    const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
+                    for (int i = 0; i < T * 8; ++i) {
+#pragma unroll
+                        for (int panel = 0; panel < kItemPanels; ++panel)
+                            *reinterpret_cast<uint4 *>(smem + slot_offset + panel * kUmmaPanelBytes + i * 16) = zero;
+                    }
+                    fence_async_proxy();
+                }
+                if (lane == 0) mbarrier_expect_bytes(bar, fetched * (unsigned)(T * 128 * kItemPanels));
+                __syncwarp();
+                if (good) {
+#pragma unroll
+                    for (int panel = 0; panel < kItemPanels; ++panel)
+                        tma_load_2d(ring + slot_offset + panel * kUmmaPanelBytes, map, (item * kItemPanels + panel) * 64, row0, bar);
+                }
             }
         }
         return true;
     };
     // copies in flight must land (or be given up, bounded) before shared memory is handed on
-    auto drain = [&](int slots, int bar_full, int count) {
-        for (int i = max(count - slots, 0); i < count; ++i)
-            (void)mbarrier_poll_bounded(misc + bar_full + (i % slots) * 8, (i / slots) & 1);
+    auto drain = [&](int bar_full, int count) {
+        for (int i = max(count - kSlots, 0); i < count; ++i)
+            (void)mbarrier_poll_bounded(misc + bar_full + (i % kSlots) * 8, (i / kSlots) & 1);
     };
 
     if (warp == kUmmaWarpK) {
@@ -436,7 +458,7 @@ grouped_attn_umma_kernel(const GroupedParams p, unsigned *ticket, const __grid_c
         int w_now = ticket_of(issue_draw());
         int w_next = ticket_of(issue_draw());
         int len_now = checked_length(w_now, issue_length(w_now));
-        int count = 0;                                  // K tiles issued so far (ring position)
+        int count = 0;                                  // K items issued so far (ring position)
         int k = 0;                                      // chunks announced so far
         bool fine = true;
         bool first = true;
@@ -483,12 +505,13 @@ grouped_attn_umma_kernel(const GroupedParams p, unsigned *ticket, const __grid_c
             if (!fine) break;
             if (lane == 0) {
                 const unsigned bar = misc + kUmmaBarQFull + qb * 8;
-                mbarrier_expect_bytes(bar, (unsigned)p.rows * 256u);
-                tma_load_4d(q_smem + qb * kUmmaQBytes, &map_q, 0, c.hk * p.group, 0, c.b, bar);
-                tma_load_4d(q_smem + qb * kUmmaQBytes + kUmmaQBytes / 2, &map_q, 64, c.hk * p.group, 0, c.b, bar);
+                mbarrier_expect_bytes(bar, (unsigned)(p.rows * D * 2));
+#pragma unroll
+                for (int panel = 0; panel < Geo::kPanels; ++panel)
+                    tma_load_4d(q_smem + qb * kQBytes + panel * kQPanelBytes, &map_q, panel * 64, c.hk * p.group, 0, c.b, bar);
             }
             ++k;
-            fine = stream_chunk(c, &map_k, 0, kUmmaKSlots, kUmmaBarKFull, kUmmaBarKEmpty, count);
+            fine = stream_chunk(c, &map_k, kKOffset, kUmmaBarKFull, kUmmaBarKEmpty, count);
         }
         if (fine) {                                     // no chunk is left: tell the others
             const int wq = k % kUmmaQueue;
@@ -503,7 +526,7 @@ grouped_attn_umma_kernel(const GroupedParams p, unsigned *ticket, const __grid_c
         }
         if (!fine) {
             if (lane == 0 && a.status) atomicOr(a.status, kFlagCopyTimeout);
-            drain(kUmmaKSlots, kUmmaBarKFull, count);
+            drain(kUmmaBarKFull, count);
         }
     } else if (warp == kUmmaWarpV) {
         // ================================ V producer ================================
@@ -517,11 +540,11 @@ grouped_attn_umma_kernel(const GroupedParams p, unsigned *ticket, const __grid_c
             __syncwarp();
             if (lane == 0) mbarrier_arrive(misc + kUmmaBarWorkEmpty + wq * 8);
             if (w < 0) break;
-            fine = stream_chunk(umma_chunk(a, w, len), &map_v, kVOffset, kUmmaVSlots, kUmmaBarVFull, kUmmaBarVEmpty, count);
+            fine = stream_chunk(umma_chunk(a, w, len), &map_v, kVOffset, kUmmaBarVFull, kUmmaBarVEmpty, count);
         }
         if (!fine) {
             if (lane == 0 && a.status) atomicOr(a.status, kFlagCopyTimeout);
-            drain(kUmmaVSlots, kUmmaBarVFull, count);
+            drain(kUmmaBarVFull, count);
         }
     } else if (warp == kUmmaWarpLogits) {
         // ================================ logit MMAs ================================
@@ -543,26 +566,34 @@ grouped_attn_umma_kernel(const GroupedParams p, unsigned *ticket, const __grid_c
                 fine = __all_sync(0xffffffffu, mbarrier_wait_bounded(misc + kUmmaBarQFull + (k & 1) * 8, (k / 2) & 1));
                 // K tile and query rows alike: rows of 128 bytes per 64-dim panel, 8-row groups 1024
                 // bytes apart, 128-byte swizzle; a k-step of 16 dims is 32 bytes along the row
-                const uint64_t q_desc = umma_desc(q_smem + (k & 1) * kUmmaQBytes, 16, 1024, 2);
+                const uint64_t q_desc = umma_desc(q_smem + (k & 1) * kQBytes, 16, 1024, 2);
                 for (int j = 0; j < n_tiles && fine; ++j, ++g) {
-                    const int slot = g % kUmmaKSlots;
-                    fine = __all_sync(0xffffffffu,
-                                      mbarrier_wait_bounded(misc + kUmmaBarKFull + slot * 8, (g / kUmmaKSlots) & 1) &&
-                                      (g < 2 || mbarrier_wait_bounded(misc + kUmmaBarSFree + (g & 1) * 8, ((g >> 1) - 1) & 1)));
-                    if (!fine) break;
-                    tc_fence_after();
-                    const uint64_t k_desc = umma_desc(ring + slot * kUmmaItemBytes, 16, 1024, 2);
-                    if (elect_one()) {
+                    if (g >= 2)
+                        fine = __all_sync(0xffffffffu, mbarrier_wait_bounded(misc + kUmmaBarSFree + (g & 1) * 8, ((g >> 1) - 1) & 1));
 #pragma unroll
-                        for (int ks = 0; ks < 8; ++ks)
-                            tc_mma_f16(tmem + (g & 1) * 16, k_desc + (uint64_t)(((ks >> 2) * kUmmaPanelBytes + (ks & 3) * 32) >> 4),
-                                       q_desc + (uint64_t)(((ks >> 2) * (kUmmaQBytes / 2) + (ks & 3) * 32) >> 4), idesc, ks > 0);
-                        tc_commit(misc + kUmmaBarSFull + (g & 1) * 8);
-                        tc_commit(misc + kUmmaBarKEmpty + slot * 8);
-                        // after the chunk's last logit MMA its query rows may be replaced
-                        if (j + 1 == n_tiles) tc_commit(misc + kUmmaBarQEmpty + (k & 1) * 8);
+                    for (int item = 0; item < kItems; ++item) {
+                        if (!fine) break;
+                        const int n = g * kItems + item, slot = n % kSlots;
+                        fine = __all_sync(0xffffffffu, mbarrier_wait_bounded(misc + kUmmaBarKFull + slot * 8, (n / kSlots) & 1));
+                        if (!fine) break;
+                        tc_fence_after();
+                        const uint64_t k_desc = umma_desc(ring + kKOffset + slot * kItemBytes, 16, 1024, 2);
+                        if (elect_one()) {
+#pragma unroll
+                            for (int ks = 0; ks < 4 * kItemPanels; ++ks)
+                                tc_mma_f16(tmem + (g & 1) * 16, k_desc + (uint64_t)(((ks >> 2) * kUmmaPanelBytes + (ks & 3) * 32) >> 4),
+                                           q_desc + (uint64_t)(((item * kItemPanels + (ks >> 2)) * kQPanelBytes + (ks & 3) * 32) >> 4),
+                                           idesc, item > 0 || ks > 0);
+                            tc_commit(misc + kUmmaBarKEmpty + slot * 8);
+                            if (item + 1 == kItems) {
+                                tc_commit(misc + kUmmaBarSFull + (g & 1) * 8);
+                                // after the chunk's last logit MMA its query rows may be replaced
+                                if (j + 1 == n_tiles) tc_commit(misc + kUmmaBarQEmpty + (k & 1) * 8);
+                            }
+                        }
+                        __syncwarp();
                     }
-                    __syncwarp();
+                    if (!fine) break;
                 }
             }
             if (!fine && lane == 0 && a.status) atomicOr(a.status, kFlagCopyTimeout);
@@ -590,26 +621,31 @@ grouped_attn_umma_kernel(const GroupedParams p, unsigned *ticket, const __grid_c
                 // the accumulator of this parity was last used two chunks ago: its epilogue must have read it
                 if (k >= 2)
                     fine = __all_sync(0xffffffffu, mbarrier_poll_bounded(misc + kUmmaBarAccFree + (k & 1) * 8, (k / 2 - 1) & 1));
-                const unsigned acc = tmem + 32 + (k & 1) * 32;
+                const unsigned acc = tmem + 32 + (k & 1) * (kAccs * 32);
                 for (int j = 0; j < n_tiles && fine; ++j, ++g) {
-                    const int slot = g % kUmmaVSlots;
-                    fine = __all_sync(0xffffffffu,
-                                      mbarrier_poll_bounded(misc + kUmmaBarVFull + slot * 8, (g / kUmmaVSlots) & 1) &&
-                                      mbarrier_poll_bounded(misc + kUmmaBarPFull, g & 1));
-                    if (!fine) break;
-                    tc_fence_after();
-                    // V tile read MN-major (M = dims): the two 64-dim panels are kUmmaPanelBytes apart
-                    // (leading offset), 8-token groups 1024 bytes apart; a k-step is 16 tokens = 2048 bytes
-                    const uint64_t v_desc = umma_desc(ring + kVOffset + slot * kUmmaItemBytes, kUmmaPanelBytes, 1024, 2);
-                    if (elect_one()) {
+                    fine = __all_sync(0xffffffffu, mbarrier_poll_bounded(misc + kUmmaBarPFull, g & 1));
 #pragma unroll
-                        for (int ks = 0; ks < 8; ++ks)
-                            tc_mma_f16(acc, v_desc + (uint64_t)((ks * 2048) >> 4), p_desc + (uint64_t)((ks * 256) >> 4), idesc,
-                                       j > 0 || ks > 0);
-                        tc_commit(misc + kUmmaBarVEmpty + slot * 8);
-                        tc_commit(misc + kUmmaBarPvDone);
+                    for (int item = 0; item < kItems; ++item) {
+                        if (!fine) break;
+                        const int n = g * kItems + item, slot = n % kSlots;
+                        fine = __all_sync(0xffffffffu, mbarrier_poll_bounded(misc + kUmmaBarVFull + slot * 8, (n / kSlots) & 1));
+                        if (!fine) break;
+                        tc_fence_after();
+                        // V item read MN-major (M = 128 dims): its two 64-dim panels are kUmmaPanelBytes
+                        // apart (leading offset), 8-token groups 1024 bytes apart; a k-step is 16 tokens
+                        // = 2048 bytes
+                        const uint64_t v_desc = umma_desc(ring + kVOffset + slot * kItemBytes, kUmmaPanelBytes, 1024, 2);
+                        if (elect_one()) {
+#pragma unroll
+                            for (int ks = 0; ks < 8; ++ks)
+                                tc_mma_f16(acc + item * 32, v_desc + (uint64_t)((ks * 2048) >> 4), p_desc + (uint64_t)((ks * 256) >> 4),
+                                           idesc, j > 0 || ks > 0);
+                            tc_commit(misc + kUmmaBarVEmpty + slot * 8);
+                            if (item + 1 == kItems) tc_commit(misc + kUmmaBarPvDone);
+                        }
+                        __syncwarp();
                     }
-                    __syncwarp();
+                    if (!fine) break;
                 }
             }
             if (!fine && lane == 0 && a.status) atomicOr(a.status, kFlagCopyTimeout);
@@ -625,35 +661,40 @@ grouped_attn_umma_kernel(const GroupedParams p, unsigned *ticket, const __grid_c
         // next chunk has been handed to the MMA, so that the tensor pipe and the copies go on
         // meanwhile; the accumulators alternate between two regions of tensor memory.
         auto epilogue = [&](const UmmaChunk &c, int parity) {
-            // Thread t owns output dim t; columns r and 16 + r are the high and low parts of row
-            // r.  Sums and accumulator both carry kGroupWeightScale.
+            // Thread t owns output dims t, 128 + t, ... (one per accumulator); columns r and 16 + r
+            // are the high and low parts of row r.
+            // Sums and accumulator both carry kGroupWeightScale.
             tc_fence_after();
-            float o_hi[16], o_lo[16];
-            tc_load16(o_hi, lane_base + 32 + parity * 32);
-            tc_load16(o_lo, lane_base + 48 + parity * 32);
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbarrier_arrive(misc + kUmmaBarAccFree + parity * 8);
             const float *sl = saved_l + parity * 64, *sm = saved_m + parity * 16;
 #pragma unroll
-            for (int r = 0; r < 16; ++r) {
-                if (r < p.rows) {
-                    const float total_w = (sl[r] + sl[16 + r]) + (sl[32 + r] + sl[48 + r]);
-                    // A row that sees no position of this chunk (causal limit before the chunk) has total 0.
-                    const bool empty = !(total_w > 0.f);
-                    const float value = empty ? 0.f : (o_hi[r] + o_lo[r]) / total_w;
-                    const float lse2 = empty ? kMinusHuge : sm[r] + log2f(total_w) - kGroupWeightLog2;
-                    if (final_writer) {
-                        const int64_t row = grouped_row_index(p, c.b, c.hk, r);
-                        a.out[row * D + t] = __float2half_rn(value);
-                        if (a.lse && t == 0) a.lse[row] = empty ? -INFINITY : lse2 * kLn2;
-                    } else {
-                        const int64_t slot = ((int64_t)c.pair * a.n_splits + c.split) * p.rows + r;
-                        a.part_o[slot * D + t] = value;
-                        if (t == 0) a.part_lse[slot] = lse2;
+            for (int acc_i = 0; acc_i < kAccs; ++acc_i) {
+                float o_hi[16], o_lo[16];
+                tc_load16(o_hi, lane_base + 32 + (parity * kAccs + acc_i) * 32);
+                tc_load16(o_lo, lane_base + 48 + (parity * kAccs + acc_i) * 32);
+                const int d = acc_i * 128 + t;
+#pragma unroll
+                for (int r = 0; r < 16; ++r) {
+                    if (r < p.rows) {
+                        const float total_w = (sl[r] + sl[16 + r]) + (sl[32 + r] + sl[48 + r]);
+                        // A row that sees no position of this chunk (causal limit before the chunk) has total 0.
+                        const bool empty = !(total_w > 0.f);
+                        const float value = empty ? 0.f : (o_hi[r] + o_lo[r]) / total_w;
+                        const float lse2 = empty ? kMinusHuge : sm[r] + log2f(total_w) - kGroupWeightLog2;
+                        if (final_writer) {
+                            const int64_t row = grouped_row_index(p, c.b, c.hk, r);
+                            a.out[row * D + d] = __float2half_rn(value);
+                            if (a.lse && d == 0) a.lse[row] = empty ? -INFINITY : lse2 * kLn2;
+                        } else {
+                            const int64_t slot = ((int64_t)c.pair * a.n_splits + c.split) * p.rows + r;
+                            a.part_o[slot * D + d] = value;
+                            if (d == 0) a.part_lse[slot] = lse2;
+                        }
                     }
                 }
             }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbarrier_arrive(misc + kUmmaBarAccFree + parity * 8);
         };
         bool aborted = false, pending = false;
         UmmaChunk before = {};                                      // the chunk whose epilogue is pending
@@ -672,7 +713,7 @@ grouped_attn_umma_kernel(const GroupedParams p, unsigned *ticket, const __grid_c
             if (w < 0) break;
             const UmmaChunk c = umma_chunk(a, w, len);
             const int n_tiles = c.n_tiles;
-            const unsigned acc = lane_base + 32 + (k & 1) * 32;     // this chunk's accumulator
+            const unsigned acc = lane_base + 32 + (k & 1) * (kAccs * 32);     // this chunk's accumulator(s)
             float m[16], l[16];
 #pragma unroll
             for (int r = 0; r < 16; ++r) {
@@ -709,14 +750,17 @@ grouped_attn_umma_kernel(const GroupedParams p, unsigned *ticket, const __grid_c
                         // The value row of a position outside the chunk gets weight zero, but its bytes
                         // may be anything (the tail of a block, a slot not fetched): 0 x NaN must not
                         // reach the accumulator, so the row is cleared once the tile has landed.
-                        const int slot = g % kUmmaVSlots;
-                        fine = mbarrier_poll_bounded(misc + kUmmaBarVFull + slot * 8, (g / kUmmaVSlots) & 1);
                         const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
-                        unsigned char *vrow = smem + kVOffset + slot * kUmmaItemBytes + t * 128;
 #pragma unroll
-                        for (int i = 0; i < 8; ++i) {
-                            *reinterpret_cast<uint4 *>(vrow + i * 16) = zero;
-                            *reinterpret_cast<uint4 *>(vrow + kUmmaPanelBytes + i * 16) = zero;
+                        for (int item = 0; item < kItems; ++item) {
+                            const int n = g * kItems + item, slot = n % kSlots;
+                            if (fine) fine = mbarrier_poll_bounded(misc + kUmmaBarVFull + slot * 8, (n / kSlots) & 1);
+                            unsigned char *vrow = smem + kVOffset + slot * kItemBytes + t * 128;
+#pragma unroll
+                            for (int panel = 0; panel < kItemPanels; ++panel) {
+#pragma unroll
+                                for (int i = 0; i < 8; ++i) *reinterpret_cast<uint4 *>(vrow + panel * kUmmaPanelBytes + i * 16) = zero;
+                            }
                         }
                     }
                 }
@@ -759,7 +803,7 @@ grouped_attn_umma_kernel(const GroupedParams p, unsigned *ticket, const __grid_c
                             tc_fence_after();
                             float o[16];
 #pragma unroll
-                            for (int half = 0; half < 2; ++half) {  // columns 0-15: high parts, 16-31: low parts
+                            for (int half = 0; half < 2 * kAccs; ++half) {  // per accumulator, columns 0-15: high parts, 16-31: low parts
                                 tc_load16(o, acc + half * 16);
 #pragma unroll
                                 for (int r = 0; r < 16; ++r) o[r] *= alpha[r];
@@ -832,7 +876,7 @@ grouped_attn_umma_kernel(const GroupedParams p, unsigned *ticket, const __grid_c
     __syncthreads();
     if (warp == kUmmaWarpLogits) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(tmem), "n"(kUmmaTmemCols) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(tmem), "n"(Geo::kTmemCols) : "memory");
     }
 }
 

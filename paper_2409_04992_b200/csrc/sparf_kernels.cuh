@@ -255,14 +255,19 @@ __device__ __forceinline__ void score_setup(const SparfParams &p, int pair, Scor
     // rounding cannot change the ranking of step 6; each logit is an fp32 sum of r exact
     // fp16 x fp16 products times that constant, i.e. within (r + 1) 2^-24 of sum |q_t k_t|.
     __syncthreads();
-    if (d == 0) {
+    if (d < 32) {                                            // warp 0: lane sums, then a butterfly
         float all = 0.f, sel = 0.f;
-        for (int e = 0; e < kHeadDim; ++e) {
+        for (int e = d; e < kHeadDim; e += 32) {
             all += ss.abs_q[e];
             if (ss.kept[e]) sel += ss.abs_q[e];
         }
+#pragma unroll
+        for (int off = 16; off >= 1; off >>= 1) {
+            all += __shfl_xor_sync(0xffffffffu, all, off);
+            sel += __shfl_xor_sync(0xffffffffu, sel, off);
+        }
         const float ratio = all > 0.f ? sel / all : 1.f;
-        ss.approx_scale = p.scale_log2e / sqrtf(ratio);
+        if (d == 0) ss.approx_scale = p.scale_log2e / sqrtf(ratio);
     }
     __syncthreads();
 }
@@ -541,7 +546,6 @@ __device__ __forceinline__ void select_row(const SparfParams &p, SelectShared &s
         sh.red_u[0][warp] = __float_as_uint(low);
     }
     for (int t = tid; t <= kLinearBins; t += NT) sh.hist[t] = 0u;
-    if (tid < 32) sh.scan_gt[tid] = 0;           // warps that do not exist count nothing in the scans
     __syncthreads();
     for (int w = 0; w < NT / 32; ++w) {
         top = fmaxf(top, sh.red_f[w]);
@@ -647,29 +651,50 @@ __device__ __forceinline__ void select_row(const SparfParams &p, SelectShared &s
     const int T = p.block_tokens;
     const int t_shift = (T & (T - 1)) == 0 ? __ffs(T) - 1 : -1;      // blocks of 2^n tokens: no division per token
     const int32_t *table_row = p.block_table + (int64_t)b * p.max_blocks_per_seq;
-    int base_gt = 0, base_eq = 0;
     float mass = 0.f;
-    // Each thread takes 4 consecutive positions; counts travel packed (greater | equal << 16).
-    float4 ahead = tid < quads ? a4[tid] : make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int start = 0; start < quads; start += NT) {
-        const int g = start + tid;
-        const float4 v = ahead;
-        if (g + NT < quads) ahead = a4[g + NT];    // next tile's loads fly over the barriers
-        float x[4] = {0.f, 0.f, 0.f, 0.f};
+    // Each warp owns a contiguous span of the row, each lane 4 consecutive positions at a time.
+    // The warps count their spans, exchange the totals once, and then emit without meeting again.
+    constexpr int kWarps = NT / 32;
+    const int span = (quads + kWarps - 1) / kWarps;
+    const int q_begin = min(warp * span, quads), q_end = min(q_begin + span, quads);
+    // counts of one thread's 4 positions travel packed (greater | equal << 16)
+    auto classify = [&](int g, const float4 &v, bool (&gt)[4], bool (&eq)[4]) -> int {
+        const float x[4] = {v.x, v.y, v.z, v.w};
+        int packed = 0;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const int i = 4 * g + e;
+            const unsigned key = key_of(i, x[e]);
+            gt[e] = i < S && key > tau;
+            eq[e] = i < S && key == tau;
+            packed += (int)gt[e] + ((int)eq[e] << 16);
+        }
+        return packed;
+    };
+    int span_gt = 0, span_eq = 0;
+    for (int g = q_begin + lane; g < q_end; g += 32) {
+        bool gt[4], eq[4];
+        const int packed = classify(g, a4[g], gt, eq);
+        span_gt += packed & 0xffff;
+        span_eq += packed >> 16;
+    }
+    span_gt = __reduce_add_sync(0xffffffffu, span_gt);
+    span_eq = __reduce_add_sync(0xffffffffu, span_eq);
+    if (lane == 0) {
+        sh.scan_gt[warp] = span_gt;
+        sh.scan_eq[warp] = span_eq;
+    }
+    __syncthreads();
+    int base_gt = __reduce_add_sync(0xffffffffu, lane < warp ? sh.scan_gt[lane] : 0);
+    int base_eq = __reduce_add_sync(0xffffffffu, lane < warp ? sh.scan_eq[lane] : 0);
+    for (int g0 = q_begin; g0 < q_end; g0 += 32) {
+        const int g = g0 + lane;
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
         bool gt[4] = {false, false, false, false}, eq[4] = {false, false, false, false};
         int mine = 0;
-        if (g < quads) {
-            x[0] = v.x; x[1] = v.y; x[2] = v.z; x[3] = v.w;
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const int i = 4 * g + e;
-                if (i < S) {
-                    const unsigned key = key_of(i, x[e]);
-                    gt[e] = key > tau;
-                    eq[e] = key == tau;
-                    mine += (int)gt[e] + ((int)eq[e] << 16);
-                }
-            }
+        if (g < q_end) {
+            v = a4[g];
+            mine = classify(g, v, gt, eq);
         }
         int incl = mine;                          // inclusive scan over the warp
 #pragma unroll
@@ -677,18 +702,9 @@ __device__ __forceinline__ void select_row(const SparfParams &p, SelectShared &s
             const int up = __shfl_up_sync(0xffffffffu, incl, off);
             if (lane >= off) incl += up;
         }
-        if (lane == 31) sh.scan_gt[warp] = incl;
-        __syncthreads();
-        const int warp_total = sh.scan_gt[lane];  // every warp scans the 32 warp totals
-        int warp_incl = warp_total;
-#pragma unroll
-        for (int off = 1; off < 32; off <<= 1) {
-            const int up = __shfl_up_sync(0xffffffffu, warp_incl, off);
-            if (lane >= off) warp_incl += up;
-        }
-        const int tile_total = __shfl_sync(0xffffffffu, warp_incl, 31);
-        const int before = __shfl_sync(0xffffffffu, warp_incl - warp_total, warp) + incl - mine;
-        int gt_before = base_gt + (before & 0xffff), eq_before = base_eq + (before >> 16);
+        const int tile_total = __shfl_sync(0xffffffffu, incl, 31);
+        int gt_before = base_gt + ((incl - mine) & 0xffff), eq_before = base_eq + ((incl - mine) >> 16);
+        const float x[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
             if (gt[e] || (eq[e] && eq_before < take_equal)) {
@@ -707,7 +723,6 @@ __device__ __forceinline__ void select_row(const SparfParams &p, SelectShared &s
         }
         base_gt += tile_total & 0xffff;
         base_eq += tile_total >> 16;
-        __syncthreads();
     }
     mass = block_sum(mass, sh.red_f);
     if (tid == 0) {

@@ -101,10 +101,10 @@ def test_chunkings(chunk, q_tokens, q_heads, kv_heads):
 
 
 @pytest.mark.parametrize("dim", [64, 256])
-@pytest.mark.parametrize("layout,tokens", [("contiguous", 0), ("paged", 16)])
+@pytest.mark.parametrize("layout,tokens", [("contiguous", 0), ("paged", 16), ("paged", 64), ("paged", 128)])
 @pytest.mark.parametrize("q_tokens,q_heads,kv_heads", [(1, 2, 2), (1, 8, 2), (2, 8, 1)])
 def test_other_head_sizes(dim, layout, tokens, q_tokens, q_heads, kv_heads):
-    for chunk in (0, 64):
+    for chunk in (0, 64, 128):
         check(make(layout, tokens, kv_heads, q_tokens, q_heads, dim=dim), chunk,
               f"D={dim} {layout} Tq={q_tokens} Hq={q_heads} Hkv={kv_heads} chunk={chunk}")
 
@@ -113,8 +113,9 @@ def test_the_tcgen05_form_is_the_one_that_runs(grouped_path):
     """On a GPU machine the driver has the tensor-map encoder, so head size 128 with a contiguous
     cache or 16/32/64-token blocks takes the tcgen05 kernel unless the warp-level one is forced."""
     want = 2 if grouped_path == 2 else 1
-    for tokens in (0, 16, 32, 64, 128, 256):
-        assert binding.grouped_path_for(128, tokens) == want
+    for dim in (128, 256):
+        for tokens in (0, 16, 32, 64, 128, 256):
+            assert binding.grouped_path_for(dim, tokens) == want
     binding.set_grouped_path(0)
     assert binding.grouped_path_for(128, 16) == 2                                 # the default
     assert binding.grouped_path_for(128, 48) == 1 and binding.grouped_path_for(128, 192) == 1
@@ -123,7 +124,7 @@ def test_the_tcgen05_form_is_the_one_that_runs(grouped_path):
         assert binding.grouped_path_for(128, 128) == 1 and binding.grouped_path_for(128, 64) == 2
     finally:
         binding.set_chunk_tokens(0)
-    assert binding.grouped_path_for(64, 16) == 1 and binding.grouped_path_for(256, 0) == 1
+    assert binding.grouped_path_for(64, 16) == 1 and binding.grouped_path_for(256, 48) == 1
     assert binding.grouped_path_for(96, 16) == 0 and binding.grouped_path_for(128, 8) == 0
 
 
