@@ -143,38 +143,43 @@ def test_tiny_contiguous_cache_smaller_than_one_tile():
     check(g, 0, "two sequences of 1 and 3 tokens, contiguous")
 
 
-def test_peaked_logits():
+@pytest.mark.parametrize("dim", [128, 256])
+def test_peaked_logits(dim):
     for chunk in (0, 64):
-        g = make("paged", 32, 2, 2, 8, lens=[700, 1500, 40])
+        g = make("paged", 32, 2, 2, 8, dim=dim, lens=[700, 1500, 40])
         g.q.mul_(3.0)                               # logits of a few tens
-        check(g, chunk, f"peaked chunk={chunk}")
+        check(g, chunk, f"peaked chunk={chunk} D={dim}")
 
 
+@pytest.mark.parametrize("dim", [128, 256, 64])
 @pytest.mark.parametrize("layout,tokens", [("contiguous", 0), ("paged", 16), ("paged", 64)])
-def test_reference_moves_in_the_middle_of_a_chunk(layout, tokens):
+def test_reference_moves_in_the_middle_of_a_chunk(layout, tokens, dim):
     """Keys aligned with the query at a few late positions, each with a logit far above all
     earlier ones: the softmax reference moves (and the accumulator is rescaled) several times
     inside one chunk, not only at its first tile."""
     lens = [1700, 900]
-    g = make(layout, tokens, 1, 1, 4, lens=lens)
+    g = make(layout, tokens, 1, 1, 4, dim=dim, lens=lens)
     c = g.base
     T = tokens
     for b, n in enumerate(lens):
-        for pos, gain in ((n // 3, 2.0), (n // 2 + 5, 4.0), (n - 140, 7.0)):
+        # (|q|^2 * scale grows like sqrt(D): the gains keep the logits tens of units apart for every D)
+        for pos, gain in ((n // 3, 2.0 * (128 / dim) ** 0.5), (n // 2 + 5, 4.0 * (128 / dim) ** 0.5),
+                          (n - 140, 7.0 * (128 / dim) ** 0.5)):
             row = (g.q[b, 0, 0].float() * gain).half()          # logit = gain * |q|^2 * scale: tens of units apart
             if c.block_table is None:
                 c.k_cache[b, 0, pos] = row
             else:
                 c.k_cache[int(c.block_table[b, pos // T]), 0, pos % T] = row
     for chunk in (0, 2048, 256):
-        check(g, chunk, f"moving reference, {layout} T={tokens} chunk={chunk}")
+        check(g, chunk, f"moving reference, {layout} T={tokens} D={dim} chunk={chunk}")
 
 
-def test_a_block_that_cannot_be_read_counts_as_zeros():
+@pytest.mark.parametrize("dim", [128, 256])
+def test_a_block_that_cannot_be_read_counts_as_zeros(dim):
     """A block id outside the pool is flagged, and the result is the oracle's on the same cache
     with that block's keys and values zeroed (every form of the kernel)."""
     lens = [200, 330]
-    g = make("paged", 16, 2, 2, 4, lens=lens)
+    g = make("paged", 16, 2, 2, 4, dim=dim, lens=lens)
     dev = to_device(g)
     c = dev.base
     # append first with the good table, then break one entry for the attention call only
