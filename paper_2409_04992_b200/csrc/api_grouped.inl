@@ -118,7 +118,7 @@ bool make_query_map(CUtensorMap *map, const void *q, int32_t batch, int32_t q_to
                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int D, bool kPaged>
+template <int D, bool kPaged, int R>
 int launch_grouped_umma(const GroupedParams &p, unsigned *ticket, const CUtensorMap &map_q, const CUtensorMap &map_k,
                         const CUtensorMap &map_v, cudaStream_t stream)
 {
@@ -126,7 +126,7 @@ int launch_grouped_umma(const GroupedParams &p, unsigned *ticket, const CUtensor
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return INSTINFER_ERR_CUDA;
     if (!done[dev]) {
-        if (cudaFuncSetAttribute(grouped_attn_umma_kernel<D, kPaged>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        if (cudaFuncSetAttribute(grouped_attn_umma_kernel<D, kPaged, R>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  UmmaGeometry<D>::kSmemBytes) != cudaSuccess) {
             (void)cudaGetLastError();
             return INSTINFER_ERR_CUDA;
@@ -140,7 +140,7 @@ int launch_grouped_umma(const GroupedParams &p, unsigned *ticket, const CUtensor
     }
     const int64_t chunks = (int64_t)p.a.pairs * p.a.n_splits;
     const unsigned grid = (unsigned)(chunks < sm_count() ? chunks : sm_count());
-    cudaError_t err = launch_overlapped(grouped_attn_umma_kernel<D, kPaged>, grid, kUmmaThreads,
+    cudaError_t err = launch_overlapped(grouped_attn_umma_kernel<D, kPaged, R>, grid, kUmmaThreads,
                                         UmmaGeometry<D>::kSmemBytes, stream, p, ticket, map_q, map_k, map_v);
     if (err != cudaSuccess || cudaGetLastError() != cudaSuccess) return INSTINFER_ERR_CUDA;
     if (p.a.n_splits > 1) {
@@ -148,6 +148,22 @@ int launch_grouped_umma(const GroupedParams &p, unsigned *ticket, const CUtensor
         if (err != cudaSuccess || cudaGetLastError() != cudaSuccess) return INSTINFER_ERR_CUDA;
     }
     return INSTINFER_OK;
+}
+
+// The instance for the cache layout and for the number of query rows per KV head (4, 8 or 16
+// rows of softmax work per token).
+template <int D>
+int launch_grouped_umma_rows(bool paged, const GroupedParams &p, unsigned *ticket, const CUtensorMap &map_q,
+                             const CUtensorMap &map_k, const CUtensorMap &map_v, cudaStream_t stream)
+{
+    if (p.rows <= 4)
+        return paged ? launch_grouped_umma<D, true, 4>(p, ticket, map_q, map_k, map_v, stream)
+                     : launch_grouped_umma<D, false, 4>(p, ticket, map_q, map_k, map_v, stream);
+    if (p.rows <= 8)
+        return paged ? launch_grouped_umma<D, true, 8>(p, ticket, map_q, map_k, map_v, stream)
+                     : launch_grouped_umma<D, false, 8>(p, ticket, map_q, map_k, map_v, stream);
+    return paged ? launch_grouped_umma<D, true, 16>(p, ticket, map_q, map_k, map_v, stream)
+                 : launch_grouped_umma<D, false, 16>(p, ticket, map_q, map_k, map_v, stream);
 }
 
 // Shape checks shared by the entry point and its workspace query.
@@ -243,11 +259,8 @@ int instinfer_decode_attention_grouped(void *out, float *lse, const void *q, con
         // the ticket counter sits in the last 256 bytes of the workspace, behind the partials
         unsigned *ticket = reinterpret_cast<unsigned *>(
             static_cast<unsigned char *>(workspace) + grouped_workspace_for(pairs, p.rows, head_dim, plan) - 256);
-        if (head_dim == 128)
-            return paged ? launch_grouped_umma<128, true>(p, ticket, map_q, map_k, map_v, stream)
-                         : launch_grouped_umma<128, false>(p, ticket, map_q, map_k, map_v, stream);
-        return paged ? launch_grouped_umma<256, true>(p, ticket, map_q, map_k, map_v, stream)
-                     : launch_grouped_umma<256, false>(p, ticket, map_q, map_k, map_v, stream);
+        return head_dim == 128 ? launch_grouped_umma_rows<128>(paged, p, ticket, map_q, map_k, map_v, stream)
+                               : launch_grouped_umma_rows<256>(paged, p, ticket, map_q, map_k, map_v, stream);
     }
     switch (head_dim) {
     case 64: return paged ? launch_grouped<64, true>(p, grid, stream) : launch_grouped<64, false>(p, grid, stream);

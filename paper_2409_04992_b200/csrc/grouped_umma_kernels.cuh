@@ -163,6 +163,30 @@ __device__ __forceinline__ void tc_load16(float (&v)[16], unsigned taddr)     //
 #pragma unroll
     for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
 }
+// The first N (4, 8 or 16) columns of this thread's lane.
+template <int N>
+__device__ __forceinline__ void tc_load(float (&v)[N], unsigned taddr)
+{
+    static_assert(N == 4 || N == 8 || N == 16, "column counts of the loads used here");
+    unsigned r[N];
+    if constexpr (N == 16) {
+        float all[16];
+        tc_load16(all, taddr);
+#pragma unroll
+        for (int i = 0; i < 16; ++i) v[i] = all[i];
+        return;
+    } else if constexpr (N == 8) {
+        asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                     : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+                     : "r"(taddr) : "memory");
+    } else {
+        asm volatile("tcgen05.ld.sync.aligned.32x32b.x4.b32 {%0, %1, %2, %3}, [%4];"
+                     : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(taddr) : "memory");
+    }
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < N; ++i) v[i] = __uint_as_float(r[i]);
+}
 __device__ __forceinline__ void tc_store16(unsigned taddr, const float (&v)[16])
 {
     asm volatile("tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
@@ -270,7 +294,10 @@ __device__ __forceinline__ UmmaChunk umma_chunk(const AttnParams &a, int w, int 
 // Persistent: one block per SM; blocks draw chunks from a ticket counter (`ticket`, zeroed by
 // the host before the launch) until the list is exhausted, and the producers stream tiles
 // across chunk boundaries, so the copy pipeline never drains between chunks.
-template <int D, bool kPaged>
+// R: the query rows per KV head the softmax warps work on (4, 8 or 16; p.rows <= R): the MMAs
+// always take 16 rows, of which those from p.rows on are zeros, but logits, exponentials and
+// weights of rows that do not exist are not computed.
+template <int D, bool kPaged, int R>
 __global__ void __launch_bounds__(kUmmaThreads, 1)
 grouped_attn_umma_kernel(const GroupedParams p, unsigned *ticket, const __grid_constant__ CUtensorMap map_q,
                          const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v)
@@ -346,6 +373,9 @@ grouped_attn_umma_kernel(const GroupedParams p, unsigned *ticket, const __grid_c
         const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
         for (int i = threadIdx.x; i < kUmmaQBuffers * kQBytes / 16; i += 128)
             *reinterpret_cast<uint4 *>(smem + kQOffset + i * 16) = zero;
+        // so does the weight buffer: the columns of rows >= R are never written
+        for (int i = threadIdx.x; i < kUmmaPBytes / 16; i += 128)
+            *reinterpret_cast<uint4 *>(smem + kPOffset + i * 16) = zero;
         fence_async_proxy();
     }
     tc_fence_before();
@@ -714,9 +744,9 @@ grouped_attn_umma_kernel(const GroupedParams p, unsigned *ticket, const __grid_c
             const UmmaChunk c = umma_chunk(a, w, len);
             const int n_tiles = c.n_tiles;
             const unsigned acc = lane_base + 32 + (k & 1) * (kAccs * 32);     // this chunk's accumulator(s)
-            float m[16], l[16];
+            float m[R], l[R];
 #pragma unroll
-            for (int r = 0; r < 16; ++r) {
+            for (int r = 0; r < R; ++r) {
                 m[r] = kMinusHuge;
                 l[r] = 0.f;
             }
@@ -725,24 +755,24 @@ grouped_attn_umma_kernel(const GroupedParams p, unsigned *ticket, const __grid_c
                 const int sb = g & 1;
                 // (warp-uniform: the tensor-memory loads below are warp-wide instructions)
                 if (fine) fine = __all_sync(0xffffffffu, mbarrier_poll_bounded(misc + kUmmaBarSFull + sb * 8, (g >> 1) & 1));
-                float s[16];
+                float s[R];
                 if (fine) {
                     tc_fence_after();
-                    tc_load16(s, lane_base + sb * 16);
+                    tc_load<R>(s, lane_base + sb * 16);
                     tc_fence_before();
                 } else {
 #pragma unroll
-                    for (int r = 0; r < 16; ++r) s[r] = 0.f;
+                    for (int r = 0; r < R; ++r) s[r] = 0.f;
                 }
                 __syncwarp();
                 if (lane == 0) mbarrier_arrive(misc + kUmmaBarSFree + sb * 8);
                 const int tile_start = c.begin + j * kUmmaTile;
                 const int tok = tile_start + t;
 #pragma unroll
-                for (int r = 0; r < 16; ++r) s[r] *= a.scale_log2e;
+                for (int r = 0; r < R; ++r) s[r] *= a.scale_log2e;
                 if (tile_start + kUmmaTile > unmasked_end) {       // uniform: last tiles of the sequence / chunk
 #pragma unroll
-                    for (int r = 0; r < 16; ++r) {
+                    for (int r = 0; r < R; ++r) {
                         const int vis = r < p.rows ? len - (p.q_tokens - 1 - r / p.group) : 0;
                         if (tok >= min(vis, c.end)) s[r] = -INFINITY;
                     }
@@ -766,7 +796,7 @@ grouped_attn_umma_kernel(const GroupedParams p, unsigned *ticket, const __grid_c
                 }
                 bool moved = false;
 #pragma unroll
-                for (int r = 0; r < 16; ++r) moved = moved || s[r] > m[r] + kGroupLag;
+                for (int r = 0; r < R; ++r) moved = moved || s[r] > m[r] + kGroupLag;
                 if (!fine) *abort_word = 1u;
                 bool waited = false;
                 if (softmax_any(moved || !fine)) {
@@ -778,16 +808,17 @@ grouped_attn_umma_kernel(const GroupedParams p, unsigned *ticket, const __grid_c
                     // accumulator (and the sums) rescaled to them.
                     float tops[16];
 #pragma unroll
-                    for (int r = 0; r < 16; ++r) tops[r] = s[r];
+                    for (int r = 0; r < 16; ++r) tops[r] = r < R ? s[r % R] : kMinusHuge;
                     const float top_mine = warp_reduce16<true>(tops, lane);
                     if ((lane & 1) == 0) red[warp * 16 + warp_reduce16_row(lane)] = top_mine;
                     softmax_sync();
                     float alpha[16];
                     bool any_change = false;
 #pragma unroll
-                    for (int r = 0; r < 16; ++r) {
+                    for (int r = 0; r < 16; ++r) alpha[r] = 1.f;
+#pragma unroll
+                    for (int r = 0; r < R; ++r) {
                         const float top = fmaxf(fmaxf(red[r], red[16 + r]), fmaxf(red[32 + r], red[48 + r]));
-                        alpha[r] = 1.f;
                         if (top > m[r] + kGroupLag) {
                             alpha[r] = fast_exp2(m[r] - top);
                             m[r] = top;
@@ -819,7 +850,9 @@ grouped_attn_umma_kernel(const GroupedParams p, unsigned *ticket, const __grid_c
                 // (MN-major: 8 columns = 16 bytes per token and column block).
                 unsigned hi[8], lo[8];
 #pragma unroll
-                for (int i = 0; i < 8; ++i) {
+                for (int i = R / 2; i < 8; ++i) hi[i] = lo[i] = 0u;
+#pragma unroll
+                for (int i = 0; i < R / 2; ++i) {
                     const float w0 = fast_exp2(s[2 * i] - (m[2 * i] - kGroupWeightLog2));
                     const float w1 = fast_exp2(s[2 * i + 1] - (m[2 * i + 1] - kGroupWeightLog2));
                     l[2 * i] += w0;
@@ -834,9 +867,11 @@ grouped_attn_umma_kernel(const GroupedParams p, unsigned *ticket, const __grid_c
                 }
                 unsigned char *prow = smem + kPOffset + t * 16;
                 *reinterpret_cast<uint4 *>(prow) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-                *reinterpret_cast<uint4 *>(prow + 2048) = make_uint4(hi[4], hi[5], hi[6], hi[7]);
                 *reinterpret_cast<uint4 *>(prow + 4096) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
-                *reinterpret_cast<uint4 *>(prow + 6144) = make_uint4(lo[4], lo[5], lo[6], lo[7]);
+                if (R > 8) {                                        // rows 8-15: the second column block of each part
+                    *reinterpret_cast<uint4 *>(prow + 2048) = make_uint4(hi[4], hi[5], hi[6], hi[7]);
+                    *reinterpret_cast<uint4 *>(prow + 6144) = make_uint4(lo[4], lo[5], lo[6], lo[7]);
+                }
                 fence_async_proxy();
                 tc_fence_before();
                 __syncwarp();
@@ -850,12 +885,15 @@ grouped_attn_umma_kernel(const GroupedParams p, unsigned *ticket, const __grid_c
             }
             if (aborted) break;
             // the chunk's references and row sums, for its epilogue
-            const float sum_mine = warp_reduce16<false>(l, lane);
+            float sums[16];
+#pragma unroll
+            for (int r = 0; r < 16; ++r) sums[r] = r < R ? l[r % R] : 0.f;
+            const float sum_mine = warp_reduce16<false>(sums, lane);
             if ((lane & 1) == 0) saved_l[(k & 1) * 64 + warp * 16 + warp_reduce16_row(lane)] = sum_mine;
-            if (t < 16) {
+            if (t < R) {
                 float mine = m[0];
 #pragma unroll
-                for (int r = 1; r < 16; ++r) mine = t == r ? m[r] : mine;
+                for (int r = 1; r < R; ++r) mine = t == r ? m[r] : mine;
                 saved_m[(k & 1) * 16 + t] = mine;
             }
             before = c;
