@@ -82,7 +82,8 @@ def check(g_cpu, chunk, what):
                            lse.reshape(B, Tq * Hq), want_lse.reshape(B, Tq * Hq), what)
 
 
-SHAPES = [(1, 3, 3), (1, 8, 2), (1, 16, 2), (1, 16, 1), (4, 4, 4), (2, 8, 2), (16, 1, 1), (3, 10, 2)]
+# (rows per KV head: 1, 4, 8, 16, 4, 8, 16, 15, and 5 and 9: just above the row counts the tcgen05 form is compiled for)
+SHAPES = [(1, 3, 3), (1, 8, 2), (1, 16, 2), (1, 16, 1), (4, 4, 4), (2, 8, 2), (16, 1, 1), (3, 10, 2), (5, 1, 1), (3, 3, 1)]
 
 
 @pytest.mark.parametrize("q_tokens,q_heads,kv_heads", SHAPES)
@@ -102,7 +103,7 @@ def test_chunkings(chunk, q_tokens, q_heads, kv_heads):
 
 @pytest.mark.parametrize("dim", [64, 256])
 @pytest.mark.parametrize("layout,tokens", [("contiguous", 0), ("paged", 16), ("paged", 64), ("paged", 128)])
-@pytest.mark.parametrize("q_tokens,q_heads,kv_heads", [(1, 2, 2), (1, 8, 2), (2, 8, 1)])
+@pytest.mark.parametrize("q_tokens,q_heads,kv_heads", [(1, 2, 2), (1, 8, 2), (2, 8, 1), (3, 3, 1), (1, 5, 1)])
 def test_other_head_sizes(dim, layout, tokens, q_tokens, q_heads, kv_heads):
     for chunk in (0, 64, 128):
         check(make(layout, tokens, kv_heads, q_tokens, q_heads, dim=dim), chunk,
